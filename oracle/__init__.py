@@ -1,0 +1,207 @@
+"""ctypes front end of the CPU oracle (``qv2_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by ``__graft_entry__.smoke()`` and by the
+``cpu_baseline`` / ``--impl reference`` legs of ``bench.py``.  The CUDA package never imports it
+and it never imports the CUDA package.  The arithmetic lives in the C file; this module only
+marshals numpy arrays and strings the per-tensor steps together in the paper's order
+(calibrate -> parameters -> fake-quantize and measure -> rank).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "qv2_oracle.c")
+_LIB = os.path.join(_HERE, "libqv2_oracle.so")
+BINS = 2048
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc.  -ffp-contract=off keeps every multiply and add a separate,
+    individually rounded operation."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True, cwd=_HERE)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = C.CDLL(build())
+    f32p, u64p, f64p, u8p, u32p = (C.POINTER(C.c_float), C.POINTER(C.c_uint64),
+                                   C.POINTER(C.c_double), C.POINTER(C.c_uint8),
+                                   C.POINTER(C.c_uint32))
+    lib.qv2o_ranges.argtypes = [f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_int,
+                                f32p, f32p, f32p, u64p]
+    lib.qv2o_ranges.restype = None
+    lib.qv2o_histogram.argtypes = [f32p, C.c_uint64, C.c_float, u64p]
+    lib.qv2o_histogram.restype = None
+    lib.qv2o_percentile_clip.argtypes = [u64p, C.c_double, C.c_float]
+    lib.qv2o_percentile_clip.restype = C.c_float
+    lib.qv2o_qparams.argtypes = [C.c_int, C.c_int, C.c_float, C.c_uint64, f32p, f32p, f32p,
+                                 f32p, f32p, f32p]
+    lib.qv2o_qparams.restype = None
+    lib.qv2o_quant_metrics.argtypes = [f32p, f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_int,
+                                       C.c_int, C.c_int, f32p, f32p, f32p, u8p,
+                                       f64p, f64p, f64p, f64p]
+    lib.qv2o_quant_metrics.restype = None
+    lib.qv2o_rank.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p,
+                              C.c_double, C.c_double, C.c_double, C.c_double,
+                              C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
+    lib.qv2o_rank.restype = None
+    _lib = lib
+    return lib
+
+
+def _p(a: Optional[np.ndarray], ct):
+    return None if a is None else a.ctypes.data_as(C.POINTER(ct))
+
+
+def _f32(a) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a
+
+
+# ------------------------------------------------------------------------------ per-step calls
+def ranges(x, outer: int, channels: int, inner: int, per_channel: bool):
+    """-> (gmin, gmax, gabsmax, nonfinite) over the groups of x viewed [outer][channels][inner]."""
+    lib = _load()
+    x = _f32(x).reshape(-1)
+    assert x.size == outer * channels * inner
+    g = channels if per_channel else 1
+    gmin = np.zeros(g, np.float32); gmax = np.zeros(g, np.float32); gabs = np.zeros(g, np.float32)
+    bad = C.c_uint64(0)
+    lib.qv2o_ranges(_p(x, C.c_float), outer, channels, inner, int(per_channel),
+                    _p(gmin, C.c_float), _p(gmax, C.c_float), _p(gabs, C.c_float), C.byref(bad))
+    return gmin, gmax, gabs, int(bad.value)
+
+
+def histogram(x, absmax: float) -> np.ndarray:
+    lib = _load()
+    x = _f32(x).reshape(-1)
+    hist = np.zeros(BINS, np.uint64)
+    lib.qv2o_histogram(_p(x, C.c_float), x.size, C.c_float(absmax), _p(hist, C.c_uint64))
+    return hist
+
+
+def percentile_clip(hist: np.ndarray, p: float, absmax: float) -> np.float32:
+    lib = _load()
+    hist = np.ascontiguousarray(hist, dtype=np.uint64)
+    return np.float32(lib.qv2o_percentile_clip(_p(hist, C.c_uint64), float(p), C.c_float(absmax)))
+
+
+def qparams(asym_u8: bool, gmin, gmax, gabsmax, clip: Optional[float] = None):
+    lib = _load()
+    gmin, gmax, gabsmax = _f32(gmin), _f32(gmax), _f32(gabsmax)
+    g = gmin.size
+    step = np.zeros(g, np.float32); inv = np.zeros(g, np.float32); off = np.zeros(g, np.float32)
+    lib.qv2o_qparams(int(asym_u8), int(clip is not None), C.c_float(0.0 if clip is None else clip),
+                     g, _p(gmin, C.c_float), _p(gmax, C.c_float), _p(gabsmax, C.c_float),
+                     _p(step, C.c_float), _p(inv, C.c_float), _p(off, C.c_float))
+    return step, inv, off
+
+
+PAIR_SELF, PAIR_REQUANT, PAIR_RAW = 0, 1, 2
+
+
+def quant_metrics(x, y, outer: int, channels: int, inner: int, per_channel: bool, asym_u8: bool,
+                  pair_mode: int, step, inv, offset, want_codes: bool = False):
+    """-> dict(sse, sig, mse, sqnr_db[, codes])."""
+    lib = _load()
+    x = _f32(x).reshape(-1)
+    yy = None if y is None else _f32(y).reshape(-1)
+    if pair_mode != PAIR_SELF:
+        assert yy is not None and yy.size == x.size
+    step, inv, offset = _f32(step), _f32(inv), _f32(offset)
+    codes = np.zeros(x.size, np.uint8) if want_codes else None
+    out = [C.c_double(0.0) for _ in range(4)]
+    lib.qv2o_quant_metrics(_p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
+                           int(per_channel), int(asym_u8), int(pair_mode),
+                           _p(step, C.c_float), _p(inv, C.c_float), _p(offset, C.c_float),
+                           _p(codes, C.c_uint8), *[C.byref(o) for o in out])
+    res = dict(sse=out[0].value, sig=out[1].value, mse=out[2].value, sqnr_db=out[3].value)
+    if want_codes:
+        res["codes"] = codes if asym_u8 else codes.view(np.int8)
+    return res
+
+
+def rank_layers(sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, w_gain=2.0, a_gain=1.0,
+                mse_factor=5.0, cap_db=200.0, select_mode=0, keep_count=0, rate_permyriad=0):
+    """-> (order[n] uint32, keep_fp32[n] uint8, n_keep)."""
+    lib = _load()
+    f = lambda a: np.ascontiguousarray(a, dtype=np.float64)
+    sqnr_w, mse_w, sqnr_a, mse_a = f(sqnr_w), f(mse_w), f(sqnr_a), f(mse_a)
+    n = sqnr_w.size
+    m = None if macs is None else np.ascontiguousarray(macs, dtype=np.uint64)
+    ps = None if pos is None else f(pos)
+    order = np.zeros(n, np.uint32); keep = np.zeros(n, np.uint8); nk = C.c_uint32(0)
+    lib.qv2o_rank(n, _p(sqnr_w, C.c_double), _p(mse_w, C.c_double), _p(sqnr_a, C.c_double),
+                  _p(mse_a, C.c_double), _p(m, C.c_uint64), _p(ps, C.c_double),
+                  w_gain, a_gain, mse_factor, cap_db, int(select_mode), int(keep_count),
+                  int(rate_permyriad), _p(order, C.c_uint32), _p(keep, C.c_uint8), C.byref(nk))
+    return order, keep, int(nk.value)
+
+
+# --------------------------------------------------------------------------- per-tensor sweep
+@dataclass
+class TensorResult:
+    gmin: np.ndarray
+    gmax: np.ndarray
+    gabsmax: np.ndarray
+    nonfinite: int
+    hist: Optional[np.ndarray]
+    clip: np.float32
+    step: np.ndarray
+    inv: np.ndarray
+    offset: np.ndarray
+    sse: float
+    sig: float
+    mse: float
+    sqnr_db: float
+    codes: Optional[np.ndarray] = None
+
+
+def calibrate_tensor(x, outer, channels, inner, per_channel, asym_u8, percentile=None):
+    """Ranges, optional |x| histogram + percentile clip, then the quantization parameters."""
+    gmin, gmax, gabs, bad = ranges(x, outer, channels, inner, per_channel)
+    A = np.float32(gabs.max()) if gabs.size else np.float32(0.0)
+    hist, clip = None, A
+    if percentile is not None:
+        hist = histogram(x, float(A))
+        clip = percentile_clip(hist, percentile, float(A))
+    step, inv, off = qparams(asym_u8, gmin, gmax, gabs, None if percentile is None else float(clip))
+    return gmin, gmax, gabs, bad, hist, clip, step, inv, off
+
+
+def sweep_tensor(x, y, outer, channels, inner, per_channel, asym_u8, percentile=None,
+                 pair_mode=None, want_codes=False) -> TensorResult:
+    """Calibrate on x, then measure: self mode when y is None, else the paired mode."""
+    gmin, gmax, gabs, bad, hist, clip, step, inv, off = calibrate_tensor(
+        x, outer, channels, inner, per_channel, asym_u8, percentile)
+    if pair_mode is None:
+        pair_mode = PAIR_SELF if y is None else PAIR_REQUANT
+    m = quant_metrics(x, y, outer, channels, inner, per_channel, asym_u8, pair_mode,
+                      step, inv, off, want_codes)
+    return TensorResult(gmin, gmax, gabs, bad, hist, clip, step, inv, off,
+                        m["sse"], m["sig"], m["mse"], m["sqnr_db"], m.get("codes"))
+
+
+def sweep_tensors(jobs: Sequence[dict], threads: int = 1) -> List[TensorResult]:
+    """Run sweep_tensor over independent tensors.  ``threads`` > 1 runs whole tensors side by
+    side (the C calls release the GIL); each tensor is still swept by the serial code above."""
+    if threads <= 1:
+        return [sweep_tensor(**j) for j in jobs]
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(lambda j: sweep_tensor(**j), jobs))

@@ -1,0 +1,417 @@
+"""Pins for the CPU oracle: each function is checked against something other than itself --
+closed forms, exact constructions in which every operation is exact, library routines on
+special cases, brute force with Python integers / fractions, and invariants.  A dropped term,
+a wrong sign or index, or a transposed operand in the oracle fails at least one test here.
+No GPU is involved."""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+
+RNG = np.random.default_rng(20250107)
+
+
+# ----------------------------------------------------------------------------------- ranges
+def test_ranges_match_numpy_per_tensor_and_per_channel():
+    o, c, i = 3, 5, 7
+    x = RNG.standard_normal((o, c, i)).astype(np.float32)
+    mn, mx, am, bad = oracle.ranges(x, o, c, i, False)
+    assert bad == 0 and mn[0] == x.min() and mx[0] == x.max()
+    assert am[0] == np.abs(x).max()
+    mn, mx, am, bad = oracle.ranges(x, o, c, i, True)
+    # channel is the MIDDLE axis: a transposed view must not match unless indexing is right
+    np.testing.assert_array_equal(mn, x.min(axis=(0, 2)))
+    np.testing.assert_array_equal(mx, x.max(axis=(0, 2)))
+    np.testing.assert_array_equal(am, np.abs(x).max(axis=(0, 2)))
+    assert not np.array_equal(mn, x.reshape(o, i, c).min(axis=(0, 1)))
+
+
+def test_ranges_planted_extremes_first_last_and_group_boundary():
+    c, i = 4, 9
+    x = np.zeros((1, c, i), np.float32)
+    x[0, 0, 0] = -3.0       # first element of the tensor
+    x[0, 3, 8] = 5.0        # last element
+    x[0, 1, 8] = 7.0        # last element of group 1
+    x[0, 2, 0] = -9.0       # first element of group 2
+    mn, mx, am, _ = oracle.ranges(x, 1, c, i, True)
+    np.testing.assert_array_equal(mn, np.float32([-3, 0, -9, 0]))
+    np.testing.assert_array_equal(mx, np.float32([0, 7, 0, 5]))
+    np.testing.assert_array_equal(am, np.float32([3, 7, 9, 5]))
+    mn, mx, am, _ = oracle.ranges(x, 1, c, i, False)
+    assert (mn[0], mx[0], am[0]) == (-9.0, 7.0, 9.0)
+
+
+def test_ranges_negative_zero_and_nonfinite():
+    x = np.float32([-0.0, -0.0, np.nan, np.inf, -np.inf, -0.0])
+    mn, mx, am, bad = oracle.ranges(x, 1, 1, 6, False)
+    assert bad == 3
+    for v in (mn[0], mx[0], am[0]):
+        assert v == 0.0 and not np.signbit(v)
+    x = np.float32([np.nan, 2.0, -1.0, np.inf])
+    mn, mx, am, bad = oracle.ranges(x, 1, 1, 4, False)
+    assert (mn[0], mx[0], am[0], bad) == (-1.0, 2.0, 2.0, 2)
+    x = np.float32([np.nan, np.nan])
+    mn, mx, am, bad = oracle.ranges(x, 1, 2, 1, True)
+    assert bad == 2 and not mn.any() and not mx.any() and not am.any()
+
+
+# -------------------------------------------------------------------------------- histogram
+def test_histogram_planted_bin_centres_and_top_edge():
+    A = 4.0  # power of two: 2048/A and every product below are exact
+    j = np.arange(2048)
+    x = ((j + 0.5) * (A / 2048)).astype(np.float32)
+    x = np.concatenate([x, -x, np.float32([A, -A])])   # |x| is what is binned
+    h = oracle.histogram(x, A)
+    expect = np.full(2048, 2, np.uint64)
+    expect[2047] += 2                                  # x = +-A lands in the last bin
+    np.testing.assert_array_equal(h, expect)
+    assert h.sum() == x.size
+
+
+def test_histogram_ramp_is_flat_and_percentile_closed_form():
+    A, per = 8.0, 16
+    n = 2048 * per
+    x = ((np.arange(n) + 0.5) * (A / n)).astype(np.float32)   # exact: A/n is a power of two
+    x[-1] = A                                                 # make A the absmax
+    h = oracle.histogram(x, A)
+    np.testing.assert_array_equal(h, np.full(2048, per, np.uint64))
+    # cumulative count reaches ceil(0.99 n) first in bin k* with (k*+1) >= 0.99*2048 = 2027.52
+    clip = oracle.percentile_clip(h, 0.99, A)
+    assert clip == np.float32(2028 * A / 2048)
+    assert oracle.percentile_clip(h, 1.0, A) == np.float32(A)       # k* = 2047 -> A itself
+    assert oracle.percentile_clip(h, 0.0, A) == np.float32(A / 2048)  # T clamps to 1 -> bin 0
+    assert oracle.percentile_clip(h, 0.5, A) == np.float32(A / 2)
+
+
+def test_histogram_zeros_nonfinite_and_degenerate():
+    x = np.zeros(1000, np.float32)
+    h = oracle.histogram(x, 0.0)
+    assert h[0] == 1000 and h[1:].sum() == 0
+    assert oracle.percentile_clip(h, 0.9999, 0.0) == 0.0
+    # half zeros (post-ReLU): the zero mass sits in bin 0 and pushes the median bin to 0
+    x = np.concatenate([np.zeros(500, np.float32), np.linspace(0.5, 1.0, 500, dtype=np.float32)])
+    h = oracle.histogram(x, 1.0)
+    assert h[0] == 500 and h.sum() == 1000 and h[1:1024].sum() == 0
+    assert oracle.percentile_clip(h, 0.5, 1.0) == np.float32(1.0 / 2048)
+    x = np.float32([np.nan, np.inf, 0.25, -np.inf, 1.0])
+    h = oracle.histogram(x, 1.0)
+    assert h.sum() == 2 and h[512] == 1 and h[2047] == 1
+
+
+def test_histogram_matches_numpy_on_random_data():
+    x = (RNG.standard_normal(50_000) * 0.7).astype(np.float32)
+    A = np.float32(np.abs(x).max())
+    h = oracle.histogram(x, float(A))
+    w = np.float32(2048) / A
+    b = np.minimum((np.abs(x) * w).astype(np.float32).astype(np.int64), 2047)
+    np.testing.assert_array_equal(h, np.bincount(b, minlength=2048).astype(np.uint64))
+    # percentile against a direct sort: the clip is the upper edge of the bin holding the
+    # T-th smallest |x|
+    p = 0.999
+    T = math.ceil(p * x.size)
+    kth = np.sort(np.abs(x))[T - 1]
+    kbin = min(int(np.float32(kth * w)), 2047)
+    clip = oracle.percentile_clip(h, p, float(A))
+    assert clip == np.float32(np.float32(kbin + 1) * np.float32(A / np.float32(2048)))
+
+
+# --------------------------------------------------------------------------------- qparams
+def test_qparams_symmetric_and_asymmetric_definitions():
+    gmin = np.float32([-1.27, 0.0, -2.0]); gmax = np.float32([0.5, 2.55, 6.0])
+    gabs = np.maximum(np.abs(gmin), np.abs(gmax))
+    step, inv, off = oracle.qparams(False, gmin, gmax, gabs)
+    np.testing.assert_array_equal(step, gabs / np.float32(127))
+    np.testing.assert_array_equal(inv, np.float32(127) / gabs)
+    assert not off.any()
+    step, inv, off = oracle.qparams(True, gmin, gmax, gabs)
+    d = gmax - gmin
+    np.testing.assert_array_equal(step, d / np.float32(255))
+    np.testing.assert_array_equal(inv, np.float32(255) / d)
+    np.testing.assert_array_equal(off, gmin)
+    # percentile clip narrows both schemes
+    step, inv, off = oracle.qparams(False, gmin, gmax, gabs, clip=1.0)
+    np.testing.assert_array_equal(step, np.minimum(gabs, 1) / np.float32(127))
+    step, inv, off = oracle.qparams(True, gmin, gmax, gabs, clip=1.0)
+    np.testing.assert_array_equal(off, np.maximum(gmin, -1))
+    np.testing.assert_array_equal(step, (np.minimum(gmax, 1) - np.maximum(gmin, -1)) / np.float32(255))
+    # degenerate ranges fall back to a unit grid
+    z = np.zeros(1, np.float32)
+    for asym in (False, True):
+        step, inv, off = oracle.qparams(asym, z, z, z)
+        assert step[0] == 1.0 and inv[0] == 1.0 and off[0] == 0.0
+
+
+# ------------------------------------------------------------------------ codes and metrics
+def _self(x, per_channel=False, asym=False, shape=None, percentile=None, codes=True):
+    x = np.asarray(x, np.float32)
+    o, c, i = shape if shape else (1, 1, x.size)
+    return oracle.sweep_tensor(x, None, o, c, i, per_channel, asym, percentile, want_codes=codes)
+
+
+def test_on_grid_tensor_has_zero_error_symmetric():
+    d = 2.0 ** -7
+    k = np.arange(-127, 128)
+    r = _self(k * d)
+    np.testing.assert_array_equal(r.codes, k.astype(np.int8))
+    assert r.step[0] == np.float32(d) and r.sse == 0.0 and r.mse == 0.0 and r.sqnr_db == math.inf
+
+
+def test_on_grid_tensor_has_zero_error_asymmetric_with_offset():
+    d = 2.0 ** -6
+    k = np.arange(0, 256)
+    lo = -1.0                      # offset is the real-valued minimum, range need not hold 0
+    r = _self(k * d + lo, asym=True)
+    np.testing.assert_array_equal(r.codes, k.astype(np.uint8))
+    assert r.offset[0] == np.float32(lo) and r.step[0] == np.float32(d)
+    assert r.sse == 0.0 and r.sqnr_db == math.inf
+
+
+def test_exact_ties_round_to_even():
+    d = 2.0 ** -7
+    k = np.arange(-126, 126)
+    x = np.concatenate([(k + 0.5) * d, [127 * d, -127 * d]])     # absmax fixes the grid
+    r = _self(x)
+    even = np.where(k % 2 == 0, k, k + 1)
+    np.testing.assert_array_equal(r.codes[:-2], even.astype(np.int8))
+    # every error is exactly half a step
+    assert r.sse == pytest.approx(k.size * (d / 2) ** 2, rel=1e-15)
+
+
+def test_saturation_beyond_percentile_clip():
+    # 9999 small values and one huge one: the 99 % clip lands far below the outlier, which
+    # must saturate at +127 (symmetric) / 255 (asymmetric) instead of wrapping
+    x = np.concatenate([np.linspace(-1, 1, 9999), [50.0, -60.0]]).astype(np.float32)
+    r = _self(x, percentile=0.99)
+    assert r.clip < 2.0 and r.codes[-2] == 127 and r.codes[-1] == -127
+    assert abs(r.codes[:-2].astype(int)).max() <= 127
+    r = _self(x, asym=True, percentile=0.99)
+    assert r.codes[-2] == 255 and r.codes[-1] == 0
+
+
+def test_power_of_two_scaling_invariance():
+    x = (RNG.standard_normal(20_000)).astype(np.float32)
+    for asym in (False, True):
+        base = _self(x, asym=asym)
+        for m in (-9, 5):
+            s = _self(x * np.float32(2.0 ** m), asym=asym)
+            np.testing.assert_array_equal(base.codes, s.codes)
+            assert s.mse == pytest.approx(base.mse * 4.0 ** m, rel=1e-14)
+            assert s.sqnr_db == pytest.approx(base.sqnr_db, abs=1e-10)
+
+
+def test_codes_agree_with_semantic_double_quantizer():
+    """rne(x / Delta) in pure double differs from the binary32 definition only where x/Delta
+    sits within rounding error of a tie."""
+    x = RNG.standard_normal(400_000).astype(np.float32)
+    r = _self(x)
+    t = x.astype(np.float64) / (float(r.gabsmax[0]) / 127.0)
+    q = np.clip(np.rint(t), -127, 127).astype(np.int64)
+    diff = q != r.codes.astype(np.int64)
+    assert diff.mean() < 1e-4
+    frac = np.abs(t - np.floor(t) - 0.5)
+    assert (frac[diff] < 1e-4).all()
+    assert np.abs(q - r.codes.astype(np.int64)).max() <= 1
+
+
+def test_mse_brute_force_python_fractions():
+    """Tiny tensor, every step redone with exact rational arithmetic."""
+    x = np.float32([0.11, -0.52, 0.9, 0.333, -1.0, 0.75, 0.0, 0.49])
+    r = _self(x)
+    step = Fraction(float(r.step[0]))
+    sse = Fraction(0); sig = Fraction(0)
+    for v, q in zip(x, r.codes):
+        e = Fraction(float(v)) - int(q) * step
+        sse += e * e
+        sig += Fraction(float(v)) ** 2
+    assert r.sse == pytest.approx(float(sse), rel=1e-15)
+    assert r.sig == pytest.approx(float(sig), rel=1e-15)
+    assert r.mse == pytest.approx(float(sse / 8), rel=1e-15)
+    assert r.sqnr_db == pytest.approx(10 * math.log10(float(sig / sse)), abs=1e-12)
+    # the codes themselves: nearest grid point, checked without the oracle's own formula
+    for v, q in zip(x, r.codes):
+        assert abs(Fraction(float(v)) - int(q) * step) <= step / 2 + Fraction(1, 10 ** 9)
+
+
+def test_uniform_noise_midpoint_construction_gives_delta_sq_over_12():
+    """M equispaced points in every full cell of the symmetric grid: the mean squared error of
+    a cell is (Delta^2/12)(1 - 1/M^2) exactly; all values and products are exact in binary32."""
+    d, M = 2.0 ** -7, 64
+    k = np.arange(-126, 127)[:, None]
+    j = np.arange(M)[None, :]
+    x = ((k - 0.5) + (j + 0.5) / M) * d
+    x = np.concatenate([x.reshape(-1), [127 * d, -127 * d]])
+    r = _self(x, codes=False)
+    n_cell = 253 * M
+    expect = (d * d / 12) * (1 - 1 / M ** 2) * n_cell / (n_cell + 2)
+    assert r.mse == pytest.approx(expect, rel=1e-13)
+
+
+def test_uniform_random_mse_and_sqnr_closed_forms():
+    n = 1 << 22
+    u = RNG.random(n)
+    xs = ((2 * u - 1) * 3.0).astype(np.float32)
+    r = _self(xs, codes=False)
+    d = float(r.step[0])
+    assert r.mse == pytest.approx(d * d / 12, rel=3e-3)
+    assert r.sqnr_db == pytest.approx(20 * math.log10(254), abs=0.02)       # 48.097 dB
+    xa = (u * 5.0).astype(np.float32)
+    r = _self(xa, asym=True, codes=False)
+    assert r.sqnr_db == pytest.approx(10 * math.log10(4 * 255 ** 2), abs=0.02)  # 54.151 dB
+    assert r.sqnr_db == pytest.approx(10 * math.log10(r.sig / (n * r.mse)), abs=1e-9)
+
+
+def test_per_channel_uses_the_middle_axis_and_own_scale():
+    o, c, i = 2, 3, 5
+    x = RNG.standard_normal((o, c, i)).astype(np.float32)
+    x[:, 1, :] *= 100.0          # one loud channel
+    r = _self(x, per_channel=True, shape=(o, c, i))
+    sse = 0.0
+    for ch in range(c):
+        sub = np.ascontiguousarray(x[:, ch, :])
+        rc = _self(sub)
+        # codes of channel ch equal a stand-alone per-tensor quantization of that channel
+        np.testing.assert_array_equal(r.codes.reshape(o, c, i)[:, ch, :].reshape(-1), rc.codes)
+        sse += rc.sse
+    assert r.sse == pytest.approx(sse, rel=1e-14)
+    rt = _self(x)                # per-tensor: the loud channel sets everyone's step
+    assert rt.mse > 2 * r.mse
+
+
+def test_pair_modes():
+    x = RNG.standard_normal(5000).astype(np.float32)
+    y = (x + 0.01 * RNG.standard_normal(5000)).astype(np.float32)
+    raw = oracle.sweep_tensor(x, y, 1, 1, 5000, False, True, pair_mode=oracle.PAIR_RAW)
+    d = x.astype(np.float64) - y.astype(np.float64)
+    assert raw.sse == pytest.approx(float((d * d).sum()), rel=1e-14)
+    assert raw.sig == pytest.approx(float((x.astype(np.float64) ** 2).sum()), rel=1e-14)
+    rq = oracle.sweep_tensor(x, y, 1, 1, 5000, False, True, want_codes=True)
+    # parameters come from x; codes are those of y on x's grid; error is x minus dequantized y
+    own = oracle.quant_metrics(y, None, 1, 1, 5000, False, True, oracle.PAIR_SELF,
+                               rq.step, rq.inv, rq.offset, want_codes=True)
+    np.testing.assert_array_equal(rq.codes, own["codes"])
+    yhat = rq.codes.astype(np.float64) * float(rq.step[0]) + float(rq.offset[0])
+    e = x.astype(np.float64) - yhat
+    assert rq.sse == pytest.approx(float((e * e).sum()), rel=1e-14)
+    # swapping the operands changes the signal term: SIG is always the reference tensor
+    sw = oracle.sweep_tensor(y, x, 1, 1, 5000, False, True, pair_mode=oracle.PAIR_RAW)
+    assert sw.sse == pytest.approx(raw.sse, rel=1e-14) and sw.sig != raw.sig
+    # y identical to an on-grid x: zero noise
+    z = oracle.sweep_tensor(x, x, 1, 1, 5000, False, True, pair_mode=oracle.PAIR_RAW)
+    assert z.sse == 0.0 and z.sqnr_db == math.inf
+    zero_sig = oracle.sweep_tensor(np.zeros(4, np.float32), np.ones(4, np.float32), 1, 1, 4,
+                                   False, True, pair_mode=oracle.PAIR_RAW)
+    assert zero_sig.sqnr_db == -math.inf and zero_sig.mse == 1.0
+
+
+# ------------------------------------------------------------------------------------- rank
+def _py_rank(sw, mw, sa, ma, pos=None, wg=2.0, ag=1.0, fac=5.0, cap=200.0):
+    """Independent restatement with Python floats and the library sort."""
+    n = len(sw)
+    cl = lambda v: max(-cap, min(cap, v))
+    score, sev = [], []
+    mean_w = sum(mw) / n; mean_a = sum(ma) / n
+    for i in range(n):
+        if i == 0:
+            dw = da = 0.0
+        else:
+            den = (pos[i] - pos[i - 1]) if pos is not None else 1.0
+            dw = (cl(sw[i]) - cl(sw[i - 1])) / den
+            da = (cl(sa[i]) - cl(sa[i - 1])) / den
+        score.append(wg * dw + ag * da)
+        rw = mw[i] / mean_w if mean_w > 0 else 0.0
+        ra = ma[i] / mean_a if mean_a > 0 else 0.0
+        sev.append(max(rw, ra))
+    out = sorted([i for i in range(n) if sev[i] > fac], key=lambda i: (-sev[i], i))
+    rest = sorted([i for i in range(n) if sev[i] <= fac], key=lambda i: (score[i], i))
+    return out + rest
+
+
+def test_rank_hand_worked_six_layers():
+    # SQNR (dB) per layer; deltas: w = [0,-5,+2,-1,+6,-8], a = [0,+1,-4,+3,-2,+1]
+    sw = [40.0, 35.0, 37.0, 36.0, 42.0, 34.0]
+    sa = [30.0, 31.0, 27.0, 30.0, 28.0, 29.0]
+    # score = 2*dw + da = [0,-9,0,1,10,-15]
+    mw = [1.0, 1.0, 1.0, 1.0, 1.0, 1.0]
+    ma = [1.0, 1.0, 1.0, 1.0, 1.0, 1.0]
+    order, keep, nk = oracle.rank_layers(sw, mw, sa, ma, keep_count=2)
+    assert order.tolist() == [5, 1, 0, 2, 3, 4]        # tie between layers 0 and 2 keeps layer order
+    assert keep.tolist() == [0, 1, 0, 0, 0, 1] and nk == 2
+    # layer 3 becomes an MSE outlier (its MSE is > 5x the mean): it jumps to the top
+    ma2 = [1.0, 1.0, 1.0, 60.0, 1.0, 1.0]              # mean 10.83, ratio 5.54
+    order, _, _ = oracle.rank_layers(sw, mw, sa, ma2)
+    assert order.tolist() == [3, 5, 1, 0, 2, 4]
+    ma3 = [1.0, 1.0, 1.0, 25.0, 1.0, 1.0]              # mean 5, ratio exactly 5: not an outlier
+    order, _, _ = oracle.rank_layers(sw, mw, sa, ma3)
+    assert order.tolist() == [5, 1, 0, 2, 3, 4]
+    # two outliers: the more severe one first, whichever list it came from
+    mw4 = [1.0, 1.0, 100.0, 1.0, 1.0, 1.0]             # ratio 100/17.5 = 5.71
+    order, _, _ = oracle.rank_layers(sw, mw4, sa, ma2)
+    assert order.tolist()[:2] == [2, 3]
+
+
+def test_rank_degenerate_variants_of_the_ablation():
+    n = 12
+    sw = RNG.uniform(20, 50, n); sa = RNG.uniform(20, 50, n)
+    ones = np.ones(n)
+    # activation gain 0 and no outliers: argsort of the weight-SQNR deltas
+    order, _, _ = oracle.rank_layers(sw, ones, sa, ones, a_gain=0.0, w_gain=1.0)
+    d = np.concatenate([[0.0], np.diff(sw)])
+    assert order.tolist() == np.argsort(d, kind="stable").tolist()
+    # feeding cumulative sums turns deltas back into raw SQNR: Weight-SQNR-Order baseline
+    csw = np.cumsum(sw)
+    order, _, _ = oracle.rank_layers(csw, ones, sa, ones, a_gain=0.0, w_gain=1.0, cap_db=1e9)
+    expect = np.argsort(np.concatenate([[0.0], sw[1:]]), kind="stable").tolist()
+    assert order.tolist() == expect
+    # positions stretch the denominator
+    pos = np.cumsum(RNG.integers(1, 4, n)).astype(float)
+    order, _, _ = oracle.rank_layers(sw, ones, sa, ones, pos=pos)
+    assert order.tolist() == _py_rank(list(sw), list(ones), list(sa), list(ones), list(pos))
+
+
+def test_rank_matches_library_sort_on_random_inputs_and_is_a_permutation():
+    for trial in range(300):
+        n = int(RNG.integers(1, 9))
+        sw = RNG.uniform(-10, 60, n).round(1)          # rounding provokes ties
+        sa = RNG.uniform(-10, 60, n).round(1)
+        mw = RNG.choice([0.0, 1e-6, 1e-5, 3e-4], n)
+        ma = RNG.choice([1e-3, 2e-3, 9e-2], n)
+        if trial % 7 == 0:
+            sw[RNG.integers(0, n)] = math.inf          # zero-noise layer, clamped to the cap
+        order, keep, nk = oracle.rank_layers(sw, mw, sa, ma)
+        assert sorted(order.tolist()) == list(range(n))
+        assert order.tolist() == _py_rank(list(sw), list(mw), list(sa), list(ma))
+        assert nk == 0 and not keep.any()
+
+
+def test_select_by_bops_rate_against_prefix_enumeration():
+    for _ in range(200):
+        n = int(RNG.integers(1, 9))
+        sw = RNG.uniform(20, 50, n); sa = RNG.uniform(20, 50, n)
+        macs = RNG.integers(0, 1000, n).astype(np.uint64)
+        rate = int(RNG.integers(0, 10001))
+        order, keep, nk = oracle.rank_layers(sw, np.ones(n), sa, np.ones(n), macs=macs,
+                                             select_mode=1, rate_permyriad=rate)
+        total = int(macs.sum())
+        best = 0
+        for k in range(n + 1):                         # every prefix, exact rationals
+            q = total - sum(int(macs[i]) for i in order[:k])
+            ok = Fraction(q * 10000) >= Fraction(rate * total)
+            if ok:
+                best = k
+            else:
+                break                                  # the rate only falls as the prefix grows
+        assert nk == best
+        assert keep.sum() == nk and all(keep[i] for i in order[:nk])
+    # 0 % keeps everything in FP32, 100 % quantizes every layer that has work
+    order, keep, nk = oracle.rank_layers([30, 20], [1, 1], [30, 20], [1, 1], macs=[5, 5],
+                                         select_mode=1, rate_permyriad=0)
+    assert nk == 2
+    order, keep, nk = oracle.rank_layers([30, 20], [1, 1], [30, 20], [1, 1], macs=[5, 5],
+                                         select_mode=1, rate_permyriad=10000)
+    assert nk == 0
+    order, keep, nk = oracle.rank_layers([30, 20], [1, 1], [30, 20], [1, 1], macs=[5, 5],
+                                         select_mode=1, rate_permyriad=5000)
+    assert nk == 1 and keep[order[0]] == 1
