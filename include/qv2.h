@@ -1,0 +1,249 @@
+/*
+ * qv2 -- local-metric sensitivity sweep of QuantuneV2 (arXiv 2501.07161) on one NVIDIA B200.
+ *
+ * For every layer of a model the sweep calibrates quantization ranges over the weight tensor and
+ * the captured activation tensor, fake-quantizes to 8 bit, reduces the quantization error to MSE
+ * and SQNR, and finally scores, ranks and selects the layers that stay in FP32 (the paper's
+ * "Sensitivity Analyzer", steps 1-4 of its overview and Algorithm 2).
+ *
+ * Conventions common to every call
+ *   - Plain C ABI.  Every function returns an int status: QV2_OK (0) or a negative QV2_ERR_*.
+ *     Nothing throws, aborts or traps on the device.
+ *   - "device" pointers are CUDA global-memory addresses valid on the context's device, "host"
+ *     pointers are ordinary process memory.  The caller owns every tensor and every output buffer;
+ *     the library owns only the scratch inside qv2_ctx (tile tables and partial sums), grown on
+ *     demand and released by qv2_destroy.
+ *   - Calls enqueue work on the context's stream and return; outputs are valid once the caller has
+ *     synchronised that stream.  Argument errors are found on the host before anything is
+ *     launched.  Exceptions: a call whose descriptor set differs from the previous call's
+ *     synchronises the stream once while it rebuilds its tile table, and qv2_sweep_model_host
+ *     synchronises before it returns.
+ *   - One context serves one stream; use it from one host thread at a time.
+ *   - Tensors are fp32, contiguous, viewed as [outer][channels][inner]; element (o,c,i) lives at
+ *     index (o*channels + c)*inner + i.  Weights: outer = 1, channels = C_out, inner = C_in/g*k*k.
+ *     Activations: outer = batch, channels = C, inner = H*W.  The quantization group of an element
+ *     is its channel c (QV2_PER_CHANNEL) or 0 (QV2_PER_TENSOR).  Per-group arrays hold the groups
+ *     of descs[0], then those of descs[1], ...; qv2_group_count gives the total.
+ *   - Non-finite input elements are counted into nonfinite[]; they are left out of ranges and
+ *     histograms, and the metrics of a tensor that has any are unspecified.
+ */
+#ifndef QV2_H_
+#define QV2_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QV2_HIST_BINS 2048
+
+enum {
+  QV2_OK = 0,
+  QV2_ERR_ARG = -1,         /* bad enum value, inconsistent sizes, percentile outside [0,1] */
+  QV2_ERR_NULL = -2,        /* a required pointer is NULL */
+  QV2_ERR_ALIGN = -3,       /* a tensor pointer is not 4-byte aligned */
+  QV2_ERR_SIZE = -4,        /* a size exceeds what the library supports (see each call) */
+  QV2_ERR_NONFINITE = -5,   /* reported by qv2_sweep_model_host when an input held NaN or Inf */
+  QV2_ERR_CUDA = -6,        /* a CUDA runtime call failed; see qv2_last_cuda_error */
+  QV2_ERR_NOMEM = -7,       /* scratch allocation failed */
+  QV2_ERR_UNSUPPORTED = -8  /* a combination the library does not implement */
+};
+
+enum { QV2_PER_TENSOR = 0, QV2_PER_CHANNEL = 1 };            /* granularity */
+enum { QV2_SYM_I8 = 0, QV2_ASYM_U8 = 1 };                    /* scheme */
+enum { QV2_ABSMAX = 0, QV2_MINMAX = 1, QV2_PERCENTILE = 2 }; /* range */
+enum { QV2_PAIR_REQUANT = 0, QV2_PAIR_RAW = 1, QV2_STORE_CODES = 2 }; /* flags (bit 0: pair mode) */
+enum { QV2_BY_COUNT = 0, QV2_BY_BOPS_RATE = 1 };             /* select_mode */
+
+typedef struct qv2_ctx qv2_ctx;
+
+/* One tensor of one layer. */
+typedef struct {
+  const float* x;        /* device (host for qv2_sweep_model_host); reference tensor; may be NULL
+                            only when the tensor has no elements */
+  const float* y;        /* nullable; the same tensor as produced by the quantized pass.  NULL
+                            selects self mode (weights): the error is x against its own
+                            dequantized copy.  Non-NULL selects pair mode (activations). */
+  uint64_t outer, channels, inner;
+  uint32_t granularity;  /* QV2_PER_TENSOR | QV2_PER_CHANNEL */
+  uint32_t scheme;       /* QV2_SYM_I8: codes in [-127,127], offset 0.
+                            QV2_ASYM_U8: codes in [0,255], real-valued offset = range minimum */
+  uint32_t range;        /* QV2_ABSMAX and QV2_MINMAX take the group's observed range (|.| max for
+                            the symmetric scheme, [min,max] for the asymmetric one);
+                            QV2_PERCENTILE additionally clips it to the tensor's |x| percentile */
+  uint32_t flags;        /* pair mode: QV2_PAIR_REQUANT (default) re-quantizes y on x's grid and
+                            measures x - dequant(q(y)); QV2_PAIR_RAW measures x - y.
+                            QV2_STORE_CODES writes the 8-bit codes (see qv2_quant_metrics). */
+  double percentile;     /* in [0,1], e.g. 0.9999; read only when range == QV2_PERCENTILE */
+} qv2_tensor_desc;
+
+/* Ranking parameters (Algorithm 2, RankLayersBySensitivity; Eq. 16; Eq. 17). */
+typedef struct {
+  double w_gain;           /* weight of the weight-SQNR delta in the score (the paper gives the
+                              weight list "more weight" without a number; 2.0 is the usual choice) */
+  double a_gain;           /* weight of the activation-SQNR delta (1.0) */
+  double mse_factor;       /* a layer whose MSE exceeds mse_factor x the mean MSE goes to the top
+                              of the list; the paper uses 5 */
+  double sqnr_cap_db;      /* SQNR values are clamped to +-cap before differencing (200) */
+  uint32_t select_mode;    /* QV2_BY_COUNT | QV2_BY_BOPS_RATE */
+  uint32_t keep_count;     /* QV2_BY_COUNT: how many list entries stay FP32 */
+  uint32_t rate_permyriad; /* QV2_BY_BOPS_RATE: requested BOPs-reduction rate, 0..10000
+                              (0 = everything FP32, 10000 = everything int8) */
+  uint32_t reserved;
+} qv2_rank_cfg;
+
+/* Creates a context bound to CUDA device `device` and to `stream` (a cudaStream_t, borrowed, may
+ * be NULL for the default stream).  Allocates a small amount of device and pinned host scratch. */
+int qv2_create(qv2_ctx** out, int device, void* stream);
+int qv2_destroy(qv2_ctx* ctx);
+/* Static, human-readable name of a status code. */
+const char* qv2_status_string(int status);
+/* cudaError_t of the most recent failing CUDA call of this context (0 when none). */
+int qv2_last_cuda_error(const qv2_ctx* ctx);
+/* Number of kernel launches this context has enqueued since it was created. */
+uint64_t qv2_launch_count(const qv2_ctx* ctx);
+/* Sum over descs of the number of quantization groups (1 or `channels`).  Host only. */
+uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n);
+
+/*
+ * Calibration: step 1 of the paper's overview ("collect statistical data on the distribution of
+ * weights and activations") together with its calibration stage (a histogram of each layer's
+ * value range), followed by the scale computation of step 2 (Eq. 4 for symmetric weights, Eq. 2
+ * for the affine form).
+ *
+ * For every group g of every tensor: gmin/gmax = min/max over the group's finite elements,
+ * gabsmax = max(|gmin|,|gmax|) (a zero is returned as +0).  For every tensor t whose range is
+ * QV2_PERCENTILE: hist[t*2048 + j] counts the elements with min(2047, trunc(|x| * fl(2048/A))) == j,
+ * A the tensor's absmax, and clip[t] is the upper edge of the bin in which the cumulative count
+ * first reaches ceil(percentile * N); for the other tensors clip[t] = A and their histogram rows
+ * are zero.  Quantization parameters per group, all in binary32 with one rounding per operation:
+ *   QV2_SYM_I8:  R = absmax_g (min(absmax_g, clip) under QV2_PERCENTILE);
+ *                step = R/127, inv = 127/R, offset = 0
+ *   QV2_ASYM_U8: lo = min_g, hi = max_g (clipped to [-clip, clip] under QV2_PERCENTILE);
+ *                step = (hi-lo)/255, inv = 255/(hi-lo), offset = lo
+ * A degenerate range gives step = inv = 1.
+ *
+ * descs: host array of n descriptors (x device pointers; y is not read here).
+ * gmin, gmax, gabsmax, step, inv, offset: device, qv2_group_count(descs,n) floats each, required.
+ * hist: device, n*2048 uint64, or NULL when the histograms are not wanted (they are then kept in
+ *       context scratch).  clip: device, n floats, required.  nonfinite: device, n uint64, required.
+ * Limits: 1 <= n <= 65535; channels and the total group count < 2^32.
+ * Errors: QV2_ERR_NULL, _ARG, _ALIGN, _SIZE, _NOMEM, _CUDA.  On an argument error nothing has
+ * been launched.
+ */
+int qv2_calibrate(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
+                  float* gmin, float* gmax, float* gabsmax,
+                  uint64_t* hist, float* clip,
+                  float* step, float* inv, float* offset,
+                  uint64_t* nonfinite);
+
+/*
+ * Fused fake-quantize + error reduction: step 3 of the overview ("measure the SQNR and MSE of each
+ * layer by comparing the weights and activations of the original and quantized models"), i.e.
+ * CalculateSQNR / CalculateMSE of Algorithm 2 over every element, with the quantizer of Eq. 1 / Eq. 5
+ * and the dequantizer of Eq. 3; SQNR is Eq. 6 and MSE is Eq. 7.
+ *
+ * Per element of the tensor v being quantized (x in self mode, y in QV2_PAIR_REQUANT):
+ *   t = fl(fl(v - offset_g) * inv_g);  q = clamp(round_half_even(t), qmin, qmax);
+ *   v^ = q*step_g + offset_g;          e = x - v^          (QV2_PAIR_RAW: e = x - y, no codes)
+ * Per tensor: sse = sum e^2, sig = sum x^2 (the signal is always the reference tensor x),
+ * mse = sse/N, sqnr_db = 10 log10(sig/sse) (+inf when sse == 0, -inf when sig == 0 < sse).
+ * Sums are accumulated in binary32 per warp and tile, then in binary64 in a fixed order, so two
+ * runs give identical bits.
+ *
+ * descs: host, n descriptors (x and, for pair mode, y device pointers).
+ * step, inv, offset: device, per-group parameters in qv2_calibrate's layout.
+ * codes: NULL, or a host array of n device pointers; for a tensor with QV2_STORE_CODES set and a
+ *        non-NULL entry, one byte per element is written (int8 for QV2_SYM_I8, uint8 otherwise).
+ * sse, sig, mse, sqnr_db: device, n doubles each, required.
+ * Errors: as qv2_calibrate, plus QV2_ERR_ARG for QV2_PAIR_RAW without y.
+ */
+int qv2_quant_metrics(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
+                      const float* step, const float* inv, const float* offset,
+                      void* const* codes,
+                      double* sse, double* sig, double* mse, double* sqnr_db);
+
+/*
+ * Sensitivity list and mixed-precision layer set: step 4 of the overview, "CalculateSQNRdeltas",
+ * "CalculateAverage" and "RankLayersBySensitivity" of Algorithm 2, the SQNR delta of Eq. 16 and
+ * the BOPs-reduction rate of Eq. 17 (normalised so that a fully quantized model is 100 %).
+ *
+ *   delta_0 = 0, delta_n = (sqnr[n]-sqnr[n-1]) / (pos[n]-pos[n-1]) after clamping sqnr to +-cap;
+ *   score_n = w_gain*delta_w_n + a_gain*delta_a_n;
+ *   severity_n = max(mse_w[n]/mean(mse_w), mse_a[n]/mean(mse_a)) (a zero mean contributes 0);
+ *   order = layers with severity > mse_factor, most severe first, then the others by ascending
+ *           score; ties keep layer order.  A NaN score sorts last, a NaN severity counts as 0.
+ *   QV2_BY_COUNT keeps order[0..keep_count) in FP32; QV2_BY_BOPS_RATE keeps the longest prefix for
+ *   which (MACs of the still-quantized layers)/(all MACs) >= rate_permyriad/10000.
+ *
+ * sqnr_w, mse_w, sqnr_a, mse_a: device, n_layers doubles.  macs: device, n_layers uint64, or NULL
+ * (every layer counts 1).  pos: device, n_layers doubles, or NULL (positions 0,1,2,...).
+ * cfg: host.  order: device uint32[n_layers]; keep_fp32: device uint8[n_layers]; n_keep: device uint32.
+ * Limits: 1 <= n_layers <= 8192 (QV2_ERR_SIZE).  Results are bit-exact functions of the inputs.
+ */
+int qv2_rank_layers(qv2_ctx* ctx, uint32_t n_layers,
+                    const double* sqnr_w, const double* mse_w,
+                    const double* sqnr_a, const double* mse_a,
+                    const uint64_t* macs, const double* pos,
+                    const qv2_rank_cfg* cfg,
+                    uint32_t* order, uint8_t* keep_fp32, uint32_t* n_keep);
+
+/* Device buffers of one full-model pass; every pointer is device memory owned by the caller. */
+typedef struct {
+  float *gmin, *gmax, *gabsmax, *step, *inv, *offset;   /* qv2_group_count floats each */
+  uint64_t* hist;                                       /* n_tensors*2048, or NULL */
+  float* clip;                                          /* n_tensors */
+  uint64_t* nonfinite;                                  /* n_tensors */
+  double *sse, *sig, *mse, *sqnr_db;                    /* n_tensors each */
+  uint32_t* order;                                      /* n_layers */
+  uint8_t* keep_fp32;                                   /* n_layers */
+  uint32_t* n_keep;                                     /* 1 */
+} qv2_sweep_buffers;
+
+/*
+ * One full sensitivity pass over a model (Algorithm 2 end to end): qv2_calibrate, qv2_quant_metrics
+ * and qv2_rank_layers chained on the context's stream.  Layout of descs: descs[l] is the weight
+ * tensor of layer l and descs[n_layers + l] its activation tensor (l < n_layers); descriptors
+ * beyond 2*n_layers are calibrated and measured but do not enter the ranking.
+ * macs, pos: device or NULL as in qv2_rank_layers.  Requires n_tensors >= 2*n_layers.
+ */
+int qv2_sweep_model(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n_tensors,
+                    uint32_t n_layers, const uint64_t* macs, const double* pos,
+                    const qv2_rank_cfg* cfg, const qv2_sweep_buffers* bufs);
+
+/* Host-side results of qv2_sweep_model_host; every pointer is host memory owned by the caller. */
+typedef struct {
+  double *mse, *sqnr_db;       /* n_tensors each */
+  uint64_t* nonfinite;         /* n_tensors */
+  uint32_t* order;             /* n_layers */
+  uint8_t* keep_fp32;          /* n_layers */
+  uint32_t* n_keep;            /* 1 */
+} qv2_host_results;
+
+/*
+ * The same pass for tensors that live in HOST memory (pinned memory makes the copies fast):
+ * every x / y of descs is a host pointer; the call copies them into `staging` (device, caller
+ * owned, at least qv2_staging_bytes(descs, n_tensors, n_layers) bytes), runs qv2_sweep_model on
+ * the copies, copies the results back into `out`, and synchronises the stream before returning.
+ * macs, pos: HOST arrays or NULL.  Returns QV2_ERR_NONFINITE (results still written) when any
+ * input element was NaN or Inf.  QV2_STORE_CODES is not available through this call.
+ */
+int qv2_sweep_model_host(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n_tensors,
+                         uint32_t n_layers, const uint64_t* macs, const double* pos,
+                         const qv2_rank_cfg* cfg, void* staging, uint64_t staging_bytes,
+                         const qv2_sweep_buffers* bufs, const qv2_host_results* out);
+uint64_t qv2_staging_bytes(const qv2_tensor_desc* descs, uint32_t n_tensors, uint32_t n_layers);
+
+/*
+ * Host-only view of the work decomposition, for tests: cuts the tensors into the tiles the
+ * kernels walk (no GPU needed, tensor pointers are not dereferenced).  Each tile is reported as
+ * 4 uint64: {tensor, first element, element count, kind (0 = one group per tile, 1 = whole rows)}.
+ * Returns the number of tiles, or a negative status; at most max_tiles are written.
+ */
+int64_t qv2_debug_plan_tiles(const qv2_tensor_desc* descs, uint32_t n, uint64_t* out, uint64_t max_tiles);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QV2_H_ */

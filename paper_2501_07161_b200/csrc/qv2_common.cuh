@@ -1,0 +1,102 @@
+// Shared declarations of the qv2 CUDA library: device-side records, the tile decomposition and
+// the launch wrappers each kernel file exports to the C-ABI layer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/qv2.h"
+
+namespace qv2 {
+
+constexpr int kThreads = 256;            // threads per CTA in the streaming kernels
+constexpr int kWarps = kThreads / 32;
+constexpr uint32_t kTileElems = 16384;   // elements per tile (64 KiB of fp32)
+constexpr uint64_t kRowTileMin = 4096;   // rows at least this long are cut into one-group tiles
+constexpr int kBins = QV2_HIST_BINS;
+constexpr uint32_t kMaxRankLayers = 8192;
+
+enum PairMode : uint32_t { kSelf = 0, kRequant = 1, kRaw = 2 };
+
+// One tensor, as the kernels see it.
+struct TensorRec {
+  const float* x;
+  const float* y;
+  uint8_t* codes;            // nullable
+  uint64_t n_elems;
+  uint64_t inner;
+  uint32_t channels;
+  uint32_t group_base;       // index of this tensor's group 0 in the per-group arrays
+  uint32_t n_groups;
+  uint32_t per_channel;
+  uint32_t asym;             // 0: symmetric int8, 1: asymmetric uint8
+  uint32_t range_mode;       // QV2_ABSMAX | QV2_MINMAX | QV2_PERCENTILE
+  uint32_t pair_mode;        // PairMode
+  uint32_t slot_first;       // first partial-sum slot of this tensor (kWarps slots per tile)
+  uint32_t slot_count;
+  uint32_t pad_;
+  double percentile;
+};
+
+// A contiguous run of elements of one tensor handled by one CTA at a time.
+//  rows == 0: every element belongs to quantization group `row0` (0 for per-tensor tensors).
+//  rows  > 0: `rows` whole rows of `inner` elements starting at row `row0`; the group of row r
+//             is r % channels.
+// `slot` is the tile's first partial-sum slot; warp w of the CTA writes slot + w.
+struct Tile {
+  uint64_t begin;
+  uint64_t row0;
+  uint32_t count;
+  uint32_t tensor;
+  uint32_t rows;
+  uint32_t slot;
+};
+static_assert(sizeof(Tile) == 32, "Tile is read as two 16-byte words");
+
+struct HostPlan {
+  std::vector<TensorRec> tensors;
+  std::vector<Tile> tiles;        // every tensor, in tensor order
+  std::vector<Tile> hist_tiles;   // flat tiles of the tensors that need a histogram
+  uint64_t total_groups = 0;
+  uint32_t total_slots = 0;
+  bool any_percentile = false;
+};
+
+// Validates the descriptors and cuts them into tiles.  `codes` may be NULL.  Returns a QV2 status.
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, HostPlan* out);
+
+// ------------------------------------------------------------------------------------------------
+// Launch wrappers (defined next to their kernels).  All enqueue on `stream` and return the
+// cudaError_t of the launch.
+struct Launch {
+  cudaStream_t stream;
+  int sm_count;
+};
+
+cudaError_t launch_range(const Launch& l, const TensorRec* tensors, const Tile* tiles,
+                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax,
+                         unsigned long long* nonfinite);
+cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
+                                  float* gmin, float* gmax, float* gabsmax, float* step, float* inv,
+                                  float* offset, float* tensor_absmax);
+cudaError_t launch_hist(const Launch& l, const TensorRec* tensors, const Tile* tiles,
+                        uint32_t n_tiles, const float* tensor_absmax,
+                        const unsigned long long* nonfinite, unsigned long long* hist);
+cudaError_t launch_clip_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
+                                 const unsigned long long* hist, const float* tensor_absmax,
+                                 const float* gmin, const float* gmax, const float* gabsmax,
+                                 float* clip, float* step, float* inv, float* offset);
+cudaError_t launch_metrics(const Launch& l, const TensorRec* tensors, const Tile* tiles,
+                           uint32_t n_tiles, const float* step, const float* inv,
+                           const float* offset, double2* partials);
+cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
+                                    const double2* partials, double* sse, double* sig, double* mse,
+                                    double* sqnr_db);
+cudaError_t launch_rank(const Launch& l, uint32_t n, const double* sqnr_w, const double* mse_w,
+                        const double* sqnr_a, const double* mse_a, const uint64_t* macs,
+                        const double* pos, qv2_rank_cfg cfg, double* score, double* severity,
+                        uint32_t* order, uint8_t* keep, uint32_t* n_keep);
+
+}  // namespace qv2

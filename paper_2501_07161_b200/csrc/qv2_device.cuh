@@ -1,0 +1,124 @@
+// Device helpers shared by the streaming kernels: streaming loads, the tile fetch, the split of
+// a flat element run into an aligned 16-byte body with scalar head/tail, and warp reductions.
+#pragma once
+
+#include "qv2_common.cuh"
+
+namespace qv2 {
+
+// Read-once data: bypass L1 allocation so the stream does not evict anything useful.
+__device__ __forceinline__ float4 ld_stream4(const float4* p) {
+  float4 v;
+  asm("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+      : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+      : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float ld_stream1(const float* p) {
+  float v;
+  asm("ld.global.nc.L1::no_allocate.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ Tile load_tile(const Tile* tiles, uint32_t i) {
+  const uint4* p = reinterpret_cast<const uint4*>(tiles + i);
+  uint4 a = __ldg(p), b = __ldg(p + 1);
+  Tile t;
+  t.begin = (uint64_t)a.x | ((uint64_t)a.y << 32);
+  t.row0 = (uint64_t)a.z | ((uint64_t)a.w << 32);
+  t.count = b.x; t.tensor = b.y; t.rows = b.z; t.slot = b.w;
+  return t;
+}
+
+// A flat run [p, p+count): `head` scalars up to the first 16-byte boundary, `nvec` float4, `tail`
+// scalars.
+struct FlatSplit {
+  uint32_t head, nvec, tail;
+};
+__device__ __forceinline__ FlatSplit split_flat(const float* p, uint32_t count) {
+  FlatSplit s;
+  uint32_t mis = (uint32_t)(((uintptr_t)p >> 2) & 3u);     // elements past a 16-byte boundary
+  uint32_t head = (4u - mis) & 3u;
+  s.head = head < count ? head : count;
+  s.nvec = (count - s.head) >> 2;
+  s.tail = count - s.head - 4u * s.nvec;
+  return s;
+}
+
+__device__ __forceinline__ float warp_min(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+// Butterfly sum: every lane ends with the same value and the order of additions is fixed.
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ uint32_t warp_sum_u32(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Order-preserving map float -> uint32 (larger float <=> larger key).  Never 0 for a non-NaN
+// input, so 0 marks "nothing recorded" in the min/max key arrays.
+__device__ __forceinline__ uint32_t f2key(float f) {
+  uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key2f(uint32_t k) {
+  uint32_t b = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+  return __uint_as_float(b);
+}
+
+// Quantization parameters of one group (Eq. 4 read as the multiplier 127/max|W|; Eq. 2 for the
+// affine form), one binary32 rounding per operation.
+__device__ __forceinline__ void make_qparams(bool asym, bool use_clip, float clip, float mn, float mx,
+                                             float am, float* step, float* inv, float* offset) {
+  float s, r, off;
+  if (!asym) {
+    float R = am;
+    if (use_clip && clip < R) R = clip;
+    s = __fdiv_rn(R, 127.0f);
+    r = __fdiv_rn(127.0f, R);
+    off = 0.0f;
+    if (!(R > 0.0f) || !isfinite(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
+  } else {
+    float lo = mn, hi = mx;
+    if (use_clip) {
+      if (-clip > lo) lo = -clip;
+      if (clip < hi) hi = clip;
+    }
+    if (lo == 0.0f) lo = 0.0f;
+    float d = __fsub_rn(hi, lo);
+    s = __fdiv_rn(d, 255.0f);
+    r = __fdiv_rn(255.0f, d);
+    off = lo;
+    if (!(d > 0.0f) || !isfinite(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
+  }
+  *step = s; *inv = r; *offset = off;
+}
+
+// Grid of a persistent streaming kernel: every SM filled with as many CTAs as fit, never more
+// CTAs than tiles.  `cache` keeps the occupancy answer of one kernel between launches.
+inline int persistent_grid(const void* kernel, int* cache, int sm_count, uint32_t n_tiles) {
+  if (*cache <= 0) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess ||
+        per_sm < 1)
+      per_sm = 1;
+    *cache = per_sm;
+  }
+  long long g = (long long)(*cache) * sm_count;
+  if (g > (long long)n_tiles) g = n_tiles;
+  return g < 1 ? 1 : (int)g;
+}
+
+}  // namespace qv2

@@ -1,0 +1,121 @@
+// Host planner: validates tensor descriptors and cuts a whole model's ragged layer list into the
+// tile table that one kernel launch per phase walks (segmented multi-layer batching).
+#include "qv2_common.cuh"
+
+namespace qv2 {
+
+static bool mul_overflows(uint64_t a, uint64_t b, uint64_t* out) {
+  if (a != 0 && b > UINT64_MAX / a) return true;
+  *out = a * b;
+  return false;
+}
+
+static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t group,
+                     std::vector<Tile>* tiles) {
+  while (count > 0) {
+    uint32_t c = count > kTileElems ? kTileElems : (uint32_t)count;
+    Tile t;
+    t.begin = begin; t.row0 = group; t.count = c; t.tensor = tensor; t.rows = 0; t.slot = 0;
+    tiles->push_back(t);
+    begin += c; count -= c;
+  }
+}
+
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, HostPlan* out) {
+  if (!descs || !out) return QV2_ERR_NULL;
+  if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
+  out->tensors.clear(); out->tiles.clear(); out->hist_tiles.clear();
+  out->total_groups = 0; out->total_slots = 0; out->any_percentile = false;
+  out->tensors.reserve(n);
+  uint64_t groups = 0, slots = 0;
+  for (uint32_t t = 0; t < n; ++t) {
+    const qv2_tensor_desc& d = descs[t];
+    if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8 || d.range > QV2_PERCENTILE)
+      return QV2_ERR_ARG;
+    if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_STORE_CODES)) return QV2_ERR_ARG;
+    if (d.range == QV2_PERCENTILE && !(d.percentile >= 0.0 && d.percentile <= 1.0))
+      return QV2_ERR_ARG;
+    uint64_t rows, ne;
+    if (mul_overflows(d.outer, d.channels, &rows) || rows > (1ull << 62)) return QV2_ERR_SIZE;
+    if (mul_overflows(rows, d.inner, &ne) || ne > (1ull << 62)) return QV2_ERR_SIZE;
+    if (d.channels >= (1ull << 32)) return QV2_ERR_SIZE;
+    if (ne > 0 && !d.x) return QV2_ERR_NULL;
+    if (((uintptr_t)d.x & 3u) || ((uintptr_t)d.y & 3u)) return QV2_ERR_ALIGN;
+    bool pair = d.y != nullptr;
+    if ((d.flags & QV2_PAIR_RAW) && !pair) return QV2_ERR_ARG;
+
+    TensorRec r;
+    r.x = d.x; r.y = d.y;
+    r.codes = (codes && (d.flags & QV2_STORE_CODES)) ? (uint8_t*)codes[t] : nullptr;
+    r.n_elems = ne; r.inner = d.inner;
+    r.channels = (uint32_t)d.channels;
+    r.per_channel = d.granularity == QV2_PER_CHANNEL;
+    r.n_groups = r.per_channel ? (uint32_t)d.channels : 1u;
+    if (groups + r.n_groups >= (1ull << 32)) return QV2_ERR_SIZE;
+    r.group_base = (uint32_t)groups;
+    groups += r.n_groups;
+    r.asym = d.scheme == QV2_ASYM_U8;
+    r.range_mode = d.range;
+    r.pair_mode = !pair ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
+    r.percentile = d.percentile;
+    r.pad_ = 0;
+
+    size_t first_tile = out->tiles.size();
+    if (d.range == QV2_PERCENTILE) out->any_percentile = true;
+    if (ne > 0) {
+      if (!r.per_channel) {
+        cut_flat(t, 0, ne, 0, &out->tiles);
+      } else if (d.inner >= kRowTileMin) {
+        for (uint64_t row = 0; row < rows; ++row)
+          cut_flat(t, row * d.inner, d.inner, row % d.channels, &out->tiles);
+      } else {
+        uint64_t per = kTileElems / d.inner;       // inner < kRowTileMin, so per >= 4
+        for (uint64_t row = 0; row < rows; row += per) {
+          uint64_t nr = rows - row < per ? rows - row : per;
+          Tile tl;
+          tl.begin = row * d.inner; tl.row0 = row; tl.count = (uint32_t)(nr * d.inner);
+          tl.tensor = t; tl.rows = (uint32_t)nr; tl.slot = 0;
+          out->tiles.push_back(tl);
+        }
+      }
+      if (d.range == QV2_PERCENTILE) cut_flat(t, 0, ne, 0, &out->hist_tiles);
+    }
+    uint64_t nt = out->tiles.size() - first_tile;
+    if (slots + nt * kWarps >= (1ull << 32)) return QV2_ERR_SIZE;
+    r.slot_first = (uint32_t)slots;
+    r.slot_count = (uint32_t)(nt * kWarps);
+    for (uint64_t i = 0; i < nt; ++i)
+      out->tiles[first_tile + i].slot = (uint32_t)(slots + i * kWarps);
+    slots += nt * kWarps;
+    out->tensors.push_back(r);
+  }
+  if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;
+  out->total_groups = groups;
+  out->total_slots = (uint32_t)slots;
+  return QV2_OK;
+}
+
+}  // namespace qv2
+
+extern "C" uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n) {
+  uint64_t g = 0;
+  if (!descs) return 0;
+  for (uint32_t t = 0; t < n; ++t)
+    g += descs[t].granularity == QV2_PER_CHANNEL ? descs[t].channels : 1;
+  return g;
+}
+
+extern "C" int64_t qv2_debug_plan_tiles(const qv2_tensor_desc* descs, uint32_t n, uint64_t* out,
+                                        uint64_t max_tiles) {
+  qv2::HostPlan plan;
+  int st = qv2::build_plan(descs, n, nullptr, &plan);
+  if (st != QV2_OK) return st;
+  uint64_t w = 0;
+  for (const qv2::Tile& t : plan.tiles) {
+    if (w >= max_tiles || !out) break;
+    out[4 * w + 0] = t.tensor; out[4 * w + 1] = t.begin; out[4 * w + 2] = t.count;
+    out[4 * w + 3] = t.rows ? 1 : 0;
+    ++w;
+  }
+  return (int64_t)plan.tiles.size();
+}

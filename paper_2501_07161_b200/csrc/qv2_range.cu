@@ -1,0 +1,177 @@
+// Range calibration: one persistent launch sweeps every tile of every tensor and records the
+// per-group minimum and maximum; a small second kernel turns them into absmax and quantization
+// parameters (step 1 and step 2 of the paper's overview, Eq. 2 and Eq. 4).
+//
+// min/max are exact and order-independent, so the per-warp results are merged with integer
+// atomicMax on an order-preserving key; no floating-point atomics are used anywhere.
+#include "qv2_device.cuh"
+
+namespace qv2 {
+
+namespace {
+
+constexpr float kInf = __builtin_huge_valf();
+
+struct RangeAcc {
+  float mn, mx;
+  float nanflag;     // fast path: becomes NaN as soon as a non-finite element is seen
+  uint32_t bad;      // careful path: count of non-finite elements
+};
+
+template <bool CAREFUL>
+__device__ __forceinline__ void range_acc(RangeAcc& a, float v) {
+  if (CAREFUL) {
+    if (isfinite(v)) { a.mn = fminf(a.mn, v); a.mx = fmaxf(a.mx, v); }
+    else ++a.bad;
+  } else {
+    a.mn = fminf(a.mn, v);
+    a.mx = fmaxf(a.mx, v);
+    a.nanflag = __fmaf_rn(v, 0.0f, a.nanflag);   // NaN*0 and Inf*0 are NaN
+  }
+}
+template <bool CAREFUL>
+__device__ __forceinline__ void range_acc4(RangeAcc& a, const float4& v) {
+  range_acc<CAREFUL>(a, v.x); range_acc<CAREFUL>(a, v.y);
+  range_acc<CAREFUL>(a, v.z); range_acc<CAREFUL>(a, v.w);
+}
+
+// This thread's share of a flat run: float4 number j for j = tid, tid+256, ...; the first
+// `head` and last `tail` scalars go to threads 0..2.
+template <bool CAREFUL>
+__device__ __forceinline__ void range_flat(const float* __restrict__ x, uint32_t count, RangeAcc& a) {
+  const FlatSplit s = split_flat(x, count);
+  const float4* xv = reinterpret_cast<const float4*>(x + s.head);
+  constexpr uint32_t U = 8;
+  uint32_t j = threadIdx.x;
+  for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
+    float4 v[U];
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) v[u] = ld_stream4(xv + j + u * kThreads);
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) range_acc4<CAREFUL>(a, v[u]);
+  }
+  for (; j < s.nvec; j += kThreads) range_acc4<CAREFUL>(a, ld_stream4(xv + j));
+  if (threadIdx.x < s.head) range_acc<CAREFUL>(a, ld_stream1(x + threadIdx.x));
+  if (threadIdx.x < s.tail) range_acc<CAREFUL>(a, ld_stream1(x + s.head + 4u * s.nvec + threadIdx.x));
+}
+
+// One row handled by one warp: lanes stride over the row.
+template <bool CAREFUL>
+__device__ __forceinline__ void range_row(const float* __restrict__ row, uint32_t inner, uint32_t lane,
+                                          RangeAcc& a) {
+  uint32_t i = lane;
+  for (; i + 96 < inner; i += 128) {
+    float v0 = ld_stream1(row + i), v1 = ld_stream1(row + i + 32), v2 = ld_stream1(row + i + 64),
+          v3 = ld_stream1(row + i + 96);
+    range_acc<CAREFUL>(a, v0); range_acc<CAREFUL>(a, v1);
+    range_acc<CAREFUL>(a, v2); range_acc<CAREFUL>(a, v3);
+  }
+  for (; i < inner; i += 32) range_acc<CAREFUL>(a, ld_stream1(row + i));
+}
+
+__device__ __forceinline__ void reset(RangeAcc& a) {
+  a.mn = kInf; a.mx = -kInf; a.nanflag = 0.0f; a.bad = 0;
+}
+
+// Warp-level merge and publication of one group's range.
+__device__ __forceinline__ void publish(RangeAcc& a, uint32_t lane, uint32_t* kmin, uint32_t* kmax,
+                                        uint32_t group, unsigned long long* nonfinite_t) {
+  float mn = warp_min(a.mn), mx = warp_max(a.mx);
+  uint32_t bad = warp_sum_u32(a.bad);
+  if (lane == 0) {
+    if (mn <= mx) {                       // false only when no finite element was seen
+      atomicMax(kmax + group, f2key(mx));
+      atomicMax(kmin + group, ~f2key(mn));
+    }
+    if (bad) atomicAdd(nonfinite_t, (unsigned long long)bad);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
+             uint32_t* kmin, uint32_t* kmax, unsigned long long* nonfinite) {
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+    const Tile tl = load_tile(tiles, ti);
+    const TensorRec* tr = tensors + tl.tensor;
+    const float* x = tr->x + tl.begin;
+    const uint32_t gbase = tr->group_base;
+    unsigned long long* nf = nonfinite + tl.tensor;
+    RangeAcc a;
+    if (tl.rows == 0) {
+      reset(a);
+      range_flat<false>(x, tl.count, a);
+      if (__any_sync(0xffffffffu, a.nanflag != a.nanflag)) {   // redo this warp's share carefully
+        reset(a);
+        range_flat<true>(x, tl.count, a);
+      }
+      publish(a, lane, kmin, kmax, gbase + (uint32_t)tl.row0, nf);
+    } else {
+      const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+      for (uint32_t r = warp; r < tl.rows; r += kWarps) {
+        const float* row = x + (uint64_t)r * inner;
+        reset(a);
+        range_row<false>(row, inner, lane, a);
+        if (__any_sync(0xffffffffu, a.nanflag != a.nanflag)) {
+          reset(a);
+          range_row<true>(row, inner, lane, a);
+        }
+        const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
+        publish(a, lane, kmin, kmax, gbase + g, nf);
+      }
+    }
+  }
+}
+
+// One CTA per tensor: decode the keys in place, write absmax, the tensor-wide absmax and -- for
+// tensors without percentile clipping -- the quantization parameters.
+__global__ void __launch_bounds__(256)
+range_finalize_kernel(const TensorRec* __restrict__ tensors, float* gmin, float* gmax, float* gabsmax,
+                      float* step, float* inv, float* offset, float* tensor_absmax) {
+  __shared__ float red[256];
+  const TensorRec tr = tensors[blockIdx.x];
+  float amax = 0.0f;
+  for (uint32_t g = threadIdx.x; g < tr.n_groups; g += blockDim.x) {
+    const uint32_t G = tr.group_base + g;
+    const uint32_t kn = reinterpret_cast<uint32_t*>(gmin)[G];
+    const uint32_t kx = reinterpret_cast<uint32_t*>(gmax)[G];
+    float mn = kn ? key2f(~kn) : 0.0f;
+    float mx = kx ? key2f(kx) : 0.0f;
+    if (mn == 0.0f) mn = 0.0f;          // -0 -> +0
+    if (mx == 0.0f) mx = 0.0f;
+    const float am = fmaxf(fabsf(mn), fabsf(mx));
+    gmin[G] = mn; gmax[G] = mx; gabsmax[G] = am;
+    amax = fmaxf(amax, am);
+    if (tr.range_mode != QV2_PERCENTILE)
+      make_qparams(tr.asym != 0, false, 0.0f, mn, mx, am, step + G, inv + G, offset + G);
+  }
+  red[threadIdx.x] = amax;
+  __syncthreads();
+  for (uint32_t o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + o]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) tensor_absmax[blockIdx.x] = red[0];
+}
+
+}  // namespace
+
+cudaError_t launch_range(const Launch& l, const TensorRec* tensors, const Tile* tiles,
+                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax,
+                         unsigned long long* nonfinite) {
+  if (n_tiles == 0) return cudaSuccess;
+  static int per_sm = 0;   // resident CTAs per SM, queried once
+  const int grid = persistent_grid((const void*)range_kernel, &per_sm, l.sm_count, n_tiles);
+  range_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, nonfinite);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
+                                  float* gmin, float* gmax, float* gabsmax, float* step, float* inv,
+                                  float* offset, float* tensor_absmax) {
+  range_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, gmin, gmax, gabsmax, step, inv,
+                                                         offset, tensor_absmax);
+  return cudaGetLastError();
+}
+
+}  // namespace qv2
