@@ -1,0 +1,339 @@
+// C-ABI layer: context, scratch management, plan caching and the call sequences of the public
+// entry points declared in include/qv2.h.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "qv2_common.cuh"
+
+using namespace qv2;
+
+struct qv2_ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  int sm_count = 1;
+  int last_cuda = 0;
+  uint64_t launches = 0;
+
+  // cached plan: rebuilt only when the descriptor bytes (or code pointers) change
+  HostPlan plan;
+  std::vector<uint8_t> plan_key;
+  bool plan_valid = false;
+
+  // device scratch
+  TensorRec* d_tensors = nullptr; size_t cap_tensors = 0;
+  Tile* d_tiles = nullptr;        size_t cap_tiles = 0;
+  Tile* d_hist_tiles = nullptr;   size_t cap_hist_tiles = 0;
+  double2* d_partials = nullptr;  size_t cap_slots = 0;
+  float* d_tensor_absmax = nullptr; size_t cap_absmax = 0;
+  unsigned long long* d_hist = nullptr; size_t cap_hist = 0;   // used when the caller passes no hist
+  double* d_rank = nullptr;                                    // 2 * kMaxRankLayers doubles
+  // pinned host staging for the plan upload
+  uint8_t* h_pinned = nullptr;    size_t cap_pinned = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+int cuda_fail(qv2_ctx* c, cudaError_t e) {
+  c->last_cuda = (int)e;
+  return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA;
+}
+
+#define QV2_CUDA(c, expr)                              \
+  do {                                                 \
+    cudaError_t e__ = (expr);                          \
+    if (e__ != cudaSuccess) return cuda_fail((c), e__);\
+  } while (0)
+
+template <class T>
+int grow(qv2_ctx* c, T** p, size_t* cap, size_t need) {
+  if (need <= *cap) return QV2_OK;
+  size_t want = need + need / 4 + 16;
+  if (*p) { QV2_CUDA(c, cudaFree(*p)); *p = nullptr; *cap = 0; }
+  QV2_CUDA(c, cudaMalloc((void**)p, want * sizeof(T)));
+  *cap = want;
+  return QV2_OK;
+}
+
+int grow_pinned(qv2_ctx* c, size_t need) {
+  if (need <= c->cap_pinned) return QV2_OK;
+  size_t want = need + need / 4 + 4096;
+  if (c->h_pinned) { QV2_CUDA(c, cudaFreeHost(c->h_pinned)); c->h_pinned = nullptr; c->cap_pinned = 0; }
+  QV2_CUDA(c, cudaMallocHost((void**)&c->h_pinned, want));
+  c->cap_pinned = want;
+  return QV2_OK;
+}
+
+// Makes ctx->plan describe (descs, codes) and resident on the device.
+int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* const* codes) {
+  if (!descs) return QV2_ERR_NULL;
+  if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
+  const size_t dbytes = (size_t)n * sizeof(qv2_tensor_desc);
+  const size_t cbytes = codes ? (size_t)n * sizeof(void*) : 0;
+  std::vector<uint8_t> key(dbytes + cbytes + 1);
+  std::memcpy(key.data(), descs, dbytes);
+  if (codes) std::memcpy(key.data() + dbytes, codes, cbytes);
+  key[dbytes + cbytes] = codes ? 1 : 0;
+  if (c->plan_valid && key == c->plan_key) return QV2_OK;
+
+  HostPlan plan;
+  int st = build_plan(descs, n, codes, &plan);
+  if (st != QV2_OK) return st;
+  // The previous upload may still be reading the pinned buffer, and buffers may be reallocated.
+  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  c->plan_valid = false;
+  const size_t nt = plan.tensors.size(), ntl = plan.tiles.size(), nh = plan.hist_tiles.size();
+  if ((st = grow(c, &c->d_tensors, &c->cap_tensors, nt)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_tiles, &c->cap_tiles, ntl ? ntl : 1)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_hist_tiles, &c->cap_hist_tiles, nh ? nh : 1)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_partials, &c->cap_slots, plan.total_slots ? plan.total_slots : 1)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_tensor_absmax, &c->cap_absmax, nt)) != QV2_OK) return st;
+  const size_t b0 = nt * sizeof(TensorRec), b1 = ntl * sizeof(Tile), b2 = nh * sizeof(Tile);
+  if ((st = grow_pinned(c, b0 + b1 + b2)) != QV2_OK) return st;
+  std::memcpy(c->h_pinned, plan.tensors.data(), b0);
+  if (b1) std::memcpy(c->h_pinned + b0, plan.tiles.data(), b1);
+  if (b2) std::memcpy(c->h_pinned + b0 + b1, plan.hist_tiles.data(), b2);
+  QV2_CUDA(c, cudaMemcpyAsync(c->d_tensors, c->h_pinned, b0, cudaMemcpyHostToDevice, c->stream));
+  if (b1) QV2_CUDA(c, cudaMemcpyAsync(c->d_tiles, c->h_pinned + b0, b1, cudaMemcpyHostToDevice, c->stream));
+  if (b2) QV2_CUDA(c, cudaMemcpyAsync(c->d_hist_tiles, c->h_pinned + b0 + b1, b2, cudaMemcpyHostToDevice, c->stream));
+  c->plan = std::move(plan);
+  c->plan_key = std::move(key);
+  c->plan_valid = true;
+  return QV2_OK;
+}
+
+Launch launch_of(qv2_ctx* c) {
+  Launch l; l.stream = c->stream; l.sm_count = c->sm_count;
+  return l;
+}
+
+}  // namespace
+
+extern "C" const char* qv2_status_string(int status) {
+  switch (status) {
+    case QV2_OK: return "QV2_OK";
+    case QV2_ERR_ARG: return "QV2_ERR_ARG: invalid argument";
+    case QV2_ERR_NULL: return "QV2_ERR_NULL: required pointer is NULL";
+    case QV2_ERR_ALIGN: return "QV2_ERR_ALIGN: pointer is not sufficiently aligned";
+    case QV2_ERR_SIZE: return "QV2_ERR_SIZE: size outside the supported range";
+    case QV2_ERR_NONFINITE: return "QV2_ERR_NONFINITE: input holds NaN or Inf";
+    case QV2_ERR_CUDA: return "QV2_ERR_CUDA: CUDA runtime call failed";
+    case QV2_ERR_NOMEM: return "QV2_ERR_NOMEM: out of memory";
+    case QV2_ERR_UNSUPPORTED: return "QV2_ERR_UNSUPPORTED: not implemented";
+    default: return "QV2: unknown status";
+  }
+}
+
+extern "C" int qv2_create(qv2_ctx** out, int device, void* stream) {
+  if (!out) return QV2_ERR_NULL;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return QV2_ERR_CUDA;
+  qv2_ctx* c = new (std::nothrow) qv2_ctx();
+  if (!c) return QV2_ERR_NOMEM;
+  c->device = device;
+  c->stream = (cudaStream_t)stream;
+  DeviceGuard guard(device);
+  int sms = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_rank, 2 * (size_t)kMaxRankLayers * sizeof(double));
+  if (e != cudaSuccess) { delete c; return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA; }
+  c->sm_count = sms > 0 ? sms : 1;
+  *out = c;
+  return QV2_OK;
+}
+
+extern "C" int qv2_destroy(qv2_ctx* c) {
+  if (!c) return QV2_ERR_NULL;
+  DeviceGuard guard(c->device);
+  cudaStreamSynchronize(c->stream);
+  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials);
+  cudaFree(c->d_tensor_absmax); cudaFree(c->d_hist); cudaFree(c->d_rank);
+  if (c->h_pinned) cudaFreeHost(c->h_pinned);
+  delete c;
+  return QV2_OK;
+}
+
+extern "C" int qv2_last_cuda_error(const qv2_ctx* c) { return c ? c->last_cuda : 0; }
+extern "C" uint64_t qv2_launch_count(const qv2_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* gmin,
+                             float* gmax, float* gabsmax, uint64_t* hist, float* clip, float* step,
+                             float* inv, float* offset, uint64_t* nonfinite) {
+  if (!c || !descs || !gmin || !gmax || !gabsmax || !clip || !step || !inv || !offset || !nonfinite)
+    return QV2_ERR_NULL;
+  DeviceGuard guard(c->device);
+  int st = ensure_plan(c, descs, n, nullptr);
+  if (st != QV2_OK) return st;
+  const HostPlan& p = c->plan;
+  unsigned long long* h = reinterpret_cast<unsigned long long*>(hist);
+  if (!h && p.any_percentile) {
+    if ((st = grow(c, &c->d_hist, &c->cap_hist, (size_t)n * kBins)) != QV2_OK) return st;
+    h = c->d_hist;
+  }
+  const Launch l = launch_of(c);
+  const size_t G = (size_t)p.total_groups;
+  if (G) {
+    QV2_CUDA(c, cudaMemsetAsync(gmin, 0, G * sizeof(float), c->stream));   // key 0 = nothing seen
+    QV2_CUDA(c, cudaMemsetAsync(gmax, 0, G * sizeof(float), c->stream));
+  }
+  QV2_CUDA(c, cudaMemsetAsync(nonfinite, 0, (size_t)n * sizeof(uint64_t), c->stream));
+  if (h) QV2_CUDA(c, cudaMemsetAsync(h, 0, (size_t)n * kBins * sizeof(uint64_t), c->stream));
+  if (!p.tiles.empty()) {
+    QV2_CUDA(c, launch_range(l, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),
+                             reinterpret_cast<uint32_t*>(gmin), reinterpret_cast<uint32_t*>(gmax),
+                             reinterpret_cast<unsigned long long*>(nonfinite)));
+    ++c->launches;
+  }
+  QV2_CUDA(c, launch_range_finalize(l, c->d_tensors, n, gmin, gmax, gabsmax, step, inv, offset,
+                                    c->d_tensor_absmax));
+  ++c->launches;
+  if (!p.hist_tiles.empty()) {
+    QV2_CUDA(c, launch_hist(l, c->d_tensors, c->d_hist_tiles, (uint32_t)p.hist_tiles.size(),
+                            c->d_tensor_absmax, reinterpret_cast<unsigned long long*>(nonfinite), h));
+    ++c->launches;
+  }
+  QV2_CUDA(c, launch_clip_finalize(l, c->d_tensors, n, h, c->d_tensor_absmax, gmin, gmax, gabsmax,
+                                   clip, step, inv, offset));
+  ++c->launches;
+  return QV2_OK;
+}
+
+extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n,
+                                 const float* step, const float* inv, const float* offset,
+                                 void* const* codes, double* sse, double* sig, double* mse,
+                                 double* sqnr_db) {
+  if (!c || !descs || !step || !inv || !offset || !sse || !sig || !mse || !sqnr_db) return QV2_ERR_NULL;
+  DeviceGuard guard(c->device);
+  bool any_codes = false;
+  if (codes)
+    for (uint32_t t = 0; t < n && n <= 65535u; ++t)
+      if ((descs[t].flags & QV2_STORE_CODES) && codes[t]) any_codes = true;
+  int st = ensure_plan(c, descs, n, any_codes ? codes : nullptr);
+  if (st != QV2_OK) return st;
+  const HostPlan& p = c->plan;
+  const Launch l = launch_of(c);
+  if (!p.tiles.empty()) {
+    QV2_CUDA(c, launch_metrics(l, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
+                               offset, c->d_partials));
+    ++c->launches;
+  }
+  QV2_CUDA(c, launch_metrics_finalize(l, c->d_tensors, n, c->d_partials, sse, sig, mse, sqnr_db));
+  ++c->launches;
+  return QV2_OK;
+}
+
+extern "C" int qv2_rank_layers(qv2_ctx* c, uint32_t n_layers, const double* sqnr_w,
+                               const double* mse_w, const double* sqnr_a, const double* mse_a,
+                               const uint64_t* macs, const double* pos, const qv2_rank_cfg* cfg,
+                               uint32_t* order, uint8_t* keep_fp32, uint32_t* n_keep) {
+  if (!c || !sqnr_w || !mse_w || !sqnr_a || !mse_a || !cfg || !order || !keep_fp32 || !n_keep)
+    return QV2_ERR_NULL;
+  if (n_layers == 0 || n_layers > kMaxRankLayers) return QV2_ERR_SIZE;
+  if (cfg->select_mode > QV2_BY_BOPS_RATE) return QV2_ERR_ARG;
+  if (cfg->select_mode == QV2_BY_BOPS_RATE && cfg->rate_permyriad > 10000u) return QV2_ERR_ARG;
+  DeviceGuard guard(c->device);
+  QV2_CUDA(c, launch_rank(launch_of(c), n_layers, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, *cfg,
+                          c->d_rank, c->d_rank + kMaxRankLayers, order, keep_fp32, n_keep));
+  ++c->launches;
+  return QV2_OK;
+}
+
+extern "C" int qv2_sweep_model(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n_tensors,
+                               uint32_t n_layers, const uint64_t* macs, const double* pos,
+                               const qv2_rank_cfg* cfg, const qv2_sweep_buffers* b) {
+  if (!c || !descs || !cfg || !b) return QV2_ERR_NULL;
+  if (n_layers == 0 || n_layers > kMaxRankLayers) return QV2_ERR_SIZE;
+  if ((uint64_t)n_tensors < 2ull * n_layers) return QV2_ERR_ARG;
+  if (!b->order || !b->keep_fp32 || !b->n_keep || !b->sse || !b->sig || !b->mse || !b->sqnr_db)
+    return QV2_ERR_NULL;
+  if (cfg->select_mode > QV2_BY_BOPS_RATE) return QV2_ERR_ARG;
+  if (cfg->select_mode == QV2_BY_BOPS_RATE && cfg->rate_permyriad > 10000u) return QV2_ERR_ARG;
+  int st = qv2_calibrate(c, descs, n_tensors, b->gmin, b->gmax, b->gabsmax, b->hist, b->clip, b->step,
+                         b->inv, b->offset, b->nonfinite);
+  if (st != QV2_OK) return st;
+  st = qv2_quant_metrics(c, descs, n_tensors, b->step, b->inv, b->offset, nullptr, b->sse, b->sig,
+                         b->mse, b->sqnr_db);
+  if (st != QV2_OK) return st;
+  return qv2_rank_layers(c, n_layers, b->sqnr_db, b->mse, b->sqnr_db + n_layers, b->mse + n_layers,
+                         macs, pos, cfg, b->order, b->keep_fp32, b->n_keep);
+}
+
+namespace {
+inline uint64_t align256(uint64_t v) { return (v + 255u) & ~(uint64_t)255u; }
+}
+
+extern "C" uint64_t qv2_staging_bytes(const qv2_tensor_desc* descs, uint32_t n_tensors,
+                                      uint32_t n_layers) {
+  if (!descs) return 0;
+  uint64_t total = 0;
+  for (uint32_t t = 0; t < n_tensors; ++t) {
+    const uint64_t bytes = align256(descs[t].outer * descs[t].channels * descs[t].inner * sizeof(float));
+    total += bytes;
+    if (descs[t].y) total += bytes;
+  }
+  total += align256((uint64_t)n_layers * sizeof(uint64_t)) + align256((uint64_t)n_layers * sizeof(double));
+  return total + 256;
+}
+
+extern "C" int qv2_sweep_model_host(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n_tensors,
+                                    uint32_t n_layers, const uint64_t* macs, const double* pos,
+                                    const qv2_rank_cfg* cfg, void* staging, uint64_t staging_bytes,
+                                    const qv2_sweep_buffers* b, const qv2_host_results* out) {
+  if (!c || !descs || !cfg || !staging || !b || !out) return QV2_ERR_NULL;
+  if (!out->mse || !out->sqnr_db || !out->nonfinite || !out->order || !out->keep_fp32 || !out->n_keep)
+    return QV2_ERR_NULL;
+  if (n_tensors == 0 || n_tensors > 65535u) return QV2_ERR_SIZE;
+  if (staging_bytes < qv2_staging_bytes(descs, n_tensors, n_layers)) return QV2_ERR_SIZE;
+  if ((uintptr_t)staging & 255u) return QV2_ERR_ALIGN;
+  DeviceGuard guard(c->device);
+  std::vector<qv2_tensor_desc> dd(descs, descs + n_tensors);
+  uint8_t* base = (uint8_t*)staging;
+  uint64_t off = 0;
+  for (uint32_t t = 0; t < n_tensors; ++t) {
+    if (dd[t].flags & QV2_STORE_CODES) return QV2_ERR_UNSUPPORTED;
+    const uint64_t bytes = descs[t].outer * descs[t].channels * descs[t].inner * sizeof(float);
+    if (bytes && !descs[t].x) return QV2_ERR_NULL;
+    dd[t].x = (const float*)(base + off);
+    if (bytes) QV2_CUDA(c, cudaMemcpyAsync(base + off, descs[t].x, bytes, cudaMemcpyHostToDevice, c->stream));
+    off += align256(bytes);
+    if (descs[t].y) {
+      dd[t].y = (const float*)(base + off);
+      if (bytes) QV2_CUDA(c, cudaMemcpyAsync(base + off, descs[t].y, bytes, cudaMemcpyHostToDevice, c->stream));
+      off += align256(bytes);
+    }
+  }
+  const uint64_t* d_macs = nullptr;
+  const double* d_pos = nullptr;
+  if (macs) {
+    d_macs = (const uint64_t*)(base + off);
+    QV2_CUDA(c, cudaMemcpyAsync(base + off, macs, (size_t)n_layers * sizeof(uint64_t), cudaMemcpyHostToDevice, c->stream));
+  }
+  off += align256((uint64_t)n_layers * sizeof(uint64_t));
+  if (pos) {
+    d_pos = (const double*)(base + off);
+    QV2_CUDA(c, cudaMemcpyAsync(base + off, pos, (size_t)n_layers * sizeof(double), cudaMemcpyHostToDevice, c->stream));
+  }
+  int st = qv2_sweep_model(c, dd.data(), n_tensors, n_layers, d_macs, d_pos, cfg, b);
+  if (st != QV2_OK) return st;
+  const cudaMemcpyKind d2h = cudaMemcpyDeviceToHost;
+  QV2_CUDA(c, cudaMemcpyAsync(out->mse, b->mse, (size_t)n_tensors * sizeof(double), d2h, c->stream));
+  QV2_CUDA(c, cudaMemcpyAsync(out->sqnr_db, b->sqnr_db, (size_t)n_tensors * sizeof(double), d2h, c->stream));
+  QV2_CUDA(c, cudaMemcpyAsync(out->nonfinite, b->nonfinite, (size_t)n_tensors * sizeof(uint64_t), d2h, c->stream));
+  QV2_CUDA(c, cudaMemcpyAsync(out->order, b->order, (size_t)n_layers * sizeof(uint32_t), d2h, c->stream));
+  QV2_CUDA(c, cudaMemcpyAsync(out->keep_fp32, b->keep_fp32, (size_t)n_layers, d2h, c->stream));
+  QV2_CUDA(c, cudaMemcpyAsync(out->n_keep, b->n_keep, sizeof(uint32_t), d2h, c->stream));
+  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  for (uint32_t t = 0; t < n_tensors; ++t)
+    if (out->nonfinite[t]) return QV2_ERR_NONFINITE;
+  return QV2_OK;
+}

@@ -96,7 +96,7 @@ __device__ __forceinline__ void make_qparams(bool asym, bool use_clip, float cli
       if (-clip > lo) lo = -clip;
       if (clip < hi) hi = clip;
     }
-    if (lo == 0.0f) lo = 0.0f;
+    lo = __fadd_rn(lo, 0.0f);            // -0 -> +0
     float d = __fsub_rn(hi, lo);
     s = __fdiv_rn(d, 255.0f);
     r = __fdiv_rn(255.0f, d);

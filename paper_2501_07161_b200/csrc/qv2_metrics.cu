@@ -1,0 +1,256 @@
+// Fused fake-quantize / dequantize / error reduction -- the memory-bound core of the sweep
+// (CalculateSQNR and CalculateMSE of Algorithm 2; quantizer Eq. 1 / Eq. 5, dequantizer Eq. 3,
+// SQNR Eq. 6, MSE Eq. 7).
+//
+// One persistent launch walks the tile table of a whole model.  Every warp reduces its share of a
+// tile in binary32 (independent accumulators per vector lane, then a fixed butterfly) and writes
+// one {sum e^2, sum x^2} pair to its own slot; a second kernel adds each tensor's slots in a fixed
+// order in binary64.  There are no floating-point atomics and no inter-CTA waits, so the result
+// is bit-identical from run to run and does not depend on the grid size.
+#include "qv2_device.cuh"
+
+namespace qv2 {
+
+namespace {
+
+struct QP {
+  float step, inv, off, qmin, qmax;
+};
+
+struct Acc {
+  float sse, sig;
+};
+
+// One element.  MODE: kSelf quantizes x, kRequant quantizes y on x's grid, kRaw compares x and y.
+//  t  = fl(fl(v - off) * inv)                      (v - 0 == v exactly, so OFF=false skips it)
+//  q  = rne(clamp(t)) == clamp(rne(t)) since the bounds are integers; the add/subtract of
+//       1.5*2^23 rounds to nearest-even for |t| <= 2^22
+//  e  = (x - off) - q*step, with x - off split exactly into (s, err) by TwoSum when off != 0 and
+//       the product folded into one fused multiply-add, so e carries a single rounding error.
+template <uint32_t MODE, bool OFF, bool CODES>
+__device__ __forceinline__ void metric_elem(float x, float y, const QP& p, Acc& a, uint8_t* code) {
+  float e;
+  if (MODE == kRaw) {
+    e = __fsub_rn(x, y);
+  } else {
+    const float v = (MODE == kRequant) ? y : x;
+    const float u = OFF ? __fsub_rn(v, p.off) : v;
+    const float t = __fmul_rn(u, p.inv);
+    const float tc = fminf(fmaxf(t, p.qmin), p.qmax);       // NaN -> qmin
+    const float q = __fsub_rn(__fadd_rn(tc, 12582912.0f), 12582912.0f);
+    if (OFF) {
+      const float b = -p.off;
+      const float s = __fadd_rn(x, b);
+      const float bb = __fsub_rn(s, x);
+      const float err = __fadd_rn(__fsub_rn(x, __fsub_rn(s, bb)), __fsub_rn(b, bb));
+      e = __fadd_rn(__fmaf_rn(-q, p.step, s), err);
+    } else {
+      e = __fmaf_rn(-q, p.step, x);
+    }
+    if (CODES) *code = (uint8_t)(int)q;
+  }
+  a.sse = __fmaf_rn(e, e, a.sse);
+  a.sig = __fmaf_rn(x, x, a.sig);
+}
+
+template <uint32_t MODE, bool OFF, bool CODES>
+__device__ __forceinline__ void metric_vec(const float4& x, const float4& y, const QP& p, Acc* a,
+                                           uint8_t* code) {
+  metric_elem<MODE, OFF, CODES>(x.x, y.x, p, a[0], code);
+  metric_elem<MODE, OFF, CODES>(x.y, y.y, p, a[1], code + 1);
+  metric_elem<MODE, OFF, CODES>(x.z, y.z, p, a[2], code + 2);
+  metric_elem<MODE, OFF, CODES>(x.w, y.w, p, a[3], code + 3);
+}
+
+// This thread's share of a flat one-group run.  `vec_y` says y has the same 16-byte phase as x.
+template <uint32_t MODE, bool OFF, bool CODES>
+__device__ __forceinline__ void metric_flat(const float* __restrict__ x, const float* __restrict__ y,
+                                            uint8_t* codes, uint32_t count, const QP& p, Acc* a) {
+  constexpr bool PAIR = MODE != kSelf;
+  const FlatSplit s = split_flat(x, count);
+  const float* xb = x + s.head;
+  const float* yb = PAIR ? y + s.head : nullptr;
+  uint8_t* cb = CODES ? codes + s.head : nullptr;
+  const bool vec_y = !PAIR || ((((uintptr_t)yb) & 15u) == 0);
+  const float4* xv = reinterpret_cast<const float4*>(xb);
+  uint32_t j = threadIdx.x;
+  if (vec_y) {
+    const float4* yv = reinterpret_cast<const float4*>(yb);
+    constexpr uint32_t U = PAIR ? 4 : 8;
+    for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
+      float4 vx[U], vy[U];
+#pragma unroll
+      for (uint32_t u = 0; u < U; ++u) {
+        vx[u] = ld_stream4(xv + j + u * kThreads);
+        if (PAIR) vy[u] = ld_stream4(yv + j + u * kThreads); else vy[u] = vx[u];
+      }
+#pragma unroll
+      for (uint32_t u = 0; u < U; ++u)
+        metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * kThreads) : nullptr);
+    }
+    for (; j < s.nvec; j += kThreads) {
+      const float4 vx = ld_stream4(xv + j);
+      const float4 vy = PAIR ? ld_stream4(yv + j) : vx;
+      metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
+    }
+  } else {
+    // x and y sit at different offsets inside their 16-byte lines: vector loads for x, scalar for y
+    for (; j < s.nvec; j += kThreads) {
+      const float4 vx = ld_stream4(xv + j);
+      float4 vy;
+      vy.x = ld_stream1(yb + 4u * j); vy.y = ld_stream1(yb + 4u * j + 1);
+      vy.z = ld_stream1(yb + 4u * j + 2); vy.w = ld_stream1(yb + 4u * j + 3);
+      metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
+    }
+  }
+  if (threadIdx.x < s.head) {
+    const uint32_t i = threadIdx.x;
+    metric_elem<MODE, OFF, CODES>(ld_stream1(x + i), PAIR ? ld_stream1(y + i) : 0.0f, p, a[0],
+                                  CODES ? codes + i : nullptr);
+  }
+  if (threadIdx.x < s.tail) {
+    const uint32_t i = s.head + 4u * s.nvec + threadIdx.x;
+    metric_elem<MODE, OFF, CODES>(ld_stream1(x + i), PAIR ? ld_stream1(y + i) : 0.0f, p, a[1],
+                                  CODES ? codes + i : nullptr);
+  }
+}
+
+// One row handled by one warp.
+template <uint32_t MODE, bool OFF, bool CODES>
+__device__ __forceinline__ void metric_row(const float* __restrict__ x, const float* __restrict__ y,
+                                           uint8_t* codes, uint32_t inner, uint32_t lane, const QP& p,
+                                           Acc* a) {
+  constexpr bool PAIR = MODE != kSelf;
+  uint32_t i = lane;
+  for (; i + 96 < inner; i += 128) {
+    float vx[4], vy[4];
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u) {
+      vx[u] = ld_stream1(x + i + 32u * u);
+      vy[u] = PAIR ? ld_stream1(y + i + 32u * u) : 0.0f;
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u)
+      metric_elem<MODE, OFF, CODES>(vx[u], vy[u], p, a[u], CODES ? codes + i + 32u * u : nullptr);
+  }
+  for (; i < inner; i += 32)
+    metric_elem<MODE, OFF, CODES>(ld_stream1(x + i), PAIR ? ld_stream1(y + i) : 0.0f, p, a[0],
+                                  CODES ? codes + i : nullptr);
+}
+
+template <uint32_t MODE, bool CODES>
+__device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
+                                            const float* __restrict__ step, const float* __restrict__ inv,
+                                            const float* __restrict__ offset, Acc* a) {
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const float* x = tr->x + tl.begin;
+  const float* y = (MODE != kSelf) ? tr->y + tl.begin : nullptr;
+  uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
+  QP p;
+  p.qmin = tr->asym ? 0.0f : -127.0f;
+  p.qmax = tr->asym ? 255.0f : 127.0f;
+  if (tl.rows == 0) {
+    const uint32_t G = tr->group_base + (uint32_t)tl.row0;
+    p.step = __ldg(step + G); p.inv = __ldg(inv + G); p.off = __ldg(offset + G);
+    if (MODE == kRaw || p.off == 0.0f) metric_flat<MODE, false, CODES>(x, y, codes, tl.count, p, a);
+    else metric_flat<MODE, true, CODES>(x, y, codes, tl.count, p, a);
+  } else {
+    const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+    for (uint32_t r = warp; r < tl.rows; r += kWarps) {
+      const uint32_t G = tr->group_base + (uint32_t)((tl.row0 + r) % channels);
+      p.step = __ldg(step + G); p.inv = __ldg(inv + G); p.off = __ldg(offset + G);
+      const uint64_t o = (uint64_t)r * inner;
+      if (MODE == kRaw || p.off == 0.0f)
+        metric_row<MODE, false, CODES>(x + o, y + o, codes + o, inner, lane, p, a);
+      else
+        metric_row<MODE, true, CODES>(x + o, y + o, codes + o, inner, lane, p, a);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
+               const float* __restrict__ step, const float* __restrict__ inv,
+               const float* __restrict__ offset, double2* __restrict__ partials) {
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+    const Tile tl = load_tile(tiles, ti);
+    const TensorRec* tr = tensors + tl.tensor;
+    Acc a[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { a[k].sse = 0.0f; a[k].sig = 0.0f; }
+    const uint32_t mode = tr->pair_mode;
+    const bool codes = tr->codes != nullptr && mode != kRaw;
+    if (mode == kSelf) {
+      if (codes) metric_tile<kSelf, true>(tl, tr, step, inv, offset, a);
+      else metric_tile<kSelf, false>(tl, tr, step, inv, offset, a);
+    } else if (mode == kRequant) {
+      if (codes) metric_tile<kRequant, true>(tl, tr, step, inv, offset, a);
+      else metric_tile<kRequant, false>(tl, tr, step, inv, offset, a);
+    } else {
+      metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
+    }
+    // thread -> warp reduction in binary32 with a fixed association
+    float sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
+    float sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
+    sse = warp_sum(sse);
+    sig = warp_sum(sig);
+    if (lane == 0) partials[tl.slot + warp] = make_double2((double)sse, (double)sig);
+  }
+}
+
+// One CTA per tensor: fixed-order binary64 sum of the tensor's slots, then MSE and SQNR.
+__global__ void __launch_bounds__(256)
+metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __restrict__ partials,
+                        double* sse_out, double* sig_out, double* mse_out, double* sqnr_out) {
+  __shared__ double sh_e[256], sh_s[256];
+  const TensorRec tr = tensors[blockIdx.x];
+  double e = 0.0, s = 0.0;
+  for (uint32_t k = threadIdx.x; k < tr.slot_count; k += 256) {
+    const double2 p = partials[tr.slot_first + k];
+    e = __dadd_rn(e, p.x);
+    s = __dadd_rn(s, p.y);
+  }
+  sh_e[threadIdx.x] = e; sh_s[threadIdx.x] = s;
+  __syncthreads();
+  for (uint32_t o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      sh_e[threadIdx.x] = __dadd_rn(sh_e[threadIdx.x], sh_e[threadIdx.x + o]);
+      sh_s[threadIdx.x] = __dadd_rn(sh_s[threadIdx.x], sh_s[threadIdx.x + o]);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const double sse = sh_e[0], sig = sh_s[0];
+    const double inf = __longlong_as_double(0x7ff0000000000000ll);
+    sse_out[blockIdx.x] = sse;
+    sig_out[blockIdx.x] = sig;
+    mse_out[blockIdx.x] = tr.n_elems ? __ddiv_rn(sse, (double)tr.n_elems) : 0.0;
+    double q;
+    if (sse == 0.0) q = inf;
+    else if (sig == 0.0) q = -inf;
+    else q = __dmul_rn(10.0, log10(__ddiv_rn(sig, sse)));
+    sqnr_out[blockIdx.x] = q;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_metrics(const Launch& l, const TensorRec* tensors, const Tile* tiles,
+                           uint32_t n_tiles, const float* step, const float* inv,
+                           const float* offset, double2* partials) {
+  if (n_tiles == 0) return cudaSuccess;
+  static int per_sm = 0;
+  const int grid = persistent_grid((const void*)metrics_kernel, &per_sm, l.sm_count, n_tiles);
+  metrics_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset, partials);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
+                                    const double2* partials, double* sse, double* sig, double* mse,
+                                    double* sqnr_db) {
+  metrics_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, partials, sse, sig, mse, sqnr_db);
+  return cudaGetLastError();
+}
+
+}  // namespace qv2

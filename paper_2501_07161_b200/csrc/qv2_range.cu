@@ -137,8 +137,8 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, float* gmin, float*
     const uint32_t kx = reinterpret_cast<uint32_t*>(gmax)[G];
     float mn = kn ? key2f(~kn) : 0.0f;
     float mx = kx ? key2f(kx) : 0.0f;
-    if (mn == 0.0f) mn = 0.0f;          // -0 -> +0
-    if (mx == 0.0f) mx = 0.0f;
+    mn = __fadd_rn(mn, 0.0f);           // -0 -> +0, every other value unchanged
+    mx = __fadd_rn(mx, 0.0f);
     const float am = fmaxf(fabsf(mn), fabsf(mx));
     gmin[G] = mn; gmax[G] = mx; gabsmax[G] = am;
     amax = fmaxf(amax, am);

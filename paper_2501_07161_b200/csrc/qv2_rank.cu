@@ -1,0 +1,104 @@
+// Sensitivity list and mixed-precision layer set (Algorithm 2: CalculateSQNRdeltas,
+// CalculateAverage, RankLayersBySensitivity; SQNR delta of Eq. 16; BOPs-reduction rate of Eq. 17).
+//
+// A model has tens of layers, so one CTA does everything.  Every binary64 operation is issued
+// through an explicit round-to-nearest intrinsic so that no multiply-add is contracted and the
+// result is a bit-exact function of the inputs.
+#include "qv2_device.cuh"
+
+namespace qv2 {
+
+namespace {
+
+__device__ __forceinline__ double clamp_cap(double v, double cap) {
+  if (v > cap) return cap;
+  if (v < -cap) return -cap;
+  return v;
+}
+
+__global__ void __launch_bounds__(256)
+rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restrict__ mse_w,
+            const double* __restrict__ sqnr_a, const double* __restrict__ mse_a,
+            const uint64_t* __restrict__ macs, const double* __restrict__ pos, qv2_rank_cfg cfg,
+            double* score, double* severity, uint32_t* order, uint8_t* keep, uint32_t* n_keep) {
+  __shared__ double mean_s[2];
+  const uint32_t tid = threadIdx.x;
+  const double inf = __longlong_as_double(0x7ff0000000000000ll);
+  if (tid == 0) {                      // means: sums in layer order, as the definition states
+    double sw = 0.0, sa = 0.0;
+    for (uint32_t i = 0; i < n; ++i) { sw = __dadd_rn(sw, mse_w[i]); sa = __dadd_rn(sa, mse_a[i]); }
+    mean_s[0] = __ddiv_rn(sw, (double)n);
+    mean_s[1] = __ddiv_rn(sa, (double)n);
+  }
+  __syncthreads();
+  const double mean_w = mean_s[0], mean_a = mean_s[1], cap = cfg.sqnr_cap_db;
+  for (uint32_t i = tid; i < n; i += blockDim.x) {
+    double dw = 0.0, da = 0.0;
+    if (i > 0) {
+      const double den = pos ? __dsub_rn(pos[i], pos[i - 1]) : 1.0;
+      dw = __ddiv_rn(__dsub_rn(clamp_cap(sqnr_w[i], cap), clamp_cap(sqnr_w[i - 1], cap)), den);
+      da = __ddiv_rn(__dsub_rn(clamp_cap(sqnr_a[i], cap), clamp_cap(sqnr_a[i - 1], cap)), den);
+    }
+    double sc = __dadd_rn(__dmul_rn(cfg.w_gain, dw), __dmul_rn(cfg.a_gain, da));
+    if (sc != sc) sc = inf;
+    const double rw = mean_w > 0.0 ? __ddiv_rn(mse_w[i], mean_w) : 0.0;
+    const double ra = mean_a > 0.0 ? __ddiv_rn(mse_a[i], mean_a) : 0.0;
+    double sv = rw > ra ? rw : ra;
+    if (sv != sv) sv = 0.0;
+    score[i] = sc; severity[i] = sv; keep[i] = 0;
+  }
+  __syncthreads();
+  // Position of layer i = number of layers that come before it: all MSE outliers precede the
+  // rest; outliers by descending severity, the rest by ascending score, ties by layer index.
+  const double fac = cfg.mse_factor;
+  for (uint32_t i = tid; i < n; i += blockDim.x) {
+    const double si = score[i], vi = severity[i];
+    const bool out_i = vi > fac;
+    uint32_t rank = 0;
+    for (uint32_t j = 0; j < n; ++j) {
+      const double vj = severity[j];
+      const bool out_j = vj > fac;
+      if (out_i) {
+        if (out_j && (vj > vi || (vj == vi && j < i))) ++rank;
+      } else {
+        if (out_j) ++rank;
+        else {
+          const double sj = score[j];
+          if (sj < si || (sj == si && j < i)) ++rank;
+        }
+      }
+    }
+    order[rank] = i;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t nk = 0;
+    if (cfg.select_mode == QV2_BY_COUNT) {
+      nk = cfg.keep_count < n ? cfg.keep_count : n;
+    } else {
+      unsigned __int128 total = 0, kept = 0;
+      for (uint32_t i = 0; i < n; ++i) total += macs ? macs[i] : 1ull;
+      for (uint32_t j = 0; j < n; ++j) {       // grow the FP32 prefix while the rate still holds
+        const unsigned __int128 m = macs ? macs[order[j]] : 1ull;
+        const unsigned __int128 quantized = total - (kept + m);
+        if (quantized * 10000u >= (unsigned __int128)cfg.rate_permyriad * total) { kept += m; nk = j + 1; }
+        else break;
+      }
+    }
+    for (uint32_t j = 0; j < nk; ++j) keep[order[j]] = 1;
+    *n_keep = nk;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_rank(const Launch& l, uint32_t n, const double* sqnr_w, const double* mse_w,
+                        const double* sqnr_a, const double* mse_a, const uint64_t* macs,
+                        const double* pos, qv2_rank_cfg cfg, double* score, double* severity,
+                        uint32_t* order, uint8_t* keep, uint32_t* n_keep) {
+  rank_kernel<<<1, 256, 0, l.stream>>>(n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, cfg, score,
+                                       severity, order, keep, n_keep);
+  return cudaGetLastError();
+}
+
+}  // namespace qv2
