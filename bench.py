@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the full-model sensitivity pass (calibrate + fake-quantize + MSE/SQNR + rank).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole path over one synthetic model (default: VGG-16 shapes, batch 64,
+per-channel int8 weights, 99.99 % percentile-clipped uint8 activations, ~7.5 GB resident, far more
+than the 126 MB L2, so nothing is served from cache between steps).  With N > 1 (torchrun) every
+rank sweeps its own replica; there is no data exchange between GPUs.  Rank 0 prints ONE JSON line.
+
+--impl reference times the CPU oracle (oracle/) on the host cores on a bounded sample of the same
+workload; it is a deliberately plain program and only a context number.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+import torch.distributed as dist
+
+import gen
+
+METRIC = "GB/s swept (calibrate+quant+MSE/SQNR), full-model sensitivity pass"
+UNIT = "GB/s"
+NS_PER_ELEM_PASS = 4.5e-9      # rough oracle cost per element and pass, used only to size samples
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="vgg16", choices=gen.CONFIG_ORDER)
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Polls SM clock, max clock, power and throttle reasons through NVML while the GPU works."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+               0x100: "display_clock_setting", 0x10: "sync_boost"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples = []
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thr = None
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _poll(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                try:
+                    watts = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                except Exception:
+                    watts = None
+                self.samples.append((time.perf_counter(), mhz, mask, watts))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._poll, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join(timeout=2)
+
+    def summary(self, t0: float, t1: float):
+        if self.nv is None or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0,
+                    "note": "NVML unavailable"}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = None
+        if not inside:                                   # very short region: take the nearest sample
+            inside = [min(self.samples, key=lambda s: abs(s[0] - (t0 + t1) / 2))]
+            note = "timed region shorter than the sampling period; nearest sample used"
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        reasons = [n for b, n in self.REASONS.items() if mask & b]
+        watts = [s[3] for s in inside if s[3] is not None]
+        out = {"sm_mhz": float(np.median([s[1] for s in inside])), "sm_max_mhz": self.max_mhz,
+               "reasons": reasons, "samples": len(inside),
+               "power_w_max": max(watts) if watts else None}
+        if note:
+            out["note"] = note
+        return out
+
+
+# -------------------------------------------------------------------------------- reference arm
+def oracle_sample_jobs(model, act_images: int, max_weight_elems: int):
+    """Oracle jobs for a bounded sample: every layer's activations restricted to the first
+    `act_images` images, and the weight tensors (in layer order) that fit the element budget (a
+    tensor larger than a quarter of the budget is left out so that no single job dominates)."""
+    cfg = model.config
+    pct = cfg.a_percentile if cfg.a_range == "percentile" else None
+    jobs, w_used, swept = [], 0, 0
+    for l in model.layers:
+        if l.w.numel() <= max_weight_elems // 4 and w_used + l.w.numel() <= max_weight_elems:
+            w_used += l.w.numel()
+            for g in cfg.w_granularity:
+                jobs.append(dict(x=l.w.detach().cpu().numpy().reshape(-1), y=None, outer=1,
+                                 channels=l.w.shape[0], inner=l.w.shape[1],
+                                 per_channel=g == "channel", asym_u8=False))
+                swept += 8 * l.w.numel()
+    for l in model.layers:
+        b = min(act_images, l.x.shape[0])
+        x = l.x[:b].detach().cpu().numpy().reshape(-1)
+        y = l.y[:b].detach().cpu().numpy().reshape(-1)
+        jobs.append(dict(x=x, y=y, outer=b, channels=l.x.shape[1], inner=l.x.shape[2],
+                         per_channel=False, asym_u8=True, percentile=pct))
+        swept += (16 if pct is not None else 12) * x.size
+    return jobs, swept, w_used
+
+
+def size_sample(name: str, batch: int, seconds_per_step: float, threads: int):
+    """Pick (images, weight-element budget) so that one oracle step takes about seconds_per_step."""
+    w, a, _ = gen.model_sizes(name, batch)
+    per_image = a // batch
+    budget = seconds_per_step * threads / NS_PER_ELEM_PASS / 3.0      # elements, ~3 passes each
+    images = int(max(1, min(batch, (budget / 2) // max(per_image, 1))))
+    return images, int(budget / 2)
+
+
+def run_oracle_steps(jobs, threads, steps, warmup):
+    import oracle
+    for _ in range(warmup):
+        oracle.sweep_tensors(jobs, threads=threads)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        res = oracle.sweep_tensors(jobs, threads=threads)
+    return (time.perf_counter() - t0) / max(steps, 1), res
+
+
+def reference_main(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    threads = os.cpu_count() or 1
+    total_steps = args.steps + args.warmup
+    per_step = min(2.0, 120.0 / max(total_steps, 1))
+    batch = args.batch or gen.CONFIGS[args.workload].batch
+    images, wbudget = size_sample(args.workload, batch, per_step, threads)
+    model = gen.make_model(args.workload, seed=0, device="cpu", batch=images)
+    jobs, swept, w_used = oracle_sample_jobs(model, images, wbudget)
+    threads = min(threads, len(jobs))
+    sec, _ = run_oracle_steps(jobs, threads, args.steps, args.warmup)
+    value = swept / sec / 1e9
+    sample = (f"{args.workload} shapes: activations of the first {images} of {batch} images for all "
+              f"{len(model.layers)} layers, weight tensors in layer order up to {w_used} elements; "
+              f"{swept / 1e9:.3f} GB swept per step")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": {"workload": args.workload, "batch": batch, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# --------------------------------------------------------------------------------------- ours
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def recorded_traffic():
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture, valid only
+    while the kernel source is unchanged since the capture."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "metrics_kernel_traffic.json")) as f:
+            rec = json.load(f)
+        h = hashlib.sha256()
+        for rel in rec["sources"]:
+            with open(os.path.join(ROOT, rel), "rb") as s:
+                h.update(s.read())
+        if h.hexdigest() != rec["sha256"]:
+            return None
+        return rec
+    except Exception:
+        return None
+
+
+def ours_main(args):
+    import paper_2501_07161_b200 as q
+    from paper_2501_07161_b200 import replicas as R
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the sweep has no CPU implementation")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rank = R.rank()
+    cfgw = gen.CONFIGS[args.workload]
+    batch = args.batch or cfgw.batch
+
+    model = gen.make_model(args.workload, seed=R.replica_seed(0, rank), device="cuda", batch=batch)
+    ctx = q.Context(local)
+    md = q.model_descs(model)
+    n, L = md.n_tensors, md.n_layers
+    rcfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
+    sb, t = ctx.alloc_sweep_buffers(md.descs, L)
+    swept = gen.swept_bytes(args.workload, batch)
+    w_elems, a_elems = model.weight_elems, model.act_elems
+    metrics_bytes = 4 * w_elems * len(cfgw.w_granularity) + 8 * a_elems   # one launch of the core kernel
+
+    lib = q.lib()
+    import ctypes as C
+    h = ctx._h
+
+    def one_step(ev=None):
+        """The three calls of the contract, back to back on the context's stream."""
+        if ev: ev[0].record()
+        st = lib.qv2_calibrate(h, md.descs, n, *[t[k].data_ptr() for k in
+                               ("gmin", "gmax", "gabsmax", "hist", "clip", "step", "inv", "offset", "nonfinite")])
+        if ev: ev[1].record()
+        st |= lib.qv2_quant_metrics(h, md.descs, n, t["step"].data_ptr(), t["inv"].data_ptr(),
+                                    t["offset"].data_ptr(), None, t["sse"].data_ptr(), t["sig"].data_ptr(),
+                                    t["mse"].data_ptr(), t["sqnr_db"].data_ptr())
+        if ev: ev[2].record()
+        st |= lib.qv2_rank_layers(h, L, t["sqnr_db"].data_ptr(), t["mse"].data_ptr(),
+                                  t["sqnr_db"].data_ptr() + 8 * L, t["mse"].data_ptr() + 8 * L,
+                                  md.macs.data_ptr(), None, C.byref(rcfg), t["order"].data_ptr(),
+                                  t["keep_fp32"].data_ptr(), t["n_keep"].data_ptr())
+        if ev: ev[3].record()
+        if st != 0:
+            raise RuntimeError(f"qv2 call failed with status {st}")
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    torch.cuda.synchronize()
+    R.barrier()
+    torch.cuda.synchronize()
+
+    K = args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    launches0 = ctx.launches
+    t_wall0 = time.perf_counter()
+    for k in range(K):
+        one_step(evs[k])
+    torch.cuda.synchronize()
+    t_wall1 = time.perf_counter()
+    R.barrier()
+    launches = ctx.launches - launches0
+    total_ms = evs[0][0].elapsed_time(evs[-1][3])
+    cal_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    met_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    rank_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
+    step_ms = sorted(e[0].elapsed_time(e[3]) for e in evs)
+    clocks = sampler.summary(t_wall0, t_wall1)
+    sampler.stop()
+
+    value, slowest_s = R.whole_job_throughput(swept * K / 1e9, total_ms / 1e3)
+    ms_per_step = slowest_s * 1e3 / K
+
+    # ------------------------------------------------------------------ end to end (host buffers)
+    e2e = None
+    if not args.no_e2e:
+        host = [(l.w.cpu().pin_memory(), l.x.cpu().pin_memory(), l.y.cpu().pin_memory()) for l in model.layers]
+
+        class _L:  # same layers, tensors in pinned host memory
+            pass
+        hl = []
+        for l, (w, x, y) in zip(model.layers, host):
+            o = _L(); o.w, o.x, o.y, o.macs = w, x, y, l.macs
+            hl.append(o)
+        hm = _L(); hm.layers = hl; hm.config = model.config
+        hd = q.model_descs(hm, host=True)
+        staging = torch.empty(q.binding.staging_bytes(hd.descs, L), dtype=torch.uint8, device="cuda")
+        out = dict(mse=np.zeros(n), sqnr_db=np.zeros(n), nonfinite=np.zeros(n, np.uint64),
+                   order=np.zeros(L, np.uint32), keep_fp32=np.zeros(L, np.uint8), n_keep=np.zeros(1, np.uint32))
+        hr = q.binding.HostResults(**{k: v.ctypes.data for k, v in out.items()})
+        ctx.sweep_model_host(hd.descs, L, hd.macs, None, rcfg, staging, sb, hr)      # warm-up
+        torch.cuda.synchronize()
+        R.barrier()
+        E = max(1, args.e2e_steps)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(E):
+            ctx.sweep_model_host(hd.descs, L, hd.macs, None, rcfg, staging, sb, hr)
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_val, _ = R.whole_job_throughput(swept * E / 1e9, e0.elapsed_time(e1) / 1e3)
+        h2d = 4 * (w_elems * len(cfgw.w_granularity) + 2 * a_elems) + 8 * L
+        d2h = sum(v.nbytes for v in out.values())
+        e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": e0.elapsed_time(e1) / E, "steps": E,
+               "api": "qv2_sweep_model_host (pinned host tensors, copies inside the timed region)"}
+        same = np.array_equal(out["order"], t["order"].cpu().numpy().view(np.uint32)[:L])
+        e2e["matches_device_path"] = bool(same)
+        del staging, host
+
+    # ------------------------------------------------------------------ CPU oracle beside it
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        threads = os.cpu_count() or 1
+        images, wbudget = size_sample(args.workload, batch, 2.0, threads)
+        jobs, s_swept, w_used = oracle_sample_jobs(model, images, wbudget)
+        threads = min(threads, len(jobs))
+        sec, _ = run_oracle_steps(jobs, threads, 1, 0)
+        cpu = {"value": s_swept / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": (f"activations of the first {images} of {batch} images for all {L} layers, weight "
+                          f"tensors in layer order up to {w_used} elements; {s_swept / 1e9:.3f} GB swept, "
+                          f"{sec:.2f} s")}
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        achieved = metrics_bytes / (met_ms * 1e-3) / 1e9
+        rec = recorded_traffic()
+        traffic = None
+        if rec is not None:
+            traffic = rec["dram_bytes_per_algorithmic_byte"] * metrics_bytes
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "batch": batch, "layers": L, "tensors": n,
+                       "weight_elems": w_elems, "act_elems": a_elems, "swept_bytes_per_step": swept,
+                       "resident_bytes": 4 * (w_elems + 2 * a_elems),
+                       "l2": "inputs larger than L2 (no flush needed)" if 4 * (w_elems + 2 * a_elems) > 4 * 126e6
+                             else "inputs fit in L2: this is an L2 number, not an HBM one",
+                       "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
+                       "seed": 0},
+            "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_min": step_ms[0],
+            "phases_ms": {"calibrate": cal_ms, "quant_metrics": met_ms, "rank": rank_ms},
+            "frac_of_measured_copy_peak": value / world / peak,
+            "frac_of_8000_nominal": value / world / 8000.0,
+            "roofline": {"kernel": "metrics_kernel (qv2_quant_metrics)", "bound": "hbm",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": metrics_bytes,
+                         "duration_ms": met_ms,
+                         "note": "duration = CUDA events around the qv2_quant_metrics call on its stream "
+                                 "(the streaming kernel plus a per-tensor finalize kernel of a few microseconds)"},
+            "clocks": clocks, "gpu_launches": int(launches),
+        }
+        if e2e is not None:
+            line["e2e"] = e2e
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        return reference_main(args)
+    return ours_main(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -221,7 +221,8 @@ void qv2o_quant_metrics(const float *x, const float *y,
  *  4. r_n = max(mse_w[n] / mean(mse_w), mse_a[n] / mean(mse_a)), a zero mean contributing 0;
  *     layers with r_n > mse_factor (5 in the paper) go to the top, most severe first.
  *  5. the remaining layers follow in ascending score (smaller delta = noise grew = more
- *     sensitive); ties keep layer order.
+ *     sensitive); ties keep layer order.  A NaN score counts as +inf, a NaN severity as 0 (the
+ *     paper does not say what an undefined metric does; this keeps the list a permutation).
  *  6. select_mode 0: the first keep_count entries stay FP32.  select_mode 1: the longest prefix
  *     stays FP32 for which the MAC-weighted share of quantized layers is still
  *     >= rate_permyriad / 10000 (integer arithmetic).
@@ -258,9 +259,11 @@ void qv2o_rank(uint32_t n, const double *sqnr_w, const double *mse_w,
         double tw = w_gain * dw;
         double ta = a_gain * da;
         score[i] = tw + ta;
+        if (isnan(score[i])) score[i] = INFINITY;      /* an undefined score sorts last */
         double rw = (mean_w > 0.0) ? mse_w[i] / mean_w : 0.0;
         double ra = (mean_a > 0.0) ? mse_a[i] / mean_a : 0.0;
         sev[i] = rw > ra ? rw : ra;
+        if (isnan(sev[i])) sev[i] = 0.0;               /* an undefined severity is no outlier */
     }
     /* selection sort, written for clarity: repeatedly take the best remaining layer */
     uint32_t filled = 0;

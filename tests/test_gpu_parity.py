@@ -1,0 +1,220 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded
+inputs, element by element.  Sizes span several 16384-element tiles and ragged tails; edge cases
+cover empty, tiny, misaligned, constant, non-finite and on-grid tensors."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2501_07161_b200 as q
+from parity import Spec, assert_metric_close, check_specs
+
+pytestmark = pytest.mark.gpu
+
+TILE = 16384
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = q.Context(0)
+    yield c
+    c.close()
+
+
+def _g(seed):
+    g = torch.Generator()
+    g.manual_seed(seed)
+    return g
+
+
+def randn(n, seed, scale=1.0):
+    return torch.randn(n, generator=_g(seed)) * scale
+
+
+# ------------------------------------------------------------------------ per-tensor, self mode
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 31, 1000, TILE - 1, TILE, TILE + 1, 3 * TILE + 777, 20 * TILE + 13])
+@pytest.mark.parametrize("asym", [False, True])
+def test_per_tensor_self_sizes(ctx, n, asym):
+    check_specs(ctx, [Spec(randn(n, n), 1, 1, n, asym=asym)])
+
+
+@pytest.mark.parametrize("mis", [1, 2, 3])
+def test_misaligned_base_pointer(ctx, mis):
+    n = 2 * TILE + 5
+    check_specs(ctx, [Spec(randn(n, 7), 1, 1, n), Spec(randn(n, 8).abs(), 1, 1, n, asym=True)],
+                misalign_x=mis)
+
+
+def test_relu_activation_has_zero_offset_and_percentile(ctx):
+    n = 5 * TILE + 99
+    x = randn(n, 11).clamp_min(0)
+    check_specs(ctx, [Spec(x, 1, 1, n, asym=True, percentile=0.9999),
+                      Spec(x, 1, 1, n, asym=True, percentile=0.99),
+                      Spec(randn(n, 12), 1, 1, n, asym=True, percentile=0.999),
+                      Spec(randn(n, 13), 1, 1, n, asym=False, percentile=0.999)])
+
+
+# --------------------------------------------------------------------------------- per channel
+@pytest.mark.parametrize("cout,k", [(7, 1), (960, 9), (64, 27), (96, 147), (130, 576), (33, 1153),
+                                    (9, 4095), (5, 4096), (5, 4097), (3, 25088), (2, 2 * TILE + 3)])
+def test_per_channel_weights(ctx, cout, k):
+    w = randn(cout * k, cout + k) * torch.exp(randn(cout, 3)).repeat_interleave(k)
+    check_specs(ctx, [Spec(w, 1, cout, k, per_channel=True),
+                      Spec(w, 1, cout, k, per_channel=True, asym=True)])
+
+
+@pytest.mark.parametrize("o,c,i", [(3, 5, 100), (2, 3, 5000), (4, 2, TILE + 7), (17, 4, 49), (2, 1, 9)])
+def test_per_channel_with_outer_dimension(ctx, o, c, i):
+    x = randn(o * c * i, o + c + i) * torch.exp(randn(c, 5)).repeat_interleave(i).repeat(o)
+    y = x + 0.01 * randn(x.numel(), 99)
+    check_specs(ctx, [Spec(x, o, c, i, per_channel=True, asym=True, y=y),
+                      Spec(x, o, c, i, per_channel=True, asym=False),
+                      Spec(x, o, c, i, per_channel=True, asym=True, percentile=0.995)])
+
+
+# ----------------------------------------------------------------------------------- pair modes
+@pytest.mark.parametrize("mx,my", [(0, 0), (1, 1), (0, 2), (3, 1)])
+def test_pair_modes_and_mixed_alignment(ctx, mx, my):
+    n = 4 * TILE + 321
+    x = randn(n, 21)
+    y = x + 0.02 * randn(n, 22)
+    xr = x.clamp_min(0)
+    yr = xr + 0.02 * randn(n, 23)
+    check_specs(ctx, [Spec(x, 1, 1, n, asym=True, y=y),               # offset != 0
+                      Spec(xr, 1, 1, n, asym=True, y=yr),             # offset == 0
+                      Spec(x, 1, 1, n, asym=True, y=y, raw=True),
+                      Spec(x, 1, 1, n, asym=False, y=y),
+                      Spec(x[: 8 * (n // 8)], 2, 4, n // 8, per_channel=True, asym=True,
+                           y=y[: 8 * (n // 8)])],
+                misalign_x=mx, misalign_y=my)
+
+
+# ----------------------------------------------------------------------------------- edge cases
+def test_empty_constant_and_zero_tensors_in_one_batch(ctx):
+    specs = [Spec(torch.zeros(0), 0, 3, 5, per_channel=True),
+             Spec(randn(100, 1), 1, 1, 100),
+             Spec(torch.zeros(0), 1, 1, 0, asym=True, percentile=0.99),
+             Spec(torch.zeros(1000), 1, 1, 1000, asym=True, percentile=0.99),
+             Spec(torch.full((1000,), 2.5), 1, 1, 1000, asym=True),
+             Spec(torch.full((1000,), -2.5), 1, 4, 250, per_channel=True),
+             Spec(-torch.zeros(8), 1, 1, 8)]
+    cal, met = check_specs(ctx, specs)
+    assert float(met.sqnr_db[0]) == math.inf and float(met.mse[0]) == 0.0
+
+
+def test_on_grid_tensor_zero_error(ctx):
+    d = 2.0 ** -7
+    k = torch.arange(-127, 128, dtype=torch.float32).repeat(300)
+    cal, met = check_specs(ctx, [Spec(k * d, 1, 1, k.numel())])
+    assert float(met.sse[0]) == 0.0 and float(met.sqnr_db[0]) == math.inf
+
+
+def test_exact_ties_round_to_even(ctx):
+    d = 2.0 ** -7
+    k = torch.arange(-126, 126, dtype=torch.float32)
+    x = torch.cat([(k + 0.5) * d, torch.tensor([127 * d, -127 * d])]).repeat(70)
+    check_specs(ctx, [Spec(x, 1, 1, x.numel())])
+
+
+def test_nonfinite_inputs_are_counted_and_excluded(ctx):
+    n = 3 * TILE + 50
+    x = randn(n, 31)
+    x[0] = float("nan"); x[5] = float("inf"); x[TILE + 3] = float("-inf"); x[n - 1] = float("nan")
+    x[2 * TILE + 17] = float("inf")
+    w = randn(40 * 300, 32)
+    w[7 * 300 + 5] = float("nan"); w[39 * 300 + 299] = float("inf")
+    cal, _ = check_specs(ctx, [Spec(x, 1, 1, n, asym=True, percentile=0.99),
+                               Spec(w, 1, 40, 300, per_channel=True),
+                               Spec(randn(1000, 33), 1, 1, 1000)], check_codes=False)
+    assert cal.nonfinite.tolist() == [5, 2, 0]
+
+
+def test_extreme_magnitudes(ctx):
+    """Squares are accumulated in binary32, so magnitudes are kept where x^2 and e^2 stay in its
+    range; the parameter path alone is also exercised with denormal and huge ranges."""
+    n = TILE + 9
+    check_specs(ctx, [Spec(randn(n, 41) * 1e-12, 1, 1, n), Spec(randn(n, 42) * 1e12, 1, 1, n, asym=True),
+                      Spec(randn(n, 44).abs() * 1e10, 1, 1, n, asym=True, percentile=0.999)])
+    # ranges / parameters / histogram stay bit-exact far outside that range
+    xs = [randn(n, 45) * 1e-42, randn(n, 46) * 1e30]
+    dev = [x.cuda() for x in xs]
+    descs = q.desc_array([q.make_desc(d, None, 1, 1, n, q.PER_TENSOR, q.ASYM_U8, q.PERCENTILE, 0.999)
+                          for d in dev])
+    cal = ctx.calibrate(descs)
+    torch.cuda.synchronize()
+    for t, x in enumerate(xs):
+        ref = oracle.calibrate_tensor(x.numpy(), 1, 1, n, False, True, 0.999)
+        gmin, gmax, gabs, bad, hist, clip, step, inv, off = ref
+        got = lambda a: a[t:t + 1].cpu().numpy().view(np.uint32)[0]
+        for a, r in ((cal.gmin, gmin), (cal.gmax, gmax), (cal.step, step), (cal.inv, inv), (cal.offset, off)):
+            assert got(a) == r.view(np.uint32)[0]
+        assert got(cal.clip) == np.float32(clip).view(np.uint32)
+        assert np.array_equal(cal.hist.cpu().numpy().view(np.uint64).reshape(-1, 2048)[t], hist)
+
+
+# ----------------------------------------------------------------------------------------- rank
+def test_rank_is_bit_exact_on_oracle_metrics(ctx):
+    rng = np.random.default_rng(5)
+    for trial in range(40):
+        n = int(rng.integers(1, 120))
+        sw = rng.uniform(-5, 60, n).round(1); sa = rng.uniform(-5, 60, n).round(1)
+        mw = rng.choice([0.0, 1e-6, 1e-5, 3e-4, 2e-3], n); ma = rng.choice([1e-3, 2e-3, 9e-2, 0.5], n)
+        if trial % 5 == 0:
+            sw[rng.integers(0, n)] = math.inf
+        macs = rng.integers(0, 10 ** 9, n).astype(np.uint64)
+        pos = np.cumsum(rng.integers(1, 4, n)).astype(np.float64) if trial % 3 == 0 else None
+        mode = trial % 2
+        rate = int(rng.integers(0, 10001)); kc = int(rng.integers(0, n + 2))
+        ro, rk, rn = oracle.rank_layers(sw, mw, sa, ma, macs=macs, pos=pos, select_mode=mode,
+                                        keep_count=kc, rate_permyriad=rate)
+        dv = lambda a: torch.from_numpy(np.asarray(a)).cuda()
+        cfg = q.default_rank_cfg(select_mode=mode, keep_count=kc, rate_permyriad=rate)
+        o, k, nk = ctx.rank_layers(dv(sw), dv(mw), dv(sa), dv(ma), dv(macs.view(np.int64)),
+                                   None if pos is None else dv(pos), cfg)
+        torch.cuda.synchronize()
+        assert o.cpu().numpy().view(np.uint32).tolist() == ro.tolist()
+        assert k.cpu().numpy().tolist() == rk.tolist() and int(nk) == rn
+
+
+def test_rank_without_macs_counts_layers(ctx):
+    sw = torch.tensor([30.0, 20.0, 25.0, 40.0], dtype=torch.float64).cuda()
+    ones = torch.ones(4, dtype=torch.float64).cuda()
+    cfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=5000)
+    o, k, nk = ctx.rank_layers(sw, ones, sw, ones, None, None, cfg)
+    ro, rk, rn = oracle.rank_layers(sw.cpu().numpy(), np.ones(4), sw.cpu().numpy(), np.ones(4),
+                                    select_mode=1, rate_permyriad=5000)
+    assert o.cpu().numpy().view(np.uint32).tolist() == ro.tolist() and int(nk) == rn == 2
+
+
+# --------------------------------------------------------------------------------- error paths
+def test_argument_errors_are_reported_before_launch(ctx):
+    x = torch.zeros(64, device="cuda")
+    good = q.make_desc(x, None, 1, 1, 64, q.PER_TENSOR, q.SYM_I8)
+    bad_enum = q.make_desc(x, None, 1, 1, 64, 7, q.SYM_I8)
+    with pytest.raises(q.binding.Qv2Error) as e:
+        ctx.calibrate(q.desc_array([good, bad_enum]))
+    assert e.value.status == -1
+    null_x = q.make_desc(None, None, 1, 1, 64, q.PER_TENSOR, q.SYM_I8)
+    with pytest.raises(q.binding.Qv2Error) as e:
+        ctx.calibrate(q.desc_array([null_x]))
+    assert e.value.status == -2
+    mis = q.make_desc(x, None, 1, 1, 32, q.PER_TENSOR, q.SYM_I8); mis.x = x.data_ptr() + 2
+    with pytest.raises(q.binding.Qv2Error) as e:
+        ctx.calibrate(q.desc_array([mis]))
+    assert e.value.status == -3
+    badp = q.make_desc(x, None, 1, 1, 64, q.PER_TENSOR, q.ASYM_U8, q.PERCENTILE, 1.5)
+    with pytest.raises(q.binding.Qv2Error) as e:
+        ctx.calibrate(q.desc_array([badp]))
+    assert e.value.status == -1
+    raw_no_y = q.make_desc(x, None, 1, 1, 64, q.PER_TENSOR, q.ASYM_U8, flags=q.PAIR_RAW)
+    with pytest.raises(q.binding.Qv2Error):
+        ctx.calibrate(q.desc_array([raw_no_y]))
+    z = torch.zeros(4, dtype=torch.float64, device="cuda")
+    with pytest.raises(q.binding.Qv2Error) as e:
+        ctx.rank_layers(z[:0], z[:0], z[:0], z[:0])
+    assert e.value.status == -4
+    # the context is still usable afterwards
+    check_specs(ctx, [Spec(randn(500, 3), 1, 1, 500)])

@@ -415,3 +415,11 @@ def test_select_by_bops_rate_against_prefix_enumeration():
     order, keep, nk = oracle.rank_layers([30, 20], [1, 1], [30, 20], [1, 1], macs=[5, 5],
                                          select_mode=1, rate_permyriad=5000)
     assert nk == 1 and keep[order[0]] == 1
+
+
+def test_rank_with_undefined_metrics_is_still_a_permutation():
+    sw = [30.0, math.nan, 25.0, 40.0]
+    sa = [30.0, 20.0, 25.0, 40.0]
+    order, _, _ = oracle.rank_layers(sw, [1, 1, 1, 1], sa, [1, math.nan, 1, 1])
+    # layers 1 and 2 have NaN deltas -> +inf score -> last, in layer order; a NaN MSE is no outlier
+    assert order.tolist() == [0, 3, 1, 2]
