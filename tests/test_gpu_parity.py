@@ -212,9 +212,9 @@ def test_argument_errors_are_reported_before_launch(ctx):
     raw_no_y = q.make_desc(x, None, 1, 1, 64, q.PER_TENSOR, q.ASYM_U8, flags=q.PAIR_RAW)
     with pytest.raises(q.binding.Qv2Error):
         ctx.calibrate(q.desc_array([raw_no_y]))
-    z = torch.zeros(4, dtype=torch.float64, device="cuda")
+    z = torch.zeros(8193, dtype=torch.float64, device="cuda")     # more layers than supported
     with pytest.raises(q.binding.Qv2Error) as e:
-        ctx.rank_layers(z[:0], z[:0], z[:0], z[:0])
+        ctx.rank_layers(z, z, z, z)
     assert e.value.status == -4
     # the context is still usable afterwards
     check_specs(ctx, [Spec(randn(500, 3), 1, 1, 500)])
