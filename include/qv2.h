@@ -149,8 +149,10 @@ int qv2_calibrate(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
  *   v^ = q*step_g + offset_g;          e = x - v^          (QV2_PAIR_RAW: e = x - y, no codes)
  * Per tensor: sse = sum e^2, sig = sum x^2 (the signal is always the reference tensor x),
  * mse = sse/N, sqnr_db = 10 log10(sig/sse) (+inf when sse == 0, -inf when sig == 0 < sse).
- * Sums are accumulated in binary32 per warp and tile, then in binary64 in a fixed order, so two
- * runs give identical bits.
+ * Squares are accumulated in binary32 within a tile (chains of 16 additions), then in binary64 in
+ * a fixed order, so two runs on the same GPU model give identical bits.  Because the first level
+ * is binary32, tensors whose x^2 or e^2 leave its range (|x| beyond roughly 1e-18 .. 1e18) lose
+ * accuracy.
  *
  * descs: host, n descriptors (x and, for pair mode, y device pointers).
  * step, inv, offset: device, per-group parameters in qv2_calibrate's layout.

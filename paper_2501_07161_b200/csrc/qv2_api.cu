@@ -12,6 +12,7 @@ struct qv2_ctx {
   int device = 0;
   cudaStream_t stream = nullptr;
   int sm_count = 1;
+  uint32_t metrics_cap = 1;   // largest useful grid of the metrics kernel on this device
   int last_cuda = 0;
   uint64_t launches = 0;
 
@@ -86,7 +87,7 @@ int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* cons
   if (c->plan_valid && key == c->plan_key) return QV2_OK;
 
   HostPlan plan;
-  int st = build_plan(descs, n, codes, &plan);
+  int st = build_plan(descs, n, codes, c->metrics_cap, &plan);
   if (st != QV2_OK) return st;
   // The previous upload may still be reading the pinned buffer, and buffers may be reallocated.
   QV2_CUDA(c, cudaStreamSynchronize(c->stream));
@@ -148,6 +149,7 @@ extern "C" int qv2_create(qv2_ctx** out, int device, void* stream) {
   if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_rank, 2 * (size_t)kMaxRankLayers * sizeof(double));
   if (e != cudaSuccess) { delete c; return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA; }
   c->sm_count = sms > 0 ? sms : 1;
+  c->metrics_cap = metrics_grid_cap(c->sm_count);
   *out = c;
   return QV2_OK;
 }
@@ -223,7 +225,7 @@ extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint3
   const HostPlan& p = c->plan;
   const Launch l = launch_of(c);
   if (!p.tiles.empty()) {
-    QV2_CUDA(c, launch_metrics(l, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
+    QV2_CUDA(c, launch_metrics(l, p.metrics_grid, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
                                offset, c->d_partials));
     ++c->launches;
   }

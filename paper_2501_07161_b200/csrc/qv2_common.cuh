@@ -34,9 +34,9 @@ struct TensorRec {
   uint32_t asym;             // 0: symmetric int8, 1: asymmetric uint8
   uint32_t range_mode;       // QV2_ABSMAX | QV2_MINMAX | QV2_PERCENTILE
   uint32_t pair_mode;        // PairMode
-  uint32_t slot_first;       // first partial-sum slot of this tensor (kWarps slots per tile)
-  uint32_t slot_count;
-  uint32_t pad_;
+  uint32_t slot_first;       // first partial-sum slot of this tensor
+  uint32_t slot_count;       // kWarps slots for every CTA of the metrics grid that owns a tile of it
+  uint32_t tile_first;       // index of this tensor's first tile in the tile table
   double percentile;
 };
 
@@ -44,14 +44,13 @@ struct TensorRec {
 //  rows == 0: every element belongs to quantization group `row0` (0 for per-tensor tensors).
 //  rows  > 0: `rows` whole rows of `inner` elements starting at row `row0`; the group of row r
 //             is r % channels.
-// `slot` is the tile's first partial-sum slot; warp w of the CTA writes slot + w.
 struct Tile {
   uint64_t begin;
   uint64_t row0;
   uint32_t count;
   uint32_t tensor;
   uint32_t rows;
-  uint32_t slot;
+  uint32_t reserved;
 };
 static_assert(sizeof(Tile) == 32, "Tile is read as two 16-byte words");
 
@@ -61,11 +60,14 @@ struct HostPlan {
   std::vector<Tile> hist_tiles;   // flat tiles of the tensors that need a histogram
   uint64_t total_groups = 0;
   uint32_t total_slots = 0;
+  uint32_t metrics_grid = 1;      // CTAs of the metrics launch; the slot layout depends on it
   bool any_percentile = false;
 };
 
-// Validates the descriptors and cuts them into tiles.  `codes` may be NULL.  Returns a QV2 status.
-int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, HostPlan* out);
+// Validates the descriptors and cuts them into tiles.  `codes` may be NULL.  `grid_cap` is the
+// largest useful grid of the metrics kernel (resident CTAs per SM x SMs).  Returns a QV2 status.
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t grid_cap,
+               HostPlan* out);
 
 // ------------------------------------------------------------------------------------------------
 // Launch wrappers (defined next to their kernels).  All enqueue on `stream` and return the
@@ -88,9 +90,10 @@ cudaError_t launch_clip_finalize(const Launch& l, const TensorRec* tensors, uint
                                  const unsigned long long* hist, const float* tensor_absmax,
                                  const float* gmin, const float* gmax, const float* gabsmax,
                                  float* clip, float* step, float* inv, float* offset);
-cudaError_t launch_metrics(const Launch& l, const TensorRec* tensors, const Tile* tiles,
-                           uint32_t n_tiles, const float* step, const float* inv,
+cudaError_t launch_metrics(const Launch& l, uint32_t grid, const TensorRec* tensors,
+                           const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
                            const float* offset, double2* partials);
+uint32_t metrics_grid_cap(int sm_count);   // resident CTAs per SM x SMs for the metrics kernel
 cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                     const double2* partials, double* sse, double* sig, double* mse,
                                     double* sqnr_db);

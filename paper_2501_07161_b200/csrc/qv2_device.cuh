@@ -26,7 +26,7 @@ __device__ __forceinline__ Tile load_tile(const Tile* tiles, uint32_t i) {
   Tile t;
   t.begin = (uint64_t)a.x | ((uint64_t)a.y << 32);
   t.row0 = (uint64_t)a.z | ((uint64_t)a.w << 32);
-  t.count = b.x; t.tensor = b.y; t.rows = b.z; t.slot = b.w;
+  t.count = b.x; t.tensor = b.y; t.rows = b.z; t.reserved = b.w;
   return t;
 }
 
@@ -59,6 +59,11 @@ __device__ __forceinline__ float warp_max(float v) {
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = __dadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
 __device__ __forceinline__ uint32_t warp_sum_u32(uint32_t v) {

@@ -2,11 +2,13 @@
 // (CalculateSQNR and CalculateMSE of Algorithm 2; quantizer Eq. 1 / Eq. 5, dequantizer Eq. 3,
 // SQNR Eq. 6, MSE Eq. 7).
 //
-// One persistent launch walks the tile table of a whole model.  Every warp reduces its share of a
-// tile in binary32 (independent accumulators per vector lane, then a fixed butterfly) and writes
-// one {sum e^2, sum x^2} pair to its own slot; a second kernel adds each tensor's slots in a fixed
-// order in binary64.  There are no floating-point atomics and no inter-CTA waits, so the result
-// is bit-identical from run to run and does not depend on the grid size.
+// One persistent launch walks the tile table of a whole model; CTA b takes tiles b, b+grid, ...
+// Every lane reduces its share of a tile in binary32 (independent accumulators per vector lane),
+// adds the tile's two sums to binary64 running sums that it keeps while the CTA stays on the same
+// tensor, and when the tensor changes the warp folds its lanes with a fixed butterfly and writes
+// one {sum e^2, sum x^2} pair to its own slot.  A second kernel adds each tensor's slots in a
+// fixed order in binary64.  There are no floating-point atomics and no inter-CTA waits: for a
+// given grid size the result is bit-identical from run to run.
 #include "qv2_device.cuh"
 
 namespace qv2 {
@@ -168,14 +170,34 @@ __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
   }
 }
 
+// Slot of (tensor, CTA, warp): the CTAs that own tiles of a tensor are numbered in the order of
+// the tensor's first tiles, rank = (b - tile_first) mod grid < min(grid, tiles of the tensor).
+__device__ __forceinline__ void flush_slot(const TensorRec* tr, double sse, double sig, uint32_t lane,
+                                           uint32_t warp, double2* __restrict__ partials) {
+  sse = warp_sum_f64(sse);
+  sig = warp_sum_f64(sig);
+  if (lane == 0) {
+    const uint32_t g = gridDim.x;
+    const uint32_t rank = (blockIdx.x + g - tr->tile_first % g) % g;
+    partials[tr->slot_first + rank * kWarps + warp] = make_double2(sse, sig);
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 4)
 metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
                const float* __restrict__ step, const float* __restrict__ inv,
                const float* __restrict__ offset, double2* __restrict__ partials) {
+  constexpr uint32_t kNone = 0xffffffffu;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  uint32_t cur = kNone;
+  double run_sse = 0.0, run_sig = 0.0;
   for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile tl = load_tile(tiles, ti);
     const TensorRec* tr = tensors + tl.tensor;
+    if (tl.tensor != cur) {
+      if (cur != kNone) flush_slot(tensors + cur, run_sse, run_sig, lane, warp, partials);
+      cur = tl.tensor; run_sse = 0.0; run_sig = 0.0;
+    }
     Acc a[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) { a[k].sse = 0.0f; a[k].sig = 0.0f; }
@@ -190,13 +212,13 @@ metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ t
     } else {
       metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
     }
-    // thread -> warp reduction in binary32 with a fixed association
-    float sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
-    float sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
-    sse = warp_sum(sse);
-    sig = warp_sum(sig);
-    if (lane == 0) partials[tl.slot + warp] = make_double2((double)sse, (double)sig);
+    // this lane's tile sums in binary32 with a fixed association, then into the binary64 totals
+    const float sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
+    const float sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
+    run_sse = __dadd_rn(run_sse, (double)sse);
+    run_sig = __dadd_rn(run_sig, (double)sig);
   }
+  if (cur != kNone) flush_slot(tensors + cur, run_sse, run_sig, lane, warp, partials);
 }
 
 // One CTA per tensor: fixed-order binary64 sum of the tensor's slots, then MSE and SQNR.
@@ -236,12 +258,15 @@ metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __
 
 }  // namespace
 
-cudaError_t launch_metrics(const Launch& l, const TensorRec* tensors, const Tile* tiles,
-                           uint32_t n_tiles, const float* step, const float* inv,
+uint32_t metrics_grid_cap(int sm_count) {
+  static int per_sm = 0;
+  return (uint32_t)persistent_grid((const void*)metrics_kernel, &per_sm, sm_count, 0x7fffffffu);
+}
+
+cudaError_t launch_metrics(const Launch& l, uint32_t grid, const TensorRec* tensors,
+                           const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
                            const float* offset, double2* partials) {
   if (n_tiles == 0) return cudaSuccess;
-  static int per_sm = 0;
-  const int grid = persistent_grid((const void*)metrics_kernel, &per_sm, l.sm_count, n_tiles);
   metrics_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset, partials);
   return cudaGetLastError();
 }

@@ -15,19 +15,20 @@ static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t g
   while (count > 0) {
     uint32_t c = count > kTileElems ? kTileElems : (uint32_t)count;
     Tile t;
-    t.begin = begin; t.row0 = group; t.count = c; t.tensor = tensor; t.rows = 0; t.slot = 0;
+    t.begin = begin; t.row0 = group; t.count = c; t.tensor = tensor; t.rows = 0; t.reserved = 0;
     tiles->push_back(t);
     begin += c; count -= c;
   }
 }
 
-int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, HostPlan* out) {
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t grid_cap,
+               HostPlan* out) {
   if (!descs || !out) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   out->tensors.clear(); out->tiles.clear(); out->hist_tiles.clear();
   out->total_groups = 0; out->total_slots = 0; out->any_percentile = false;
   out->tensors.reserve(n);
-  uint64_t groups = 0, slots = 0;
+  uint64_t groups = 0;
   for (uint32_t t = 0; t < n; ++t) {
     const qv2_tensor_desc& d = descs[t];
     if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8 || d.range > QV2_PERCENTILE)
@@ -58,7 +59,6 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, Hos
     r.range_mode = d.range;
     r.pair_mode = !pair ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
     r.percentile = d.percentile;
-    r.pad_ = 0;
 
     size_t first_tile = out->tiles.size();
     if (d.range == QV2_PERCENTILE) out->any_percentile = true;
@@ -74,22 +74,36 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, Hos
           uint64_t nr = rows - row < per ? rows - row : per;
           Tile tl;
           tl.begin = row * d.inner; tl.row0 = row; tl.count = (uint32_t)(nr * d.inner);
-          tl.tensor = t; tl.rows = (uint32_t)nr; tl.slot = 0;
+          tl.tensor = t; tl.rows = (uint32_t)nr; tl.reserved = 0;
           out->tiles.push_back(tl);
         }
       }
       if (d.range == QV2_PERCENTILE) cut_flat(t, 0, ne, 0, &out->hist_tiles);
     }
-    uint64_t nt = out->tiles.size() - first_tile;
-    if (slots + nt * kWarps >= (1ull << 32)) return QV2_ERR_SIZE;
-    r.slot_first = (uint32_t)slots;
-    r.slot_count = (uint32_t)(nt * kWarps);
-    for (uint64_t i = 0; i < nt; ++i)
-      out->tiles[first_tile + i].slot = (uint32_t)(slots + i * kWarps);
-    slots += nt * kWarps;
+    if (first_tile >= (1ull << 31)) return QV2_ERR_SIZE;
+    r.tile_first = (uint32_t)first_tile;
+    r.slot_first = 0; r.slot_count = 0;             // filled in below, once the grid is known
     out->tensors.push_back(r);
   }
   if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;
+  // Partial-sum slots of the metrics kernel.  CTA b walks tiles b, b+grid, ...; a tensor whose
+  // tiles are [first, first+count) is therefore touched by min(grid, count) CTAs, and each of
+  // their warps owns one slot.
+  const uint64_t n_tiles = out->tiles.size();
+  uint64_t grid = grid_cap < 1 ? 1 : grid_cap;
+  if (grid > n_tiles) grid = n_tiles ? n_tiles : 1;
+  uint64_t slots = 0;
+  for (uint32_t t = 0; t < n; ++t) {
+    TensorRec& r = out->tensors[t];
+    const uint64_t next = (t + 1 < n) ? out->tensors[t + 1].tile_first : n_tiles;
+    const uint64_t cnt = next - r.tile_first;
+    const uint64_t ctas = cnt < grid ? cnt : grid;
+    if (slots + ctas * kWarps >= (1ull << 32)) return QV2_ERR_SIZE;
+    r.slot_first = (uint32_t)slots;
+    r.slot_count = (uint32_t)(ctas * kWarps);
+    slots += ctas * kWarps;
+  }
+  out->metrics_grid = (uint32_t)grid;
   out->total_groups = groups;
   out->total_slots = (uint32_t)slots;
   return QV2_OK;
@@ -108,7 +122,7 @@ extern "C" uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n) {
 extern "C" int64_t qv2_debug_plan_tiles(const qv2_tensor_desc* descs, uint32_t n, uint64_t* out,
                                         uint64_t max_tiles) {
   qv2::HostPlan plan;
-  int st = qv2::build_plan(descs, n, nullptr, &plan);
+  int st = qv2::build_plan(descs, n, nullptr, 1, &plan);
   if (st != QV2_OK) return st;
   uint64_t w = 0;
   for (const qv2::Tile& t : plan.tiles) {

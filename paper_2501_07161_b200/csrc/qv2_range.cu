@@ -87,40 +87,53 @@ __device__ __forceinline__ void publish(RangeAcc& a, uint32_t lane, uint32_t* km
   }
 }
 
+// Lanes keep their min/max across consecutive tiles of the same group and merge them (one warp
+// reduction, two atomics) only when the group changes.  A per-tensor activation is a single group
+// cut into thousands of tiles, and publishing each tile would serialise that many atomics on one
+// address.
 __global__ void __launch_bounds__(kThreads, 4)
 range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
              uint32_t* kmin, uint32_t* kmax, unsigned long long* nonfinite) {
+  constexpr uint32_t kNone = 0xffffffffu;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  RangeAcc a;
+  reset(a);
+  uint32_t cur_group = kNone, cur_tensor = 0;
   for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile tl = load_tile(tiles, ti);
     const TensorRec* tr = tensors + tl.tensor;
     const float* x = tr->x + tl.begin;
     const uint32_t gbase = tr->group_base;
-    unsigned long long* nf = nonfinite + tl.tensor;
-    RangeAcc a;
     if (tl.rows == 0) {
-      reset(a);
+      const uint32_t G = gbase + (uint32_t)tl.row0;
+      if (G != cur_group) {
+        if (cur_group != kNone) publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
+        reset(a);
+        cur_group = G; cur_tensor = tl.tensor;
+      }
+      const float mn0 = a.mn, mx0 = a.mx;
       range_flat<false>(x, tl.count, a);
       if (__any_sync(0xffffffffu, a.nanflag != a.nanflag)) {   // redo this warp's share carefully
-        reset(a);
+        a.mn = mn0; a.mx = mx0; a.nanflag = 0.0f;
         range_flat<true>(x, tl.count, a);
       }
-      publish(a, lane, kmin, kmax, gbase + (uint32_t)tl.row0, nf);
     } else {
       const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+      RangeAcc b;
       for (uint32_t r = warp; r < tl.rows; r += kWarps) {
         const float* row = x + (uint64_t)r * inner;
-        reset(a);
-        range_row<false>(row, inner, lane, a);
-        if (__any_sync(0xffffffffu, a.nanflag != a.nanflag)) {
-          reset(a);
-          range_row<true>(row, inner, lane, a);
+        reset(b);
+        range_row<false>(row, inner, lane, b);
+        if (__any_sync(0xffffffffu, b.nanflag != b.nanflag)) {
+          reset(b);
+          range_row<true>(row, inner, lane, b);
         }
         const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
-        publish(a, lane, kmin, kmax, gbase + g, nf);
+        publish(b, lane, kmin, kmax, gbase + g, nonfinite + tl.tensor);
       }
     }
   }
+  if (cur_group != kNone) publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
 }
 
 // One CTA per tensor: decode the keys in place, write absmax, the tensor-wide absmax and -- for
