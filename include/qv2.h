@@ -238,6 +238,44 @@ int qv2_sweep_model_host(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n_
 uint64_t qv2_staging_bytes(const qv2_tensor_desc* descs, uint32_t n_tensors, uint32_t n_layers);
 
 /*
+ * The fake-quantize + error reduction of qv2_quant_metrics for ONE tensor, for callers that must
+ * not allocate.  (The paper has no counterpart to this call; it exists for the library's users.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits -- inside a region whose
+ * memory footprint was fixed up front (a serving process that has handed all device memory to its
+ * own pool), in a latency-critical loop where an allocation would stall the device, or in a host
+ * callback.  The regular entry points keep tile tables and partial sums in context scratch that
+ * grows with cudaMalloc; this one takes no context and calls no allocator of any kind.  Instead
+ * its partial sums (one pair of doubles per warp and per 16384-element tile) live in a fixed
+ * 1 MiB array that is part of the library image: every GPU that loads the library holds that
+ * 1 MiB until the process ends, whether or not this call is ever used.
+ *
+ * desc: host, one descriptor (x and, for pair mode, y are device pointers; QV2_STORE_CODES is not
+ * accepted).  step, inv, offset: device, this tensor's per-group parameters (group 0 first), e.g.
+ * a slice of qv2_calibrate's output.  result4: device, 4 doubles {sse, sig, mse, sqnr_db}, defined
+ * as in qv2_quant_metrics.  stream: cudaStream_t or NULL.  The work is enqueued and the call
+ * returns; results are valid once the stream has been synchronised.
+ *
+ * Limit: outer*channels*inner <= QV2_NOALLOC_MAX_ELEMS, and no more than
+ * QV2_NOALLOC_MAX_ELEMS/16384 tiles (per-channel rows of 4096 elements or more are cut at row
+ * boundaries, so very ragged shapes reach the tile limit earlier).  Larger tensors are refused
+ * with QV2_ERR_SIZE before anything is launched; split them or use qv2_quant_metrics.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and the
+ * SM count; make that first call outside any stream capture.  All calls on a device share the one
+ * array, which still holds the previous call's partial sums: each call overwrites every slot it
+ * later reads, so nothing has to be cleared, but two calls that overlap on the GPU (different
+ * streams, or host threads racing) corrupt each other -- serialise them.  Sums are added in a
+ * different order than in qv2_quant_metrics, so the two agree to rounding (the same tolerances:
+ * 1e-5 relative on MSE, 1e-3 dB on SQNR), not bit for bit.
+ * Errors: QV2_ERR_NULL, _ARG, _ALIGN, _SIZE, _CUDA.
+ */
+#define QV2_NOALLOC_MAX_ELEMS (134217728ull) /* 2^27 elements = 8192 tiles -> 65536 slots = 1 MiB */
+int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_tensor_desc* desc,
+                              const float* step, const float* inv, const float* offset,
+                              double* result4);
+
+/*
  * Host-only view of the work decomposition, for tests: cuts the tensors into the tiles the
  * kernels walk (no GPU needed, tensor pointers are not dereferenced).  Each tile is reported as
  * 4 uint64: {tensor, first element, element count, kind (0 = one group per tile, 1 = whole rows)}.

@@ -24,7 +24,8 @@ OK = 0
 EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_error",
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
-           "qv2_debug_plan_tiles"]
+           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc"]
+NOALLOC_MAX_ELEMS = 1 << 27
 
 
 class TensorDesc(C.Structure):
@@ -83,6 +84,8 @@ def lib() -> C.CDLL:
     L.qv2_sweep_model_host.restype = i32
     L.qv2_staging_bytes.argtypes = [dp, u32, u32]; L.qv2_staging_bytes.restype = u64
     L.qv2_debug_plan_tiles.argtypes = [dp, u32, vp, u64]; L.qv2_debug_plan_tiles.restype = C.c_int64
+    L.qv2_quant_metrics_noalloc.argtypes = [i32, vp, dp, vp, vp, vp, vp]
+    L.qv2_quant_metrics_noalloc.restype = i32
     _lib = L
     return L
 
@@ -247,6 +250,18 @@ class Context:
         if st not in (OK, -5):
             raise Qv2Error(st, "qv2_sweep_model_host")
         return st
+
+
+def quant_metrics_noalloc(desc: TensorDesc, step: torch.Tensor, inv: torch.Tensor, offset: torch.Tensor,
+                          result4: torch.Tensor, device: int = 0,
+                          stream: Optional[torch.cuda.Stream] = None) -> int:
+    """qv2_quant_metrics_noalloc for one tensor: no context, no allocation inside the library.
+    `result4` is a caller-owned float64[4] device tensor that receives {sse, sig, mse, sqnr_db}.
+    Returns the status instead of raising so that callers can test the size limit."""
+    s = stream if stream is not None else torch.cuda.current_stream(device)
+    arr = (TensorDesc * 1)(desc)
+    return int(lib().qv2_quant_metrics_noalloc(device, C.c_void_p(s.cuda_stream), arr, _ptr(step),
+                                               _ptr(inv), _ptr(offset), _ptr(result4)))
 
 
 def staging_bytes(descs, n_layers: int) -> int:

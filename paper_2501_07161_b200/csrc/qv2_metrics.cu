@@ -279,3 +279,197 @@ cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, u
 }
 
 }  // namespace qv2
+
+// ================================================================================================
+// qv2_quant_metrics_noalloc: the fused fake-quantize + error reduction for ONE tensor with no
+// allocation of any kind.  Its partial sums live in a fixed array inside the loaded library image
+// instead of context scratch, and the tensor is described to the kernel by value instead of
+// through uploaded tables.  The per-element arithmetic is the code above, unchanged.
+// ================================================================================================
+namespace qv2 {
+namespace {
+
+// One {sum e^2, sum x^2} pair per warp and tile.  1 MiB per GPU that loads the library, held
+// until the process exits.  Every slot a call reads is written by that same call first, so the
+// array needs no clearing between calls; it does keep the previous call's contents.
+constexpr uint32_t kNoAllocMaxTiles = QV2_NOALLOC_MAX_ELEMS / kTileElems;
+static __device__ __align__(256) double2 g_noalloc_slots[kNoAllocMaxTiles * kWarps];
+
+struct NoAllocJob {
+  TensorRec tr;
+  uint64_t rows;            // outer * channels
+  uint32_t n_tiles;
+  uint32_t cut;             // 0: flat run, 1: long rows cut at row boundaries, 2: whole short rows
+  uint32_t tiles_per_row;   // cut 1
+  uint32_t rows_per_tile;   // cut 2
+};
+
+// The same decomposition as the host planner, evaluated on the fly for one tensor.
+__device__ __forceinline__ Tile noalloc_tile(const NoAllocJob& j, uint32_t ti) {
+  Tile t;
+  t.tensor = 0; t.reserved = 0;
+  if (j.cut == 0) {
+    t.begin = (uint64_t)ti * kTileElems;
+    const uint64_t left = j.tr.n_elems - t.begin;
+    t.count = left > kTileElems ? kTileElems : (uint32_t)left;
+    t.row0 = 0; t.rows = 0;
+  } else if (j.cut == 1) {
+    const uint64_t row = ti / j.tiles_per_row;
+    const uint64_t piece = ti % j.tiles_per_row;
+    t.begin = row * j.tr.inner + piece * kTileElems;
+    const uint64_t left = j.tr.inner - piece * kTileElems;
+    t.count = left > kTileElems ? kTileElems : (uint32_t)left;
+    t.row0 = row % j.tr.channels; t.rows = 0;
+  } else {
+    const uint64_t row = (uint64_t)ti * j.rows_per_tile;
+    const uint64_t left = j.rows - row;
+    t.rows = left > j.rows_per_tile ? j.rows_per_tile : (uint32_t)left;
+    t.begin = row * j.tr.inner; t.row0 = row;
+    t.count = (uint32_t)(t.rows * j.tr.inner);
+  }
+  return t;
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+metrics_noalloc_kernel(const __grid_constant__ NoAllocJob job, const float* __restrict__ step,
+                       const float* __restrict__ inv, const float* __restrict__ offset,
+                       double2* __restrict__ slots) {
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const TensorRec* tr = &job.tr;
+  for (uint32_t ti = blockIdx.x; ti < job.n_tiles; ti += gridDim.x) {
+    const Tile tl = noalloc_tile(job, ti);
+    Acc a[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { a[k].sse = 0.0f; a[k].sig = 0.0f; }
+    if (tr->pair_mode == kSelf) metric_tile<kSelf, false>(tl, tr, step, inv, offset, a);
+    else if (tr->pair_mode == kRequant) metric_tile<kRequant, false>(tl, tr, step, inv, offset, a);
+    else metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
+    float sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
+    float sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
+    sse = warp_sum(sse);
+    sig = warp_sum(sig);
+    if (lane == 0) slots[(size_t)ti * kWarps + warp] = make_double2((double)sse, (double)sig);
+  }
+}
+
+// One CTA: fixed-order binary64 sum of the n_tiles * kWarps slots, then MSE and SQNR.
+__global__ void __launch_bounds__(1024)
+metrics_noalloc_finalize_kernel(uint32_t n_slots, uint64_t n_elems, const double2* __restrict__ slots,
+                                double* out4) {
+  __shared__ double sh_e[1024], sh_s[1024];
+  double e = 0.0, s = 0.0;
+  for (uint32_t k = threadIdx.x; k < n_slots; k += 1024) {
+    const double2 p = slots[k];
+    e = __dadd_rn(e, p.x);
+    s = __dadd_rn(s, p.y);
+  }
+  sh_e[threadIdx.x] = e; sh_s[threadIdx.x] = s;
+  __syncthreads();
+  for (uint32_t o = 512; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      sh_e[threadIdx.x] = __dadd_rn(sh_e[threadIdx.x], sh_e[threadIdx.x + o]);
+      sh_s[threadIdx.x] = __dadd_rn(sh_s[threadIdx.x], sh_s[threadIdx.x + o]);
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const double sse = sh_e[0], sig = sh_s[0];
+    const double inf = __longlong_as_double(0x7ff0000000000000ll);
+    out4[0] = sse;
+    out4[1] = sig;
+    out4[2] = n_elems ? __ddiv_rn(sse, (double)n_elems) : 0.0;
+    out4[3] = sse == 0.0 ? inf : (sig == 0.0 ? -inf : __dmul_rn(10.0, log10(__ddiv_rn(sig, sse))));
+  }
+}
+
+// Per-device set-up state.  The array's name is only a handle on the host; its device address
+// has to be asked for, once per device, with that device current.
+constexpr int kMaxDevices = 64;
+struct NoAllocDevice {
+  bool ready = false;
+  double2* slots = nullptr;
+  int grid_cap = 1;
+};
+NoAllocDevice g_noalloc_dev[kMaxDevices];
+
+}  // namespace
+}  // namespace qv2
+
+extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_tensor_desc* desc,
+                                         const float* step, const float* inv, const float* offset,
+                                         double* result4) {
+  using namespace qv2;
+  if (!desc || !step || !inv || !offset || !result4) return QV2_ERR_NULL;
+  if (device < 0 || device >= kMaxDevices) return QV2_ERR_ARG;
+  const qv2_tensor_desc& d = *desc;
+  if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8 || d.range > QV2_PERCENTILE)
+    return QV2_ERR_ARG;
+  if (d.flags & ~(uint32_t)QV2_PAIR_RAW) return QV2_ERR_ARG;          // no code output here
+  if ((d.flags & QV2_PAIR_RAW) && !d.y) return QV2_ERR_ARG;
+  if (d.channels >= (1ull << 32)) return QV2_ERR_SIZE;
+  // sizes: reject anything whose partial sums would not fit the fixed array
+  if (d.outer && d.channels > QV2_NOALLOC_MAX_ELEMS / d.outer) return QV2_ERR_SIZE;
+  const uint64_t rows = d.outer * d.channels;
+  if (rows && d.inner > QV2_NOALLOC_MAX_ELEMS / rows) return QV2_ERR_SIZE;
+  const uint64_t ne = rows * d.inner;
+  if (ne > 0 && !d.x) return QV2_ERR_NULL;
+  if (((uintptr_t)d.x & 3u) || ((uintptr_t)d.y & 3u)) return QV2_ERR_ALIGN;
+
+  NoAllocJob job;
+  job.tr.x = d.x; job.tr.y = d.y; job.tr.codes = nullptr;
+  job.tr.n_elems = ne; job.tr.inner = d.inner; job.tr.channels = (uint32_t)d.channels;
+  job.tr.group_base = 0;
+  job.tr.per_channel = d.granularity == QV2_PER_CHANNEL;
+  job.tr.n_groups = job.tr.per_channel ? (uint32_t)d.channels : 1u;
+  job.tr.asym = d.scheme == QV2_ASYM_U8;
+  job.tr.range_mode = d.range;
+  job.tr.pair_mode = !d.y ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
+  job.tr.slot_first = 0; job.tr.slot_count = 0; job.tr.tile_first = 0;
+  job.tr.percentile = d.percentile;
+  job.rows = rows; job.tiles_per_row = 1; job.rows_per_tile = 1;
+  uint64_t n_tiles;
+  if (!job.tr.per_channel || ne == 0) {
+    job.cut = 0;
+    n_tiles = (ne + kTileElems - 1) / kTileElems;
+  } else if (d.inner >= kRowTileMin) {
+    job.cut = 1;
+    job.tiles_per_row = (uint32_t)((d.inner + kTileElems - 1) / kTileElems);
+    n_tiles = rows * job.tiles_per_row;
+  } else {
+    job.cut = 2;
+    job.rows_per_tile = (uint32_t)(kTileElems / d.inner);
+    n_tiles = (rows + job.rows_per_tile - 1) / job.rows_per_tile;
+  }
+  if (n_tiles > kNoAllocMaxTiles) return QV2_ERR_SIZE;     // ragged rows can need more tiles than N/16384
+  job.n_tiles = (uint32_t)n_tiles;
+
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return QV2_ERR_CUDA;
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) return QV2_ERR_CUDA;
+  int status = QV2_OK;
+  NoAllocDevice& nd = g_noalloc_dev[device];
+  if (!nd.ready) {                        // first call on this device: resolve the array's address
+    double2* p = nullptr;
+    int sms = 0, per_sm = 0;
+    if (cudaGetSymbolAddress((void**)&p, g_noalloc_slots) != cudaSuccess || !p ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+      status = QV2_ERR_CUDA;
+    } else {
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)metrics_noalloc_kernel,
+                                                        kThreads, 0) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+      nd.slots = p; nd.grid_cap = per_sm * (sms > 0 ? sms : 1); nd.ready = true;
+    }
+  }
+  if (status == QV2_OK) {
+    cudaStream_t s = (cudaStream_t)stream;
+    if (job.n_tiles) {
+      const uint32_t grid = job.n_tiles < (uint32_t)nd.grid_cap ? job.n_tiles : (uint32_t)nd.grid_cap;
+      metrics_noalloc_kernel<<<grid, kThreads, 0, s>>>(job, step, inv, offset, nd.slots);
+    }
+    metrics_noalloc_finalize_kernel<<<1, 1024, 0, s>>>(job.n_tiles * kWarps, ne, nd.slots, result4);
+    if (cudaGetLastError() != cudaSuccess) status = QV2_ERR_CUDA;
+  }
+  if (prev != device) cudaSetDevice(prev);
+  return status;
+}
