@@ -208,18 +208,24 @@ def measured_peak():
 
 
 def recorded_traffic():
-    """DRAM bytes per launch of the dominant kernel from the committed ncu capture, valid only
-    while the kernel source is unchanged since the capture."""
+    """DRAM bytes per algorithmic byte of the dominant kernel from the committed ncu capture
+    (profiles/metrics_kernel_traffic.txt), valid only while the kernel sources are unchanged
+    since the capture."""
     try:
-        with open(os.path.join(ROOT, "profiles", "metrics_kernel_traffic.json")) as f:
-            rec = json.load(f)
+        rec = {}
+        with open(os.path.join(ROOT, "profiles", "metrics_kernel_traffic.txt")) as f:
+            for ln in f:
+                if ln.startswith("#") or ":" not in ln:
+                    continue
+                k, v = ln.split(":", 1)
+                rec[k.strip()] = v.strip()
         h = hashlib.sha256()
-        for rel in rec["sources"]:
+        for rel in rec["sources"].split():
             with open(os.path.join(ROOT, rel), "rb") as s:
                 h.update(s.read())
         if h.hexdigest() != rec["sha256"]:
             return None
-        return rec
+        return float(rec["dram_bytes_per_algorithmic_byte"])
     except Exception:
         return None
 
@@ -353,10 +359,8 @@ def ours_main(args):
     if rank == 0:
         peak, peak_src = measured_peak()
         achieved = metrics_bytes / (met_ms * 1e-3) / 1e9
-        rec = recorded_traffic()
-        traffic = None
-        if rec is not None:
-            traffic = rec["dram_bytes_per_algorithmic_byte"] * metrics_bytes
+        ratio = recorded_traffic()
+        traffic = None if ratio is None else ratio * metrics_bytes
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
