@@ -13,6 +13,7 @@ struct qv2_ctx {
   cudaStream_t stream = nullptr;
   int sm_count = 1;
   uint32_t metrics_cap = 1;   // largest useful grid of the metrics kernel on this device
+  uint32_t range_cap = 1;     // the same for the range kernel
   int last_cuda = 0;
   uint64_t launches = 0;
 
@@ -26,6 +27,7 @@ struct qv2_ctx {
   Tile* d_tiles = nullptr;        size_t cap_tiles = 0;
   Tile* d_hist_tiles = nullptr;   size_t cap_hist_tiles = 0;
   double2* d_partials = nullptr;  size_t cap_slots = 0;
+  uint2* d_rslots = nullptr;      size_t cap_rslots = 0;
   float* d_tensor_absmax = nullptr; size_t cap_absmax = 0;
   unsigned long long* d_hist = nullptr; size_t cap_hist = 0;   // used when the caller passes no hist
   double* d_rank = nullptr;                                    // 2 * kMaxRankLayers doubles
@@ -87,7 +89,7 @@ int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* cons
   if (c->plan_valid && key == c->plan_key) return QV2_OK;
 
   HostPlan plan;
-  int st = build_plan(descs, n, codes, c->metrics_cap, &plan);
+  int st = build_plan(descs, n, codes, c->metrics_cap, c->range_cap, &plan);
   if (st != QV2_OK) return st;
   // The previous upload may still be reading the pinned buffer, and buffers may be reallocated.
   QV2_CUDA(c, cudaStreamSynchronize(c->stream));
@@ -97,6 +99,7 @@ int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* cons
   if ((st = grow(c, &c->d_tiles, &c->cap_tiles, ntl ? ntl : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_hist_tiles, &c->cap_hist_tiles, nh ? nh : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_partials, &c->cap_slots, plan.total_slots ? plan.total_slots : 1)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_rslots, &c->cap_rslots, plan.total_rslots ? plan.total_rslots : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_tensor_absmax, &c->cap_absmax, nt)) != QV2_OK) return st;
   const size_t b0 = nt * sizeof(TensorRec), b1 = ntl * sizeof(Tile), b2 = nh * sizeof(Tile);
   if ((st = grow_pinned(c, b0 + b1 + b2)) != QV2_OK) return st;
@@ -150,6 +153,7 @@ extern "C" int qv2_create(qv2_ctx** out, int device, void* stream) {
   if (e != cudaSuccess) { delete c; return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA; }
   c->sm_count = sms > 0 ? sms : 1;
   c->metrics_cap = metrics_grid_cap(c->sm_count);
+  c->range_cap = range_grid_cap(c->sm_count);
   *out = c;
   return QV2_OK;
 }
@@ -158,7 +162,7 @@ extern "C" int qv2_destroy(qv2_ctx* c) {
   if (!c) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
-  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials);
+  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials); cudaFree(c->d_rslots);
   cudaFree(c->d_tensor_absmax); cudaFree(c->d_hist); cudaFree(c->d_rank);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
   delete c;
@@ -191,12 +195,12 @@ extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t 
   QV2_CUDA(c, cudaMemsetAsync(nonfinite, 0, (size_t)n * sizeof(uint64_t), c->stream));
   if (h) QV2_CUDA(c, cudaMemsetAsync(h, 0, (size_t)n * kBins * sizeof(uint64_t), c->stream));
   if (!p.tiles.empty()) {
-    QV2_CUDA(c, launch_range(l, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),
+    QV2_CUDA(c, launch_range(l, p.range_grid, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),
                              reinterpret_cast<uint32_t*>(gmin), reinterpret_cast<uint32_t*>(gmax),
-                             reinterpret_cast<unsigned long long*>(nonfinite)));
+                             c->d_rslots, reinterpret_cast<unsigned long long*>(nonfinite)));
     ++c->launches;
   }
-  QV2_CUDA(c, launch_range_finalize(l, c->d_tensors, n, gmin, gmax, gabsmax, step, inv, offset,
+  QV2_CUDA(c, launch_range_finalize(l, c->d_tensors, n, c->d_rslots, gmin, gmax, gabsmax, step, inv, offset,
                                     c->d_tensor_absmax));
   ++c->launches;
   if (!p.hist_tiles.empty()) {

@@ -37,6 +37,8 @@ struct TensorRec {
   uint32_t slot_first;       // first partial-sum slot of this tensor
   uint32_t slot_count;       // kWarps slots for every CTA of the metrics grid that owns a tile of it
   uint32_t tile_first;       // index of this tensor's first tile in the tile table
+  uint32_t rslot_first;      // per-tensor tensors: first {min,max} key slot written by the range kernel,
+  uint32_t rslot_count;      //   one per CTA of the range grid that owns a tile of the tensor
   double percentile;
 };
 
@@ -61,13 +63,16 @@ struct HostPlan {
   uint64_t total_groups = 0;
   uint32_t total_slots = 0;
   uint32_t metrics_grid = 1;      // CTAs of the metrics launch; the slot layout depends on it
+  uint32_t total_rslots = 0;
+  uint32_t range_grid = 1;        // CTAs of the range launch; the range-slot layout depends on it
   bool any_percentile = false;
 };
 
-// Validates the descriptors and cuts them into tiles.  `codes` may be NULL.  `grid_cap` is the
-// largest useful grid of the metrics kernel (resident CTAs per SM x SMs).  Returns a QV2 status.
-int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t grid_cap,
-               HostPlan* out);
+// Validates the descriptors and cuts them into tiles.  `codes` may be NULL.  `metrics_cap` and
+// `range_cap` are the largest useful grids of those kernels (resident CTAs per SM x SMs).
+// Returns a QV2 status.
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
+               uint32_t range_cap, HostPlan* out);
 
 // ------------------------------------------------------------------------------------------------
 // Launch wrappers (defined next to their kernels).  All enqueue on `stream` and return the
@@ -77,12 +82,13 @@ struct Launch {
   int sm_count;
 };
 
-cudaError_t launch_range(const Launch& l, const TensorRec* tensors, const Tile* tiles,
-                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax,
+cudaError_t launch_range(const Launch& l, uint32_t grid, const TensorRec* tensors, const Tile* tiles,
+                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax, uint2* rslots,
                          unsigned long long* nonfinite);
+uint32_t range_grid_cap(int sm_count);     // resident CTAs per SM x SMs for the range kernel
 cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                  float* gmin, float* gmax, float* gabsmax, float* step, float* inv,
-                                  float* offset, float* tensor_absmax);
+                                  const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
+                                  float* step, float* inv, float* offset, float* tensor_absmax);
 cudaError_t launch_hist(const Launch& l, const TensorRec* tensors, const Tile* tiles,
                         uint32_t n_tiles, const float* tensor_absmax,
                         const unsigned long long* nonfinite, unsigned long long* hist);

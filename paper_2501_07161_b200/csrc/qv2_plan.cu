@@ -21,8 +21,8 @@ static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t g
   }
 }
 
-int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t grid_cap,
-               HostPlan* out) {
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
+               uint32_t range_cap, HostPlan* out) {
   if (!descs || !out) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   out->tensors.clear(); out->tiles.clear(); out->hist_tiles.clear();
@@ -82,28 +82,41 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     }
     if (first_tile >= (1ull << 31)) return QV2_ERR_SIZE;
     r.tile_first = (uint32_t)first_tile;
-    r.slot_first = 0; r.slot_count = 0;             // filled in below, once the grid is known
+    r.slot_first = 0; r.slot_count = 0;             // filled in below, once the grids are known
+    r.rslot_first = 0; r.rslot_count = 0;
     out->tensors.push_back(r);
   }
   if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;
-  // Partial-sum slots of the metrics kernel.  CTA b walks tiles b, b+grid, ...; a tensor whose
-  // tiles are [first, first+count) is therefore touched by min(grid, count) CTAs, and each of
-  // their warps owns one slot.
+  // Slots written with plain stores instead of atomics.  In both persistent kernels CTA b walks
+  // tiles b, b+grid, ...; a tensor whose tiles are [first, first+count) is therefore touched by
+  // min(grid, count) CTAs.  The metrics kernel gives each warp of those CTAs one partial-sum slot;
+  // the range kernel gives each of those CTAs one {min,max} slot for per-tensor tensors (a single
+  // group shared by thousands of tiles; per-channel groups are merged with atomics).
   const uint64_t n_tiles = out->tiles.size();
-  uint64_t grid = grid_cap < 1 ? 1 : grid_cap;
-  if (grid > n_tiles) grid = n_tiles ? n_tiles : 1;
-  uint64_t slots = 0;
+  uint64_t mgrid = metrics_cap < 1 ? 1 : metrics_cap, rgrid = range_cap < 1 ? 1 : range_cap;
+  if (mgrid > n_tiles) mgrid = n_tiles ? n_tiles : 1;
+  if (rgrid > n_tiles) rgrid = n_tiles ? n_tiles : 1;
+  uint64_t slots = 0, rslots = 0;
   for (uint32_t t = 0; t < n; ++t) {
     TensorRec& r = out->tensors[t];
     const uint64_t next = (t + 1 < n) ? out->tensors[t + 1].tile_first : n_tiles;
     const uint64_t cnt = next - r.tile_first;
-    const uint64_t ctas = cnt < grid ? cnt : grid;
+    const uint64_t ctas = cnt < mgrid ? cnt : mgrid;
     if (slots + ctas * kWarps >= (1ull << 32)) return QV2_ERR_SIZE;
     r.slot_first = (uint32_t)slots;
     r.slot_count = (uint32_t)(ctas * kWarps);
     slots += ctas * kWarps;
+    if (!r.per_channel) {
+      const uint64_t rc = cnt < rgrid ? cnt : rgrid;
+      if (rslots + rc >= (1ull << 32)) return QV2_ERR_SIZE;
+      r.rslot_first = (uint32_t)rslots;
+      r.rslot_count = (uint32_t)rc;
+      rslots += rc;
+    }
   }
-  out->metrics_grid = (uint32_t)grid;
+  out->metrics_grid = (uint32_t)mgrid;
+  out->range_grid = (uint32_t)rgrid;
+  out->total_rslots = (uint32_t)rslots;
   out->total_groups = groups;
   out->total_slots = (uint32_t)slots;
   return QV2_OK;
@@ -122,7 +135,7 @@ extern "C" uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n) {
 extern "C" int64_t qv2_debug_plan_tiles(const qv2_tensor_desc* descs, uint32_t n, uint64_t* out,
                                         uint64_t max_tiles) {
   qv2::HostPlan plan;
-  int st = qv2::build_plan(descs, n, nullptr, 1, &plan);
+  int st = qv2::build_plan(descs, n, nullptr, 1, 1, &plan);
   if (st != QV2_OK) return st;
   uint64_t w = 0;
   for (const qv2::Tile& t : plan.tiles) {

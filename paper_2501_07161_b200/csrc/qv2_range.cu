@@ -87,18 +87,42 @@ __device__ __forceinline__ void publish(RangeAcc& a, uint32_t lane, uint32_t* km
   }
 }
 
-// Lanes keep their min/max across consecutive tiles of the same group and merge them (one warp
-// reduction, two atomics) only when the group changes.  A per-tensor activation is a single group
-// cut into thousands of tiles, and publishing each tile would serialise that many atomics on one
-// address.
+// Lanes keep their min/max across consecutive tiles of the same group and merge them only when
+// the group changes.  A per-tensor tensor is ONE group cut into thousands of tiles: its CTAs
+// combine their warps through shared memory and store one {min,max} key pair into the CTA's own
+// slot (atomics from every warp of every CTA on that single address would serialise).  Per-channel
+// groups are touched by one or two CTAs each and are merged with atomics.
+__device__ __forceinline__ void publish_slot(RangeAcc& a, uint32_t lane, uint32_t warp, const TensorRec* tr,
+                                             uint2* rslots, unsigned long long* nonfinite_t, float* sh) {
+  const float mn = warp_min(a.mn), mx = warp_max(a.mx);
+  const uint32_t bad = warp_sum_u32(a.bad);
+  if (lane == 0) {
+    sh[warp] = mn; sh[kWarps + warp] = mx;
+    if (bad) atomicAdd(nonfinite_t, (unsigned long long)bad);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m0 = sh[0], m1 = sh[kWarps];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) { m0 = fminf(m0, sh[w]); m1 = fmaxf(m1, sh[kWarps + w]); }
+    const uint32_t g = gridDim.x;
+    const uint32_t rank = (blockIdx.x + g - tr->tile_first % g) % g;
+    // 0 = "no finite element seen" (m0 > m1 only in that case)
+    rslots[tr->rslot_first + rank] = (m0 <= m1) ? make_uint2(~f2key(m0), f2key(m1)) : make_uint2(0u, 0u);
+  }
+  __syncthreads();
+}
+
 __global__ void __launch_bounds__(kThreads, 4)
 range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
-             uint32_t* kmin, uint32_t* kmax, unsigned long long* nonfinite) {
+             uint32_t* kmin, uint32_t* kmax, uint2* rslots, unsigned long long* nonfinite) {
   constexpr uint32_t kNone = 0xffffffffu;
+  __shared__ float sh[2 * kWarps];
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   RangeAcc a;
   reset(a);
   uint32_t cur_group = kNone, cur_tensor = 0;
+  bool cur_slot = false;           // the pending group belongs to a per-tensor tensor
   for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile tl = load_tile(tiles, ti);
     const TensorRec* tr = tensors + tl.tensor;
@@ -106,10 +130,13 @@ range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ til
     const uint32_t gbase = tr->group_base;
     if (tl.rows == 0) {
       const uint32_t G = gbase + (uint32_t)tl.row0;
-      if (G != cur_group) {
-        if (cur_group != kNone) publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
+      if (G != cur_group) {        // block-uniform: every warp of the CTA takes this branch together
+        if (cur_group != kNone) {
+          if (cur_slot) publish_slot(a, lane, warp, tensors + cur_tensor, rslots, nonfinite + cur_tensor, sh);
+          else publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
+        }
         reset(a);
-        cur_group = G; cur_tensor = tl.tensor;
+        cur_group = G; cur_tensor = tl.tensor; cur_slot = tr->per_channel == 0;
       }
       const float mn0 = a.mn, mx0 = a.mx;
       range_flat<false>(x, tl.count, a);
@@ -133,16 +160,43 @@ range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ til
       }
     }
   }
-  if (cur_group != kNone) publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
+  if (cur_group != kNone) {
+    if (cur_slot) publish_slot(a, lane, warp, tensors + cur_tensor, rslots, nonfinite + cur_tensor, sh);
+    else publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
+  }
 }
 
-// One CTA per tensor: decode the keys in place, write absmax, the tensor-wide absmax and -- for
-// tensors without percentile clipping -- the quantization parameters.
+// One CTA per tensor: fold the CTA slots of a per-tensor tensor, decode the keys in place, write
+// absmax, the tensor-wide absmax and -- for tensors without percentile clipping -- the
+// quantization parameters.
 __global__ void __launch_bounds__(256)
-range_finalize_kernel(const TensorRec* __restrict__ tensors, float* gmin, float* gmax, float* gabsmax,
-                      float* step, float* inv, float* offset, float* tensor_absmax) {
+range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __restrict__ rslots,
+                      float* gmin, float* gmax, float* gabsmax, float* step, float* inv, float* offset,
+                      float* tensor_absmax) {
   __shared__ float red[256];
+  __shared__ uint32_t kred[2][256];
   const TensorRec tr = tensors[blockIdx.x];
+  if (!tr.per_channel) {                 // keys of the single group come from the slots
+    uint32_t kn = 0, kx = 0;             // both arrays hold "larger is better" keys, 0 = empty
+    for (uint32_t k = threadIdx.x; k < tr.rslot_count; k += blockDim.x) {
+      const uint2 v = rslots[tr.rslot_first + k];
+      kn = max(kn, v.x); kx = max(kx, v.y);
+    }
+    kred[0][threadIdx.x] = kn; kred[1][threadIdx.x] = kx;
+    __syncthreads();
+    for (uint32_t o = 128; o > 0; o >>= 1) {
+      if (threadIdx.x < o) {
+        kred[0][threadIdx.x] = max(kred[0][threadIdx.x], kred[0][threadIdx.x + o]);
+        kred[1][threadIdx.x] = max(kred[1][threadIdx.x], kred[1][threadIdx.x + o]);
+      }
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      reinterpret_cast<uint32_t*>(gmin)[tr.group_base] = kred[0][0];
+      reinterpret_cast<uint32_t*>(gmax)[tr.group_base] = kred[1][0];
+    }
+    __syncthreads();
+  }
   float amax = 0.0f;
   for (uint32_t g = threadIdx.x; g < tr.n_groups; g += blockDim.x) {
     const uint32_t G = tr.group_base + g;
@@ -169,21 +223,24 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, float* gmin, float*
 
 }  // namespace
 
-cudaError_t launch_range(const Launch& l, const TensorRec* tensors, const Tile* tiles,
-                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax,
+uint32_t range_grid_cap(int sm_count) {
+  static int per_sm = 0;
+  return (uint32_t)persistent_grid((const void*)range_kernel, &per_sm, sm_count, 0x7fffffffu);
+}
+
+cudaError_t launch_range(const Launch& l, uint32_t grid, const TensorRec* tensors, const Tile* tiles,
+                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax, uint2* rslots,
                          unsigned long long* nonfinite) {
   if (n_tiles == 0) return cudaSuccess;
-  static int per_sm = 0;   // resident CTAs per SM, queried once
-  const int grid = persistent_grid((const void*)range_kernel, &per_sm, l.sm_count, n_tiles);
-  range_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, nonfinite);
+  range_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, rslots, nonfinite);
   return cudaGetLastError();
 }
 
 cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                  float* gmin, float* gmax, float* gabsmax, float* step, float* inv,
-                                  float* offset, float* tensor_absmax) {
-  range_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, gmin, gmax, gabsmax, step, inv,
-                                                         offset, tensor_absmax);
+                                  const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
+                                  float* step, float* inv, float* offset, float* tensor_absmax) {
+  range_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, rslots, gmin, gmax, gabsmax, step,
+                                                         inv, offset, tensor_absmax);
   return cudaGetLastError();
 }
 

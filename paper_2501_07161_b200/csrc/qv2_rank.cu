@@ -21,12 +21,29 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
             const double* __restrict__ sqnr_a, const double* __restrict__ mse_a,
             const uint64_t* __restrict__ macs, const double* __restrict__ pos, qv2_rank_cfg cfg,
             double* score, double* severity, uint32_t* order, uint8_t* keep, uint32_t* n_keep) {
+  // Models have tens of layers: up to kStage layers the serial parts below run out of shared
+  // memory instead of paying a global-memory latency per step.
+  constexpr uint32_t kStage = 1024;
   __shared__ double mean_s[2];
+  __shared__ double st_a[kStage], st_b[kStage];
+  __shared__ unsigned long long st_macs[kStage];
+  __shared__ uint32_t st_order[kStage];
   const uint32_t tid = threadIdx.x;
+  const bool staged = n <= kStage;
   const double inf = __longlong_as_double(0x7ff0000000000000ll);
+  if (staged) {
+    for (uint32_t i = tid; i < n; i += blockDim.x) {
+      st_a[i] = mse_w[i]; st_b[i] = mse_a[i];
+      st_macs[i] = macs ? macs[i] : 1ull;
+    }
+    __syncthreads();
+  }
   if (tid == 0) {                      // means: sums in layer order, as the definition states
     double sw = 0.0, sa = 0.0;
-    for (uint32_t i = 0; i < n; ++i) { sw = __dadd_rn(sw, mse_w[i]); sa = __dadd_rn(sa, mse_a[i]); }
+    for (uint32_t i = 0; i < n; ++i) {
+      sw = __dadd_rn(sw, staged ? st_a[i] : mse_w[i]);
+      sa = __dadd_rn(sa, staged ? st_b[i] : mse_a[i]);
+    }
     mean_s[0] = __ddiv_rn(sw, (double)n);
     mean_s[1] = __ddiv_rn(sa, (double)n);
   }
@@ -71,21 +88,26 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
     order[rank] = i;
   }
   __syncthreads();
+  if (staged) {
+    for (uint32_t i = tid; i < n; i += blockDim.x) st_order[i] = order[i];
+    __syncthreads();
+  }
   if (tid == 0) {
     uint32_t nk = 0;
     if (cfg.select_mode == QV2_BY_COUNT) {
       nk = cfg.keep_count < n ? cfg.keep_count : n;
     } else {
       unsigned __int128 total = 0, kept = 0;
-      for (uint32_t i = 0; i < n; ++i) total += macs ? macs[i] : 1ull;
+      for (uint32_t i = 0; i < n; ++i) total += staged ? st_macs[i] : (macs ? macs[i] : 1ull);
       for (uint32_t j = 0; j < n; ++j) {       // grow the FP32 prefix while the rate still holds
-        const unsigned __int128 m = macs ? macs[order[j]] : 1ull;
+        const uint32_t l = staged ? st_order[j] : order[j];
+        const unsigned __int128 m = staged ? st_macs[l] : (macs ? macs[l] : 1ull);
         const unsigned __int128 quantized = total - (kept + m);
         if (quantized * 10000u >= (unsigned __int128)cfg.rate_permyriad * total) { kept += m; nk = j + 1; }
         else break;
       }
     }
-    for (uint32_t j = 0; j < nk; ++j) keep[order[j]] = 1;
+    for (uint32_t j = 0; j < nk; ++j) keep[staged ? st_order[j] : order[j]] = 1;
     *n_keep = nk;
   }
 }
