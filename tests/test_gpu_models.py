@@ -185,3 +185,42 @@ def test_full_size_benchmark_workload_sampled_against_oracle(ctx):
     md2, t2 = run_sweep(ctx, model)
     for k in ("sse", "sig", "mse", "sqnr_db"):
         assert torch.equal(t[k].view(torch.int64), t2[k].view(torch.int64))
+
+
+def test_sweep_can_be_captured_in_a_cuda_graph_and_replayed():
+    """Once the tile table of a descriptor set is resident, a pass enqueues only kernels and
+    memsets on the context's stream: it can be captured once and replayed (one launch per pass,
+    which matters for small models whose pass is launch-bound)."""
+    s = torch.cuda.Stream()
+    gctx = q.Context(0, stream=s)
+    try:
+        model = gen.make_model("squeezenet", seed=5, device="cuda", batch=1)
+        md = q.model_descs(model)
+        cfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
+        sb, t = gctx.alloc_sweep_buffers(md.descs, md.n_layers)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s):
+            gctx.sweep_model(md.descs, md.n_layers, md.macs, None, cfg, sb)     # warm-up: builds the plan
+        s.synchronize()
+        ref = {k: t[k].clone() for k in ("mse", "sqnr_db", "order", "keep_fp32", "n_keep", "step", "hist")}
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            gctx.sweep_model(md.descs, md.n_layers, md.macs, None, cfg, sb)
+        for k in ("mse", "sqnr_db", "order", "step", "hist"):
+            t[k].zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for k, v in ref.items():
+            assert torch.equal(t[k].view(torch.uint8), v.view(torch.uint8)), k
+        # new inputs, same buffers: the replay recomputes everything
+        model.layers[3].x.mul_(1.5)
+        g.replay()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s):
+            sb2, t2 = gctx.alloc_sweep_buffers(md.descs, md.n_layers)
+            gctx.sweep_model(md.descs, md.n_layers, md.macs, None, cfg, sb2)
+        torch.cuda.synchronize()
+        assert torch.equal(t["mse"].view(torch.int64), t2["mse"].view(torch.int64))
+        assert not torch.equal(t["mse"].view(torch.int64), ref["mse"].view(torch.int64))
+    finally:
+        gctx.close()
