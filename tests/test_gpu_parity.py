@@ -218,3 +218,58 @@ def test_argument_errors_are_reported_before_launch(ctx):
     assert e.value.status == -4
     # the context is still usable afterwards
     check_specs(ctx, [Spec(randn(500, 3), 1, 1, 500)])
+
+
+def test_rank_at_the_maximum_layer_count(ctx):
+    rng = np.random.default_rng(11)
+    n = 8192
+    sw = rng.uniform(10, 60, n).round(2); sa = rng.uniform(10, 60, n).round(2)
+    mw = rng.uniform(1e-6, 1e-4, n); ma = rng.uniform(1e-4, 1e-2, n)
+    ma[[5, 4000, 8191]] = [3.0, 5.0, 4.0]                       # three MSE outliers
+    macs = rng.integers(1, 2 ** 40, n).astype(np.uint64)
+    ro, rk, rn = oracle.rank_layers(sw, mw, sa, ma, macs=macs, select_mode=1, rate_permyriad=7000)
+    dv = lambda a: torch.from_numpy(np.asarray(a)).cuda()
+    cfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=7000)
+    o, k, nk = ctx.rank_layers(dv(sw), dv(mw), dv(sa), dv(ma), dv(macs.view(np.int64)), None, cfg)
+    torch.cuda.synchronize()
+    assert o.cpu().numpy().view(np.uint32).tolist() == ro.tolist()
+    assert ro.tolist()[:3] == [4000, 8191, 5]
+    assert k.cpu().numpy().tolist() == rk.tolist() and int(nk) == rn
+
+
+def test_tensor_with_more_than_2_to_32_elements(ctx):
+    """64-bit element indexing: a 17 GB tensor whose extremes sit beyond element 2^32, checked by
+    invariants (the oracle would need minutes): planted min/max, histogram total, and the sum of
+    squared errors of the whole against those of its two halves under the same parameters."""
+    n = (1 << 32) + 3 * TILE + 5
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2 ** 30:
+        pytest.skip("needs about 40 GiB of free device memory")
+    g = torch.Generator(device="cuda"); g.manual_seed(17)
+    x = torch.empty(n, dtype=torch.float32, device="cuda")
+    step_n = 1 << 28
+    for s in range(0, n, step_n):
+        e = min(n, s + step_n)
+        x[s:e].normal_(generator=g)
+    x[(1 << 32) + 7] = -9.5
+    x[n - 1] = 11.25
+    d_whole = q.make_desc(x, None, 1, 1, n, q.PER_TENSOR, q.ASYM_U8, q.PERCENTILE, 0.9999)
+    cal = ctx.calibrate(q.desc_array([d_whole]))
+    torch.cuda.synchronize()
+    assert float(cal.gmin[0]) == -9.5 and float(cal.gmax[0]) == 11.25 and int(cal.nonfinite[0]) == 0
+    hist = cal.hist.cpu().numpy().view(np.uint64)[:2048]
+    assert int(hist.sum()) == n and hist[2047] >= 1
+    h1 = 1 << 31
+    halves = [q.make_desc(x, None, 1, 1, n, q.PER_TENSOR, q.ASYM_U8, q.MINMAX),
+              q.make_desc(x[:h1], None, 1, 1, h1, q.PER_TENSOR, q.ASYM_U8, q.MINMAX),
+              q.make_desc(x[h1:], None, 1, 1, n - h1, q.PER_TENSOR, q.ASYM_U8, q.MINMAX)]
+    rep = lambda t: t[:1].repeat(3)
+    met = ctx.quant_metrics(q.desc_array(halves), rep(cal.step), rep(cal.inv), rep(cal.offset))
+    torch.cuda.synchronize()
+    sse, sig = met.sse.tolist(), met.sig.tolist()
+    assert abs(sse[0] - (sse[1] + sse[2])) <= 1e-7 * sse[0]
+    assert abs(sig[0] - (sig[1] + sig[2])) <= 1e-7 * sig[0]
+    assert abs(sig[0] / n - 1.0) < 1e-3                         # unit-variance data
+    assert abs(float(met.mse[0]) - sse[0] / n) <= 1e-15 * sse[0]
+    del x
+    torch.cuda.empty_cache()
