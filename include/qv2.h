@@ -167,6 +167,22 @@ int qv2_quant_metrics(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
                       double* sse, double* sig, double* mse, double* sqnr_db);
 
 /*
+ * qv2_quant_metrics with one more local metric: the cosine similarity of Eq. 8, one of the
+ * metrics the paper evaluates beside SQNR and MSE (and then sets aside).  cosine[t] =
+ * A.B / (|A| |B|) with A the reference tensor x and B the tensor it is compared with: the
+ * dequantized copy of x (self mode), the dequantized re-quantization of y (QV2_PAIR_REQUANT) or y
+ * itself (QV2_PAIR_RAW).  It costs one more fused multiply-add per element: with e = A - B,
+ * A.B = sig - sum(x e) and |B|^2 = sig - 2 sum(x e) + sse.  A zero vector gives 0.  Accuracy:
+ * 1e-7 absolute in general; when B is a quantized copy of A (cos within 1e-2 of 1) the distance
+ * 1 - cos is good to 1e-4 relative.
+ * cosine: device, n doubles, or NULL (then this is exactly qv2_quant_metrics).
+ */
+int qv2_quant_metrics_ex(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
+                         const float* step, const float* inv, const float* offset,
+                         void* const* codes,
+                         double* sse, double* sig, double* mse, double* sqnr_db, double* cosine);
+
+/*
  * Sensitivity list and mixed-precision layer set: step 4 of the overview, "CalculateSQNRdeltas",
  * "CalculateAverage" and "RankLayersBySensitivity" of Algorithm 2, the SQNR delta of Eq. 16 and
  * the BOPs-reduction rate of Eq. 17 (normalised so that a fully quantized model is 100 %).

@@ -24,7 +24,7 @@ OK = 0
 EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_error",
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
-           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc"]
+           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex"]
 NOALLOC_MAX_ELEMS = 1 << 27
 
 
@@ -74,6 +74,8 @@ def lib() -> C.CDLL:
     L.qv2_calibrate.argtypes = [vp, dp, u32] + [vp] * 9; L.qv2_calibrate.restype = i32
     L.qv2_quant_metrics.argtypes = [vp, dp, u32, vp, vp, vp, C.POINTER(vp), vp, vp, vp, vp]
     L.qv2_quant_metrics.restype = i32
+    L.qv2_quant_metrics_ex.argtypes = [vp, dp, u32, vp, vp, vp, C.POINTER(vp), vp, vp, vp, vp, vp]
+    L.qv2_quant_metrics_ex.restype = i32
     L.qv2_rank_layers.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, C.POINTER(RankCfg), vp, vp, vp]
     L.qv2_rank_layers.restype = i32
     L.qv2_sweep_model.argtypes = [vp, dp, u32, u32, vp, vp, C.POINTER(RankCfg),
@@ -151,6 +153,7 @@ class MetricsOut:
     mse: torch.Tensor
     sqnr_db: torch.Tensor
     codes: Optional[List[Optional[torch.Tensor]]] = None
+    cosine: Optional[torch.Tensor] = None
 
 
 class Context:
@@ -212,14 +215,20 @@ class Context:
                                    _ptr(out.offset), _ptr(out.nonfinite)), "qv2_calibrate")
         return out
 
-    def quant_metrics(self, descs, step, inv, offset, codes: Optional[Sequence[Optional[torch.Tensor]]] = None
-                      ) -> MetricsOut:
+    def quant_metrics(self, descs, step, inv, offset, codes: Optional[Sequence[Optional[torch.Tensor]]] = None,
+                      want_cosine: bool = False) -> MetricsOut:
         n = len(descs)
         d = lambda: self._empty(n, torch.float64)
         out = MetricsOut(d(), d(), d(), d(), list(codes) if codes is not None else None)
         cp = None
         if codes is not None:
             cp = (C.c_void_p * n)(*[_ptr(c) for c in codes])
+        if want_cosine:
+            out.cosine = d()
+            _check(lib().qv2_quant_metrics_ex(self._h, descs, n, _ptr(step), _ptr(inv), _ptr(offset), cp,
+                                              _ptr(out.sse), _ptr(out.sig), _ptr(out.mse), _ptr(out.sqnr_db),
+                                              _ptr(out.cosine)), "qv2_quant_metrics_ex")
+            return out
         _check(lib().qv2_quant_metrics(self._h, descs, n, _ptr(step), _ptr(inv), _ptr(offset), cp,
                                        _ptr(out.sse), _ptr(out.sig), _ptr(out.mse), _ptr(out.sqnr_db)),
                "qv2_quant_metrics")

@@ -28,6 +28,7 @@ struct qv2_ctx {
   Tile* d_hist_tiles = nullptr;   size_t cap_hist_tiles = 0;
   double2* d_partials = nullptr;  size_t cap_slots = 0;
   uint2* d_rslots = nullptr;      size_t cap_rslots = 0;
+  double* d_partials_xe = nullptr; size_t cap_slots_xe = 0;   // sum x*e slots, cosine only
   float* d_tensor_absmax = nullptr; size_t cap_absmax = 0;
   unsigned long long* d_hist = nullptr; size_t cap_hist = 0;   // used when the caller passes no hist
   double* d_rank = nullptr;                                    // 2 * kMaxRankLayers doubles
@@ -162,7 +163,7 @@ extern "C" int qv2_destroy(qv2_ctx* c) {
   if (!c) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
-  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials); cudaFree(c->d_rslots);
+  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials); cudaFree(c->d_rslots); cudaFree(c->d_partials_xe);
   cudaFree(c->d_tensor_absmax); cudaFree(c->d_hist); cudaFree(c->d_rank);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
   delete c;
@@ -214,10 +215,10 @@ extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t 
   return QV2_OK;
 }
 
-extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n,
-                                 const float* step, const float* inv, const float* offset,
-                                 void* const* codes, double* sse, double* sig, double* mse,
-                                 double* sqnr_db) {
+extern "C" int qv2_quant_metrics_ex(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n,
+                                    const float* step, const float* inv, const float* offset,
+                                    void* const* codes, double* sse, double* sig, double* mse,
+                                    double* sqnr_db, double* cosine) {
   if (!c || !descs || !step || !inv || !offset || !sse || !sig || !mse || !sqnr_db) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
   bool any_codes = false;
@@ -227,15 +228,28 @@ extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint3
   int st = ensure_plan(c, descs, n, any_codes ? codes : nullptr);
   if (st != QV2_OK) return st;
   const HostPlan& p = c->plan;
+  double* xe = nullptr;
+  if (cosine) {                        // third slot array, only when the cosine is wanted
+    if ((st = grow(c, &c->d_partials_xe, &c->cap_slots_xe, p.total_slots ? p.total_slots : 1)) != QV2_OK)
+      return st;
+    xe = c->d_partials_xe;
+  }
   const Launch l = launch_of(c);
   if (!p.tiles.empty()) {
     QV2_CUDA(c, launch_metrics(l, p.metrics_grid, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
-                               offset, c->d_partials));
+                               offset, c->d_partials, xe));
     ++c->launches;
   }
-  QV2_CUDA(c, launch_metrics_finalize(l, c->d_tensors, n, c->d_partials, sse, sig, mse, sqnr_db));
+  QV2_CUDA(c, launch_metrics_finalize(l, c->d_tensors, n, c->d_partials, xe, sse, sig, mse, sqnr_db, cosine));
   ++c->launches;
   return QV2_OK;
+}
+
+extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n,
+                                 const float* step, const float* inv, const float* offset,
+                                 void* const* codes, double* sse, double* sig, double* mse,
+                                 double* sqnr_db) {
+  return qv2_quant_metrics_ex(c, descs, n, step, inv, offset, codes, sse, sig, mse, sqnr_db, nullptr);
 }
 
 extern "C" int qv2_rank_layers(qv2_ctx* c, uint32_t n_layers, const double* sqnr_w,

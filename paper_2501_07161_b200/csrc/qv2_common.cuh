@@ -98,11 +98,11 @@ cudaError_t launch_clip_finalize(const Launch& l, const TensorRec* tensors, uint
                                  float* clip, float* step, float* inv, float* offset);
 cudaError_t launch_metrics(const Launch& l, uint32_t grid, const TensorRec* tensors,
                            const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
-                           const float* offset, double2* partials);
+                           const float* offset, double2* partials, double* partials_xe);
 uint32_t metrics_grid_cap(int sm_count);   // resident CTAs per SM x SMs for the metrics kernel
 cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                    const double2* partials, double* sse, double* sig, double* mse,
-                                    double* sqnr_db);
+                                    const double2* partials, const double* partials_xe, double* sse,
+                                    double* sig, double* mse, double* sqnr_db, double* cosine);
 cudaError_t launch_rank(const Launch& l, uint32_t n, const double* sqnr_w, const double* mse_w,
                         const double* sqnr_a, const double* mse_a, const uint64_t* macs,
                         const double* pos, qv2_rank_cfg cfg, double* score, double* severity,

@@ -9,6 +9,8 @@
 // one {sum e^2, sum x^2} pair to its own slot.  A second kernel adds each tensor's slots in a
 // fixed order in binary64.  There are no floating-point atomics and no inter-CTA waits: for a
 // given grid size the result is bit-identical from run to run.
+#include <type_traits>
+
 #include "qv2_device.cuh"
 
 namespace qv2 {
@@ -19,8 +21,24 @@ struct QP {
   float step, inv, off, qmin, qmax;
 };
 
+// Per-lane accumulators of one tile.  AccCos also carries sum x*e, from which the cosine
+// similarity of Eq. 8 follows without a second pass: A.B = sig - xe, |B|^2 = sig - 2 xe + sse.
 struct Acc {
   float sse, sig;
+  __device__ __forceinline__ void clear() { sse = 0.0f; sig = 0.0f; }
+  __device__ __forceinline__ void add(float x, float e) {
+    sse = __fmaf_rn(e, e, sse);
+    sig = __fmaf_rn(x, x, sig);
+  }
+};
+struct AccCos {
+  float sse, sig, xe;
+  __device__ __forceinline__ void clear() { sse = 0.0f; sig = 0.0f; xe = 0.0f; }
+  __device__ __forceinline__ void add(float x, float e) {
+    sse = __fmaf_rn(e, e, sse);
+    sig = __fmaf_rn(x, x, sig);
+    xe = __fmaf_rn(x, e, xe);
+  }
 };
 
 // One element.  MODE: kSelf quantizes x, kRequant quantizes y on x's grid, kRaw compares x and y.
@@ -29,8 +47,8 @@ struct Acc {
 //       1.5*2^23 rounds to nearest-even for |t| <= 2^22
 //  e  = (x - off) - q*step, with x - off split exactly into (s, err) by TwoSum when off != 0 and
 //       the product folded into one fused multiply-add, so e carries a single rounding error.
-template <uint32_t MODE, bool OFF, bool CODES>
-__device__ __forceinline__ void metric_elem(float x, float y, const QP& p, Acc& a, uint8_t* code) {
+template <uint32_t MODE, bool OFF, bool CODES, class ACC>
+__device__ __forceinline__ void metric_elem(float x, float y, const QP& p, ACC& a, uint8_t* code) {
   float e;
   if (MODE == kRaw) {
     e = __fsub_rn(x, y);
@@ -51,12 +69,11 @@ __device__ __forceinline__ void metric_elem(float x, float y, const QP& p, Acc& 
     }
     if (CODES) *code = (uint8_t)(int)q;
   }
-  a.sse = __fmaf_rn(e, e, a.sse);
-  a.sig = __fmaf_rn(x, x, a.sig);
+  a.add(x, e);
 }
 
-template <uint32_t MODE, bool OFF, bool CODES>
-__device__ __forceinline__ void metric_vec(const float4& x, const float4& y, const QP& p, Acc* a,
+template <uint32_t MODE, bool OFF, bool CODES, class ACC>
+__device__ __forceinline__ void metric_vec(const float4& x, const float4& y, const QP& p, ACC* a,
                                            uint8_t* code) {
   metric_elem<MODE, OFF, CODES>(x.x, y.x, p, a[0], code);
   metric_elem<MODE, OFF, CODES>(x.y, y.y, p, a[1], code + 1);
@@ -65,9 +82,9 @@ __device__ __forceinline__ void metric_vec(const float4& x, const float4& y, con
 }
 
 // This thread's share of a flat one-group run.  `vec_y` says y has the same 16-byte phase as x.
-template <uint32_t MODE, bool OFF, bool CODES>
+template <uint32_t MODE, bool OFF, bool CODES, class ACC>
 __device__ __forceinline__ void metric_flat(const float* __restrict__ x, const float* __restrict__ y,
-                                            uint8_t* codes, uint32_t count, const QP& p, Acc* a) {
+                                            uint8_t* codes, uint32_t count, const QP& p, ACC* a) {
   constexpr bool PAIR = MODE != kSelf;
   const FlatSplit s = split_flat(x, count);
   const float* xb = x + s.head;
@@ -118,10 +135,10 @@ __device__ __forceinline__ void metric_flat(const float* __restrict__ x, const f
 }
 
 // One row handled by one warp.
-template <uint32_t MODE, bool OFF, bool CODES>
+template <uint32_t MODE, bool OFF, bool CODES, class ACC>
 __device__ __forceinline__ void metric_row(const float* __restrict__ x, const float* __restrict__ y,
                                            uint8_t* codes, uint32_t inner, uint32_t lane, const QP& p,
-                                           Acc* a) {
+                                           ACC* a) {
   constexpr bool PAIR = MODE != kSelf;
   uint32_t i = lane;
   for (; i + 96 < inner; i += 128) {
@@ -140,10 +157,10 @@ __device__ __forceinline__ void metric_row(const float* __restrict__ x, const fl
                                   CODES ? codes + i : nullptr);
 }
 
-template <uint32_t MODE, bool CODES>
+template <uint32_t MODE, bool CODES, class ACC>
 __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
                                             const float* __restrict__ step, const float* __restrict__ inv,
-                                            const float* __restrict__ offset, Acc* a) {
+                                            const float* __restrict__ offset, ACC* a) {
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const float* x = tr->x + tl.begin;
   const float* y = (MODE != kSelf) ? tr->y + tl.begin : nullptr;
@@ -172,35 +189,44 @@ __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
 
 // Slot of (tensor, CTA, warp): the CTAs that own tiles of a tensor are numbered in the order of
 // the tensor's first tiles, rank = (b - tile_first) mod grid < min(grid, tiles of the tensor).
-__device__ __forceinline__ void flush_slot(const TensorRec* tr, double sse, double sig, uint32_t lane,
-                                           uint32_t warp, double2* __restrict__ partials) {
-  sse = warp_sum_f64(sse);
-  sig = warp_sum_f64(sig);
-  if (lane == 0) {
-    const uint32_t g = gridDim.x;
-    const uint32_t rank = (blockIdx.x + g - tr->tile_first % g) % g;
-    partials[tr->slot_first + rank * kWarps + warp] = make_double2(sse, sig);
-  }
+__device__ __forceinline__ uint32_t slot_of(const TensorRec* tr, uint32_t warp) {
+  const uint32_t g = gridDim.x;
+  const uint32_t rank = (blockIdx.x + g - tr->tile_first % g) % g;
+  return tr->slot_first + rank * kWarps + warp;
 }
 
+// COS adds the sum x*e (third slot array) needed for the cosine similarity.
+template <bool COS>
 __global__ void __launch_bounds__(kThreads, 4)
 metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
                const float* __restrict__ step, const float* __restrict__ inv,
-               const float* __restrict__ offset, double2* __restrict__ partials) {
+               const float* __restrict__ offset, double2* __restrict__ partials,
+               double* __restrict__ partials_xe) {
+  using ACC = typename std::conditional<COS, AccCos, Acc>::type;
   constexpr uint32_t kNone = 0xffffffffu;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   uint32_t cur = kNone;
-  double run_sse = 0.0, run_sig = 0.0;
+  double run_sse = 0.0, run_sig = 0.0, run_xe = 0.0;
+  auto flush = [&](const TensorRec* tr) {
+    const double sse = warp_sum_f64(run_sse), sig = warp_sum_f64(run_sig);
+    double xe = 0.0;
+    if (COS) xe = warp_sum_f64(run_xe);
+    if (lane == 0) {
+      const uint32_t slot = slot_of(tr, warp);
+      partials[slot] = make_double2(sse, sig);
+      if (COS) partials_xe[slot] = xe;
+    }
+  };
   for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile tl = load_tile(tiles, ti);
     const TensorRec* tr = tensors + tl.tensor;
     if (tl.tensor != cur) {
-      if (cur != kNone) flush_slot(tensors + cur, run_sse, run_sig, lane, warp, partials);
-      cur = tl.tensor; run_sse = 0.0; run_sig = 0.0;
+      if (cur != kNone) flush(tensors + cur);
+      cur = tl.tensor; run_sse = 0.0; run_sig = 0.0; run_xe = 0.0;
     }
-    Acc a[4];
+    ACC a[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) { a[k].sse = 0.0f; a[k].sig = 0.0f; }
+    for (int k = 0; k < 4; ++k) a[k].clear();
     const uint32_t mode = tr->pair_mode;
     const bool codes = tr->codes != nullptr && mode != kRaw;
     if (mode == kSelf) {
@@ -217,28 +243,37 @@ metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ t
     const float sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
     run_sse = __dadd_rn(run_sse, (double)sse);
     run_sig = __dadd_rn(run_sig, (double)sig);
+    if constexpr (COS) {
+      const float xe = __fadd_rn(__fadd_rn(a[0].xe, a[1].xe), __fadd_rn(a[2].xe, a[3].xe));
+      run_xe = __dadd_rn(run_xe, (double)xe);
+    }
   }
-  if (cur != kNone) flush_slot(tensors + cur, run_sse, run_sig, lane, warp, partials);
+  if (cur != kNone) flush(tensors + cur);
 }
 
-// One CTA per tensor: fixed-order binary64 sum of the tensor's slots, then MSE and SQNR.
+// One CTA per tensor: fixed-order binary64 sum of the tensor's slots, then MSE (Eq. 7), SQNR
+// (Eq. 6) and, when asked for, the cosine similarity (Eq. 8) between the reference tensor A = x
+// and the compared tensor B = x - e:  A.B = sig - xe,  |B|^2 = sig - 2 xe + sse.
 __global__ void __launch_bounds__(256)
 metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __restrict__ partials,
-                        double* sse_out, double* sig_out, double* mse_out, double* sqnr_out) {
-  __shared__ double sh_e[256], sh_s[256];
+                        const double* __restrict__ partials_xe, double* sse_out, double* sig_out,
+                        double* mse_out, double* sqnr_out, double* cos_out) {
+  __shared__ double sh_e[256], sh_s[256], sh_x[256];
   const TensorRec tr = tensors[blockIdx.x];
-  double e = 0.0, s = 0.0;
+  double e = 0.0, s = 0.0, xe = 0.0;
   for (uint32_t k = threadIdx.x; k < tr.slot_count; k += 256) {
     const double2 p = partials[tr.slot_first + k];
     e = __dadd_rn(e, p.x);
     s = __dadd_rn(s, p.y);
+    if (cos_out) xe = __dadd_rn(xe, partials_xe[tr.slot_first + k]);
   }
-  sh_e[threadIdx.x] = e; sh_s[threadIdx.x] = s;
+  sh_e[threadIdx.x] = e; sh_s[threadIdx.x] = s; sh_x[threadIdx.x] = xe;
   __syncthreads();
   for (uint32_t o = 128; o > 0; o >>= 1) {
     if (threadIdx.x < o) {
       sh_e[threadIdx.x] = __dadd_rn(sh_e[threadIdx.x], sh_e[threadIdx.x + o]);
       sh_s[threadIdx.x] = __dadd_rn(sh_s[threadIdx.x], sh_s[threadIdx.x + o]);
+      sh_x[threadIdx.x] = __dadd_rn(sh_x[threadIdx.x], sh_x[threadIdx.x + o]);
     }
     __syncthreads();
   }
@@ -253,6 +288,12 @@ metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __
     else if (sig == 0.0) q = -inf;
     else q = __dmul_rn(10.0, log10(__ddiv_rn(sig, sse)));
     sqnr_out[blockIdx.x] = q;
+    if (cos_out) {
+      const double ab = sig - sh_x[0];
+      const double bb = sig - 2.0 * sh_x[0] + sse;
+      const double den = sqrt(sig) * sqrt(bb > 0.0 ? bb : 0.0);
+      cos_out[blockIdx.x] = den > 0.0 ? ab / den : 0.0;       // a zero vector has no direction
+    }
   }
 }
 
@@ -260,21 +301,27 @@ metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __
 
 uint32_t metrics_grid_cap(int sm_count) {
   static int per_sm = 0;
-  return (uint32_t)persistent_grid((const void*)metrics_kernel, &per_sm, sm_count, 0x7fffffffu);
+  return (uint32_t)persistent_grid((const void*)metrics_kernel<false>, &per_sm, sm_count, 0x7fffffffu);
 }
 
 cudaError_t launch_metrics(const Launch& l, uint32_t grid, const TensorRec* tensors,
                            const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
-                           const float* offset, double2* partials) {
+                           const float* offset, double2* partials, double* partials_xe) {
   if (n_tiles == 0) return cudaSuccess;
-  metrics_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset, partials);
+  if (partials_xe)
+    metrics_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset,
+                                                          partials, partials_xe);
+  else
+    metrics_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset,
+                                                           partials, nullptr);
   return cudaGetLastError();
 }
 
 cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                    const double2* partials, double* sse, double* sig, double* mse,
-                                    double* sqnr_db) {
-  metrics_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, partials, sse, sig, mse, sqnr_db);
+                                    const double2* partials, const double* partials_xe, double* sse,
+                                    double* sig, double* mse, double* sqnr_db, double* cosine) {
+  metrics_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, partials, partials_xe, sse, sig,
+                                                           mse, sqnr_db, cosine);
   return cudaGetLastError();
 }
 
@@ -340,7 +387,7 @@ metrics_noalloc_kernel(const __grid_constant__ NoAllocJob job, const float* __re
     const Tile tl = noalloc_tile(job, ti);
     Acc a[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) { a[k].sse = 0.0f; a[k].sig = 0.0f; }
+    for (int k = 0; k < 4; ++k) a[k].clear();
     if (tr->pair_mode == kSelf) metric_tile<kSelf, false>(tl, tr, step, inv, offset, a);
     else if (tr->pair_mode == kRequant) metric_tile<kRequant, false>(tl, tr, step, inv, offset, a);
     else metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
