@@ -57,6 +57,9 @@ def _load():
                                        C.c_int, C.c_int, f32p, f32p, f32p, u8p,
                                        f64p, f64p, f64p, f64p]
     lib.qv2o_quant_metrics.restype = None
+    lib.qv2o_cosine.argtypes = [f32p, f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_int, C.c_int,
+                                C.c_int, f32p, f32p, f32p]
+    lib.qv2o_cosine.restype = C.c_double
     lib.qv2o_rank.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p,
                               C.c_double, C.c_double, C.c_double, C.c_double,
                               C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
@@ -135,6 +138,18 @@ def quant_metrics(x, y, outer: int, channels: int, inner: int, per_channel: bool
     if want_codes:
         res["codes"] = codes if asym_u8 else codes.view(np.int8)
     return res
+
+
+def cosine(x, y, outer: int, channels: int, inner: int, per_channel: bool, asym_u8: bool,
+           pair_mode: int, step, inv, offset) -> float:
+    """Cosine similarity between x and the tensor it is compared with (see quant_metrics)."""
+    lib = _load()
+    x = _f32(x).reshape(-1)
+    yy = None if y is None else _f32(y).reshape(-1)
+    step, inv, offset = _f32(step), _f32(inv), _f32(offset)
+    return float(lib.qv2o_cosine(_p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
+                                 int(per_channel), int(asym_u8), int(pair_mode), _p(step, C.c_float),
+                                 _p(inv, C.c_float), _p(offset, C.c_float)))
 
 
 def rank_layers(sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, w_gain=2.0, a_gain=1.0,

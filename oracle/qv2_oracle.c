@@ -213,6 +213,38 @@ void qv2o_quant_metrics(const float *x, const float *y,
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * Cosine similarity (Eq. 8): A.B / (|A| |B|) with A the reference tensor x and B the tensor it is
+ * compared with -- the dequantized copy of x (pair_mode 0), the dequantized re-quantization of y
+ * (pair_mode 1) or y itself (pair_mode 2).  Written straight from the definition, three sums in
+ * long double.  A zero vector has no direction: the result is then 0.
+ * ------------------------------------------------------------------------------------------- */
+double qv2o_cosine(const float *x, const float *y,
+                   uint64_t outer, uint64_t channels, uint64_t inner, int per_channel,
+                   int asym_u8, int pair_mode,
+                   const float *step, const float *inv, const float *offset)
+{
+    int32_t qmin = asym_u8 ? 0 : -127, qmax = asym_u8 ? 255 : 127;
+    long double ab = 0.0L, aa = 0.0L, bb = 0.0L;
+    for (uint64_t o = 0; o < outer; ++o)
+        for (uint64_t c = 0; c < channels; ++c)
+            for (uint64_t i = 0; i < inner; ++i) {
+                uint64_t k = (o * channels + c) * inner + i;
+                uint64_t g = per_channel ? c : 0;
+                long double a = (long double)x[k], b;
+                if (pair_mode == 2) {
+                    b = (long double)y[k];
+                } else {
+                    float v = (pair_mode == 1) ? y[k] : x[k];
+                    int32_t q = quant_code(v, inv[g], offset[g], qmin, qmax);
+                    b = (long double)q * (long double)step[g] + (long double)offset[g];
+                }
+                ab += a * b; aa += a * a; bb += b * b;
+            }
+    long double den = sqrtl(aa) * sqrtl(bb);
+    return den > 0.0L ? (double)(ab / den) : 0.0;
+}
+
+/* ---------------------------------------------------------------------------------------------
  * Sensitivity list (Algorithm 2 with RankLayersBySensitivity, Eq. 16 for the SQNR delta) and
  * the FP32-kept set for a requested quantization level (Eq. 17, normalised).
  *  1. every SQNR is clamped to [-cap, cap].

@@ -273,3 +273,42 @@ def test_tensor_with_more_than_2_to_32_elements(ctx):
     assert abs(float(met.mse[0]) - sse[0] / n) <= 1e-15 * sse[0]
     del x
     torch.cuda.empty_cache()
+
+
+# --------------------------------------------------------------------------------------- cosine
+def test_cosine_similarity_matches_oracle(ctx):
+    """Eq. 8 through qv2_quant_metrics_ex.  The three sums behind it (sig, sse, sum x*e) each carry
+    the relative error of a 16-term binary32 chain (~1e-7 at worst), so cos agrees to 1e-7
+    absolute whatever the operands; for quantization error proper cos sits within ~1e-5 of 1 and
+    the sums that matter are tiny against sig, so 1 - cos is compared too, to 1e-4 relative."""
+    from parity import make_descs, to_dev
+    n = 6 * TILE + 77
+    x = randn(n, 61); y = x + 0.05 * randn(n, 62)
+    xr = x.clamp_min(0)
+    w = randn(70 * 1153, 63) * torch.exp(randn(70, 64)).repeat_interleave(1153)
+    specs = [Spec(x, 1, 1, n), Spec(x, 1, 1, n, asym=True), Spec(xr, 1, 1, n, asym=True, percentile=0.999),
+             Spec(x, 1, 1, n, asym=True, y=y), Spec(x, 1, 1, n, asym=True, y=y, raw=True),
+             Spec(x, 1, 1, n, asym=True, y=-y, raw=True),
+             Spec(w, 1, 70, 1153, per_channel=True), Spec(torch.zeros(100), 1, 1, 100)]
+    dx = [to_dev(s.x) for s in specs]; dy = [to_dev(s.y) for s in specs]
+    descs = make_descs(specs, dx, dy, store_codes=False)
+    cal = ctx.calibrate(descs)
+    plain = ctx.quant_metrics(descs, cal.step, cal.inv, cal.offset)
+    met = ctx.quant_metrics(descs, cal.step, cal.inv, cal.offset, want_cosine=True)
+    torch.cuda.synchronize()
+    for k in ("sse", "sig", "mse", "sqnr_db"):        # the extra accumulator changes nothing else
+        assert torch.equal(getattr(plain, k).view(torch.int64), getattr(met, k).view(torch.int64)), k
+    g = 0
+    for t, s in enumerate(specs):
+        ng = s.channels if s.per_channel else 1
+        sl = slice(g, g + ng); g += ng
+        mode = oracle.PAIR_SELF if s.y is None else (oracle.PAIR_RAW if s.raw else oracle.PAIR_REQUANT)
+        ref = oracle.cosine(s.x.numpy(), None if s.y is None else s.y.numpy(), s.outer, s.channels, s.inner,
+                            s.per_channel, s.asym, mode, cal.step[sl].cpu().numpy(), cal.inv[sl].cpu().numpy(),
+                            cal.offset[sl].cpu().numpy())
+        got = float(met.cosine[t])
+        assert abs(got - ref) <= 1e-7, (t, got, ref)
+        if 1e-9 < abs(1 - ref) < 1e-2:
+            assert abs((1 - got) - (1 - ref)) <= 1e-4 * abs(1 - ref), (t, 1 - got, 1 - ref)
+    assert float(met.cosine[5]) < -0.99 and float(met.cosine[7]) == 0.0
+    assert 0.9999 < float(met.cosine[0]) < 1.0

@@ -423,3 +423,35 @@ def test_rank_with_undefined_metrics_is_still_a_permutation():
     order, _, _ = oracle.rank_layers(sw, [1, 1, 1, 1], sa, [1, math.nan, 1, 1])
     # layers 1 and 2 have NaN deltas -> +inf score -> last, in layer order; a NaN MSE is no outlier
     assert order.tolist() == [0, 3, 1, 2]
+
+
+# ---------------------------------------------------------------------------------- cosine
+def test_cosine_closed_forms_and_library_dot_product():
+    one = np.ones(1, np.float32); zero = np.zeros(1, np.float32)
+    raw = lambda a, b: oracle.cosine(np.float32(a), np.float32(b), 1, 1, len(a), False, True,
+                                     oracle.PAIR_RAW, one, one, zero)
+    assert raw([1, 0], [0, 1]) == 0.0                       # orthogonal
+    assert raw([1, 2, 3], [2, 4, 6]) == pytest.approx(1.0, abs=1e-15)    # parallel, any length
+    assert raw([1, 2, 3], [-1, -2, -3]) == pytest.approx(-1.0, abs=1e-15)
+    assert raw([1, 1], [1, 0]) == pytest.approx(1 / math.sqrt(2), abs=1e-15)
+    assert raw([0, 0], [1, 2]) == 0.0 and raw([1, 2], [0, 0]) == 0.0     # a zero vector
+    x = RNG.standard_normal(10_000).astype(np.float32)
+    y = (x + 0.1 * RNG.standard_normal(10_000)).astype(np.float32)
+    xd, yd = x.astype(np.float64), y.astype(np.float64)
+    assert raw(x, y) == pytest.approx(xd @ yd / (np.linalg.norm(xd) * np.linalg.norm(yd)), abs=1e-14)
+    assert raw(x, y) == pytest.approx(raw(y, x), abs=1e-15)              # symmetric
+    # self mode: B is the dequantized tensor; on-grid data reproduces itself exactly
+    d = 2.0 ** -7
+    g = (np.arange(-127, 128) * d).astype(np.float32)
+    r = _self(g)
+    c1 = oracle.cosine(g, None, 1, 1, g.size, False, False, oracle.PAIR_SELF, r.step, r.inv, r.offset)
+    assert c1 == pytest.approx(1.0, abs=1e-15)
+    # and in general equals the dot-product form built from the codes
+    r = _self(x)
+    xh = r.codes.astype(np.float64) * float(r.step[0])
+    got = oracle.cosine(x, None, 1, 1, x.size, False, False, oracle.PAIR_SELF, r.step, r.inv, r.offset)
+    assert got == pytest.approx(xd @ xh / (np.linalg.norm(xd) * np.linalg.norm(xh)), abs=1e-14)
+    # identity used by the GPU path: A.B = sig - sum(x e), |B|^2 = sig - 2 sum(x e) + sse
+    e = xd - xh
+    xe = float(xd @ e)
+    assert got == pytest.approx((r.sig - xe) / math.sqrt(r.sig * (r.sig - 2 * xe + r.sse)), abs=1e-13)
