@@ -332,3 +332,62 @@ void qv2o_rank(uint32_t n, const double *sqnr_w, const double *mse_w,
     *n_keep = nk;
     free(score); free(sev); free(taken);
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Fusion-aware sensitivity list.  The paper says only that fusion-capable operators (convolution,
+ * batch normalisation, add, ReLU) may have their positions in the list adjusted so that they can
+ * be fused and share one bit-width.  Reading taken here: fuse_group[i] names the fusion group of
+ * layer i (QV2O_NO_GROUP = on its own).  The base list is qv2o_rank's; walking it from the top,
+ * the first time a member of a group is met the whole group is emitted at that place in layer
+ * order, and later members are skipped.  The FP32-kept prefix never splits a group: by count it
+ * is the longest run of whole groups with at most keep_count layers; by rate it grows group by
+ * group while the MAC-weighted share of still-quantized layers is >= rate_permyriad / 10000.
+ * ------------------------------------------------------------------------------------------- */
+#define QV2O_NO_GROUP 0xFFFFFFFFu
+
+void qv2o_rank_fused(uint32_t n, const double *sqnr_w, const double *mse_w,
+                     const double *sqnr_a, const double *mse_a,
+                     const uint64_t *macs, const double *pos, const uint32_t *fuse_group,
+                     double w_gain, double a_gain, double mse_factor, double cap,
+                     int select_mode, uint32_t keep_count, uint32_t rate_permyriad,
+                     uint32_t *order, uint8_t *keep, uint32_t *n_keep)
+{
+    if (n == 0) { *n_keep = 0; return; }
+    uint32_t *base = (uint32_t *)malloc(n * sizeof(uint32_t));
+    uint8_t *tmp_keep = (uint8_t *)malloc(n);
+    uint32_t tmp_nk;
+    qv2o_rank(n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, w_gain, a_gain, mse_factor, cap,
+              0, 0, 0, base, tmp_keep, &tmp_nk);
+    uint8_t *done = (uint8_t *)calloc(n, 1);
+    uint32_t filled = 0;
+    for (uint32_t j = 0; j < n; ++j) {
+        uint32_t l = base[j];
+        if (done[l]) continue;
+        uint32_t g = fuse_group ? fuse_group[l] : QV2O_NO_GROUP;
+        if (g == QV2O_NO_GROUP) { order[filled++] = l; done[l] = 1; continue; }
+        for (uint32_t m = 0; m < n; ++m)            /* the whole group, in layer order */
+            if (fuse_group[m] == g) { order[filled++] = m; done[m] = 1; }
+    }
+    unsigned __int128 total = 0, kept = 0;
+    for (uint32_t i = 0; i < n; ++i) total += macs ? macs[i] : 1;
+    uint32_t nk = 0, j = 0;
+    while (j < n) {                                  /* one whole group at a time */
+        uint32_t g = fuse_group ? fuse_group[order[j]] : QV2O_NO_GROUP;
+        uint32_t e = j + 1;
+        if (g != QV2O_NO_GROUP) while (e < n && fuse_group[order[e]] == g) ++e;
+        if (select_mode == 0) {
+            if (e <= keep_count) nk = e; else break;
+        } else {
+            unsigned __int128 m = 0;
+            for (uint32_t k = j; k < e; ++k) m += macs ? macs[order[k]] : 1;
+            unsigned __int128 quantized = total - (kept + m);
+            if (quantized * 10000 >= (unsigned __int128)rate_permyriad * total) { kept += m; nk = e; }
+            else break;
+        }
+        j = e;
+    }
+    for (uint32_t i = 0; i < n; ++i) keep[i] = 0;
+    for (uint32_t k = 0; k < nk; ++k) keep[order[k]] = 1;
+    *n_keep = nk;
+    free(base); free(tmp_keep); free(done);
+}

@@ -455,3 +455,71 @@ def test_cosine_closed_forms_and_library_dot_product():
     e = xd - xh
     xe = float(xd @ e)
     assert got == pytest.approx((r.sig - xe) / math.sqrt(r.sig * (r.sig - 2 * xe + r.sse)), abs=1e-13)
+
+
+# ------------------------------------------------------------------------ fusion-aware list
+def test_fused_rank_hand_example_and_properties():
+    NG = oracle.NO_GROUP
+    sw = [40.0, 35.0, 37.0, 36.0, 42.0, 34.0]          # base order (see the hand-worked test): 5 1 0 2 3 4
+    sa = [30.0, 31.0, 27.0, 30.0, 28.0, 29.0]
+    one = [1.0] * 6
+    base, _, _ = oracle.rank_layers(sw, one, sa, one)
+    assert base.tolist() == [5, 1, 0, 2, 3, 4]
+    # no groups at all, or everyone alone: the base list
+    for fg in (None, [NG] * 6, [10, 11, 12, 13, 14, 15]):
+        o, k, nk = oracle.rank_layers_fused(sw, one, sa, one, fg, keep_count=2)
+        assert o.tolist() == base.tolist() and nk == 2 and k.tolist() == [0, 1, 0, 0, 0, 1]
+    # layers 4 and 5 fuse (say conv + relu): 4 is pulled up beside 5, in layer order
+    fg = [NG, NG, NG, NG, 7, 7]
+    o, k, nk = oracle.rank_layers_fused(sw, one, sa, one, fg, keep_count=2)
+    assert o.tolist() == [4, 5, 1, 0, 2, 3] and nk == 2 and k.tolist() == [0, 0, 0, 0, 1, 1]
+    # a cut that would split the group keeps neither member
+    o, k, nk = oracle.rank_layers_fused(sw, one, sa, one, fg, keep_count=1)
+    assert nk == 0 and not k.any()
+    o, k, nk = oracle.rank_layers_fused(sw, one, sa, one, fg, keep_count=3)
+    assert nk == 3 and k.tolist() == [0, 1, 0, 0, 1, 1]
+    # two groups: ordered by their best-ranked member (group {0,3} via layer 0 at base place 2,
+    # group {1,2} via layer 1 at base place 1)
+    fg = [3, 9, 9, 3, NG, NG]
+    o, _, _ = oracle.rank_layers_fused(sw, one, sa, one, fg)
+    assert o.tolist() == [5, 1, 2, 0, 3, 4]
+
+
+def test_fused_rank_random_against_python_walk():
+    NG = oracle.NO_GROUP
+    for trial in range(200):
+        n = int(RNG.integers(1, 12))
+        sw = RNG.uniform(10, 60, n).round(1); sa = RNG.uniform(10, 60, n).round(1)
+        mw = RNG.choice([1e-6, 1e-5, 3e-4], n); ma = RNG.choice([1e-3, 2e-3, 9e-2], n)
+        fg = RNG.choice([NG, NG, 1, 2, 3], n).astype(np.uint32)
+        macs = RNG.integers(0, 1000, n).astype(np.uint64)
+        rate = int(RNG.integers(0, 10001)); kc = int(RNG.integers(0, n + 2)); mode = trial % 2
+        base, _, _ = oracle.rank_layers(sw, mw, sa, ma)
+        o, k, nk = oracle.rank_layers_fused(sw, mw, sa, ma, fg, macs=macs, select_mode=mode,
+                                            keep_count=kc, rate_permyriad=rate)
+        exp, seen = [], set()
+        for l in base.tolist():
+            if l in seen:
+                continue
+            members = [l] if fg[l] == NG else [m for m in range(n) if fg[m] == fg[l]]
+            exp += members; seen.update(members)
+        assert o.tolist() == exp and sorted(exp) == list(range(n))
+        # selection: enumerate group boundaries
+        bounds, j = [0], 0
+        while j < n:
+            e = j + 1
+            while fg[exp[j]] != NG and e < n and fg[exp[e]] == fg[exp[j]]:
+                e += 1
+            bounds.append(e); j = e
+        total = int(macs.sum()); best = 0
+        for b in bounds[1:]:
+            if mode == 0:
+                ok = b <= kc
+            else:
+                q = total - sum(int(macs[i]) for i in exp[:b])
+                ok = Fraction(q * 10000) >= Fraction(rate * total)
+            if ok:
+                best = b
+            else:
+                break
+        assert nk == best and k.sum() == nk and all(k[i] for i in exp[:nk])
