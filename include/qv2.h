@@ -207,6 +207,25 @@ int qv2_rank_layers(qv2_ctx* ctx, uint32_t n_layers,
                     const qv2_rank_cfg* cfg,
                     uint32_t* order, uint8_t* keep_fp32, uint32_t* n_keep);
 
+/*
+ * qv2_rank_layers with fusion groups.  The paper notes that fusion-capable operators (convolution,
+ * batch normalisation, add, ReLU) may have their places in the list adjusted so that they can be
+ * fused and share one bit-width, without saying how; this library's reading: fuse_group[i] is the
+ * id of layer i's fusion group or QV2_NO_GROUP.  The list of qv2_rank_layers is walked from the
+ * top; where the first member of a group stands, the whole group is placed in layer order, and
+ * its other members leave their old places.  The FP32-kept prefix never splits a group: by count
+ * it is the longest run of whole groups with at most keep_count layers, by rate it grows group
+ * by group while the rate still holds.
+ * fuse_group: device, n_layers uint32, or NULL (then this is exactly qv2_rank_layers).
+ */
+#define QV2_NO_GROUP 0xFFFFFFFFu
+int qv2_rank_layers_ex(qv2_ctx* ctx, uint32_t n_layers,
+                       const double* sqnr_w, const double* mse_w,
+                       const double* sqnr_a, const double* mse_a,
+                       const uint64_t* macs, const double* pos, const uint32_t* fuse_group,
+                       const qv2_rank_cfg* cfg,
+                       uint32_t* order, uint8_t* keep_fp32, uint32_t* n_keep);
+
 /* Device buffers of one full-model pass; every pointer is device memory owned by the caller. */
 typedef struct {
   float *gmin, *gmax, *gabsmax, *step, *inv, *offset;   /* qv2_group_count floats each */

@@ -24,7 +24,8 @@ OK = 0
 EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_error",
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
-           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex"]
+           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex"]
+NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
 
 
@@ -78,6 +79,8 @@ def lib() -> C.CDLL:
     L.qv2_quant_metrics_ex.restype = i32
     L.qv2_rank_layers.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, C.POINTER(RankCfg), vp, vp, vp]
     L.qv2_rank_layers.restype = i32
+    L.qv2_rank_layers_ex.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(RankCfg), vp, vp, vp]
+    L.qv2_rank_layers_ex.restype = i32
     L.qv2_sweep_model.argtypes = [vp, dp, u32, u32, vp, vp, C.POINTER(RankCfg),
                                   C.POINTER(SweepBuffers)]
     L.qv2_sweep_model.restype = i32
@@ -234,12 +237,18 @@ class Context:
                "qv2_quant_metrics")
         return out
 
-    def rank_layers(self, sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, cfg: Optional[RankCfg] = None):
+    def rank_layers(self, sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, cfg: Optional[RankCfg] = None,
+                    fuse_group: Optional[torch.Tensor] = None):
         n = sqnr_w.numel()
         cfg = cfg or default_rank_cfg()
         order = self._empty(n, torch.int32)
         keep = self._empty(n, torch.uint8)
         nk = self._empty(1, torch.int32)
+        if fuse_group is not None:
+            _check(lib().qv2_rank_layers_ex(self._h, n, _ptr(sqnr_w), _ptr(mse_w), _ptr(sqnr_a), _ptr(mse_a),
+                                            _ptr(macs), _ptr(pos), _ptr(fuse_group), C.byref(cfg),
+                                            _ptr(order), _ptr(keep), _ptr(nk)), "qv2_rank_layers_ex")
+            return order, keep, nk
         _check(lib().qv2_rank_layers(self._h, n, _ptr(sqnr_w), _ptr(mse_w), _ptr(sqnr_a), _ptr(mse_a),
                                      _ptr(macs), _ptr(pos), C.byref(cfg), _ptr(order), _ptr(keep),
                                      _ptr(nk)), "qv2_rank_layers")

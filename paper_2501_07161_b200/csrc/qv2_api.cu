@@ -150,7 +150,7 @@ extern "C" int qv2_create(qv2_ctx** out, int device, void* stream) {
   DeviceGuard guard(device);
   int sms = 0;
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_rank, 2 * (size_t)kMaxRankLayers * sizeof(double));
+  if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_rank, kRankScratchDoubles * sizeof(double));
   if (e != cudaSuccess) { delete c; return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA; }
   c->sm_count = sms > 0 ? sms : 1;
   c->metrics_cap = metrics_grid_cap(c->sm_count);
@@ -252,20 +252,29 @@ extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint3
   return qv2_quant_metrics_ex(c, descs, n, step, inv, offset, codes, sse, sig, mse, sqnr_db, nullptr);
 }
 
-extern "C" int qv2_rank_layers(qv2_ctx* c, uint32_t n_layers, const double* sqnr_w,
-                               const double* mse_w, const double* sqnr_a, const double* mse_a,
-                               const uint64_t* macs, const double* pos, const qv2_rank_cfg* cfg,
-                               uint32_t* order, uint8_t* keep_fp32, uint32_t* n_keep) {
+extern "C" int qv2_rank_layers_ex(qv2_ctx* c, uint32_t n_layers, const double* sqnr_w,
+                                  const double* mse_w, const double* sqnr_a, const double* mse_a,
+                                  const uint64_t* macs, const double* pos, const uint32_t* fuse_group,
+                                  const qv2_rank_cfg* cfg, uint32_t* order, uint8_t* keep_fp32,
+                                  uint32_t* n_keep) {
   if (!c || !sqnr_w || !mse_w || !sqnr_a || !mse_a || !cfg || !order || !keep_fp32 || !n_keep)
     return QV2_ERR_NULL;
   if (n_layers == 0 || n_layers > kMaxRankLayers) return QV2_ERR_SIZE;
   if (cfg->select_mode > QV2_BY_BOPS_RATE) return QV2_ERR_ARG;
   if (cfg->select_mode == QV2_BY_BOPS_RATE && cfg->rate_permyriad > 10000u) return QV2_ERR_ARG;
   DeviceGuard guard(c->device);
-  QV2_CUDA(c, launch_rank(launch_of(c), n_layers, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, *cfg,
-                          c->d_rank, c->d_rank + kMaxRankLayers, order, keep_fp32, n_keep));
+  QV2_CUDA(c, launch_rank(launch_of(c), n_layers, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, fuse_group,
+                          *cfg, c->d_rank, order, keep_fp32, n_keep));
   ++c->launches;
   return QV2_OK;
+}
+
+extern "C" int qv2_rank_layers(qv2_ctx* c, uint32_t n_layers, const double* sqnr_w,
+                               const double* mse_w, const double* sqnr_a, const double* mse_a,
+                               const uint64_t* macs, const double* pos, const qv2_rank_cfg* cfg,
+                               uint32_t* order, uint8_t* keep_fp32, uint32_t* n_keep) {
+  return qv2_rank_layers_ex(c, n_layers, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, nullptr, cfg, order,
+                            keep_fp32, n_keep);
 }
 
 extern "C" int qv2_sweep_model(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n_tensors,

@@ -105,7 +105,8 @@ cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, u
                                     double* sig, double* mse, double* sqnr_db, double* cosine);
 cudaError_t launch_rank(const Launch& l, uint32_t n, const double* sqnr_w, const double* mse_w,
                         const double* sqnr_a, const double* mse_a, const uint64_t* macs,
-                        const double* pos, qv2_rank_cfg cfg, double* score, double* severity,
+                        const double* pos, const uint32_t* fuse_group, qv2_rank_cfg cfg, double* scratch,
                         uint32_t* order, uint8_t* keep, uint32_t* n_keep);
+constexpr size_t kRankScratchDoubles = 3 * (size_t)kMaxRankLayers;   // see launch_rank
 
 }  // namespace qv2

@@ -312,3 +312,33 @@ def test_cosine_similarity_matches_oracle(ctx):
             assert abs((1 - got) - (1 - ref)) <= 1e-4 * abs(1 - ref), (t, 1 - got, 1 - ref)
     assert float(met.cosine[5]) < -0.99 and float(met.cosine[7]) == 0.0
     assert 0.9999 < float(met.cosine[0]) < 1.0
+
+
+# ------------------------------------------------------------------------ fusion-aware ranking
+def test_fused_rank_is_bit_exact_on_oracle_metrics(ctx):
+    rng = np.random.default_rng(23)
+    NG = oracle.NO_GROUP
+    for trial in range(40):
+        n = int(rng.integers(1, 150)) if trial < 38 else (1024, 2000)[trial - 38]
+        sw = rng.uniform(-5, 60, n).round(1); sa = rng.uniform(-5, 60, n).round(1)
+        mw = rng.choice([0.0, 1e-6, 1e-5, 3e-4, 2e-3], n); ma = rng.choice([1e-3, 2e-3, 9e-2, 0.5], n)
+        n_groups = max(1, n // 4)
+        fg = np.where(rng.random(n) < 0.5, NG, rng.integers(0, n_groups, n)).astype(np.uint32)
+        macs = rng.integers(0, 10 ** 9, n).astype(np.uint64)
+        mode = trial % 2
+        rate = int(rng.integers(0, 10001)); kc = int(rng.integers(0, n + 2))
+        ro, rk, rn = oracle.rank_layers_fused(sw, mw, sa, ma, fg, macs=macs, select_mode=mode,
+                                              keep_count=kc, rate_permyriad=rate)
+        dv = lambda a: torch.from_numpy(np.asarray(a)).cuda()
+        cfg = q.default_rank_cfg(select_mode=mode, keep_count=kc, rate_permyriad=rate)
+        o, k, nk = ctx.rank_layers(dv(sw), dv(mw), dv(sa), dv(ma), dv(macs.view(np.int64)), None, cfg,
+                                   fuse_group=dv(fg.view(np.int32)))
+        torch.cuda.synchronize()
+        assert o.cpu().numpy().view(np.uint32).tolist() == ro.tolist(), trial
+        assert k.cpu().numpy().tolist() == rk.tolist() and int(nk) == rn, trial
+    # everyone alone: identical to the plain call
+    fg = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+    a = ctx.rank_layers(dv(sw), dv(mw), dv(sa), dv(ma), dv(macs.view(np.int64)), None, cfg)
+    b = ctx.rank_layers(dv(sw), dv(mw), dv(sa), dv(ma), dv(macs.view(np.int64)), None, cfg, fuse_group=fg)
+    torch.cuda.synchronize()
+    assert all(torch.equal(u, v) for u, v in zip(a, b))
