@@ -388,7 +388,8 @@ def ours_main(args):
     if rank == 0:
         peak, peak_src = measured_peak()
         achieved = metrics_bytes / (met_ms * 1e-3) / 1e9
-        ratio = recorded_traffic()
+        # the capture was taken on the default workload; DRAM traffic is reported for it only
+        ratio = recorded_traffic() if (args.workload == "vgg16" and batch == cfgw.batch) else None
         traffic = None if ratio is None else ratio * metrics_bytes
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
