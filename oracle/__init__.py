@@ -64,6 +64,12 @@ def _load():
                               C.c_double, C.c_double, C.c_double, C.c_double,
                               C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
     lib.qv2o_rank.restype = None
+    lib.qv2o_qparams_bits.argtypes = [C.c_int] + list(lib.qv2o_qparams.argtypes)
+    lib.qv2o_qparams_bits.restype = None
+    lib.qv2o_quant_metrics_bits.argtypes = [C.c_int] + list(lib.qv2o_quant_metrics.argtypes)
+    lib.qv2o_quant_metrics_bits.restype = None
+    lib.qv2o_cosine_bits.argtypes = [C.c_int] + list(lib.qv2o_cosine.argtypes)
+    lib.qv2o_cosine_bits.restype = C.c_double
     lib.qv2o_rank_fused.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p, u32p,
                                     C.c_double, C.c_double, C.c_double, C.c_double,
                                     C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
@@ -109,12 +115,12 @@ def percentile_clip(hist: np.ndarray, p: float, absmax: float) -> np.float32:
     return np.float32(lib.qv2o_percentile_clip(_p(hist, C.c_uint64), float(p), C.c_float(absmax)))
 
 
-def qparams(asym_u8: bool, gmin, gmax, gabsmax, clip: Optional[float] = None):
+def qparams(asym_u8: bool, gmin, gmax, gabsmax, clip: Optional[float] = None, bits: int = 8):
     lib = _load()
     gmin, gmax, gabsmax = _f32(gmin), _f32(gmax), _f32(gabsmax)
     g = gmin.size
     step = np.zeros(g, np.float32); inv = np.zeros(g, np.float32); off = np.zeros(g, np.float32)
-    lib.qv2o_qparams(int(asym_u8), int(clip is not None), C.c_float(0.0 if clip is None else clip),
+    lib.qv2o_qparams_bits(int(bits), int(asym_u8), int(clip is not None), C.c_float(0.0 if clip is None else clip),
                      g, _p(gmin, C.c_float), _p(gmax, C.c_float), _p(gabsmax, C.c_float),
                      _p(step, C.c_float), _p(inv, C.c_float), _p(off, C.c_float))
     return step, inv, off
@@ -124,7 +130,7 @@ PAIR_SELF, PAIR_REQUANT, PAIR_RAW = 0, 1, 2
 
 
 def quant_metrics(x, y, outer: int, channels: int, inner: int, per_channel: bool, asym_u8: bool,
-                  pair_mode: int, step, inv, offset, want_codes: bool = False):
+                  pair_mode: int, step, inv, offset, want_codes: bool = False, bits: int = 8):
     """-> dict(sse, sig, mse, sqnr_db[, codes])."""
     lib = _load()
     x = _f32(x).reshape(-1)
@@ -134,7 +140,7 @@ def quant_metrics(x, y, outer: int, channels: int, inner: int, per_channel: bool
     step, inv, offset = _f32(step), _f32(inv), _f32(offset)
     codes = np.zeros(x.size, np.uint8) if want_codes else None
     out = [C.c_double(0.0) for _ in range(4)]
-    lib.qv2o_quant_metrics(_p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
+    lib.qv2o_quant_metrics_bits(int(bits), _p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
                            int(per_channel), int(asym_u8), int(pair_mode),
                            _p(step, C.c_float), _p(inv, C.c_float), _p(offset, C.c_float),
                            _p(codes, C.c_uint8), *[C.byref(o) for o in out])
@@ -145,13 +151,13 @@ def quant_metrics(x, y, outer: int, channels: int, inner: int, per_channel: bool
 
 
 def cosine(x, y, outer: int, channels: int, inner: int, per_channel: bool, asym_u8: bool,
-           pair_mode: int, step, inv, offset) -> float:
+           pair_mode: int, step, inv, offset, bits: int = 8) -> float:
     """Cosine similarity between x and the tensor it is compared with (see quant_metrics)."""
     lib = _load()
     x = _f32(x).reshape(-1)
     yy = None if y is None else _f32(y).reshape(-1)
     step, inv, offset = _f32(step), _f32(inv), _f32(offset)
-    return float(lib.qv2o_cosine(_p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
+    return float(lib.qv2o_cosine_bits(int(bits), _p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
                                  int(per_channel), int(asym_u8), int(pair_mode), _p(step, C.c_float),
                                  _p(inv, C.c_float), _p(offset, C.c_float)))
 
@@ -215,7 +221,7 @@ class TensorResult:
     codes: Optional[np.ndarray] = None
 
 
-def calibrate_tensor(x, outer, channels, inner, per_channel, asym_u8, percentile=None):
+def calibrate_tensor(x, outer, channels, inner, per_channel, asym_u8, percentile=None, bits=8):
     """Ranges, optional |x| histogram + percentile clip, then the quantization parameters."""
     gmin, gmax, gabs, bad = ranges(x, outer, channels, inner, per_channel)
     A = np.float32(gabs.max()) if gabs.size else np.float32(0.0)
@@ -223,19 +229,19 @@ def calibrate_tensor(x, outer, channels, inner, per_channel, asym_u8, percentile
     if percentile is not None:
         hist = histogram(x, float(A))
         clip = percentile_clip(hist, percentile, float(A))
-    step, inv, off = qparams(asym_u8, gmin, gmax, gabs, None if percentile is None else float(clip))
+    step, inv, off = qparams(asym_u8, gmin, gmax, gabs, None if percentile is None else float(clip), bits)
     return gmin, gmax, gabs, bad, hist, clip, step, inv, off
 
 
 def sweep_tensor(x, y, outer, channels, inner, per_channel, asym_u8, percentile=None,
-                 pair_mode=None, want_codes=False) -> TensorResult:
+                 pair_mode=None, want_codes=False, bits=8) -> TensorResult:
     """Calibrate on x, then measure: self mode when y is None, else the paired mode."""
     gmin, gmax, gabs, bad, hist, clip, step, inv, off = calibrate_tensor(
-        x, outer, channels, inner, per_channel, asym_u8, percentile)
+        x, outer, channels, inner, per_channel, asym_u8, percentile, bits)
     if pair_mode is None:
         pair_mode = PAIR_SELF if y is None else PAIR_REQUANT
     m = quant_metrics(x, y, outer, channels, inner, per_channel, asym_u8, pair_mode,
-                      step, inv, off, want_codes)
+                      step, inv, off, want_codes, bits)
     return TensorResult(gmin, gmax, gabs, bad, hist, clip, step, inv, off,
                         m["sse"], m["sig"], m["mse"], m["sqnr_db"], m.get("codes"))
 

@@ -121,17 +121,22 @@ float qv2o_percentile_clip(const uint64_t *hist, double p, float A)
  * Eq. 1 and Eq. 3, not an integer zero point).
  * Degenerate range (zero, or a reciprocal that is not finite): step = inv = 1.
  * ------------------------------------------------------------------------------------------- */
-void qv2o_qparams(int asym_u8, int use_clip, float clip, uint64_t groups,
+/* Levels of a b-bit quantizer: Eq. 4's 2^(b-1) - 1 for the symmetric scheme (codes in
+ * [-qmax, qmax]), Eq. 2's N - 1 with N = 2^b levels for the affine one (codes in [0, qmax]). */
+static int32_t top_code(int asym, int bits) { return asym ? (1 << bits) - 1 : (1 << (bits - 1)) - 1; }
+
+void qv2o_qparams_bits(int bits, int asym_u8, int use_clip, float clip, uint64_t groups,
                   const float *gmin, const float *gmax, const float *gabsmax,
                   float *step, float *inv, float *offset)
 {
+    const float top = (float)top_code(asym_u8, bits);      /* 127 or 255 for 8 bits */
     for (uint64_t g = 0; g < groups; ++g) {
         float s, r, off;
         if (!asym_u8) {
             float R = gabsmax[g];
             if (use_clip && clip < R) R = clip;
-            s = fl_div(R, 127.0f);
-            r = fl_div(127.0f, R);
+            s = fl_div(R, top);
+            r = fl_div(top, R);
             off = 0.0f;
             if (!(R > 0.0f) || !finite_f(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
         } else {
@@ -142,13 +147,20 @@ void qv2o_qparams(int asym_u8, int use_clip, float clip, uint64_t groups,
             }
             if (lo == 0.0f) lo = 0.0f;
             float d = fl_sub(hi, lo);
-            s = fl_div(d, 255.0f);
-            r = fl_div(255.0f, d);
+            s = fl_div(d, top);
+            r = fl_div(top, d);
             off = lo;
             if (!(d > 0.0f) || !finite_f(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
         }
         step[g] = s; inv[g] = r; offset[g] = off;
     }
+}
+
+void qv2o_qparams(int asym_u8, int use_clip, float clip, uint64_t groups,
+                  const float *gmin, const float *gmax, const float *gabsmax,
+                  float *step, float *inv, float *offset)
+{
+    qv2o_qparams_bits(8, asym_u8, use_clip, clip, groups, gmin, gmax, gabsmax, step, inv, offset);
 }
 
 /* One code (Eq. 1 / Eq. 5): t = fl(fl(v - offset) * inv); q = clamp(rne(t), qmin, qmax), the
@@ -173,16 +185,17 @@ static int32_t quant_code(float v, float inv, float offset, int32_t qmin, int32_
  * SSE = sum e^2 (P_noise), SIG = sum x^2 (P_signal, always the reference tensor);
  * MSE = SSE / N;  SQNR = 10 log10(SIG / SSE), +inf when SSE == 0, -inf when SIG == 0 < SSE.
  * Metrics are per tensor even when the parameters are per channel.
- * codes (nullable) receives one byte per element: int8 for the symmetric scheme, uint8 else.
+ * codes (nullable) receives one byte per element: int8 for the symmetric scheme, uint8 else
+ * (the low byte of the code; meaningful for bit widths up to 8).
  * ------------------------------------------------------------------------------------------- */
-void qv2o_quant_metrics(const float *x, const float *y,
+void qv2o_quant_metrics_bits(int bits, const float *x, const float *y,
                         uint64_t outer, uint64_t channels, uint64_t inner, int per_channel,
                         int asym_u8, int pair_mode,
                         const float *step, const float *inv, const float *offset,
                         uint8_t *codes, double *sse_out, double *sig_out,
                         double *mse_out, double *sqnr_out)
 {
-    int32_t qmin = asym_u8 ? 0 : -127, qmax = asym_u8 ? 255 : 127;
+    int32_t qmax = top_code(asym_u8, bits), qmin = asym_u8 ? 0 : -qmax;
     long double sse = 0.0L, sig = 0.0L;
     uint64_t n = outer * channels * inner;
     for (uint64_t o = 0; o < outer; ++o)
@@ -212,18 +225,29 @@ void qv2o_quant_metrics(const float *x, const float *y,
     else *sqnr_out = 10.0 * log10(dsig / dsse);
 }
 
+void qv2o_quant_metrics(const float *x, const float *y,
+                        uint64_t outer, uint64_t channels, uint64_t inner, int per_channel,
+                        int asym_u8, int pair_mode,
+                        const float *step, const float *inv, const float *offset,
+                        uint8_t *codes, double *sse_out, double *sig_out,
+                        double *mse_out, double *sqnr_out)
+{
+    qv2o_quant_metrics_bits(8, x, y, outer, channels, inner, per_channel, asym_u8, pair_mode, step, inv,
+                            offset, codes, sse_out, sig_out, mse_out, sqnr_out);
+}
+
 /* ---------------------------------------------------------------------------------------------
  * Cosine similarity (Eq. 8): A.B / (|A| |B|) with A the reference tensor x and B the tensor it is
  * compared with -- the dequantized copy of x (pair_mode 0), the dequantized re-quantization of y
  * (pair_mode 1) or y itself (pair_mode 2).  Written straight from the definition, three sums in
  * long double.  A zero vector has no direction: the result is then 0.
  * ------------------------------------------------------------------------------------------- */
-double qv2o_cosine(const float *x, const float *y,
+double qv2o_cosine_bits(int bits, const float *x, const float *y,
                    uint64_t outer, uint64_t channels, uint64_t inner, int per_channel,
                    int asym_u8, int pair_mode,
                    const float *step, const float *inv, const float *offset)
 {
-    int32_t qmin = asym_u8 ? 0 : -127, qmax = asym_u8 ? 255 : 127;
+    int32_t qmax = top_code(asym_u8, bits), qmin = asym_u8 ? 0 : -qmax;
     long double ab = 0.0L, aa = 0.0L, bb = 0.0L;
     for (uint64_t o = 0; o < outer; ++o)
         for (uint64_t c = 0; c < channels; ++c)
@@ -242,6 +266,14 @@ double qv2o_cosine(const float *x, const float *y,
             }
     long double den = sqrtl(aa) * sqrtl(bb);
     return den > 0.0L ? (double)(ab / den) : 0.0;
+}
+
+double qv2o_cosine(const float *x, const float *y,
+                   uint64_t outer, uint64_t channels, uint64_t inner, int per_channel,
+                   int asym_u8, int pair_mode,
+                   const float *step, const float *inv, const float *offset)
+{
+    return qv2o_cosine_bits(8, x, y, outer, channels, inner, per_channel, asym_u8, pair_mode, step, inv, offset);
 }
 
 /* ---------------------------------------------------------------------------------------------

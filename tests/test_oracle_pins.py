@@ -523,3 +523,37 @@ def test_fused_rank_random_against_python_walk():
             else:
                 break
         assert nk == best and k.sum() == nk and all(k[i] for i in exp[:nk])
+
+
+# ------------------------------------------------------------------------------- bit widths
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 8, 12, 16])
+def test_bit_width_levels_on_grid_and_sqnr_closed_form(bits):
+    qs, qa = 2 ** (bits - 1) - 1, 2 ** bits - 1               # Eq. 4's 2^(b-1)-1 and Eq. 2's N-1
+    d = 2.0 ** -10
+    k = np.arange(-qs, qs + 1)
+    r = oracle.sweep_tensor((k * d).astype(np.float32), None, 1, 1, k.size, False, False,
+                            want_codes=bits <= 8, bits=bits)
+    assert r.step[0] == np.float32(d) and r.sse == 0.0 and r.sqnr_db == math.inf
+    if bits <= 8:
+        np.testing.assert_array_equal(r.codes, k.astype(np.int8))
+    ka = np.arange(0, qa + 1)
+    r = oracle.sweep_tensor((ka * d + 0.5).astype(np.float32), None, 1, 1, ka.size, False, True, bits=bits)
+    assert r.step[0] == np.float32(d) and r.offset[0] == 0.5 and r.sse == 0.0
+    # full-range uniform data: SQNR = 20 log10(2 qmax) symmetric, 10 log10(4 qmax^2) affine on [0,R]
+    u = np.random.default_rng(bits).random(1 << 20)
+    r = oracle.sweep_tensor(((2 * u - 1) * 3).astype(np.float32), None, 1, 1, u.size, False, False, bits=bits)
+    assert r.sqnr_db == pytest.approx(20 * math.log10(2 * qs), abs=0.05)
+    assert r.mse == pytest.approx(float(r.step[0]) ** 2 / 12, rel=2e-2 if bits > 2 else 0.2)
+    if bits <= 12:      # beyond that the binary32 inputs themselves are coarser than the grid
+        r = oracle.sweep_tensor((u * 5).astype(np.float32), None, 1, 1, u.size, False, True, bits=bits)
+        assert r.sqnr_db == pytest.approx(10 * math.log10(4 * qa ** 2), abs=0.05)
+
+
+def test_eight_bit_entry_points_are_the_bits_8_case():
+    x = RNG.standard_normal(5000).astype(np.float32)
+    a = oracle.sweep_tensor(x, None, 1, 1, 5000, False, True, want_codes=True)
+    b = oracle.sweep_tensor(x, None, 1, 1, 5000, False, True, want_codes=True, bits=8)
+    assert a.sse == b.sse and np.array_equal(a.codes, b.codes) and a.step[0] == b.step[0]
+    c = oracle.sweep_tensor(x, None, 1, 1, 5000, False, True, bits=4)
+    assert c.step[0] == np.float32(np.float32(a.gmax[0] - a.gmin[0]) / np.float32(15))
+    assert c.mse > 200 * a.mse            # 4 fewer bits: about 2^8 = 256 times the noise power
