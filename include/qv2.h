@@ -55,6 +55,13 @@ enum { QV2_SYM_I8 = 0, QV2_ASYM_U8 = 1 };                    /* scheme */
 enum { QV2_ABSMAX = 0, QV2_MINMAX = 1, QV2_PERCENTILE = 2 }; /* range */
 enum { QV2_PAIR_REQUANT = 0, QV2_PAIR_RAW = 1, QV2_STORE_CODES = 2 }; /* flags (bit 0: pair mode) */
 enum { QV2_BY_COUNT = 0, QV2_BY_BOPS_RATE = 1 };             /* select_mode */
+/* Code width other than 8 bits, OR-ed into qv2_tensor_desc.flags: QV2_BITS(b), 2 <= b <= 16.  The
+ * largest code is 2^(b-1) - 1 for QV2_SYM_I8 (Eq. 4) and 2^b - 1 for QV2_ASYM_U8 (Eq. 2 with
+ * N = 2^b levels); wherever this header says 127 or 255 read that value.  No QV2_BITS means 8.
+ * QV2_STORE_CODES needs b <= 8 (codes are one byte), else QV2_ERR_UNSUPPORTED. */
+#define QV2_BITS(b) ((uint32_t)(b) << 8)
+#define QV2_BITS_MASK 0xFF00u
+#define QV2_DESC_BITS(flags) (((flags) & QV2_BITS_MASK) ? (((uint32_t)(flags) & QV2_BITS_MASK) >> 8) : 8u)
 
 typedef struct qv2_ctx qv2_ctx;
 

@@ -112,14 +112,14 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
 
 def make_desc(x: Optional[torch.Tensor], y: Optional[torch.Tensor], outer: int, channels: int,
               inner: int, granularity: int, scheme: int, range_mode: int = ABSMAX,
-              percentile: float = 0.0, flags: int = 0) -> TensorDesc:
+              percentile: float = 0.0, flags: int = 0, bits: int = 8) -> TensorDesc:
     d = TensorDesc()
     d.x = _ptr(x) if x is not None and x.numel() else None
     d.y = _ptr(y) if y is not None and y.numel() else None
     if y is not None and not y.numel():
         d.y = None
     d.outer, d.channels, d.inner = outer, channels, inner
-    d.granularity, d.scheme, d.range, d.flags = granularity, scheme, range_mode, flags
+    d.granularity, d.scheme, d.range, d.flags = granularity, scheme, range_mode, flags | (0 if bits == 8 else bits << 8)
     d.percentile = percentile
     return d
 

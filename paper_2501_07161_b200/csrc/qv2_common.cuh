@@ -39,6 +39,7 @@ struct TensorRec {
   uint32_t tile_first;       // index of this tensor's first tile in the tile table
   uint32_t rslot_first;      // per-tensor tensors: first {min,max} key slot written by the range kernel,
   uint32_t rslot_count;      //   one per CTA of the range grid that owns a tile of the tensor
+  uint32_t bits;             // code width, 2..16 (8 unless the descriptor asks otherwise)
   double percentile;
 };
 

@@ -85,14 +85,18 @@ __device__ __forceinline__ float key2f(uint32_t k) {
 
 // Quantization parameters of one group (Eq. 4 read as the multiplier 127/max|W|; Eq. 2 for the
 // affine form), one binary32 rounding per operation.
-__device__ __forceinline__ void make_qparams(bool asym, bool use_clip, float clip, float mn, float mx,
-                                             float am, float* step, float* inv, float* offset) {
+// `top` is the largest code: 2^(b-1) - 1 (symmetric) or 2^b - 1 (affine); 127 / 255 at 8 bits.
+__device__ __host__ __forceinline__ float top_code(bool asym, uint32_t bits) {
+  return (float)(asym ? (1u << bits) - 1u : (1u << (bits - 1u)) - 1u);
+}
+__device__ __forceinline__ void make_qparams(bool asym, float top, bool use_clip, float clip, float mn,
+                                             float mx, float am, float* step, float* inv, float* offset) {
   float s, r, off;
   if (!asym) {
     float R = am;
     if (use_clip && clip < R) R = clip;
-    s = __fdiv_rn(R, 127.0f);
-    r = __fdiv_rn(127.0f, R);
+    s = __fdiv_rn(R, top);
+    r = __fdiv_rn(top, R);
     off = 0.0f;
     if (!(R > 0.0f) || !isfinite(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
   } else {
@@ -103,8 +107,8 @@ __device__ __forceinline__ void make_qparams(bool asym, bool use_clip, float cli
     }
     lo = __fadd_rn(lo, 0.0f);            // -0 -> +0
     float d = __fsub_rn(hi, lo);
-    s = __fdiv_rn(d, 255.0f);
-    r = __fdiv_rn(255.0f, d);
+    s = __fdiv_rn(d, top);
+    r = __fdiv_rn(top, d);
     off = lo;
     if (!(d > 0.0f) || !isfinite(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
   }

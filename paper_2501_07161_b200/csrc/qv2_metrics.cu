@@ -166,8 +166,8 @@ __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
   const float* y = (MODE != kSelf) ? tr->y + tl.begin : nullptr;
   uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
   QP p;
-  p.qmin = tr->asym ? 0.0f : -127.0f;
-  p.qmax = tr->asym ? 255.0f : 127.0f;
+  p.qmax = top_code(tr->asym != 0, tr->bits);
+  p.qmin = tr->asym ? 0.0f : -p.qmax;
   if (tl.rows == 0) {
     const uint32_t G = tr->group_base + (uint32_t)tl.row0;
     p.step = __ldg(step + G); p.inv = __ldg(inv + G); p.off = __ldg(offset + G);
@@ -451,7 +451,8 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   const qv2_tensor_desc& d = *desc;
   if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8 || d.range > QV2_PERCENTILE)
     return QV2_ERR_ARG;
-  if (d.flags & ~(uint32_t)QV2_PAIR_RAW) return QV2_ERR_ARG;          // no code output here
+  if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_BITS_MASK)) return QV2_ERR_ARG;   // no code output here
+  if (QV2_DESC_BITS(d.flags) < 2 || QV2_DESC_BITS(d.flags) > 16) return QV2_ERR_ARG;
   if ((d.flags & QV2_PAIR_RAW) && !d.y) return QV2_ERR_ARG;
   if (d.channels >= (1ull << 32)) return QV2_ERR_SIZE;
   // sizes: reject anything whose partial sums would not fit the fixed array
@@ -473,6 +474,8 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   job.tr.pair_mode = !d.y ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
   job.tr.slot_first = 0; job.tr.slot_count = 0; job.tr.tile_first = 0;
   job.tr.percentile = d.percentile;
+  job.tr.rslot_first = 0; job.tr.rslot_count = 0;
+  job.tr.bits = QV2_DESC_BITS(d.flags);
   job.rows = rows; job.tiles_per_row = 1; job.rows_per_tile = 1;
   uint64_t n_tiles;
   if (!job.tr.per_channel || ne == 0) {

@@ -33,7 +33,10 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     const qv2_tensor_desc& d = descs[t];
     if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8 || d.range > QV2_PERCENTILE)
       return QV2_ERR_ARG;
-    if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_STORE_CODES)) return QV2_ERR_ARG;
+    if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_STORE_CODES | QV2_BITS_MASK)) return QV2_ERR_ARG;
+    const uint32_t bits = QV2_DESC_BITS(d.flags);
+    if (bits < 2 || bits > 16) return QV2_ERR_ARG;
+    if ((d.flags & QV2_STORE_CODES) && bits > 8) return QV2_ERR_UNSUPPORTED;   // codes are one byte
     if (d.range == QV2_PERCENTILE && !(d.percentile >= 0.0 && d.percentile <= 1.0))
       return QV2_ERR_ARG;
     uint64_t rows, ne;
@@ -59,6 +62,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     r.range_mode = d.range;
     r.pair_mode = !pair ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
     r.percentile = d.percentile;
+    r.bits = bits;
 
     size_t first_tile = out->tiles.size();
     if (d.range == QV2_PERCENTILE) out->any_percentile = true;

@@ -31,6 +31,7 @@ class Spec:
     y: Optional[torch.Tensor] = None
     raw: bool = False
     name: str = ""
+    bits: int = 8
 
 
 def bits(a) -> np.ndarray:
@@ -53,12 +54,12 @@ def to_dev(t: Optional[torch.Tensor], misalign: int = 0):
 def make_descs(specs: List[Spec], dev_x, dev_y, store_codes=True):
     descs = []
     for s, dx, dy in zip(specs, dev_x, dev_y):
-        flags = (q.PAIR_RAW if s.raw else 0) | (q.STORE_CODES if store_codes and not s.raw else 0)
+        flags = (q.PAIR_RAW if s.raw else 0) | (q.STORE_CODES if store_codes and not s.raw and s.bits <= 8 else 0)
         descs.append(q.make_desc(dx, dy, s.outer, s.channels, s.inner,
                                  q.PER_CHANNEL if s.per_channel else q.PER_TENSOR,
                                  q.ASYM_U8 if s.asym else q.SYM_I8,
                                  q.PERCENTILE if s.percentile is not None else (q.MINMAX if s.asym else q.ABSMAX),
-                                 s.percentile or 0.0, flags))
+                                 s.percentile or 0.0, flags, s.bits))
     return q.desc_array(descs)
 
 
@@ -69,7 +70,7 @@ def oracle_tensor(s: Spec, want_codes=True):
     if y is not None:
         mode = oracle.PAIR_RAW if s.raw else oracle.PAIR_REQUANT
     return oracle.sweep_tensor(x, y, s.outer, s.channels, s.inner, s.per_channel, s.asym,
-                               s.percentile, pair_mode=mode, want_codes=want_codes and not s.raw)
+                               s.percentile, pair_mode=mode, want_codes=want_codes and not s.raw, bits=s.bits)
 
 
 def assert_metric_close(got_mse, got_sqnr, ref_mse, ref_sqnr, what=""):
@@ -127,7 +128,7 @@ def check_specs(ctx, specs: List[Spec], misalign_x=0, misalign_y=0, check_codes=
             assert_metric_close(float(met.mse[t]), float(met.sqnr_db[t]), ref.mse, ref.sqnr_db, name)
             if ref.sig > 0:
                 assert abs(float(met.sig[t]) - ref.sig) <= MSE_RTOL * ref.sig, f"{name}: sig"
-            if check_codes and not s.raw and s.x.numel():
+            if check_codes and not s.raw and s.x.numel() and s.bits <= 8:
                 got = codes[t][: s.x.numel()].cpu().numpy()
                 exp = ref.codes.view(np.uint8)
                 nbad = int((got != exp).sum())

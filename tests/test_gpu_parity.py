@@ -342,3 +342,28 @@ def test_fused_rank_is_bit_exact_on_oracle_metrics(ctx):
     b = ctx.rank_layers(dv(sw), dv(mw), dv(sa), dv(ma), dv(macs.view(np.int64)), None, cfg, fuse_group=fg)
     torch.cuda.synchronize()
     assert all(torch.equal(u, v) for u, v in zip(a, b))
+
+
+# ---------------------------------------------------------------------------------- bit widths
+@pytest.mark.parametrize("bits", [2, 3, 4, 6, 7, 12, 16])
+def test_other_bit_widths(ctx, bits):
+    n = 3 * TILE + 123
+    x = randn(n, 70 + bits); y = x + 0.02 * randn(n, 90 + bits)
+    w = randn(40 * 300, 71 + bits) * torch.exp(randn(40, 72)).repeat_interleave(300)
+    check_specs(ctx, [Spec(x, 1, 1, n, bits=bits), Spec(x, 1, 1, n, asym=True, bits=bits),
+                      Spec(x.clamp_min(0), 1, 1, n, asym=True, percentile=0.999, bits=bits),
+                      Spec(x, 1, 1, n, asym=True, y=y, bits=bits),
+                      Spec(w, 1, 40, 300, per_channel=True, bits=bits)])
+
+
+def test_bit_width_argument_errors(ctx):
+    x = torch.zeros(64, device="cuda")
+    for bad in (1, 17, 200):
+        d = q.make_desc(x, None, 1, 1, 64, q.PER_TENSOR, q.SYM_I8, bits=bad)
+        with pytest.raises(q.binding.Qv2Error) as e:
+            ctx.calibrate(q.desc_array([d]))
+        assert e.value.status == -1
+    d = q.make_desc(x, None, 1, 1, 64, q.PER_TENSOR, q.SYM_I8, flags=q.STORE_CODES, bits=12)
+    with pytest.raises(q.binding.Qv2Error) as e:
+        ctx.calibrate(q.desc_array([d]))
+    assert e.value.status == -8
