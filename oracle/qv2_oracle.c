@@ -120,6 +120,12 @@ float qv2o_percentile_clip(const uint64_t *hist, double p, float A)
  * d = fl(hi - lo); step = fl(d / 255), inv = fl(255 / d), offset = lo (the real-valued x_min of
  * Eq. 1 and Eq. 3, not an integer zero point).
  * Degenerate range (zero, or a reciprocal that is not finite): step = inv = 1.
+ * Affine form with an INTEGER zero point (scheme 2; what an integer-only accelerator runs, the
+ * target the paper's compiler extension names): the range is first widened to contain 0,
+ * lo' = min(lo, 0), hi' = max(hi, 0); d = fl(hi' - lo'); step = fl(d / top), inv = fl(top / d);
+ * z = clamp(rne(fl(-lo' / step)), 0, top); the offset slot then carries z.  Codes are
+ * q = clamp(rne(fl(v * inv)) + z, 0, top) and the dequantized value is (q - z) * step, so that
+ * 0 is represented exactly.
  * ------------------------------------------------------------------------------------------- */
 /* Levels of a b-bit quantizer: Eq. 4's 2^(b-1) - 1 for the symmetric scheme (codes in
  * [-qmax, qmax]), Eq. 2's N - 1 with N = 2^b levels for the affine one (codes in [0, qmax]). */
@@ -145,12 +151,22 @@ void qv2o_qparams_bits(int bits, int asym_u8, int use_clip, float clip, uint64_t
                 if (-clip > lo) lo = -clip;
                 if (clip < hi) hi = clip;
             }
+            if (asym_u8 == 2) {                  /* integer zero point: the range must hold 0 */
+                if (lo > 0.0f) lo = 0.0f;
+                if (hi < 0.0f) hi = 0.0f;
+            }
             if (lo == 0.0f) lo = 0.0f;
             float d = fl_sub(hi, lo);
             s = fl_div(d, top);
             r = fl_div(top, d);
             off = lo;
-            if (!(d > 0.0f) || !finite_f(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
+            if (!(d > 0.0f) || !finite_f(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; if (asym_u8 == 2) off = 0.0f; }
+            else if (asym_u8 == 2) {
+                double z = nearbyint((double)fl_div(-lo, s));
+                if (!(z >= 0.0)) z = 0.0;
+                if (z > (double)top) z = (double)top;
+                off = (float)z;
+            }
         }
         step[g] = s; inv[g] = r; offset[g] = off;
     }
@@ -171,6 +187,17 @@ static int32_t quant_code(float v, float inv, float offset, int32_t qmin, int32_
     if (isnan(t)) return qmin;
     double r = nearbyint((double)t);       /* default rounding mode: ties to even */
     if (r < (double)qmin) return qmin;
+    if (r > (double)qmax) return qmax;
+    return (int32_t)r;
+}
+
+/* One code with an integer zero point z: q = clamp(rne(fl(v * inv)) + z, 0, qmax). */
+static int32_t quant_code_zp(float v, float inv, int32_t z, int32_t qmax)
+{
+    float t = fl_mul(v, inv);
+    if (isnan(t)) return 0;
+    double r = nearbyint((double)t) + (double)z;
+    if (r < 0.0) return 0;
     if (r > (double)qmax) return qmax;
     return (int32_t)r;
 }
@@ -208,8 +235,16 @@ void qv2o_quant_metrics_bits(int bits, const float *x, const float *y,
                     e = xr - (double)y[k];
                 } else {
                     float v = (pair_mode == 1) ? y[k] : x[k];
-                    int32_t q = quant_code(v, inv[g], offset[g], qmin, qmax);
-                    double deq = (double)q * (double)step[g] + (double)offset[g];
+                    int32_t q;
+                    double deq;
+                    if (asym_u8 == 2) {
+                        int32_t z = (int32_t)offset[g];
+                        q = quant_code_zp(v, inv[g], z, qmax);
+                        deq = (double)(q - z) * (double)step[g];
+                    } else {
+                        q = quant_code(v, inv[g], offset[g], qmin, qmax);
+                        deq = (double)q * (double)step[g] + (double)offset[g];
+                    }
                     e = xr - deq;
                     if (codes) codes[k] = (uint8_t)(q & 0xFF);
                 }
@@ -259,8 +294,14 @@ double qv2o_cosine_bits(int bits, const float *x, const float *y,
                     b = (long double)y[k];
                 } else {
                     float v = (pair_mode == 1) ? y[k] : x[k];
-                    int32_t q = quant_code(v, inv[g], offset[g], qmin, qmax);
-                    b = (long double)q * (long double)step[g] + (long double)offset[g];
+                    if (asym_u8 == 2) {
+                        int32_t z = (int32_t)offset[g];
+                        int32_t q = quant_code_zp(v, inv[g], z, qmax);
+                        b = (long double)(q - z) * (long double)step[g];
+                    } else {
+                        int32_t q = quant_code(v, inv[g], offset[g], qmin, qmax);
+                        b = (long double)q * (long double)step[g] + (long double)offset[g];
+                    }
                 }
                 ab += a * b; aa += a * a; bb += b * b;
             }

@@ -557,3 +557,67 @@ def test_eight_bit_entry_points_are_the_bits_8_case():
     c = oracle.sweep_tensor(x, None, 1, 1, 5000, False, True, bits=4)
     assert c.step[0] == np.float32(np.float32(a.gmax[0] - a.gmin[0]) / np.float32(15))
     assert c.mse > 200 * a.mse            # 4 fewer bits: about 2^8 = 256 times the noise power
+
+
+# ------------------------------------------------------------------- integer zero point (scheme 2)
+ZP = 2
+
+
+def _zp(x, percentile=None, bits=8, y=None):
+    x = np.asarray(x, np.float32)
+    return oracle.sweep_tensor(x, y, 1, 1, x.size, False, ZP, percentile, want_codes=True, bits=bits)
+
+
+def test_zero_point_represents_zero_exactly_and_widens_the_range():
+    x = np.concatenate([np.zeros(50), RNG.uniform(-0.37, 1.91, 5000)]).astype(np.float32)
+    r = _zp(x)
+    z = int(r.offset[0])
+    assert 0 < z < 255 and float(r.offset[0]) == z             # an integer, stored in the offset slot
+    assert (r.codes[:50] == z).all()                           # x = 0 -> code z -> dequantized 0
+    d = np.float32(r.gmax[0] - r.gmin[0])
+    assert r.step[0] == d / np.float32(255) and r.inv[0] == np.float32(255) / d
+    assert z == int(np.rint(np.float32(-r.gmin[0]) / r.step[0]))
+    # an all-positive tensor: the range is widened down to 0, so z = 0 and step = max / 255
+    pos = RNG.uniform(2.0, 5.0, 1000).astype(np.float32)
+    r = _zp(pos)
+    assert r.offset[0] == 0.0 and r.step[0] == np.float32(pos.max()) / np.float32(255) and r.codes.min() >= 102
+    neg = -pos
+    r = _zp(neg)
+    assert r.offset[0] == 255.0 and r.codes.max() <= 153
+    r = _zp(np.zeros(10))
+    assert r.step[0] == 1.0 and r.offset[0] == 0.0 and r.sse == 0.0
+
+
+def test_zero_point_equals_real_offset_when_the_minimum_is_on_the_grid():
+    d = 2.0 ** -6
+    x = (RNG.integers(-64, 192, 4000) * d + RNG.uniform(-0.4, 0.4, 4000) * d).astype(np.float32)
+    x = np.clip(x, np.float32(-64 * d), np.float32(191 * d))
+    x[0], x[1] = -64 * d, 191 * d                               # lo = -64 step, hi - lo = 255 step
+    a = oracle.sweep_tensor(x, None, 1, 1, x.size, False, True, want_codes=True)
+    b = _zp(x)
+    assert a.step[0] == b.step[0] == np.float32(d) and b.offset[0] == 64.0 and a.offset[0] == np.float32(-64 * d)
+    np.testing.assert_array_equal(a.codes, b.codes)
+    assert b.sse == pytest.approx(a.sse, rel=1e-12)
+
+
+def test_zero_point_against_library_quantizer_and_fractions():
+    import torch
+    x = (RNG.standard_normal(200_000) * 0.8 + 0.3).astype(np.float32)
+    r = _zp(x)
+    z = int(r.offset[0])
+    qt = torch.quantize_per_tensor(torch.from_numpy(x), float(r.step[0]), z, torch.quint8).int_repr().numpy()
+    diff = qt != r.codes
+    assert diff.mean() < 1e-4 and np.abs(qt.astype(int) - r.codes.astype(int)).max() <= 1
+    step = Fraction(float(r.step[0]))
+    sse = Fraction(0)
+    for v, q in zip(x[:300], r.codes[:300]):
+        e = Fraction(float(v)) - (int(q) - z) * step
+        assert abs(e) <= step / 2 + Fraction(1, 10 ** 6) or q in (0, 255)
+        sse += e * e
+    part = oracle.quant_metrics(x[:300], None, 1, 1, 300, False, ZP, oracle.PAIR_SELF, r.step, r.inv, r.offset)
+    assert part["sse"] == pytest.approx(float(sse), rel=1e-14)
+    # bit widths and saturation
+    r4 = _zp(x, bits=4)
+    assert r4.codes.max() == 15 and r4.codes.min() == 0 and 0 <= r4.offset[0] <= 15
+    rc = _zp(np.concatenate([x, [40.0, -40.0]]), percentile=0.999)
+    assert rc.codes[-2] == 255 and rc.codes[-1] == 0
