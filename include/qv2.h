@@ -51,7 +51,7 @@ enum {
 };
 
 enum { QV2_PER_TENSOR = 0, QV2_PER_CHANNEL = 1 };            /* granularity */
-enum { QV2_SYM_I8 = 0, QV2_ASYM_U8 = 1 };                    /* scheme */
+enum { QV2_SYM_I8 = 0, QV2_ASYM_U8 = 1, QV2_ASYM_U8_ZP = 2 }; /* scheme */
 enum { QV2_ABSMAX = 0, QV2_MINMAX = 1, QV2_PERCENTILE = 2 }; /* range */
 enum { QV2_PAIR_REQUANT = 0, QV2_PAIR_RAW = 1, QV2_STORE_CODES = 2 }; /* flags (bit 0: pair mode) */
 enum { QV2_BY_COUNT = 0, QV2_BY_BOPS_RATE = 1 };             /* select_mode */
@@ -75,7 +75,11 @@ typedef struct {
   uint64_t outer, channels, inner;
   uint32_t granularity;  /* QV2_PER_TENSOR | QV2_PER_CHANNEL */
   uint32_t scheme;       /* QV2_SYM_I8: codes in [-127,127], offset 0.
-                            QV2_ASYM_U8: codes in [0,255], real-valued offset = range minimum */
+                            QV2_ASYM_U8: codes in [0,255], real-valued offset = range minimum
+                            QV2_ASYM_U8_ZP: codes in [0,255] with an integer zero point z (what an
+                            integer-only accelerator runs): the range is widened to contain 0,
+                            z = clamp(round(-lo/step), 0, 255), q = clamp(round(v*inv) + z, 0, 255),
+                            v^ = (q - z)*step; the offset[] slot of the group then holds z */
   uint32_t range;        /* QV2_ABSMAX and QV2_MINMAX take the group's observed range (|.| max for
                             the symmetric scheme, [min,max] for the asymmetric one);
                             QV2_PERCENTILE additionally clips it to the tensor's |x| percentile */

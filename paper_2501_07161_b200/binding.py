@@ -14,7 +14,7 @@ import torch
 from . import build as _build
 
 PER_TENSOR, PER_CHANNEL = 0, 1
-SYM_I8, ASYM_U8 = 0, 1
+SYM_I8, ASYM_U8, ASYM_U8_ZP = 0, 1, 2
 ABSMAX, MINMAX, PERCENTILE = 0, 1, 2
 PAIR_REQUANT, PAIR_RAW, STORE_CODES = 0, 1, 2
 BY_COUNT, BY_BOPS_RATE = 0, 1

@@ -31,7 +31,7 @@ struct TensorRec {
   uint32_t group_base;       // index of this tensor's group 0 in the per-group arrays
   uint32_t n_groups;
   uint32_t per_channel;
-  uint32_t asym;             // 0: symmetric int8, 1: asymmetric uint8
+  uint32_t asym;             // 0: symmetric, 1: affine with real offset, 2: affine with integer zero point
   uint32_t range_mode;       // QV2_ABSMAX | QV2_MINMAX | QV2_PERCENTILE
   uint32_t pair_mode;        // PairMode
   uint32_t slot_first;       // first partial-sum slot of this tensor

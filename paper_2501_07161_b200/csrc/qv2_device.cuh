@@ -89,8 +89,11 @@ __device__ __forceinline__ float key2f(uint32_t k) {
 __device__ __host__ __forceinline__ float top_code(bool asym, uint32_t bits) {
   return (float)(asym ? (1u << bits) - 1u : (1u << (bits - 1u)) - 1u);
 }
-__device__ __forceinline__ void make_qparams(bool asym, float top, bool use_clip, float clip, float mn,
+// scheme: 0 symmetric, 1 affine with the real-valued minimum as offset, 2 affine with an integer
+// zero point (range widened to hold 0; the offset slot then carries z = clamp(rne(-lo/step), 0, top)).
+__device__ __forceinline__ void make_qparams(uint32_t scheme, float top, bool use_clip, float clip, float mn,
                                              float mx, float am, float* step, float* inv, float* offset) {
+  const bool asym = scheme != 0;
   float s, r, off;
   if (!asym) {
     float R = am;
@@ -105,12 +108,23 @@ __device__ __forceinline__ void make_qparams(bool asym, float top, bool use_clip
       if (-clip > lo) lo = -clip;
       if (clip < hi) hi = clip;
     }
+    if (scheme == 2) {
+      if (lo > 0.0f) lo = 0.0f;
+      if (hi < 0.0f) hi = 0.0f;
+    }
     lo = __fadd_rn(lo, 0.0f);            // -0 -> +0
     float d = __fsub_rn(hi, lo);
     s = __fdiv_rn(d, top);
     r = __fdiv_rn(top, d);
     off = lo;
-    if (!(d > 0.0f) || !isfinite(r) || !(s > 0.0f)) { s = 1.0f; r = 1.0f; }
+    if (!(d > 0.0f) || !isfinite(r) || !(s > 0.0f)) {
+      s = 1.0f; r = 1.0f;
+      if (scheme == 2) off = 0.0f;
+    } else if (scheme == 2) {
+      float z = rintf(__fdiv_rn(-lo, s));          // round half to even
+      if (!(z >= 0.0f)) z = 0.0f;
+      off = fminf(z, top);
+    }
   }
   *step = s; *inv = r; *offset = off;
 }

@@ -152,7 +152,7 @@ clip_finalize_kernel(const TensorRec* __restrict__ tensors, const unsigned long 
   if (tid == 0) clip[t] = c;
   for (uint32_t g = tid; g < tr.n_groups; g += blockDim.x) {
     const uint32_t G = tr.group_base + g;
-    make_qparams(tr.asym != 0, top_code(tr.asym != 0, tr.bits), true, c, gmin[G], gmax[G], gabsmax[G], step + G, inv + G, offset + G);
+    make_qparams(tr.asym, top_code(tr.asym != 0, tr.bits), true, c, gmin[G], gmax[G], gabsmax[G], step + G, inv + G, offset + G);
   }
 }
 

@@ -19,6 +19,7 @@ namespace {
 
 struct QP {
   float step, inv, off, qmin, qmax;
+  float bias;   // added to the rounded value to form the stored code (the zero point, else 0)
 };
 
 // Per-lane accumulators of one tile.  AccCos also carries sum x*e, from which the cosine
@@ -67,7 +68,7 @@ __device__ __forceinline__ void metric_elem(float x, float y, const QP& p, ACC& 
     } else {
       e = __fmaf_rn(-q, p.step, x);
     }
-    if (CODES) *code = (uint8_t)(int)q;
+    if (CODES) *code = (uint8_t)(int)(q + p.bias);
   }
   a.add(x, e);
 }
@@ -166,18 +167,25 @@ __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
   const float* y = (MODE != kSelf) ? tr->y + tl.begin : nullptr;
   uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
   QP p;
-  p.qmax = top_code(tr->asym != 0, tr->bits);
-  p.qmin = tr->asym ? 0.0f : -p.qmax;
-  if (tl.rows == 0) {
-    const uint32_t G = tr->group_base + (uint32_t)tl.row0;
+  const float top = top_code(tr->asym != 0, tr->bits);
+  const bool zp = tr->asym == 2;      // integer zero point: codes are rne(v*inv) + z, clamped to [0, top]
+  p.qmax = top;
+  p.qmin = tr->asym ? 0.0f : -top;
+  p.bias = 0.0f;
+  // With a zero point z the arithmetic is the offset-free path on d = q - z: clamp to [-z, top-z],
+  // e = x - d*step; only the stored code differs (d + z).
+  auto load_params = [&](uint32_t G) {
     p.step = __ldg(step + G); p.inv = __ldg(inv + G); p.off = __ldg(offset + G);
+    if (zp) { p.bias = p.off; p.qmin = -p.off; p.qmax = top - p.off; p.off = 0.0f; }
+  };
+  if (tl.rows == 0) {
+    load_params(tr->group_base + (uint32_t)tl.row0);
     if (MODE == kRaw || p.off == 0.0f) metric_flat<MODE, false, CODES>(x, y, codes, tl.count, p, a);
     else metric_flat<MODE, true, CODES>(x, y, codes, tl.count, p, a);
   } else {
     const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
     for (uint32_t r = warp; r < tl.rows; r += kWarps) {
-      const uint32_t G = tr->group_base + (uint32_t)((tl.row0 + r) % channels);
-      p.step = __ldg(step + G); p.inv = __ldg(inv + G); p.off = __ldg(offset + G);
+      load_params(tr->group_base + (uint32_t)((tl.row0 + r) % channels));
       const uint64_t o = (uint64_t)r * inner;
       if (MODE == kRaw || p.off == 0.0f)
         metric_row<MODE, false, CODES>(x + o, y + o, codes + o, inner, lane, p, a);
@@ -449,7 +457,7 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   if (!desc || !step || !inv || !offset || !result4) return QV2_ERR_NULL;
   if (device < 0 || device >= kMaxDevices) return QV2_ERR_ARG;
   const qv2_tensor_desc& d = *desc;
-  if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8 || d.range > QV2_PERCENTILE)
+  if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE)
     return QV2_ERR_ARG;
   if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_BITS_MASK)) return QV2_ERR_ARG;   // no code output here
   if (QV2_DESC_BITS(d.flags) < 2 || QV2_DESC_BITS(d.flags) > 16) return QV2_ERR_ARG;
@@ -469,7 +477,7 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   job.tr.group_base = 0;
   job.tr.per_channel = d.granularity == QV2_PER_CHANNEL;
   job.tr.n_groups = job.tr.per_channel ? (uint32_t)d.channels : 1u;
-  job.tr.asym = d.scheme == QV2_ASYM_U8;
+  job.tr.asym = d.scheme;
   job.tr.range_mode = d.range;
   job.tr.pair_mode = !d.y ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
   job.tr.slot_first = 0; job.tr.slot_count = 0; job.tr.tile_first = 0;

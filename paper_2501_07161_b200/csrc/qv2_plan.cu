@@ -31,7 +31,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
   uint64_t groups = 0;
   for (uint32_t t = 0; t < n; ++t) {
     const qv2_tensor_desc& d = descs[t];
-    if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8 || d.range > QV2_PERCENTILE)
+    if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE)
       return QV2_ERR_ARG;
     if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_STORE_CODES | QV2_BITS_MASK)) return QV2_ERR_ARG;
     const uint32_t bits = QV2_DESC_BITS(d.flags);
@@ -58,7 +58,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     if (groups + r.n_groups >= (1ull << 32)) return QV2_ERR_SIZE;
     r.group_base = (uint32_t)groups;
     groups += r.n_groups;
-    r.asym = d.scheme == QV2_ASYM_U8;
+    r.asym = d.scheme;                  // 0 symmetric, 1 affine with real offset, 2 affine with zero point
     r.range_mode = d.range;
     r.pair_mode = !pair ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
     r.percentile = d.percentile;

@@ -32,6 +32,7 @@ class Spec:
     raw: bool = False
     name: str = ""
     bits: int = 8
+    zp: bool = False                   # affine scheme with an integer zero point (implies asym)
 
 
 def bits(a) -> np.ndarray:
@@ -57,8 +58,8 @@ def make_descs(specs: List[Spec], dev_x, dev_y, store_codes=True):
         flags = (q.PAIR_RAW if s.raw else 0) | (q.STORE_CODES if store_codes and not s.raw and s.bits <= 8 else 0)
         descs.append(q.make_desc(dx, dy, s.outer, s.channels, s.inner,
                                  q.PER_CHANNEL if s.per_channel else q.PER_TENSOR,
-                                 q.ASYM_U8 if s.asym else q.SYM_I8,
-                                 q.PERCENTILE if s.percentile is not None else (q.MINMAX if s.asym else q.ABSMAX),
+                                 q.ASYM_U8_ZP if s.zp else (q.ASYM_U8 if s.asym else q.SYM_I8),
+                                 q.PERCENTILE if s.percentile is not None else (q.MINMAX if (s.asym or s.zp) else q.ABSMAX),
                                  s.percentile or 0.0, flags, s.bits))
     return q.desc_array(descs)
 
@@ -69,7 +70,7 @@ def oracle_tensor(s: Spec, want_codes=True):
     mode = None
     if y is not None:
         mode = oracle.PAIR_RAW if s.raw else oracle.PAIR_REQUANT
-    return oracle.sweep_tensor(x, y, s.outer, s.channels, s.inner, s.per_channel, s.asym,
+    return oracle.sweep_tensor(x, y, s.outer, s.channels, s.inner, s.per_channel, 2 if s.zp else s.asym,
                                s.percentile, pair_mode=mode, want_codes=want_codes and not s.raw, bits=s.bits)
 
 

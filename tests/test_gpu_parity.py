@@ -367,3 +367,25 @@ def test_bit_width_argument_errors(ctx):
     with pytest.raises(q.binding.Qv2Error) as e:
         ctx.calibrate(q.desc_array([d]))
     assert e.value.status == -8
+
+
+# --------------------------------------------------------------------------- integer zero point
+@pytest.mark.parametrize("bits", [8, 4])
+def test_integer_zero_point_scheme(ctx, bits):
+    n = 4 * TILE + 57
+    x = randn(n, 110) * 0.8 + 0.3; y = x + 0.02 * randn(n, 111)
+    xr = x.clamp_min(0)
+    pos = randn(n, 112).abs() + 2.0
+    w = randn(30 * 500, 113) * torch.exp(randn(30, 114)).repeat_interleave(500) + 0.1
+    specs = [Spec(x, 1, 1, n, zp=True, asym=True, bits=bits),
+             Spec(xr, 1, 1, n, zp=True, asym=True, percentile=0.999, bits=bits),
+             Spec(pos, 1, 1, n, zp=True, asym=True, bits=bits),            # range widened down to 0
+             Spec(-pos, 1, 1, n, zp=True, asym=True, bits=bits),
+             Spec(x, 1, 1, n, zp=True, asym=True, y=y, bits=bits),
+             Spec(w, 1, 30, 500, per_channel=True, zp=True, asym=True, bits=bits),
+             Spec(torch.zeros(500), 1, 1, 500, zp=True, asym=True, bits=bits)]
+    cal, met = check_specs(ctx, specs)
+    top = float(2 ** bits - 1)
+    z = cal.offset.cpu().numpy()
+    assert (z == np.rint(z)).all() and z.min() >= 0 and z.max() <= top     # zero points are integer codes
+    assert z[2] == 0.0 and z[3] == top
