@@ -70,6 +70,9 @@ def _load():
     lib.qv2o_quant_metrics_bits.restype = None
     lib.qv2o_cosine_bits.argtypes = [C.c_int] + list(lib.qv2o_cosine.argtypes)
     lib.qv2o_cosine_bits.restype = C.c_double
+    lib.qv2o_kl_bits.argtypes = [C.c_int, f32p, f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_int, C.c_int,
+                                 C.c_int, f32p, f32p, f32p, C.c_float, u64p, u64p]
+    lib.qv2o_kl_bits.restype = C.c_double
     lib.qv2o_rank_fused.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p, u32p,
                                     C.c_double, C.c_double, C.c_double, C.c_double,
                                     C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
@@ -160,6 +163,24 @@ def cosine(x, y, outer: int, channels: int, inner: int, per_channel: bool, asym_
     return float(lib.qv2o_cosine_bits(int(bits), _p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
                                  int(per_channel), int(asym_u8), int(pair_mode), _p(step, C.c_float),
                                  _p(inv, C.c_float), _p(offset, C.c_float)))
+
+
+KL_BINS = 128
+
+
+def kl_divergence(x, y, outer: int, channels: int, inner: int, per_channel: bool, asym_u8, pair_mode: int,
+                  step, inv, offset, absmax: float, bits: int = 8):
+    """-> (kl in nats, hist of |x| [128], hist of the compared tensor [128]); see qv2o_kl_bits."""
+    lib = _load()
+    x = _f32(x).reshape(-1)
+    yy = None if y is None else _f32(y).reshape(-1)
+    step, inv, offset = _f32(step), _f32(inv), _f32(offset)
+    hp = np.zeros(KL_BINS, np.uint64); hq = np.zeros(KL_BINS, np.uint64)
+    kl = lib.qv2o_kl_bits(int(bits), _p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
+                          int(per_channel), int(asym_u8), int(pair_mode), _p(step, C.c_float),
+                          _p(inv, C.c_float), _p(offset, C.c_float), C.c_float(absmax),
+                          _p(hp, C.c_uint64), _p(hq, C.c_uint64))
+    return float(kl), hp, hq
 
 
 def rank_layers(sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, w_gain=2.0, a_gain=1.0,

@@ -318,6 +318,73 @@ double qv2o_cosine(const float *x, const float *y,
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * KL divergence (Eq. 9): sum_x P(x) log(P(x) / Q(x)), P the distribution of the original tensor's
+ * values and Q that of the tensor it is compared with (dequantized x, dequantized re-quantized y,
+ * or y).  The paper gives no discretisation; the reading taken here: both tensors are binned on
+ * the same QV2O_KL_BINS = 128 linear bins of |value| over [0, A], A the reference tensor's
+ * absmax (values beyond A fall in the last bin); w = fl(128 / A), bin(v) = min(127,
+ * trunc(fl(|v| * w))); counts get add-one smoothing, P_j = (hp_j + 1) / (N + 128), same for Q;
+ * the result is in nats.  The compared value is formed in binary32 so that its bin is a fixed
+ * function of the inputs: b = fl(fl(q * step) + offset) (offset 0 adds nothing; with an integer
+ * zero point b = fl((q - z) * step)); in raw mode b = y.  Non-finite values are skipped.
+ * hp / hq (nullable) receive the two 128-bin histograms.
+ * ------------------------------------------------------------------------------------------- */
+#define QV2O_KL_BINS 128
+
+static uint32_t kl_bin(float v, float w)
+{
+    float f = fl_mul(fabsf(v), w);
+    if (!(f < (float)QV2O_KL_BINS)) return QV2O_KL_BINS - 1;
+    return (uint32_t)f;
+}
+
+double qv2o_kl_bits(int bits, const float *x, const float *y,
+                    uint64_t outer, uint64_t channels, uint64_t inner, int per_channel,
+                    int asym_u8, int pair_mode,
+                    const float *step, const float *inv, const float *offset, float A,
+                    uint64_t *hp_out, uint64_t *hq_out)
+{
+    int32_t qmax = top_code(asym_u8, bits), qmin = asym_u8 ? 0 : -qmax;
+    uint64_t hp[QV2O_KL_BINS] = {0}, hq[QV2O_KL_BINS] = {0};
+    float w = (A > 0.0f) ? fl_div((float)QV2O_KL_BINS, A) : 0.0f;
+    if (!finite_f(w)) w = 0.0f;
+    uint64_t n = 0;
+    for (uint64_t o = 0; o < outer; ++o)
+        for (uint64_t c = 0; c < channels; ++c)
+            for (uint64_t i = 0; i < inner; ++i) {
+                uint64_t k = (o * channels + c) * inner + i;
+                uint64_t g = per_channel ? c : 0;
+                float b;
+                if (pair_mode == 2) {
+                    b = y[k];
+                } else {
+                    float v = (pair_mode == 1) ? y[k] : x[k];
+                    if (asym_u8 == 2) {
+                        int32_t z = (int32_t)offset[g];
+                        int32_t q = quant_code_zp(v, inv[g], z, qmax);
+                        b = fl_mul((float)(q - z), step[g]);
+                    } else {
+                        int32_t q = quant_code(v, inv[g], offset[g], qmin, qmax);
+                        b = fl_mul((float)q, step[g]);
+                        b = (float)((double)b + (double)offset[g]);
+                    }
+                }
+                if (!finite_f(x[k]) || !finite_f(b)) continue;
+                hp[kl_bin(x[k], w)] += 1;
+                hq[kl_bin(b, w)] += 1;
+                ++n;
+            }
+    double kl = 0.0, den = (double)n + (double)QV2O_KL_BINS;
+    for (int j = 0; j < QV2O_KL_BINS; ++j) {
+        double p = ((double)hp[j] + 1.0) / den, q = ((double)hq[j] + 1.0) / den;
+        kl += p * log(p / q);
+    }
+    if (hp_out) memcpy(hp_out, hp, sizeof(hp));
+    if (hq_out) memcpy(hq_out, hq, sizeof(hq));
+    return kl;
+}
+
+/* ---------------------------------------------------------------------------------------------
  * Sensitivity list (Algorithm 2 with RankLayersBySensitivity, Eq. 16 for the SQNR delta) and
  * the FP32-kept set for a requested quantization level (Eq. 17, normalised).
  *  1. every SQNR is clamped to [-cap, cap].

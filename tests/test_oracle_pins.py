@@ -621,3 +621,54 @@ def test_zero_point_against_library_quantizer_and_fractions():
     assert r4.codes.max() == 15 and r4.codes.min() == 0 and 0 <= r4.offset[0] <= 15
     rc = _zp(np.concatenate([x, [40.0, -40.0]]), percentile=0.999)
     assert rc.codes[-2] == 255 and rc.codes[-1] == 0
+
+
+# ------------------------------------------------------------------------------ KL divergence
+def _kl_raw(a, b, A):
+    one = np.ones(1, np.float32); zero = np.zeros(1, np.float32)
+    a = np.float32(a); b = np.float32(b)
+    return oracle.kl_divergence(a, b, 1, 1, a.size, False, True, oracle.PAIR_RAW, one, one, zero, A)
+
+
+def test_kl_closed_forms_and_scipy():
+    from scipy.special import rel_entr
+    x = RNG.uniform(-4, 4, 50_000).astype(np.float32)
+    kl, hp, hq = _kl_raw(x, x, 4.0)
+    assert kl == 0.0 and np.array_equal(hp, hq) and hp.sum() == x.size        # identical -> 0
+    kl, hp, hq = _kl_raw(x, -x, 4.0)
+    assert kl == 0.0                                                          # |.| is what is binned
+    y = (x * 0.5).astype(np.float32)                                          # mass moves to the lower half
+    kl, hp, hq = _kl_raw(x, y, 4.0)
+    assert hq[64:].sum() == 0 and hq.sum() == hp.sum() == x.size
+    p = (hp + 1.0) / (x.size + 128); qq = (hq + 1.0) / (x.size + 128)
+    assert kl == pytest.approx(float(rel_entr(p, qq).sum()), rel=1e-12) and kl > 0.5
+    kl_rev, _, _ = _kl_raw(y, x, 4.0)
+    assert kl_rev != pytest.approx(kl, rel=1e-3)                              # not symmetric
+    # bins: planted centres with a power-of-two range are exact
+    j = np.arange(128)
+    c = ((j + 0.5) * (8.0 / 128)).astype(np.float32)
+    kl, hp, hq = _kl_raw(c, c[::-1].copy(), 8.0)
+    assert (hp == 1).all() and (hq == 1).all() and kl == 0.0
+    kl, hp, hq = _kl_raw(np.float32([8.0, 100.0, np.nan, 1.0]), np.float32([8.0, 8.0, 1.0, np.inf]), 8.0)
+    assert hp.sum() == 2 and hp[127] == 2 and hq[127] == 2                    # beyond A -> last bin; non-finite skipped
+    # two-bin closed form: P = (3+1, 1+1)/(4+128) on bins 0 and 127 ... checked through the formula
+    kl, hp, hq = _kl_raw(np.float32([0.0, 0.0, 0.0, 8.0]), np.float32([0.0, 8.0, 8.0, 8.0]), 8.0)
+    den = 4 + 128
+    exp = (4 / den) * math.log(4 / 2) + (2 / den) * math.log(2 / 4)
+    assert kl == pytest.approx(exp, rel=1e-13)
+
+
+def test_kl_of_quantized_tensor_uses_the_dequantized_values():
+    x = RNG.standard_normal(100_000).astype(np.float32)
+    r = _self(x)
+    A = float(r.gabsmax[0])
+    kl, hp, hq = oracle.kl_divergence(x, None, 1, 1, x.size, False, False, oracle.PAIR_SELF,
+                                      r.step, r.inv, r.offset, A)
+    xh = (r.codes.astype(np.float32) * r.step[0]).astype(np.float32)          # fl(q * step), offset 0
+    w = np.float32(128) / np.float32(A)
+    bins = lambda v: np.minimum((np.abs(v) * w).astype(np.float32).astype(np.int64), 127)
+    assert np.array_equal(hp, np.bincount(bins(x), minlength=128)) and np.array_equal(hq, np.bincount(bins(xh), minlength=128))
+    assert 0 < kl < 0.05                                                      # 8 bits: close distributions
+    kl4, _, _ = oracle.kl_divergence(x, None, 1, 1, x.size, False, False, oracle.PAIR_SELF,
+                                     *oracle.qparams(False, r.gmin, r.gmax, r.gabsmax, bits=4), A, bits=4)
+    assert kl4 > 5 * kl                                                       # coarser grid, further apart
