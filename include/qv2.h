@@ -194,6 +194,26 @@ int qv2_quant_metrics_ex(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
                          double* sse, double* sig, double* mse, double* sqnr_db, double* cosine);
 
 /*
+ * KL divergence (Eq. 9), the fourth local metric the paper considers (and sets aside):
+ * kl[t] = sum_j P_j ln(P_j / Q_j) in nats, P the distribution of the reference tensor x and Q that
+ * of the tensor it is compared with (dequantized x, dequantized re-quantized y, or y under
+ * QV2_PAIR_RAW).  The paper gives no discretisation; here both are binned on the same
+ * QV2_KL_BINS = 128 linear bins of |value| over [0, A], A the tensor-wide absmax of x
+ * (bin = min(127, trunc(|v| * fl(128/A))), values beyond A in the last bin), with add-one
+ * smoothing: P_j = (count_j + 1) / (N + 128).  The compared value is formed in binary32 as
+ * fl(fl(q*step) + offset) (fl((q - z)*step) with a zero point).  Non-finite values are skipped.
+ * This is a separate pass over the tensors (4 or 8 bytes per element) and not part of qv2_sweep_model.
+ *
+ * step, inv, offset, gabsmax: device, per group, as produced by qv2_calibrate.
+ * kl: device, n doubles.  hists: device, n*2*128 uint64 (per tensor the histogram of x, then that
+ * of the compared tensor), or NULL (kept in context scratch).
+ */
+#define QV2_KL_BINS 128
+int qv2_kl_divergence(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
+                      const float* step, const float* inv, const float* offset, const float* gabsmax,
+                      double* kl, uint64_t* hists);
+
+/*
  * Sensitivity list and mixed-precision layer set: step 4 of the overview, "CalculateSQNRdeltas",
  * "CalculateAverage" and "RankLayersBySensitivity" of Algorithm 2, the SQNR delta of Eq. 16 and
  * the BOPs-reduction rate of Eq. 17 (normalised so that a fully quantized model is 100 %).

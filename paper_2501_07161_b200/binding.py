@@ -24,7 +24,8 @@ OK = 0
 EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_error",
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
-           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex"]
+           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence"]
+KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
 
@@ -79,6 +80,8 @@ def lib() -> C.CDLL:
     L.qv2_quant_metrics_ex.restype = i32
     L.qv2_rank_layers.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, C.POINTER(RankCfg), vp, vp, vp]
     L.qv2_rank_layers.restype = i32
+    L.qv2_kl_divergence.argtypes = [vp, dp, u32, vp, vp, vp, vp, vp, vp]
+    L.qv2_kl_divergence.restype = i32
     L.qv2_rank_layers_ex.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(RankCfg), vp, vp, vp]
     L.qv2_rank_layers_ex.restype = i32
     L.qv2_sweep_model.argtypes = [vp, dp, u32, u32, vp, vp, C.POINTER(RankCfg),
@@ -236,6 +239,15 @@ class Context:
                                        _ptr(out.sse), _ptr(out.sig), _ptr(out.mse), _ptr(out.sqnr_db)),
                "qv2_quant_metrics")
         return out
+
+    def kl_divergence(self, descs, step, inv, offset, gabsmax, want_hists: bool = True):
+        """-> (kl float64[n], hists int64[n, 2, 128] or None)."""
+        n = len(descs)
+        kl = self._empty(n, torch.float64)
+        h = self._empty(n * 2 * KL_BINS, torch.int64) if want_hists else None
+        _check(lib().qv2_kl_divergence(self._h, descs, n, _ptr(step), _ptr(inv), _ptr(offset), _ptr(gabsmax),
+                                       _ptr(kl), _ptr(h)), "qv2_kl_divergence")
+        return kl, (None if h is None else h.view(n, 2, KL_BINS))
 
     def rank_layers(self, sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, cfg: Optional[RankCfg] = None,
                     fuse_group: Optional[torch.Tensor] = None):

@@ -29,6 +29,7 @@ struct qv2_ctx {
   double2* d_partials = nullptr;  size_t cap_slots = 0;
   uint2* d_rslots = nullptr;      size_t cap_rslots = 0;
   double* d_partials_xe = nullptr; size_t cap_slots_xe = 0;   // sum x*e slots, cosine only
+  unsigned long long* d_kl_hist = nullptr; size_t cap_kl_hist = 0;   // used when the caller passes no hists
   float* d_tensor_absmax = nullptr; size_t cap_absmax = 0;
   unsigned long long* d_hist = nullptr; size_t cap_hist = 0;   // used when the caller passes no hist
   double* d_rank = nullptr;                                    // 2 * kMaxRankLayers doubles
@@ -163,7 +164,7 @@ extern "C" int qv2_destroy(qv2_ctx* c) {
   if (!c) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
-  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials); cudaFree(c->d_rslots); cudaFree(c->d_partials_xe);
+  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials); cudaFree(c->d_rslots); cudaFree(c->d_partials_xe); cudaFree(c->d_kl_hist);
   cudaFree(c->d_tensor_absmax); cudaFree(c->d_hist); cudaFree(c->d_rank);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
   delete c;
@@ -250,6 +251,27 @@ extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint3
                                  void* const* codes, double* sse, double* sig, double* mse,
                                  double* sqnr_db) {
   return qv2_quant_metrics_ex(c, descs, n, step, inv, offset, codes, sse, sig, mse, sqnr_db, nullptr);
+}
+
+extern "C" int qv2_kl_divergence(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, const float* step,
+                                 const float* inv, const float* offset, const float* gabsmax, double* kl,
+                                 uint64_t* hists) {
+  if (!c || !descs || !step || !inv || !offset || !gabsmax || !kl) return QV2_ERR_NULL;
+  DeviceGuard guard(c->device);
+  int st = ensure_plan(c, descs, n, nullptr);
+  if (st != QV2_OK) return st;
+  const HostPlan& p = c->plan;
+  unsigned long long* h = reinterpret_cast<unsigned long long*>(hists);
+  const size_t cells = (size_t)n * 2 * QV2_KL_BINS;
+  if (!h) {
+    if ((st = grow(c, &c->d_kl_hist, &c->cap_kl_hist, cells)) != QV2_OK) return st;
+    h = c->d_kl_hist;
+  }
+  QV2_CUDA(c, cudaMemsetAsync(h, 0, cells * sizeof(unsigned long long), c->stream));
+  QV2_CUDA(c, launch_kl(launch_of(c), c->d_tensors, n, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
+                        offset, gabsmax, c->d_tensor_absmax, h, kl));
+  c->launches += p.tiles.empty() ? 2 : 3;
+  return QV2_OK;
 }
 
 extern "C" int qv2_rank_layers_ex(qv2_ctx* c, uint32_t n_layers, const double* sqnr_w,

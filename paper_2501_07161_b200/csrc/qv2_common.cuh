@@ -104,6 +104,9 @@ uint32_t metrics_grid_cap(int sm_count);   // resident CTAs per SM x SMs for the
 cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                     const double2* partials, const double* partials_xe, double* sse,
                                     double* sig, double* mse, double* sqnr_db, double* cosine);
+cudaError_t launch_kl(const Launch& l, const TensorRec* tensors, uint32_t n_tensors, const Tile* tiles,
+                      uint32_t n_tiles, const float* step, const float* inv, const float* offset,
+                      const float* gabsmax, float* tensor_absmax, unsigned long long* hists, double* kl);
 cudaError_t launch_rank(const Launch& l, uint32_t n, const double* sqnr_w, const double* mse_w,
                         const double* sqnr_a, const double* mse_a, const uint64_t* macs,
                         const double* pos, const uint32_t* fuse_group, qv2_rank_cfg cfg, double* scratch,

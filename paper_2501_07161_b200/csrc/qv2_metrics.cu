@@ -25,6 +25,7 @@ struct QP {
 // Per-lane accumulators of one tile.  AccCos also carries sum x*e, from which the cosine
 // similarity of Eq. 8 follows without a second pass: A.B = sig - xe, |B|^2 = sig - 2 xe + sse.
 struct Acc {
+  static constexpr bool kWantsB = false;     // needs (x, e) only
   float sse, sig;
   __device__ __forceinline__ void clear() { sse = 0.0f; sig = 0.0f; }
   __device__ __forceinline__ void add(float x, float e) {
@@ -33,6 +34,7 @@ struct Acc {
   }
 };
 struct AccCos {
+  static constexpr bool kWantsB = false;
   float sse, sig, xe;
   __device__ __forceinline__ void clear() { sse = 0.0f; sig = 0.0f; xe = 0.0f; }
   __device__ __forceinline__ void add(float x, float e) {
@@ -69,8 +71,15 @@ __device__ __forceinline__ void metric_elem(float x, float y, const QP& p, ACC& 
       e = __fmaf_rn(-q, p.step, x);
     }
     if (CODES) *code = (uint8_t)(int)(q + p.bias);
+    if constexpr (ACC::kWantsB) {
+      // the compared value itself, in binary32 with fixed rounding points: fl(fl(q*step) + off)
+      const float b = OFF ? __fadd_rn(__fmul_rn(q, p.step), p.off) : __fmul_rn(q, p.step);
+      a.add_b(x, b);
+      return;
+    }
   }
-  a.add(x, e);
+  if constexpr (ACC::kWantsB) a.add_b(x, y);
+  else a.add(x, e);
 }
 
 template <uint32_t MODE, bool OFF, bool CODES, class ACC>
@@ -305,6 +314,109 @@ metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// KL divergence (Eq. 9) between the distribution of x and that of the tensor it is compared with,
+// both binned on kKlBins linear bins of |value| over [0, absmax of x].  Same tile walk and
+// quantizer as the metrics kernel; the accumulator bins instead of summing.  Each warp owns a
+// private pair of histograms in shared memory; they are merged into the 64-bit global ones when
+// the CTA moves to another tensor.  Counts are integers: the result does not depend on order.
+constexpr uint32_t kKlBins = QV2_KL_BINS;
+
+struct AccKL {
+  static constexpr bool kWantsB = true;
+  uint32_t* hp;      // this warp's histogram of |x|
+  uint32_t* hq;      // ... and of |b|
+  float w;           // fl(kKlBins / absmax)
+  __device__ __forceinline__ static uint32_t bin(float v, float w) {
+    const float f = __fmul_rn(fabsf(v), w);
+    const uint32_t b = __float_as_uint(__fadd_rz(f, 8388608.0f)) - 0x4B000000u;   // trunc for 0 <= f < 2^23
+    return min(b, kKlBins - 1u);
+  }
+  __device__ __forceinline__ void add_b(float x, float b) {
+    if (!isfinite(x) || !isfinite(b)) return;
+    atomicAdd(hp + bin(x, w), 1u);
+    atomicAdd(hq + bin(b, w), 1u);
+  }
+};
+
+__global__ void __launch_bounds__(kThreads, 2)
+kl_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
+          const float* __restrict__ step, const float* __restrict__ inv, const float* __restrict__ offset,
+          const float* __restrict__ tensor_absmax, unsigned long long* hists) {
+  __shared__ uint32_t sh[kWarps * 2 * kKlBins];
+  constexpr uint32_t kNone = 0xffffffffu;
+  const uint32_t warp = threadIdx.x >> 5;
+  for (uint32_t b = threadIdx.x; b < kWarps * 2 * kKlBins; b += kThreads) sh[b] = 0;
+  __syncthreads();
+  uint32_t cur = kNone, since_flush = 0;
+  float w = 0.0f;
+  for (uint32_t ti = blockIdx.x;; ti += gridDim.x) {
+    const bool more = ti < n_tiles;
+    Tile tl;
+    if (more) tl = load_tile(tiles, ti);
+    if (cur != kNone && (!more || tl.tensor != cur || since_flush >= 16384u)) {
+      __syncthreads();                               // every warp is done with its last tile
+      unsigned long long* h = hists + (size_t)cur * 2 * kKlBins;
+      for (uint32_t b = threadIdx.x; b < kWarps * 2 * kKlBins; b += kThreads) {
+        const uint32_t c = sh[b];
+        if (c) { atomicAdd(h + (b % (2 * kKlBins)), (unsigned long long)c); sh[b] = 0; }
+      }
+      __syncthreads();
+      since_flush = 0;
+    }
+    if (!more) break;
+    const TensorRec* tr = tensors + tl.tensor;
+    if (tl.tensor != cur) {
+      cur = tl.tensor;
+      const float A = tensor_absmax[cur];
+      w = (A > 0.0f) ? __fdiv_rn((float)kKlBins, A) : 0.0f;
+      if (!isfinite(w)) w = 0.0f;
+    }
+    AccKL a[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { a[k].hp = sh + warp * 2 * kKlBins; a[k].hq = a[k].hp + kKlBins; a[k].w = w; }
+    const uint32_t mode = tr->pair_mode;
+    if (mode == kSelf) metric_tile<kSelf, false>(tl, tr, step, inv, offset, a);
+    else if (mode == kRequant) metric_tile<kRequant, false>(tl, tr, step, inv, offset, a);
+    else metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
+    ++since_flush;
+  }
+}
+
+// One CTA per tensor: the tensor-wide absmax from the per-group values.
+__global__ void __launch_bounds__(256)
+tensor_absmax_kernel(const TensorRec* __restrict__ tensors, const float* __restrict__ gabsmax, float* out) {
+  __shared__ float red[256];
+  const TensorRec tr = tensors[blockIdx.x];
+  float m = 0.0f;
+  for (uint32_t g = threadIdx.x; g < tr.n_groups; g += 256) m = fmaxf(m, gabsmax[tr.group_base + g]);
+  red[threadIdx.x] = m;
+  __syncthreads();
+  for (uint32_t o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + o]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[blockIdx.x] = red[0];
+}
+
+// One thread per tensor: add-one smoothing, then the sum in bin order.
+__global__ void kl_finalize_kernel(uint32_t n, const unsigned long long* __restrict__ hists, double* kl_out) {
+  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  const unsigned long long* hp = hists + (size_t)t * 2 * kKlBins;
+  const unsigned long long* hq = hp + kKlBins;
+  unsigned long long cnt = 0;
+  for (uint32_t j = 0; j < kKlBins; ++j) cnt += hp[j];
+  const double den = __dadd_rn((double)cnt, (double)kKlBins);
+  double kl = 0.0;
+  for (uint32_t j = 0; j < kKlBins; ++j) {
+    const double p = __ddiv_rn(__dadd_rn((double)hp[j], 1.0), den);
+    const double q = __ddiv_rn(__dadd_rn((double)hq[j], 1.0), den);
+    kl = __dadd_rn(kl, __dmul_rn(p, log(__ddiv_rn(p, q))));
+  }
+  kl_out[t] = kl;
+}
+
 }  // namespace
 
 uint32_t metrics_grid_cap(int sm_count) {
@@ -333,6 +445,21 @@ cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, u
   return cudaGetLastError();
 }
 
+}  // namespace qv2
+
+namespace qv2 {
+cudaError_t launch_kl(const Launch& l, const TensorRec* tensors, uint32_t n_tensors, const Tile* tiles,
+                      uint32_t n_tiles, const float* step, const float* inv, const float* offset,
+                      const float* gabsmax, float* tensor_absmax, unsigned long long* hists, double* kl) {
+  tensor_absmax_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, gabsmax, tensor_absmax);
+  if (n_tiles) {
+    static int per_sm = 0;
+    const int grid = persistent_grid((const void*)kl_kernel, &per_sm, l.sm_count, n_tiles);
+    kl_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset, tensor_absmax, hists);
+  }
+  kl_finalize_kernel<<<(n_tensors + 63) / 64, 64, 0, l.stream>>>(n_tensors, hists, kl);
+  return cudaGetLastError();
+}
 }  // namespace qv2
 
 // ================================================================================================

@@ -389,3 +389,43 @@ def test_integer_zero_point_scheme(ctx, bits):
     z = cal.offset.cpu().numpy()
     assert (z == np.rint(z)).all() and z.min() >= 0 and z.max() <= top     # zero points are integer codes
     assert z[2] == 0.0 and z[3] == top
+
+
+# ------------------------------------------------------------------------------- KL divergence
+def test_kl_divergence_matches_oracle(ctx):
+    """Eq. 9 on 128 smoothed bins: the two histograms are integers and must match exactly; the
+    divergence itself differs only through log() (1 ulp) and is compared to 1e-12 absolute."""
+    from parity import make_descs, to_dev
+    n = 5 * TILE + 311
+    x = randn(n, 131); y = x + 0.05 * randn(n, 132)
+    xr = x.clamp_min(0)
+    w = randn(50 * 700, 133) * torch.exp(randn(50, 134)).repeat_interleave(700)
+    xn = x.clone(); xn[7] = float("nan"); xn[TILE + 1] = float("inf")
+    specs = [Spec(x, 1, 1, n), Spec(x, 1, 1, n, asym=True), Spec(x, 1, 1, n, asym=True, zp=True),
+             Spec(xr, 1, 1, n, asym=True, percentile=0.999), Spec(x, 1, 1, n, asym=True, y=y),
+             Spec(x, 1, 1, n, asym=True, y=y, raw=True), Spec(x, 1, 1, n, bits=4),
+             Spec(w, 1, 50, 700, per_channel=True), Spec(x[: 6 * (n // 6)], 2, 3, n // 6, per_channel=True, asym=True),
+             Spec(torch.zeros(300), 1, 1, 300), Spec(xn, 1, 1, n, asym=True, y=y, raw=True)]
+    dx = [to_dev(s.x) for s in specs]; dy = [to_dev(s.y) for s in specs]
+    descs = make_descs(specs, dx, dy, store_codes=False)
+    cal = ctx.calibrate(descs)
+    kl, hists = ctx.kl_divergence(descs, cal.step, cal.inv, cal.offset, cal.gabsmax)
+    kl2, _ = ctx.kl_divergence(descs, cal.step, cal.inv, cal.offset, cal.gabsmax, want_hists=False)
+    torch.cuda.synchronize()
+    assert torch.equal(kl.view(torch.int64), kl2.view(torch.int64))
+    hists = hists.cpu().numpy().view(np.uint64)
+    g = 0
+    for t, s in enumerate(specs):
+        ng = s.channels if s.per_channel else 1
+        sl = slice(g, g + ng); g += ng
+        mode = oracle.PAIR_SELF if s.y is None else (oracle.PAIR_RAW if s.raw else oracle.PAIR_REQUANT)
+        A = float(cal.gabsmax[sl].max())
+        ref, hp, hq = oracle.kl_divergence(s.x.numpy(), None if s.y is None else s.y.numpy(), s.outer,
+                                           s.channels, s.inner, s.per_channel, 2 if s.zp else s.asym, mode,
+                                           cal.step[sl].cpu().numpy(), cal.inv[sl].cpu().numpy(),
+                                           cal.offset[sl].cpu().numpy(), A, bits=s.bits)
+        assert np.array_equal(hists[t, 0], hp), (t, "hist of x")
+        assert np.array_equal(hists[t, 1], hq), (t, "hist of the compared tensor")
+        assert abs(float(kl[t]) - ref) <= 1e-12, (t, float(kl[t]), ref)
+    assert float(kl[6]) > 5 * float(kl[0]) > 0                 # 4 bits is further from x than 8 bits
+    assert int(hists[10, 0].sum()) == n - 2                    # non-finite elements are skipped
