@@ -118,6 +118,20 @@ uint64_t qv2_launch_count(const qv2_ctx* ctx);
 uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n);
 
 /*
+ * Convolution + batch-normalisation folding, Eq. 10-12: the pre-pass that produces the weights of
+ * the fused graph, on which the mixed-precision decision is applied.  Per output channel c:
+ *   s_c = gamma_c / sqrt(var_c);  w_out[c][k] = s_c * w[c][k];  bias_out[c] = s_c*(bias_c - mean_c) + beta_c
+ * each operation rounded once in binary32, in that order.  As printed in the paper there is no
+ * epsilon under the root: the caller adds it to var if its framework uses one; var_c <= 0 gives
+ * Inf/NaN in that channel.
+ * w, w_out: device, [channels][inner] fp32 (w_out may alias w).  bias: device [channels] or NULL
+ * (zeros).  gamma, beta, mean, var: device [channels].  bias_out: device [channels] or NULL.
+ */
+int qv2_fold_batchnorm(qv2_ctx* ctx, const float* w, const float* bias, const float* gamma,
+                       const float* beta, const float* mean, const float* var,
+                       uint64_t channels, uint64_t inner, float* w_out, float* bias_out);
+
+/*
  * Calibration: step 1 of the paper's overview ("collect statistical data on the distribution of
  * weights and activations") together with its calibration stage (a histogram of each layer's
  * value range), followed by the scale computation of step 2 (Eq. 4 for symmetric weights, Eq. 2

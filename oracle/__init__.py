@@ -73,6 +73,8 @@ def _load():
     lib.qv2o_kl_bits.argtypes = [C.c_int, f32p, f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_int, C.c_int,
                                  C.c_int, f32p, f32p, f32p, C.c_float, u64p, u64p]
     lib.qv2o_kl_bits.restype = C.c_double
+    lib.qv2o_fold_batchnorm.argtypes = [f32p] * 6 + [C.c_uint64, C.c_uint64, f32p, f32p]
+    lib.qv2o_fold_batchnorm.restype = None
     lib.qv2o_rank_fused.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p, u32p,
                                     C.c_double, C.c_double, C.c_double, C.c_double,
                                     C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
@@ -163,6 +165,20 @@ def cosine(x, y, outer: int, channels: int, inner: int, per_channel: bool, asym_
     return float(lib.qv2o_cosine_bits(int(bits), _p(x, C.c_float), _p(yy, C.c_float), outer, channels, inner,
                                  int(per_channel), int(asym_u8), int(pair_mode), _p(step, C.c_float),
                                  _p(inv, C.c_float), _p(offset, C.c_float)))
+
+
+def fold_batchnorm(w, bias, gamma, beta, mean, var):
+    """Eq. 10-12: -> (folded weights [C, K] float32, folded bias [C] float32)."""
+    lib = _load()
+    w = _f32(w)
+    c, k = w.shape
+    b = None if bias is None else _f32(bias)
+    gamma, beta, mean, var = _f32(gamma), _f32(beta), _f32(mean), _f32(var)
+    w_out = np.zeros((c, k), np.float32); b_out = np.zeros(c, np.float32)
+    lib.qv2o_fold_batchnorm(_p(w, C.c_float), _p(b, C.c_float), _p(gamma, C.c_float), _p(beta, C.c_float),
+                            _p(mean, C.c_float), _p(var, C.c_float), c, k, _p(w_out, C.c_float),
+                            _p(b_out, C.c_float))
+    return w_out, b_out
 
 
 KL_BINS = 128

@@ -531,3 +531,24 @@ void qv2o_rank_fused(uint32_t n, const double *sqnr_w, const double *mse_w,
     *n_keep = nk;
     free(base); free(tmp_keep); free(done);
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Convolution + batch-normalisation folding (Eq. 10-12): A_c = gamma_c / sqrt(var_c) * W_c,
+ * C_c = gamma_c (B_c - mean_c) / sqrt(var_c) + beta_c.  The outputs are binary32 tensors that feed
+ * the sweep, so every operation is one binary32 rounding, in this order: r = sqrt(var),
+ * s = gamma / r, A = s * W, C = (s * (B - mean)) + beta.  bias may be NULL (zeros).
+ * ------------------------------------------------------------------------------------------- */
+void qv2o_fold_batchnorm(const float *w, const float *bias, const float *gamma, const float *beta,
+                         const float *mean, const float *var, uint64_t channels, uint64_t inner,
+                         float *w_out, float *bias_out)
+{
+    for (uint64_t c = 0; c < channels; ++c) {
+        float r = (float)sqrt((double)var[c]);          /* correctly rounded: 53 >= 2*24 + 2 */
+        float s = fl_div(gamma[c], r);
+        for (uint64_t k = 0; k < inner; ++k) w_out[c * inner + k] = fl_mul(s, w[c * inner + k]);
+        if (bias_out) {
+            float b = bias ? bias[c] : 0.0f;
+            bias_out[c] = (float)((double)fl_mul(s, fl_sub(b, mean[c])) + (double)beta[c]);
+        }
+    }
+}

@@ -24,7 +24,7 @@ OK = 0
 EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_error",
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
-           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence"]
+           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm"]
 KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
     L.qv2_rank_layers.restype = i32
     L.qv2_kl_divergence.argtypes = [vp, dp, u32, vp, vp, vp, vp, vp, vp]
     L.qv2_kl_divergence.restype = i32
+    L.qv2_fold_batchnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, u64, u64, vp, vp]
+    L.qv2_fold_batchnorm.restype = i32
     L.qv2_rank_layers_ex.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(RankCfg), vp, vp, vp]
     L.qv2_rank_layers_ex.restype = i32
     L.qv2_sweep_model.argtypes = [vp, dp, u32, u32, vp, vp, C.POINTER(RankCfg),
@@ -239,6 +241,15 @@ class Context:
                                        _ptr(out.sse), _ptr(out.sig), _ptr(out.mse), _ptr(out.sqnr_db)),
                "qv2_quant_metrics")
         return out
+
+    def fold_batchnorm(self, w, bias, gamma, beta, mean, var):
+        """Eq. 10-12: -> (folded weights [C, K], folded bias [C])."""
+        c, k = w.shape
+        w_out = torch.empty_like(w)
+        b_out = self._empty(c, torch.float32)
+        _check(lib().qv2_fold_batchnorm(self._h, _ptr(w), _ptr(bias), _ptr(gamma), _ptr(beta), _ptr(mean),
+                                        _ptr(var), c, k, _ptr(w_out), _ptr(b_out)), "qv2_fold_batchnorm")
+        return w_out, b_out[:c]
 
     def kl_divergence(self, descs, step, inv, offset, gabsmax, want_hists: bool = True):
         """-> (kl float64[n], hists int64[n, 2, 128] or None)."""

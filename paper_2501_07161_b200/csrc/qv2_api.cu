@@ -274,6 +274,19 @@ extern "C" int qv2_kl_divergence(qv2_ctx* c, const qv2_tensor_desc* descs, uint3
   return QV2_OK;
 }
 
+extern "C" int qv2_fold_batchnorm(qv2_ctx* c, const float* w, const float* bias, const float* gamma,
+                                  const float* beta, const float* mean, const float* var,
+                                  uint64_t channels, uint64_t inner, float* w_out, float* bias_out) {
+  if (!c || !gamma || !beta || !mean || !var) return QV2_ERR_NULL;
+  if (channels && inner && (!w || !w_out)) return QV2_ERR_NULL;
+  if (channels != 0 && inner > (1ull << 62) / channels) return QV2_ERR_SIZE;
+  if ((((uintptr_t)w) | ((uintptr_t)w_out)) & 3u) return QV2_ERR_ALIGN;
+  DeviceGuard guard(c->device);
+  QV2_CUDA(c, launch_fold(launch_of(c), w, bias, gamma, beta, mean, var, channels, inner, w_out, bias_out));
+  c->launches += (channels && inner ? (channels + 65534) / 65535 : 0) + (bias_out && channels ? 1 : 0);
+  return QV2_OK;
+}
+
 extern "C" int qv2_rank_layers_ex(qv2_ctx* c, uint32_t n_layers, const double* sqnr_w,
                                   const double* mse_w, const double* sqnr_a, const double* mse_a,
                                   const uint64_t* macs, const double* pos, const uint32_t* fuse_group,

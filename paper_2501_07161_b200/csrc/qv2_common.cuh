@@ -107,6 +107,9 @@ cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, u
 cudaError_t launch_kl(const Launch& l, const TensorRec* tensors, uint32_t n_tensors, const Tile* tiles,
                       uint32_t n_tiles, const float* step, const float* inv, const float* offset,
                       const float* gabsmax, float* tensor_absmax, unsigned long long* hists, double* kl);
+cudaError_t launch_fold(const Launch& l, const float* w, const float* bias, const float* gamma,
+                        const float* beta, const float* mean, const float* var, uint64_t channels,
+                        uint64_t inner, float* w_out, float* bias_out);
 cudaError_t launch_rank(const Launch& l, uint32_t n, const double* sqnr_w, const double* mse_w,
                         const double* sqnr_a, const double* mse_a, const uint64_t* macs,
                         const double* pos, const uint32_t* fuse_group, qv2_rank_cfg cfg, double* scratch,

@@ -429,3 +429,23 @@ def test_kl_divergence_matches_oracle(ctx):
         assert abs(float(kl[t]) - ref) <= 1e-12, (t, float(kl[t]), ref)
     assert float(kl[6]) > 5 * float(kl[0]) > 0                 # 4 bits is further from x than 8 bits
     assert int(hists[10, 0].sum()) == n - 2                    # non-finite elements are skipped
+
+
+# ----------------------------------------------------------------------------- Conv+BN folding
+@pytest.mark.parametrize("c,k,mis", [(64, 576, 0), (37, 1153, 0), (5, 25088, 0), (960, 9, 0), (16, 64, 1)])
+def test_fold_batchnorm_is_bit_exact(ctx, c, k, mis):
+    from parity import to_dev
+    w = randn(c * k, 140 + c).reshape(c, k); b = randn(c, 141)
+    gamma = torch.rand(c, generator=_g(142)) * 1.5 + 0.5; beta = randn(c, 143)
+    mean = randn(c, 144); var = torch.rand(c, generator=_g(145)) * 3 + 0.05
+    ra, rc = oracle.fold_batchnorm(w.numpy(), b.numpy(), gamma.numpy(), beta.numpy(), mean.numpy(), var.numpy())
+    dw = to_dev(w, mis).view(c, k)
+    a, cc = ctx.fold_batchnorm(dw, b.cuda(), gamma.cuda(), beta.cuda(), mean.cuda(), var.cuda())
+    a0, c0 = ctx.fold_batchnorm(dw, None, gamma.cuda(), beta.cuda(), mean.cuda(), var.cuda())
+    torch.cuda.synchronize()
+    assert np.array_equal(a.cpu().numpy().view(np.uint32), ra.view(np.uint32))
+    assert np.array_equal(cc.cpu().numpy().view(np.uint32), rc.view(np.uint32))
+    r0 = oracle.fold_batchnorm(w.numpy(), None, gamma.numpy(), beta.numpy(), mean.numpy(), var.numpy())[1]
+    assert torch.equal(a0, a) and np.array_equal(c0.cpu().numpy().view(np.uint32), r0.view(np.uint32))
+    # the folded weights feed the sweep like any other weight tensor
+    check_specs(ctx, [Spec(a.cpu(), 1, c, k, per_channel=True)], twice=False)

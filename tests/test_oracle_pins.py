@@ -672,3 +672,26 @@ def test_kl_of_quantized_tensor_uses_the_dequantized_values():
     kl4, _, _ = oracle.kl_divergence(x, None, 1, 1, x.size, False, False, oracle.PAIR_SELF,
                                      *oracle.qparams(False, r.gmin, r.gmax, r.gabsmax, bits=4), A, bits=4)
     assert kl4 > 5 * kl                                                       # coarser grid, further apart
+
+
+# -------------------------------------------------------------------------- Conv+BN folding
+def test_fold_batchnorm_identity_equivalence_and_float32_ops():
+    c, k = 7, 33
+    w = RNG.standard_normal((c, k)).astype(np.float32); b = RNG.standard_normal(c).astype(np.float32)
+    one = np.ones(c, np.float32); zero = np.zeros(c, np.float32)
+    a, cc = oracle.fold_batchnorm(w, b, one, zero, zero, one)           # identity normalisation
+    assert np.array_equal(a, w) and np.array_equal(cc, b)
+    gamma = RNG.uniform(0.5, 2, c).astype(np.float32); beta = RNG.standard_normal(c).astype(np.float32)
+    mean = RNG.standard_normal(c).astype(np.float32); var = RNG.uniform(0.1, 3, c).astype(np.float32)
+    a, cc = oracle.fold_batchnorm(w, b, gamma, beta, mean, var)
+    # functional meaning (Eq. 10 = Eq. 11): BN(W x + B) == A x + C for any input x
+    x = RNG.standard_normal(k)
+    conv = w.astype(np.float64) @ x + b
+    bn = gamma * (conv - mean) / np.sqrt(var.astype(np.float64)) + beta
+    np.testing.assert_allclose(a.astype(np.float64) @ x + cc, bn, rtol=0, atol=5e-6)
+    # the same sequence of correctly rounded binary32 operations in numpy
+    s = gamma / np.sqrt(var)                                               # float32 sqrt and divide
+    assert np.array_equal(a, s[:, None] * w)
+    assert np.array_equal(cc, s * (b - mean) + beta)
+    a0, c0 = oracle.fold_batchnorm(w, None, gamma, beta, mean, var)        # no conv bias
+    assert np.array_equal(a0, a) and np.array_equal(c0, s * (zero - mean) + beta)
