@@ -224,3 +224,40 @@ def test_sweep_can_be_captured_in_a_cuda_graph_and_replayed():
         assert not torch.equal(t["mse"].view(torch.int64), ref["mse"].view(torch.int64))
     finally:
         gctx.close()
+
+
+def test_two_contexts_on_two_streams_do_not_interfere():
+    """The library keeps no global state besides per-kernel occupancy caches: two contexts, each on
+    its own stream, sweeping different models at the same time give the results each gives alone."""
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    c1, c2 = q.Context(0, stream=s1), q.Context(0, stream=s2)
+    try:
+        m1 = gen.make_model("squeezenet", seed=11, device="cuda", batch=2)
+        m2 = gen.make_model("resnet18", seed=12, device="cuda", batch=1)
+        torch.cuda.synchronize()
+        alone = []
+        for c, s, m in ((c1, s1, m1), (c2, s2, m2)):
+            with torch.cuda.stream(s):
+                md, t = run_sweep(c, m)
+            alone.append({k: t[k].clone() for k in ("mse", "sqnr_db", "order", "step", "clip")})
+        runs = []
+        for _ in range(3):                              # interleave launches of the two streams
+            with torch.cuda.stream(s1):
+                md1 = q.model_descs(m1); sb1, t1 = c1.alloc_sweep_buffers(md1.descs, md1.n_layers)
+            with torch.cuda.stream(s2):
+                md2 = q.model_descs(m2); sb2, t2 = c2.alloc_sweep_buffers(md2.descs, md2.n_layers)
+            torch.cuda.synchronize()
+            cfg1 = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md1.rate_permyriad)
+            cfg2 = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md2.rate_permyriad)
+            c1.sweep_model(md1.descs, md1.n_layers, md1.macs, None, cfg1, sb1)
+            c2.sweep_model(md2.descs, md2.n_layers, md2.macs, None, cfg2, sb2)
+            c1.sweep_model(md1.descs, md1.n_layers, md1.macs, None, cfg1, sb1)
+            c2.sweep_model(md2.descs, md2.n_layers, md2.macs, None, cfg2, sb2)
+            torch.cuda.synchronize()
+            runs.append((t1, t2))
+        for t1, t2 in runs:
+            for ref, t in ((alone[0], t1), (alone[1], t2)):
+                for k, v in ref.items():
+                    assert torch.equal(t[k].view(torch.uint8), v.view(torch.uint8)), k
+    finally:
+        c1.close(); c2.close()
