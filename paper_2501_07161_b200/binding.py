@@ -24,7 +24,8 @@ OK = 0
 EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_error",
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
-           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm"]
+           "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm", "qv2_sweep_graph_create", "qv2_sweep_graph_launch",
+           "qv2_sweep_graph_destroy"]
 KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
@@ -82,6 +83,11 @@ def lib() -> C.CDLL:
     L.qv2_rank_layers.restype = i32
     L.qv2_kl_divergence.argtypes = [vp, dp, u32, vp, vp, vp, vp, vp, vp]
     L.qv2_kl_divergence.restype = i32
+    L.qv2_sweep_graph_create.argtypes = [vp, dp, u32, u32, vp, vp, C.POINTER(RankCfg), C.POINTER(SweepBuffers),
+                                         C.POINTER(vp)]
+    L.qv2_sweep_graph_create.restype = i32
+    L.qv2_sweep_graph_launch.argtypes = [vp]; L.qv2_sweep_graph_launch.restype = i32
+    L.qv2_sweep_graph_destroy.argtypes = [vp]; L.qv2_sweep_graph_destroy.restype = i32
     L.qv2_fold_batchnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, u64, u64, vp, vp]
     L.qv2_fold_batchnorm.restype = i32
     L.qv2_rank_layers_ex.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(RankCfg), vp, vp, vp]
@@ -281,6 +287,13 @@ class Context:
         _check(lib().qv2_sweep_model(self._h, descs, len(descs), n_layers, _ptr(macs), _ptr(pos),
                                      C.byref(cfg), C.byref(bufs)), "qv2_sweep_model")
 
+    def sweep_graph(self, descs, n_layers: int, macs, pos, cfg: RankCfg, bufs: SweepBuffers) -> "SweepGraph":
+        """Captures the pass once (the context must be on a non-default stream)."""
+        h = C.c_void_p()
+        _check(lib().qv2_sweep_graph_create(self._h, descs, len(descs), n_layers, _ptr(macs), _ptr(pos),
+                                            C.byref(cfg), C.byref(bufs), C.byref(h)), "qv2_sweep_graph_create")
+        return SweepGraph(h, (descs, macs, pos, cfg, bufs))
+
     def sweep_model_host(self, host_descs, n_layers: int, macs_host, pos_host, cfg: RankCfg,
                          staging: torch.Tensor, bufs: SweepBuffers, out: HostResults) -> int:
         """Returns the status (OK or ERR_NONFINITE); other errors raise."""
@@ -303,6 +316,28 @@ def quant_metrics_noalloc(desc: TensorDesc, step: torch.Tensor, inv: torch.Tenso
     arr = (TensorDesc * 1)(desc)
     return int(lib().qv2_quant_metrics_noalloc(device, C.c_void_p(s.cuda_stream), arr, _ptr(step),
                                                _ptr(inv), _ptr(offset), _ptr(result4)))
+
+
+class SweepGraph:
+    """A captured pass; launch() replays it on the owning context's stream."""
+
+    def __init__(self, handle, keepalive):
+        self._h = handle
+        self._keep = keepalive
+
+    def launch(self):
+        _check(lib().qv2_sweep_graph_launch(self._h), "qv2_sweep_graph_launch")
+
+    def close(self):
+        if self._h:
+            lib().qv2_sweep_graph_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def staging_bytes(descs, n_layers: int) -> int:

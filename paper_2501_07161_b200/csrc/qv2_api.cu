@@ -401,3 +401,64 @@ extern "C" int qv2_sweep_model_host(qv2_ctx* c, const qv2_tensor_desc* descs, ui
     if (out->nonfinite[t]) return QV2_ERR_NONFINITE;
   return QV2_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// A whole pass captured once in a CUDA graph and replayed with one launch.
+struct qv2_graph {
+  qv2_ctx* ctx = nullptr;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  uint64_t launches_per_replay = 0;
+};
+
+extern "C" int qv2_sweep_graph_create(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n_tensors,
+                                      uint32_t n_layers, const uint64_t* macs, const double* pos,
+                                      const qv2_rank_cfg* cfg, const qv2_sweep_buffers* bufs,
+                                      qv2_graph** out) {
+  if (!out) return QV2_ERR_NULL;
+  *out = nullptr;
+  if (!c) return QV2_ERR_NULL;
+  if (c->stream == nullptr || c->stream == cudaStreamLegacy) return QV2_ERR_UNSUPPORTED;  // cannot be captured
+  DeviceGuard guard(c->device);
+  // First an ordinary pass: validates the arguments, makes the tile tables resident and sizes
+  // every scratch buffer, so that the captured pass allocates and uploads nothing.
+  const uint64_t before = c->launches;
+  int st = qv2_sweep_model(c, descs, n_tensors, n_layers, macs, pos, cfg, bufs);
+  if (st != QV2_OK) return st;
+  const uint64_t per_pass = c->launches - before;
+  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  qv2_graph* g = new (std::nothrow) qv2_graph();
+  if (!g) return QV2_ERR_NOMEM;
+  g->ctx = c; g->launches_per_replay = per_pass;
+  cudaError_t e = cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal);
+  if (e != cudaSuccess) { delete g; return cuda_fail(c, e); }
+  st = qv2_sweep_model(c, descs, n_tensors, n_layers, macs, pos, cfg, bufs);
+  c->launches -= (st == QV2_OK) ? per_pass : 0;        // captured, not executed
+  e = cudaStreamEndCapture(c->stream, &g->graph);
+  if (st != QV2_OK || e != cudaSuccess || !g->graph) {
+    if (g->graph) cudaGraphDestroy(g->graph);
+    delete g;
+    return st != QV2_OK ? st : cuda_fail(c, e != cudaSuccess ? e : cudaErrorUnknown);
+  }
+  e = cudaGraphInstantiate(&g->exec, g->graph, 0);
+  if (e != cudaSuccess) { cudaGraphDestroy(g->graph); delete g; return cuda_fail(c, e); }
+  *out = g;
+  return QV2_OK;
+}
+
+extern "C" int qv2_sweep_graph_launch(qv2_graph* g) {
+  if (!g || !g->ctx || !g->exec) return QV2_ERR_NULL;
+  DeviceGuard guard(g->ctx->device);
+  QV2_CUDA(g->ctx, cudaGraphLaunch(g->exec, g->ctx->stream));
+  g->ctx->launches += g->launches_per_replay;
+  return QV2_OK;
+}
+
+extern "C" int qv2_sweep_graph_destroy(qv2_graph* g) {
+  if (!g) return QV2_ERR_NULL;
+  if (g->ctx) { DeviceGuard guard(g->ctx->device); cudaStreamSynchronize(g->ctx->stream); }
+  if (g->exec) cudaGraphExecDestroy(g->exec);
+  if (g->graph) cudaGraphDestroy(g->graph);
+  delete g;
+  return QV2_OK;
+}

@@ -261,3 +261,42 @@ def test_two_contexts_on_two_streams_do_not_interfere():
                     assert torch.equal(t[k].view(torch.uint8), v.view(torch.uint8)), k
     finally:
         c1.close(); c2.close()
+
+
+def test_library_sweep_graph_replays_the_pass():
+    """qv2_sweep_graph_create / _launch: same bits as the ordinary call, new inputs picked up in
+    place, and the default-stream context is refused."""
+    s = torch.cuda.Stream()
+    gctx = q.Context(0, stream=s)
+    dctx = q.Context(0)                                   # torch's default stream: cannot be captured
+    try:
+        model = gen.make_model("squeezenet", seed=8, device="cuda", batch=1)
+        md = q.model_descs(model)
+        cfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s):
+            sb, t = gctx.alloc_sweep_buffers(md.descs, md.n_layers)
+            sb_ref, t_ref = gctx.alloc_sweep_buffers(md.descs, md.n_layers)
+            gctx.sweep_model(md.descs, md.n_layers, md.macs, None, cfg, sb_ref)
+            g = gctx.sweep_graph(md.descs, md.n_layers, md.macs, None, cfg, sb)
+            n0 = gctx.launches
+            for k in ("mse", "sqnr_db", "order", "hist"):
+                t[k].zero_()
+            g.launch()
+            s.synchronize()
+            assert gctx.launches - n0 == 7
+            for k in ("mse", "sqnr_db", "order", "keep_fp32", "n_keep", "step", "hist", "clip"):
+                assert torch.equal(t[k].view(torch.uint8), t_ref[k].view(torch.uint8)), k
+            model.layers[5].x.mul_(0.5)                   # refill a tensor in place
+            g.launch(); g.launch()
+            gctx.sweep_model(md.descs, md.n_layers, md.macs, None, cfg, sb_ref)
+            s.synchronize()
+            assert torch.equal(t["mse"].view(torch.int64), t_ref["mse"].view(torch.int64))
+            g.close()
+        sb2, _ = dctx.alloc_sweep_buffers(md.descs, md.n_layers)
+        if torch.cuda.current_stream().cuda_stream == 0:
+            with pytest.raises(q.binding.Qv2Error) as e:
+                dctx.sweep_graph(md.descs, md.n_layers, md.macs, None, cfg, sb2)
+            assert e.value.status == -8
+    finally:
+        gctx.close(); dctx.close()
