@@ -178,9 +178,13 @@ class Context:
         self.device = torch.device("cuda", device)
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
         self.stream = s
+        self._graphs = []          # captured passes must be destroyed before their context
         _check(lib().qv2_create(C.byref(self._h), device, C.c_void_p(s.cuda_stream)), "qv2_create")
 
     def close(self):
+        for g in getattr(self, "_graphs", []):
+            g.close()
+        self._graphs = []
         if self._h:
             lib().qv2_destroy(self._h)
             self._h = C.c_void_p()
@@ -292,7 +296,9 @@ class Context:
         h = C.c_void_p()
         _check(lib().qv2_sweep_graph_create(self._h, descs, len(descs), n_layers, _ptr(macs), _ptr(pos),
                                             C.byref(cfg), C.byref(bufs), C.byref(h)), "qv2_sweep_graph_create")
-        return SweepGraph(h, (descs, macs, pos, cfg, bufs))
+        g = SweepGraph(h, (descs, macs, pos, cfg, bufs))
+        self._graphs.append(g)
+        return g
 
     def sweep_model_host(self, host_descs, n_layers: int, macs_host, pos_host, cfg: RankCfg,
                          staging: torch.Tensor, bufs: SweepBuffers, out: HostResults) -> int:
