@@ -164,6 +164,15 @@ int qv2_calibrate(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
                   uint64_t* nonfinite);
 
 /*
+ * Turns the device-side non-finite counters of qv2_calibrate into a status: synchronises the
+ * context's stream, reads nonfinite[0..n) (device) and returns QV2_ERR_NONFINITE if any tensor
+ * held a NaN or Inf (first_bad, host, nullable, receives the index of the first such tensor),
+ * else QV2_OK.  The other calls never synchronise for this; data errors are reported only here
+ * and by qv2_sweep_model_host.
+ */
+int qv2_check_nonfinite(qv2_ctx* ctx, const uint64_t* nonfinite, uint32_t n, uint32_t* first_bad);
+
+/*
  * Fused fake-quantize + error reduction: step 3 of the overview ("measure the SQNR and MSE of each
  * layer by comparing the weights and activations of the original and quantized models"), i.e.
  * CalculateSQNR / CalculateMSE of Algorithm 2 over every element, with the quantizer of Eq. 1 / Eq. 5

@@ -25,7 +25,7 @@ EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_erro
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
            "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm", "qv2_sweep_graph_create", "qv2_sweep_graph_launch",
-           "qv2_sweep_graph_destroy"]
+           "qv2_sweep_graph_destroy", "qv2_check_nonfinite"]
 KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
     L.qv2_rank_layers.restype = i32
     L.qv2_kl_divergence.argtypes = [vp, dp, u32, vp, vp, vp, vp, vp, vp]
     L.qv2_kl_divergence.restype = i32
+    L.qv2_check_nonfinite.argtypes = [vp, vp, u32, C.POINTER(u32)]; L.qv2_check_nonfinite.restype = i32
     L.qv2_sweep_graph_create.argtypes = [vp, dp, u32, u32, vp, vp, C.POINTER(RankCfg), C.POINTER(SweepBuffers),
                                          C.POINTER(vp)]
     L.qv2_sweep_graph_create.restype = i32
@@ -251,6 +252,14 @@ class Context:
                                        _ptr(out.sse), _ptr(out.sig), _ptr(out.mse), _ptr(out.sqnr_db)),
                "qv2_quant_metrics")
         return out
+
+    def check_nonfinite(self, nonfinite: torch.Tensor):
+        """-> (status, index of the first tensor with NaN/Inf or None); synchronises the stream."""
+        bad = C.c_uint32(0xFFFFFFFF)
+        st = int(lib().qv2_check_nonfinite(self._h, _ptr(nonfinite), nonfinite.numel(), C.byref(bad)))
+        if st not in (OK, -5):
+            raise Qv2Error(st, "qv2_check_nonfinite")
+        return st, (int(bad.value) if st == -5 else None)
 
     def fold_batchnorm(self, w, bias, gamma, beta, mean, var):
         """Eq. 10-12: -> (folded weights [C, K], folded bias [C])."""

@@ -274,6 +274,19 @@ extern "C" int qv2_kl_divergence(qv2_ctx* c, const qv2_tensor_desc* descs, uint3
   return QV2_OK;
 }
 
+extern "C" int qv2_check_nonfinite(qv2_ctx* c, const uint64_t* nonfinite, uint32_t n, uint32_t* first_bad) {
+  if (!c || !nonfinite) return QV2_ERR_NULL;
+  if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
+  DeviceGuard guard(c->device);
+  std::vector<uint64_t> host(n);
+  QV2_CUDA(c, cudaMemcpyAsync(host.data(), nonfinite, (size_t)n * sizeof(uint64_t), cudaMemcpyDeviceToHost,
+                              c->stream));
+  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  for (uint32_t t = 0; t < n; ++t)
+    if (host[t]) { if (first_bad) *first_bad = t; return QV2_ERR_NONFINITE; }
+  return QV2_OK;
+}
+
 extern "C" int qv2_fold_batchnorm(qv2_ctx* c, const float* w, const float* bias, const float* gamma,
                                   const float* beta, const float* mean, const float* var,
                                   uint64_t channels, uint64_t inner, float* w_out, float* bias_out) {

@@ -130,6 +130,8 @@ def test_nonfinite_inputs_are_counted_and_excluded(ctx):
                                Spec(w, 1, 40, 300, per_channel=True),
                                Spec(randn(1000, 33), 1, 1, 1000)], check_codes=False)
     assert cal.nonfinite.tolist() == [5, 2, 0]
+    assert ctx.check_nonfinite(cal.nonfinite) == (-5, 0)
+    assert ctx.check_nonfinite(cal.nonfinite[2:]) == (0, None)
 
 
 def test_extreme_magnitudes(ctx):
