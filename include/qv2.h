@@ -59,6 +59,15 @@ enum { QV2_BY_COUNT = 0, QV2_BY_BOPS_RATE = 1 };             /* select_mode */
  * largest code is 2^(b-1) - 1 for QV2_SYM_I8 (Eq. 4) and 2^b - 1 for QV2_ASYM_U8 (Eq. 2 with
  * N = 2^b levels); wherever this header says 127 or 255 read that value.  No QV2_BITS means 8.
  * QV2_STORE_CODES needs b <= 8 (codes are one byte), else QV2_ERR_UNSUPPORTED. */
+/* Element type of the tensors x and y, OR-ed into flags.  The default is binary32.  With
+ * QV2_IN_F16 / QV2_IN_BF16 the pointers x and y (declared const float* for the ABI) address
+ * IEEE binary16 / bfloat16 data, 2-byte aligned; every value is widened exactly to binary32 and
+ * all arithmetic is as documented for binary32, so the pass moves half the bytes.  Not accepted
+ * by qv2_quant_metrics_noalloc. */
+#define QV2_IN_F32 0u
+#define QV2_IN_F16 (1u << 16)
+#define QV2_IN_BF16 (2u << 16)
+#define QV2_IN_MASK (3u << 16)
 #define QV2_BITS(b) ((uint32_t)(b) << 8)
 #define QV2_BITS_MASK 0xFF00u
 #define QV2_DESC_BITS(flags) (((flags) & QV2_BITS_MASK) ? (((uint32_t)(flags) & QV2_BITS_MASK) >> 8) : 8u)

@@ -19,6 +19,8 @@ constexpr int kBins = QV2_HIST_BINS;
 constexpr uint32_t kMaxRankLayers = 8192;
 
 enum PairMode : uint32_t { kSelf = 0, kRequant = 1, kRaw = 2 };
+enum DType : uint32_t { kF32 = 0, kF16 = 1, kBF16 = 2 };
+inline uint32_t dtype_size(uint32_t dtype) { return dtype == kF32 ? 4u : 2u; }
 
 // One tensor, as the kernels see it.
 struct TensorRec {
@@ -40,6 +42,7 @@ struct TensorRec {
   uint32_t rslot_first;      // per-tensor tensors: first {min,max} key slot written by the range kernel,
   uint32_t rslot_count;      //   one per CTA of the range grid that owns a tile of the tensor
   uint32_t bits;             // code width, 2..16 (8 unless the descriptor asks otherwise)
+  uint32_t dtype;            // element type of x and y: 0 binary32, 1 binary16, 2 bfloat16
   double percentile;
 };
 

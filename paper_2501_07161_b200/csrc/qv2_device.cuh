@@ -2,6 +2,9 @@
 // a flat element run into an aligned 16-byte body with scalar head/tail, and warp reductions.
 #pragma once
 
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include "qv2_common.cuh"
 
 namespace qv2 {
@@ -20,6 +23,45 @@ __device__ __forceinline__ float ld_stream1(const float* p) {
   return v;
 }
 
+// Element access by type: four consecutive elements widened to binary32 (the address must be a
+// multiple of four elements), or one element.  binary16 and bfloat16 widen exactly.
+template <class T> struct Ld;
+template <> struct Ld<float> {
+  static __device__ __forceinline__ float4 vec(const float* p) { return ld_stream4(reinterpret_cast<const float4*>(p)); }
+  static __device__ __forceinline__ float one(const float* p) { return ld_stream1(p); }
+};
+__device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
+  uint2 v;
+  asm("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ unsigned short ld_stream_u16(const void* p) {
+  unsigned short v;
+  asm("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
+  return v;
+}
+template <> struct Ld<__half> {
+  static __device__ __forceinline__ float4 vec(const __half* p) {
+    const uint2 r = ld_stream_u2(p);
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&r.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&r.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+  static __device__ __forceinline__ float one(const __half* p) {
+    return __half2float(__ushort_as_half(ld_stream_u16(p)));
+  }
+};
+template <> struct Ld<__nv_bfloat16> {      // a bfloat16 is the upper half of a binary32
+  static __device__ __forceinline__ float4 vec(const __nv_bfloat16* p) {
+    const uint2 r = ld_stream_u2(p);
+    return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u),
+                       __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
+  }
+  static __device__ __forceinline__ float one(const __nv_bfloat16* p) {
+    return __uint_as_float((uint32_t)ld_stream_u16(p) << 16);
+  }
+};
+
 __device__ __forceinline__ Tile load_tile(const Tile* tiles, uint32_t i) {
   const uint4* p = reinterpret_cast<const uint4*>(tiles + i);
   uint4 a = __ldg(p), b = __ldg(p + 1);
@@ -30,14 +72,15 @@ __device__ __forceinline__ Tile load_tile(const Tile* tiles, uint32_t i) {
   return t;
 }
 
-// A flat run [p, p+count): `head` scalars up to the first 16-byte boundary, `nvec` float4, `tail`
-// scalars.
+// A flat run [p, p+count): `head` scalars up to the first address that is a multiple of four
+// elements (16 bytes of binary32, 8 of the 16-bit types), `nvec` groups of four, `tail` scalars.
 struct FlatSplit {
   uint32_t head, nvec, tail;
 };
-__device__ __forceinline__ FlatSplit split_flat(const float* p, uint32_t count) {
+template <class T>
+__device__ __forceinline__ FlatSplit split_flat(const T* p, uint32_t count) {
   FlatSplit s;
-  uint32_t mis = (uint32_t)(((uintptr_t)p >> 2) & 3u);     // elements past a 16-byte boundary
+  uint32_t mis = (uint32_t)(((uintptr_t)p / sizeof(T)) & 3u);   // elements past a 4-element boundary
   uint32_t head = (4u - mis) & 3u;
   s.head = head < count ? head : count;
   s.nvec = (count - s.head) >> 2;

@@ -33,7 +33,9 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     const qv2_tensor_desc& d = descs[t];
     if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE)
       return QV2_ERR_ARG;
-    if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_STORE_CODES | QV2_BITS_MASK)) return QV2_ERR_ARG;
+    if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_STORE_CODES | QV2_BITS_MASK | QV2_IN_MASK)) return QV2_ERR_ARG;
+    const uint32_t dtype = (d.flags & QV2_IN_MASK) >> 16;
+    if (dtype > kBF16) return QV2_ERR_ARG;
     const uint32_t bits = QV2_DESC_BITS(d.flags);
     if (bits < 2 || bits > 16) return QV2_ERR_ARG;
     if ((d.flags & QV2_STORE_CODES) && bits > 8) return QV2_ERR_UNSUPPORTED;   // codes are one byte
@@ -44,7 +46,8 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     if (mul_overflows(rows, d.inner, &ne) || ne > (1ull << 62)) return QV2_ERR_SIZE;
     if (d.channels >= (1ull << 32)) return QV2_ERR_SIZE;
     if (ne > 0 && !d.x) return QV2_ERR_NULL;
-    if (((uintptr_t)d.x & 3u) || ((uintptr_t)d.y & 3u)) return QV2_ERR_ALIGN;
+    const uintptr_t amask = dtype_size(dtype) - 1u;
+    if (((uintptr_t)d.x & amask) || ((uintptr_t)d.y & amask)) return QV2_ERR_ALIGN;
     bool pair = d.y != nullptr;
     if ((d.flags & QV2_PAIR_RAW) && !pair) return QV2_ERR_ARG;
 
@@ -63,6 +66,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     r.pair_mode = !pair ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
     r.percentile = d.percentile;
     r.bits = bits;
+    r.dtype = dtype;
 
     size_t first_tile = out->tiles.size();
     if (d.range == QV2_PERCENTILE) out->any_percentile = true;

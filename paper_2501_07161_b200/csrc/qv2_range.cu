@@ -35,38 +35,38 @@ __device__ __forceinline__ void range_acc4(RangeAcc& a, const float4& v) {
   range_acc<CAREFUL>(a, v.z); range_acc<CAREFUL>(a, v.w);
 }
 
-// This thread's share of a flat run: float4 number j for j = tid, tid+256, ...; the first
-// `head` and last `tail` scalars go to threads 0..2.
-template <bool CAREFUL>
-__device__ __forceinline__ void range_flat(const float* __restrict__ x, uint32_t count, RangeAcc& a) {
+// This thread's share of a flat run: group of four number j for j = tid, tid+256, ...; the first
+// `head` and last `tail` scalars go to threads 0..2.  T is the element type in memory.
+template <bool CAREFUL, class T>
+__device__ __forceinline__ void range_flat(const T* __restrict__ x, uint32_t count, RangeAcc& a) {
   const FlatSplit s = split_flat(x, count);
-  const float4* xv = reinterpret_cast<const float4*>(x + s.head);
-  constexpr uint32_t U = 8;
+  const T* xv = x + s.head;
+  constexpr uint32_t U = sizeof(T) == 4 ? 8 : 16;       // the same bytes in flight for 16-bit types
   uint32_t j = threadIdx.x;
   for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
     float4 v[U];
 #pragma unroll
-    for (uint32_t u = 0; u < U; ++u) v[u] = ld_stream4(xv + j + u * kThreads);
+    for (uint32_t u = 0; u < U; ++u) v[u] = Ld<T>::vec(xv + 4u * (j + u * kThreads));
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) range_acc4<CAREFUL>(a, v[u]);
   }
-  for (; j < s.nvec; j += kThreads) range_acc4<CAREFUL>(a, ld_stream4(xv + j));
-  if (threadIdx.x < s.head) range_acc<CAREFUL>(a, ld_stream1(x + threadIdx.x));
-  if (threadIdx.x < s.tail) range_acc<CAREFUL>(a, ld_stream1(x + s.head + 4u * s.nvec + threadIdx.x));
+  for (; j < s.nvec; j += kThreads) range_acc4<CAREFUL>(a, Ld<T>::vec(xv + 4u * j));
+  if (threadIdx.x < s.head) range_acc<CAREFUL>(a, Ld<T>::one(x + threadIdx.x));
+  if (threadIdx.x < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(x + s.head + 4u * s.nvec + threadIdx.x));
 }
 
 // One row handled by one warp: lanes stride over the row.
-template <bool CAREFUL>
-__device__ __forceinline__ void range_row(const float* __restrict__ row, uint32_t inner, uint32_t lane,
+template <bool CAREFUL, class T>
+__device__ __forceinline__ void range_row(const T* __restrict__ row, uint32_t inner, uint32_t lane,
                                           RangeAcc& a) {
   uint32_t i = lane;
   for (; i + 96 < inner; i += 128) {
-    float v0 = ld_stream1(row + i), v1 = ld_stream1(row + i + 32), v2 = ld_stream1(row + i + 64),
-          v3 = ld_stream1(row + i + 96);
+    float v0 = Ld<T>::one(row + i), v1 = Ld<T>::one(row + i + 32), v2 = Ld<T>::one(row + i + 64),
+          v3 = Ld<T>::one(row + i + 96);
     range_acc<CAREFUL>(a, v0); range_acc<CAREFUL>(a, v1);
     range_acc<CAREFUL>(a, v2); range_acc<CAREFUL>(a, v3);
   }
-  for (; i < inner; i += 32) range_acc<CAREFUL>(a, ld_stream1(row + i));
+  for (; i < inner; i += 32) range_acc<CAREFUL>(a, Ld<T>::one(row + i));
 }
 
 __device__ __forceinline__ void reset(RangeAcc& a) {
@@ -84,6 +84,38 @@ __device__ __forceinline__ void publish(RangeAcc& a, uint32_t lane, uint32_t* km
       atomicMax(kmin + group, ~f2key(mn));
     }
     if (bad) atomicAdd(nonfinite_t, (unsigned long long)bad);
+  }
+}
+
+// One flat tile into the running accumulator; a warp that meets a NaN or Inf redoes its share
+// of the tile with exact per-element checks.
+template <class T>
+__device__ __forceinline__ void range_flat_tile(const T* x, uint32_t count, RangeAcc& a) {
+  const float mn0 = a.mn, mx0 = a.mx;
+  range_flat<false>(x, count, a);
+  if (__any_sync(0xffffffffu, a.nanflag != a.nanflag)) {
+    a.mn = mn0; a.mx = mx0; a.nanflag = 0.0f;
+    range_flat<true>(x, count, a);
+  }
+}
+
+// A tile of whole short rows: one warp per row, one publication per row.
+template <class T>
+__device__ __forceinline__ void range_rows_tile(const T* x, const Tile& tl, const TensorRec* tr, uint32_t lane,
+                                                uint32_t warp, uint32_t* kmin, uint32_t* kmax,
+                                                unsigned long long* nonfinite) {
+  const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+  RangeAcc b;
+  for (uint32_t r = warp; r < tl.rows; r += kWarps) {
+    const T* row = x + (uint64_t)r * inner;
+    reset(b);
+    range_row<false>(row, inner, lane, b);
+    if (__any_sync(0xffffffffu, b.nanflag != b.nanflag)) {
+      reset(b);
+      range_row<true>(row, inner, lane, b);
+    }
+    const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
+    publish(b, lane, kmin, kmax, tr->group_base + g, nonfinite + tl.tensor);
   }
 }
 
@@ -126,7 +158,6 @@ range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ til
   for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile tl = load_tile(tiles, ti);
     const TensorRec* tr = tensors + tl.tensor;
-    const float* x = tr->x + tl.begin;
     const uint32_t gbase = tr->group_base;
     if (tl.rows == 0) {
       const uint32_t G = gbase + (uint32_t)tl.row0;
@@ -138,26 +169,16 @@ range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ til
         reset(a);
         cur_group = G; cur_tensor = tl.tensor; cur_slot = tr->per_channel == 0;
       }
-      const float mn0 = a.mn, mx0 = a.mx;
-      range_flat<false>(x, tl.count, a);
-      if (__any_sync(0xffffffffu, a.nanflag != a.nanflag)) {   // redo this warp's share carefully
-        a.mn = mn0; a.mx = mx0; a.nanflag = 0.0f;
-        range_flat<true>(x, tl.count, a);
-      }
+      if (tr->dtype == kF32) range_flat_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, a);
+      else if (tr->dtype == kF16) range_flat_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, a);
+      else range_flat_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, a);
     } else {
-      const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
-      RangeAcc b;
-      for (uint32_t r = warp; r < tl.rows; r += kWarps) {
-        const float* row = x + (uint64_t)r * inner;
-        reset(b);
-        range_row<false>(row, inner, lane, b);
-        if (__any_sync(0xffffffffu, b.nanflag != b.nanflag)) {
-          reset(b);
-          range_row<true>(row, inner, lane, b);
-        }
-        const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
-        publish(b, lane, kmin, kmax, gbase + g, nonfinite + tl.tensor);
-      }
+      if (tr->dtype == kF32)
+        range_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
+      else if (tr->dtype == kF16)
+        range_rows_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
+      else
+        range_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
     }
   }
   if (cur_group != kNone) {
