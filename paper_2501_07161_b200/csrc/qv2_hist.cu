@@ -27,17 +27,17 @@ __device__ __forceinline__ void hist_elem(float v, float w, uint32_t* sh, uint32
   else atomicAdd(sh + b, 1u);
 }
 
-template <bool CAREFUL>
-__device__ __forceinline__ void hist_flat(const float* __restrict__ x, uint32_t count, float w,
+template <bool CAREFUL, class T>
+__device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t count, float w,
                                           uint32_t* sh, uint32_t& zeros) {
   const FlatSplit s = split_flat(x, count);
-  const float4* xv = reinterpret_cast<const float4*>(x + s.head);
+  const T* xv = x + s.head;
   constexpr uint32_t U = 4;
   uint32_t j = threadIdx.x;
   for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
     float4 v[U];
 #pragma unroll
-    for (uint32_t u = 0; u < U; ++u) v[u] = ld_stream4(xv + j + u * kThreads);
+    for (uint32_t u = 0; u < U; ++u) v[u] = Ld<T>::vec(xv + 4u * (j + u * kThreads));
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) {
       hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
@@ -45,13 +45,20 @@ __device__ __forceinline__ void hist_flat(const float* __restrict__ x, uint32_t 
     }
   }
   for (; j < s.nvec; j += kThreads) {
-    const float4 v = ld_stream4(xv + j);
+    const float4 v = Ld<T>::vec(xv + 4u * j);
     hist_elem<CAREFUL>(v.x, w, sh, zeros); hist_elem<CAREFUL>(v.y, w, sh, zeros);
     hist_elem<CAREFUL>(v.z, w, sh, zeros); hist_elem<CAREFUL>(v.w, w, sh, zeros);
   }
-  if (threadIdx.x < s.head) hist_elem<CAREFUL>(ld_stream1(x + threadIdx.x), w, sh, zeros);
+  if (threadIdx.x < s.head) hist_elem<CAREFUL>(Ld<T>::one(x + threadIdx.x), w, sh, zeros);
   if (threadIdx.x < s.tail)
-    hist_elem<CAREFUL>(ld_stream1(x + s.head + 4u * s.nvec + threadIdx.x), w, sh, zeros);
+    hist_elem<CAREFUL>(Ld<T>::one(x + s.head + 4u * s.nvec + threadIdx.x), w, sh, zeros);
+}
+
+template <class T>
+__device__ __forceinline__ void hist_tile(const T* x, uint32_t count, float w, bool careful, uint32_t* sh,
+                                          uint32_t& zeros) {
+  if (careful) hist_flat<true>(x, count, w, sh, zeros);
+  else hist_flat<false>(x, count, w, sh, zeros);
 }
 
 __global__ void __launch_bounds__(kThreads, 4)
@@ -91,9 +98,10 @@ hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tile
       if (!isfinite(w)) w = 0.0f;
       careful = nonfinite[cur] != 0ull;
     }
-    const float* x = tensors[cur].x + tl.begin;
-    if (careful) hist_flat<true>(x, tl.count, w, sh, zeros);
-    else hist_flat<false>(x, tl.count, w, sh, zeros);
+    const TensorRec* tr = tensors + cur;
+    if (tr->dtype == kF32) hist_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+    else if (tr->dtype == kF16) hist_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+    else hist_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
     ++since_flush;
   }
 }
