@@ -91,62 +91,61 @@ __device__ __forceinline__ void metric_vec(const float4& x, const float4& y, con
   metric_elem<MODE, OFF, CODES>(x.w, y.w, p, a[3], code + 3);
 }
 
-// This thread's share of a flat one-group run.  `vec_y` says y has the same 16-byte phase as x.
-template <uint32_t MODE, bool OFF, bool CODES, class ACC>
-__device__ __forceinline__ void metric_flat(const float* __restrict__ x, const float* __restrict__ y,
+// This thread's share of a flat one-group run.  T is the element type of x and y in memory;
+// `vec_y` says y has the same phase as x inside its group of four elements.
+template <uint32_t MODE, bool OFF, bool CODES, class ACC, class T>
+__device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __restrict__ y,
                                             uint8_t* codes, uint32_t count, const QP& p, ACC* a) {
   constexpr bool PAIR = MODE != kSelf;
   const FlatSplit s = split_flat(x, count);
-  const float* xb = x + s.head;
-  const float* yb = PAIR ? y + s.head : nullptr;
+  const T* xb = x + s.head;
+  const T* yb = PAIR ? y + s.head : nullptr;
   uint8_t* cb = CODES ? codes + s.head : nullptr;
-  const bool vec_y = !PAIR || ((((uintptr_t)yb) & 15u) == 0);
-  const float4* xv = reinterpret_cast<const float4*>(xb);
+  const bool vec_y = !PAIR || ((((uintptr_t)yb) & (4u * sizeof(T) - 1u)) == 0);
   uint32_t j = threadIdx.x;
   if (vec_y) {
-    const float4* yv = reinterpret_cast<const float4*>(yb);
     constexpr uint32_t U = PAIR ? 4 : 8;
     for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
       float4 vx[U], vy[U];
 #pragma unroll
       for (uint32_t u = 0; u < U; ++u) {
-        vx[u] = ld_stream4(xv + j + u * kThreads);
-        if (PAIR) vy[u] = ld_stream4(yv + j + u * kThreads); else vy[u] = vx[u];
+        vx[u] = Ld<T>::vec(xb + 4u * (j + u * kThreads));
+        if (PAIR) vy[u] = Ld<T>::vec(yb + 4u * (j + u * kThreads)); else vy[u] = vx[u];
       }
 #pragma unroll
       for (uint32_t u = 0; u < U; ++u)
         metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * kThreads) : nullptr);
     }
     for (; j < s.nvec; j += kThreads) {
-      const float4 vx = ld_stream4(xv + j);
-      const float4 vy = PAIR ? ld_stream4(yv + j) : vx;
+      const float4 vx = Ld<T>::vec(xb + 4u * j);
+      const float4 vy = PAIR ? Ld<T>::vec(yb + 4u * j) : vx;
       metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
     }
   } else {
-    // x and y sit at different offsets inside their 16-byte lines: vector loads for x, scalar for y
+    // x and y sit at different offsets inside their groups of four: vector loads for x, scalar for y
     for (; j < s.nvec; j += kThreads) {
-      const float4 vx = ld_stream4(xv + j);
+      const float4 vx = Ld<T>::vec(xb + 4u * j);
       float4 vy;
-      vy.x = ld_stream1(yb + 4u * j); vy.y = ld_stream1(yb + 4u * j + 1);
-      vy.z = ld_stream1(yb + 4u * j + 2); vy.w = ld_stream1(yb + 4u * j + 3);
+      vy.x = Ld<T>::one(yb + 4u * j); vy.y = Ld<T>::one(yb + 4u * j + 1);
+      vy.z = Ld<T>::one(yb + 4u * j + 2); vy.w = Ld<T>::one(yb + 4u * j + 3);
       metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
     }
   }
   if (threadIdx.x < s.head) {
     const uint32_t i = threadIdx.x;
-    metric_elem<MODE, OFF, CODES>(ld_stream1(x + i), PAIR ? ld_stream1(y + i) : 0.0f, p, a[0],
+    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[0],
                                   CODES ? codes + i : nullptr);
   }
   if (threadIdx.x < s.tail) {
     const uint32_t i = s.head + 4u * s.nvec + threadIdx.x;
-    metric_elem<MODE, OFF, CODES>(ld_stream1(x + i), PAIR ? ld_stream1(y + i) : 0.0f, p, a[1],
+    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[1],
                                   CODES ? codes + i : nullptr);
   }
 }
 
 // One row handled by one warp.
-template <uint32_t MODE, bool OFF, bool CODES, class ACC>
-__device__ __forceinline__ void metric_row(const float* __restrict__ x, const float* __restrict__ y,
+template <uint32_t MODE, bool OFF, bool CODES, class ACC, class T>
+__device__ __forceinline__ void metric_row(const T* __restrict__ x, const T* __restrict__ y,
                                            uint8_t* codes, uint32_t inner, uint32_t lane, const QP& p,
                                            ACC* a) {
   constexpr bool PAIR = MODE != kSelf;
@@ -155,25 +154,25 @@ __device__ __forceinline__ void metric_row(const float* __restrict__ x, const fl
     float vx[4], vy[4];
 #pragma unroll
     for (uint32_t u = 0; u < 4; ++u) {
-      vx[u] = ld_stream1(x + i + 32u * u);
-      vy[u] = PAIR ? ld_stream1(y + i + 32u * u) : 0.0f;
+      vx[u] = Ld<T>::one(x + i + 32u * u);
+      vy[u] = PAIR ? Ld<T>::one(y + i + 32u * u) : 0.0f;
     }
 #pragma unroll
     for (uint32_t u = 0; u < 4; ++u)
       metric_elem<MODE, OFF, CODES>(vx[u], vy[u], p, a[u], CODES ? codes + i + 32u * u : nullptr);
   }
   for (; i < inner; i += 32)
-    metric_elem<MODE, OFF, CODES>(ld_stream1(x + i), PAIR ? ld_stream1(y + i) : 0.0f, p, a[0],
+    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[0],
                                   CODES ? codes + i : nullptr);
 }
 
-template <uint32_t MODE, bool CODES, class ACC>
-__device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
-                                            const float* __restrict__ step, const float* __restrict__ inv,
-                                            const float* __restrict__ offset, ACC* a) {
+template <uint32_t MODE, bool CODES, class T, class ACC>
+__device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRec* tr,
+                                                  const float* __restrict__ step, const float* __restrict__ inv,
+                                                  const float* __restrict__ offset, ACC* a) {
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-  const float* x = tr->x + tl.begin;
-  const float* y = (MODE != kSelf) ? tr->y + tl.begin : nullptr;
+  const T* x = reinterpret_cast<const T*>(tr->x) + tl.begin;
+  const T* y = (MODE != kSelf) ? reinterpret_cast<const T*>(tr->y) + tl.begin : nullptr;
   uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
   QP p;
   const float top = top_code(tr->asym != 0, tr->bits);
@@ -202,6 +201,16 @@ __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
         metric_row<MODE, true, CODES>(x + o, y + o, codes + o, inner, lane, p, a);
     }
   }
+}
+
+// Dispatch on the element type of the tensor.
+template <uint32_t MODE, bool CODES, class ACC>
+__device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
+                                            const float* __restrict__ step, const float* __restrict__ inv,
+                                            const float* __restrict__ offset, ACC* a) {
+  if (tr->dtype == kF32) metric_tile_typed<MODE, CODES, float>(tl, tr, step, inv, offset, a);
+  else if (tr->dtype == kF16) metric_tile_typed<MODE, CODES, __half>(tl, tr, step, inv, offset, a);
+  else metric_tile_typed<MODE, CODES, __nv_bfloat16>(tl, tr, step, inv, offset, a);
 }
 
 // Slot of (tensor, CTA, warp): the CTAs that own tiles of a tensor are numbered in the order of
@@ -611,6 +620,7 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   job.tr.percentile = d.percentile;
   job.tr.rslot_first = 0; job.tr.rslot_count = 0;
   job.tr.bits = QV2_DESC_BITS(d.flags);
+  job.tr.dtype = kF32;                  // this entry point takes binary32 tensors only
   job.rows = rows; job.tiles_per_row = 1; job.rows_per_tile = 1;
   uint64_t n_tiles;
   if (!job.tr.per_channel || ne == 0) {
