@@ -18,6 +18,8 @@ SYM_I8, ASYM_U8, ASYM_U8_ZP = 0, 1, 2
 ABSMAX, MINMAX, PERCENTILE = 0, 1, 2
 PAIR_REQUANT, PAIR_RAW, STORE_CODES = 0, 1, 2
 BY_COUNT, BY_BOPS_RATE = 0, 1
+IN_F32, IN_F16, IN_BF16 = 0, 1 << 16, 2 << 16
+_DTYPE_FLAG = {torch.float32: IN_F32, torch.float16: IN_F16, torch.bfloat16: IN_BF16}
 HIST_BINS = 2048
 OK = 0
 
@@ -126,6 +128,10 @@ def make_desc(x: Optional[torch.Tensor], y: Optional[torch.Tensor], outer: int, 
               inner: int, granularity: int, scheme: int, range_mode: int = ABSMAX,
               percentile: float = 0.0, flags: int = 0, bits: int = 8) -> TensorDesc:
     d = TensorDesc()
+    if x is not None:                     # the element type travels in the flags
+        if x.dtype not in _DTYPE_FLAG or (y is not None and y.dtype != x.dtype):
+            raise TypeError("x and y must both be float32, float16 or bfloat16")
+        flags |= _DTYPE_FLAG[x.dtype]
     d.x = _ptr(x) if x is not None and x.numel() else None
     d.y = _ptr(y) if y is not None and y.numel() else None
     if y is not None and not y.numel():

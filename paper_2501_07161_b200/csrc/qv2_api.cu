@@ -354,7 +354,8 @@ extern "C" uint64_t qv2_staging_bytes(const qv2_tensor_desc* descs, uint32_t n_t
   if (!descs) return 0;
   uint64_t total = 0;
   for (uint32_t t = 0; t < n_tensors; ++t) {
-    const uint64_t bytes = align256(descs[t].outer * descs[t].channels * descs[t].inner * sizeof(float));
+    const uint64_t esz = dtype_size((descs[t].flags & QV2_IN_MASK) >> 16);
+    const uint64_t bytes = align256(descs[t].outer * descs[t].channels * descs[t].inner * esz);
     total += bytes;
     if (descs[t].y) total += bytes;
   }
@@ -378,7 +379,8 @@ extern "C" int qv2_sweep_model_host(qv2_ctx* c, const qv2_tensor_desc* descs, ui
   uint64_t off = 0;
   for (uint32_t t = 0; t < n_tensors; ++t) {
     if (dd[t].flags & QV2_STORE_CODES) return QV2_ERR_UNSUPPORTED;
-    const uint64_t bytes = descs[t].outer * descs[t].channels * descs[t].inner * sizeof(float);
+    const uint64_t bytes = descs[t].outer * descs[t].channels * descs[t].inner *
+                           dtype_size((descs[t].flags & QV2_IN_MASK) >> 16);
     if (bytes && !descs[t].x) return QV2_ERR_NULL;
     dd[t].x = (const float*)(base + off);
     if (bytes) QV2_CUDA(c, cudaMemcpyAsync(base + off, descs[t].x, bytes, cudaMemcpyHostToDevice, c->stream));

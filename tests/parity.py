@@ -32,6 +32,7 @@ class Spec:
     raw: bool = False
     name: str = ""
     bits: int = 8
+    dtype: torch.dtype = torch.float32  # element type the GPU side stores x and y in
     zp: bool = False                   # affine scheme with an integer zero point (implies asym)
 
 
@@ -39,15 +40,15 @@ def bits(a) -> np.ndarray:
     return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
 
 
-def to_dev(t: Optional[torch.Tensor], misalign: int = 0):
+def to_dev(t: Optional[torch.Tensor], misalign: int = 0, dtype: torch.dtype = torch.float32):
     """Copy to the GPU; `misalign` (0..3) shifts the start by that many elements past a
     256-byte boundary so that vector loads need a scalar head."""
     if t is None:
         return None
-    flat = t.reshape(-1).to(torch.float32)
+    flat = t.reshape(-1).to(dtype)
     if misalign == 0:
         return flat.cuda().contiguous()
-    buf = torch.empty(flat.numel() + misalign, dtype=torch.float32, device="cuda")
+    buf = torch.empty(flat.numel() + misalign, dtype=dtype, device="cuda")
     buf[misalign:].copy_(flat)
     return buf[misalign:]
 
@@ -65,8 +66,9 @@ def make_descs(specs: List[Spec], dev_x, dev_y, store_codes=True):
 
 
 def oracle_tensor(s: Spec, want_codes=True):
-    x = s.x.detach().cpu().numpy().reshape(-1)
-    y = None if s.y is None else s.y.detach().cpu().numpy().reshape(-1)
+    # the oracle sees exactly the values the GPU side stores: rounded to the storage type, widened back
+    x = s.x.detach().cpu().to(s.dtype).to(torch.float32).numpy().reshape(-1)
+    y = None if s.y is None else s.y.detach().cpu().to(s.dtype).to(torch.float32).numpy().reshape(-1)
     mode = None
     if y is not None:
         mode = oracle.PAIR_RAW if s.raw else oracle.PAIR_REQUANT
@@ -89,8 +91,8 @@ def assert_metric_close(got_mse, got_sqnr, ref_mse, ref_sqnr, what=""):
 def check_specs(ctx, specs: List[Spec], misalign_x=0, misalign_y=0, check_codes=True,
                 twice=True):
     """Calibrate + measure every spec in ONE batched call each, compare with the oracle."""
-    dev_x = [to_dev(s.x, misalign_x) for s in specs]
-    dev_y = [to_dev(s.y, misalign_y) for s in specs]
+    dev_x = [to_dev(s.x, misalign_x, s.dtype) for s in specs]
+    dev_y = [to_dev(s.y, misalign_y, s.dtype) for s in specs]
     descs = make_descs(specs, dev_x, dev_y, store_codes=check_codes)
     cal = ctx.calibrate(descs)
     codes = None

@@ -451,3 +451,35 @@ def test_fold_batchnorm_is_bit_exact(ctx, c, k, mis):
     assert torch.equal(a0, a) and np.array_equal(c0.cpu().numpy().view(np.uint32), r0.view(np.uint32))
     # the folded weights feed the sweep like any other weight tensor
     check_specs(ctx, [Spec(a.cpu(), 1, c, k, per_channel=True)], twice=False)
+
+
+# ----------------------------------------------------------------------------- 16-bit input types
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("mis", [0, 1, 3])
+def test_half_precision_inputs(ctx, dtype, mis):
+    """binary16 / bfloat16 tensors: values are widened exactly, everything else is the binary32
+    definition, so the oracle is fed the stored values and the same bars apply."""
+    n = 4 * TILE + 203
+    x = randn(n, 150); y = x + 0.03 * randn(n, 151)
+    xr = x.clamp_min(0)
+    w = randn(48 * 577, 152) * torch.exp(randn(48, 153)).repeat_interleave(577)
+    wl = randn(3 * 20001, 154)
+    specs = [Spec(x, 1, 1, n, dtype=dtype), Spec(x, 1, 1, n, asym=True, dtype=dtype),
+             Spec(xr, 1, 1, n, asym=True, percentile=0.999, dtype=dtype),
+             Spec(x, 1, 1, n, asym=True, y=y, dtype=dtype), Spec(x, 1, 1, n, asym=True, y=y, raw=True, dtype=dtype),
+             Spec(w, 1, 48, 577, per_channel=True, dtype=dtype), Spec(wl, 1, 3, 20001, per_channel=True, dtype=dtype),
+             Spec(x, 1, 1, n, asym=True, zp=True, bits=4, dtype=dtype), Spec(x[:7], 1, 1, 7, dtype=dtype)]
+    check_specs(ctx, specs, misalign_x=mis, misalign_y=(mis + 2) % 4 if mis else 0)
+
+
+def test_half_precision_nonfinite_and_mixed_batch(ctx):
+    n = 2 * TILE + 11
+    x = randn(n, 160)
+    xh = x.clone(); xh[3] = float("inf"); xh[n - 2] = float("nan")
+    cal, _ = check_specs(ctx, [Spec(xh, 1, 1, n, asym=True, percentile=0.99, dtype=torch.float16),
+                               Spec(x, 1, 1, n, dtype=torch.float32), Spec(x, 1, 1, n, dtype=torch.bfloat16)],
+                         check_codes=False)
+    assert cal.nonfinite.tolist() == [2, 0, 0]
+    big = torch.tensor([70000.0, 1.0]).repeat(50)            # overflows binary16: stored as Inf
+    cal, _ = check_specs(ctx, [Spec(big, 1, 1, 100, dtype=torch.float16)], check_codes=False)
+    assert int(cal.nonfinite[0]) == 50
