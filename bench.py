@@ -47,6 +47,8 @@ def parse():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--input-dtype", default="f32", choices=["f32", "f16", "bf16"],
+                    help="element type the tensors are stored in (the default workload is f32)")
     ap.add_argument("--graph", action="store_true",
                     help="capture one pass in a CUDA graph and time its replays (per-phase times are then not available)")
     return ap.parse_args()
@@ -137,14 +139,14 @@ def oracle_sample_jobs(model, act_images: int, max_weight_elems: int):
         if l.w.numel() <= max_weight_elems // 4 and w_used + l.w.numel() <= max_weight_elems:
             w_used += l.w.numel()
             for g in cfg.w_granularity:
-                jobs.append(dict(x=l.w.detach().cpu().numpy().reshape(-1), y=None, outer=1,
+                jobs.append(dict(x=l.w.detach().cpu().float().numpy().reshape(-1), y=None, outer=1,
                                  channels=l.w.shape[0], inner=l.w.shape[1],
                                  per_channel=g == "channel", asym_u8=False))
                 swept += 8 * l.w.numel()
     for l in model.layers:
         b = min(act_images, l.x.shape[0])
-        x = l.x[:b].detach().cpu().numpy().reshape(-1)
-        y = l.y[:b].detach().cpu().numpy().reshape(-1)
+        x = l.x[:b].detach().cpu().float().numpy().reshape(-1)
+        y = l.y[:b].detach().cpu().float().numpy().reshape(-1)
         jobs.append(dict(x=x, y=y, outer=b, channels=l.x.shape[1], inner=l.x.shape[2],
                          per_channel=False, asym_u8=True, percentile=pct))
         swept += (16 if pct is not None else 12) * x.size
@@ -248,6 +250,12 @@ def ours_main(args):
     batch = args.batch or cfgw.batch
 
     model = gen.make_model(args.workload, seed=R.replica_seed(0, rank), device="cuda", batch=batch)
+    esz = 4
+    if args.input_dtype != "f32":        # same values, stored in 16 bits: half the bytes to sweep
+        tdt = torch.float16 if args.input_dtype == "f16" else torch.bfloat16
+        esz = 2
+        for l in model.layers:
+            l.w, l.x, l.y = l.w.to(tdt), l.x.to(tdt), l.y.to(tdt)
     # a captured pass needs a non-default stream; everything of this rank then runs on it
     stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
     torch.cuda.set_stream(stream)
@@ -256,9 +264,9 @@ def ours_main(args):
     n, L = md.n_tensors, md.n_layers
     rcfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
     sb, t = ctx.alloc_sweep_buffers(md.descs, L)
-    swept = gen.swept_bytes(args.workload, batch)
+    swept = gen.swept_bytes(args.workload, batch) * esz // 4
     w_elems, a_elems = model.weight_elems, model.act_elems
-    metrics_bytes = 4 * w_elems * len(cfgw.w_granularity) + 8 * a_elems   # one launch of the core kernel
+    metrics_bytes = (4 * w_elems * len(cfgw.w_granularity) + 8 * a_elems) * esz // 4   # one launch of the core kernel
 
     lib = q.lib()
     import ctypes as C
@@ -362,7 +370,7 @@ def ours_main(args):
         e1.record()
         torch.cuda.synchronize()
         e2e_val, _ = R.whole_job_throughput(swept * E / 1e9, e0.elapsed_time(e1) / 1e3)
-        h2d = 4 * (w_elems * len(cfgw.w_granularity) + 2 * a_elems) + 8 * L
+        h2d = esz * (w_elems * len(cfgw.w_granularity) + 2 * a_elems) + 8 * L
         d2h = sum(v.nbytes for v in out.values())
         e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": e0.elapsed_time(e1) / E, "steps": E,
@@ -388,15 +396,16 @@ def ours_main(args):
         peak, peak_src = measured_peak()
         achieved = metrics_bytes / (met_ms * 1e-3) / 1e9
         # the capture was taken on the default workload; DRAM traffic is reported for it only
-        ratio = recorded_traffic() if (args.workload == "vgg16" and batch == cfgw.batch) else None
+        ratio = recorded_traffic() if (args.workload == "vgg16" and batch == cfgw.batch and esz == 4) else None
         traffic = None if ratio is None else ratio * metrics_bytes
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "batch": batch, "layers": L, "tensors": n,
+                       "stored_as": args.input_dtype,
                        "weight_elems": w_elems, "act_elems": a_elems, "swept_bytes_per_step": swept,
-                       "resident_bytes": 4 * (w_elems + 2 * a_elems),
+                       "resident_bytes": esz * (w_elems + 2 * a_elems),
                        "l2": "inputs larger than L2 (no flush needed)" if 4 * (w_elems + 2 * a_elems) > 4 * 126e6
                              else "inputs fit in L2: this is an L2 number, not an HBM one",
                        "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
