@@ -197,7 +197,7 @@ extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t 
   QV2_CUDA(c, cudaMemsetAsync(nonfinite, 0, (size_t)n * sizeof(uint64_t), c->stream));
   if (h) QV2_CUDA(c, cudaMemsetAsync(h, 0, (size_t)n * kBins * sizeof(uint64_t), c->stream));
   if (!p.tiles.empty()) {
-    QV2_CUDA(c, launch_range(l, p.range_grid, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),
+    QV2_CUDA(c, launch_range(l, p.range_grid, p.any_16bit, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),
                              reinterpret_cast<uint32_t*>(gmin), reinterpret_cast<uint32_t*>(gmax),
                              c->d_rslots, reinterpret_cast<unsigned long long*>(nonfinite)));
     ++c->launches;
@@ -206,7 +206,7 @@ extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t 
                                     c->d_tensor_absmax));
   ++c->launches;
   if (!p.hist_tiles.empty()) {
-    QV2_CUDA(c, launch_hist(l, c->d_tensors, c->d_hist_tiles, (uint32_t)p.hist_tiles.size(),
+    QV2_CUDA(c, launch_hist(l, p.any_16bit, c->d_tensors, c->d_hist_tiles, (uint32_t)p.hist_tiles.size(),
                             c->d_tensor_absmax, reinterpret_cast<unsigned long long*>(nonfinite), h));
     ++c->launches;
   }
@@ -237,7 +237,7 @@ extern "C" int qv2_quant_metrics_ex(qv2_ctx* c, const qv2_tensor_desc* descs, ui
   }
   const Launch l = launch_of(c);
   if (!p.tiles.empty()) {
-    QV2_CUDA(c, launch_metrics(l, p.metrics_grid, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
+    QV2_CUDA(c, launch_metrics(l, p.metrics_grid, p.any_16bit, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
                                offset, c->d_partials, xe));
     ++c->launches;
   }

@@ -70,6 +70,7 @@ struct HostPlan {
   uint32_t total_rslots = 0;
   uint32_t range_grid = 1;        // CTAs of the range launch; the range-slot layout depends on it
   bool any_percentile = false;
+  bool any_16bit = false;         // some tensor is stored in binary16 / bfloat16
 };
 
 // Validates the descriptors and cuts them into tiles.  `codes` may be NULL.  `metrics_cap` and
@@ -86,21 +87,21 @@ struct Launch {
   int sm_count;
 };
 
-cudaError_t launch_range(const Launch& l, uint32_t grid, const TensorRec* tensors, const Tile* tiles,
+cudaError_t launch_range(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors, const Tile* tiles,
                          uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax, uint2* rslots,
                          unsigned long long* nonfinite);
 uint32_t range_grid_cap(int sm_count);     // resident CTAs per SM x SMs for the range kernel
 cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                   const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
                                   float* step, float* inv, float* offset, float* tensor_absmax);
-cudaError_t launch_hist(const Launch& l, const TensorRec* tensors, const Tile* tiles,
+cudaError_t launch_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
                         uint32_t n_tiles, const float* tensor_absmax,
                         const unsigned long long* nonfinite, unsigned long long* hist);
 cudaError_t launch_clip_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                  const unsigned long long* hist, const float* tensor_absmax,
                                  const float* gmin, const float* gmax, const float* gabsmax,
                                  float* clip, float* step, float* inv, float* offset);
-cudaError_t launch_metrics(const Launch& l, uint32_t grid, const TensorRec* tensors,
+cudaError_t launch_metrics(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors,
                            const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
                            const float* offset, double2* partials, double* partials_xe);
 uint32_t metrics_grid_cap(int sm_count);   // resident CTAs per SM x SMs for the metrics kernel

@@ -26,6 +26,10 @@ __device__ __forceinline__ float ld_stream1(const float* p) {
 // Element access by type: four consecutive elements widened to binary32 (the address must be a
 // multiple of four elements), or one element.  binary16 and bfloat16 widen exactly.
 template <class T> struct Ld;
+// vec_at(base, j): the j-th group of four after `base`; the index is widened before it is scaled
+// so that the address is one multiply-add.
+template <class T>
+__device__ __forceinline__ float4 ld_vec_at(const T* base, uint32_t j) { return Ld<T>::vec(base + 4 * (size_t)j); }
 template <> struct Ld<float> {
   static __device__ __forceinline__ float4 vec(const float* p) { return ld_stream4(reinterpret_cast<const float4*>(p)); }
   static __device__ __forceinline__ float one(const float* p) { return ld_stream1(p); }

@@ -37,7 +37,7 @@ __device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t coun
   for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
     float4 v[U];
 #pragma unroll
-    for (uint32_t u = 0; u < U; ++u) v[u] = Ld<T>::vec(xv + 4u * (j + u * kThreads));
+    for (uint32_t u = 0; u < U; ++u) v[u] = ld_vec_at(xv, j + u * kThreads);
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) {
       hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
@@ -45,7 +45,7 @@ __device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t coun
     }
   }
   for (; j < s.nvec; j += kThreads) {
-    const float4 v = Ld<T>::vec(xv + 4u * j);
+    const float4 v = ld_vec_at(xv, j);
     hist_elem<CAREFUL>(v.x, w, sh, zeros); hist_elem<CAREFUL>(v.y, w, sh, zeros);
     hist_elem<CAREFUL>(v.z, w, sh, zeros); hist_elem<CAREFUL>(v.w, w, sh, zeros);
   }
@@ -61,6 +61,7 @@ __device__ __forceinline__ void hist_tile(const T* x, uint32_t count, float w, b
   else hist_flat<false>(x, count, w, sh, zeros);
 }
 
+template <bool ANY16>      // false: every tensor is binary32, no element-type dispatch
 __global__ void __launch_bounds__(kThreads, 4)
 hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
             const float* __restrict__ tensor_absmax, const unsigned long long* __restrict__ nonfinite,
@@ -99,7 +100,7 @@ hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tile
       careful = nonfinite[cur] != 0ull;
     }
     const TensorRec* tr = tensors + cur;
-    if (tr->dtype == kF32) hist_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+    if (!ANY16 || tr->dtype == kF32) hist_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
     else if (tr->dtype == kF16) hist_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
     else hist_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
     ++since_flush;
@@ -166,13 +167,14 @@ clip_finalize_kernel(const TensorRec* __restrict__ tensors, const unsigned long 
 
 }  // namespace
 
-cudaError_t launch_hist(const Launch& l, const TensorRec* tensors, const Tile* tiles,
+cudaError_t launch_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
                         uint32_t n_tiles, const float* tensor_absmax,
                         const unsigned long long* nonfinite, unsigned long long* hist) {
   if (n_tiles == 0) return cudaSuccess;
   static int per_sm = 0;
-  const int grid = persistent_grid((const void*)hist_kernel, &per_sm, l.sm_count, n_tiles);
-  hist_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, tensor_absmax, nonfinite, hist);
+  const int grid = persistent_grid((const void*)hist_kernel<false>, &per_sm, l.sm_count, n_tiles);
+  if (any16) hist_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, tensor_absmax, nonfinite, hist);
+  else hist_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, tensor_absmax, nonfinite, hist);
   return cudaGetLastError();
 }
 

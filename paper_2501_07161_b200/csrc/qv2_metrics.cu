@@ -109,22 +109,22 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
       float4 vx[U], vy[U];
 #pragma unroll
       for (uint32_t u = 0; u < U; ++u) {
-        vx[u] = Ld<T>::vec(xb + 4u * (j + u * kThreads));
-        if (PAIR) vy[u] = Ld<T>::vec(yb + 4u * (j + u * kThreads)); else vy[u] = vx[u];
+        vx[u] = ld_vec_at(xb, j + u * kThreads);
+        if (PAIR) vy[u] = ld_vec_at(yb, j + u * kThreads); else vy[u] = vx[u];
       }
 #pragma unroll
       for (uint32_t u = 0; u < U; ++u)
         metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * kThreads) : nullptr);
     }
     for (; j < s.nvec; j += kThreads) {
-      const float4 vx = Ld<T>::vec(xb + 4u * j);
-      const float4 vy = PAIR ? Ld<T>::vec(yb + 4u * j) : vx;
+      const float4 vx = ld_vec_at(xb, j);
+      const float4 vy = PAIR ? ld_vec_at(yb, j) : vx;
       metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
     }
   } else {
     // x and y sit at different offsets inside their groups of four: vector loads for x, scalar for y
     for (; j < s.nvec; j += kThreads) {
-      const float4 vx = Ld<T>::vec(xb + 4u * j);
+      const float4 vx = ld_vec_at(xb, j);
       float4 vy;
       vy.x = Ld<T>::one(yb + 4u * j); vy.y = Ld<T>::one(yb + 4u * j + 1);
       vy.z = Ld<T>::one(yb + 4u * j + 2); vy.w = Ld<T>::one(yb + 4u * j + 3);
@@ -176,15 +176,17 @@ __device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRe
   uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
   QP p;
   const float top = top_code(tr->asym != 0, tr->bits);
-  const bool zp = tr->asym == 2;      // integer zero point: codes are rne(v*inv) + z, clamped to [0, top]
-  p.qmax = top;
-  p.qmin = tr->asym ? 0.0f : -top;
-  p.bias = 0.0f;
-  // With a zero point z the arithmetic is the offset-free path on d = q - z: clamp to [-z, top-z],
-  // e = x - d*step; only the stored code differs (d + z).
+  const float qmin0 = tr->asym ? 0.0f : -top;
+  // Integer zero point z (tr->asym == 2, the offset slot carries z): the arithmetic is the
+  // offset-free path on d = q - z -- clamp to [-z, top - z], e = x - d*step -- and only the
+  // stored code differs (d + z).  Written without branches: z is 0 for the other schemes.
+  const bool zp = tr->asym == 2;
   auto load_params = [&](uint32_t G) {
-    p.step = __ldg(step + G); p.inv = __ldg(inv + G); p.off = __ldg(offset + G);
-    if (zp) { p.bias = p.off; p.qmin = -p.off; p.qmax = top - p.off; p.off = 0.0f; }
+    p.step = __ldg(step + G); p.inv = __ldg(inv + G);
+    const float off = __ldg(offset + G);
+    const float z = zp ? off : 0.0f;
+    p.off = zp ? 0.0f : off;
+    p.bias = z; p.qmin = qmin0 - z; p.qmax = top - z;
   };
   if (tl.rows == 0) {
     load_params(tr->group_base + (uint32_t)tl.row0);
@@ -203,12 +205,12 @@ __device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRe
   }
 }
 
-// Dispatch on the element type of the tensor.
-template <uint32_t MODE, bool CODES, class ACC>
+// Dispatch on the element type of the tensor (compiled out when ANY16 is false: all binary32).
+template <uint32_t MODE, bool CODES, bool ANY16 = true, class ACC>
 __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
                                             const float* __restrict__ step, const float* __restrict__ inv,
                                             const float* __restrict__ offset, ACC* a) {
-  if (tr->dtype == kF32) metric_tile_typed<MODE, CODES, float>(tl, tr, step, inv, offset, a);
+  if (!ANY16 || tr->dtype == kF32) metric_tile_typed<MODE, CODES, float>(tl, tr, step, inv, offset, a);
   else if (tr->dtype == kF16) metric_tile_typed<MODE, CODES, __half>(tl, tr, step, inv, offset, a);
   else metric_tile_typed<MODE, CODES, __nv_bfloat16>(tl, tr, step, inv, offset, a);
 }
@@ -222,8 +224,8 @@ __device__ __forceinline__ uint32_t slot_of(const TensorRec* tr, uint32_t warp) 
 }
 
 // COS adds the sum x*e (third slot array) needed for the cosine similarity.
-template <bool COS>
-__global__ void __launch_bounds__(kThreads, 4)
+template <bool COS, bool ANY16>
+__global__ void __launch_bounds__(kThreads, 3)       // 85 registers: nothing spills; 4 CTAs per SM did not run faster
 metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
                const float* __restrict__ step, const float* __restrict__ inv,
                const float* __restrict__ offset, double2* __restrict__ partials,
@@ -256,13 +258,13 @@ metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ t
     const uint32_t mode = tr->pair_mode;
     const bool codes = tr->codes != nullptr && mode != kRaw;
     if (mode == kSelf) {
-      if (codes) metric_tile<kSelf, true>(tl, tr, step, inv, offset, a);
-      else metric_tile<kSelf, false>(tl, tr, step, inv, offset, a);
+      if (codes) metric_tile<kSelf, true, ANY16>(tl, tr, step, inv, offset, a);
+      else metric_tile<kSelf, false, ANY16>(tl, tr, step, inv, offset, a);
     } else if (mode == kRequant) {
-      if (codes) metric_tile<kRequant, true>(tl, tr, step, inv, offset, a);
-      else metric_tile<kRequant, false>(tl, tr, step, inv, offset, a);
+      if (codes) metric_tile<kRequant, true, ANY16>(tl, tr, step, inv, offset, a);
+      else metric_tile<kRequant, false, ANY16>(tl, tr, step, inv, offset, a);
     } else {
-      metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
+      metric_tile<kRaw, false, ANY16>(tl, tr, step, inv, offset, a);
     }
     // this lane's tile sums in binary32 with a fixed association, then into the binary64 totals
     const float sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
@@ -430,19 +432,18 @@ __global__ void kl_finalize_kernel(uint32_t n, const unsigned long long* __restr
 
 uint32_t metrics_grid_cap(int sm_count) {
   static int per_sm = 0;
-  return (uint32_t)persistent_grid((const void*)metrics_kernel<false>, &per_sm, sm_count, 0x7fffffffu);
+  return (uint32_t)persistent_grid((const void*)metrics_kernel<false, false>, &per_sm, sm_count, 0x7fffffffu);
 }
 
-cudaError_t launch_metrics(const Launch& l, uint32_t grid, const TensorRec* tensors,
+cudaError_t launch_metrics(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors,
                            const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
                            const float* offset, double2* partials, double* partials_xe) {
   if (n_tiles == 0) return cudaSuccess;
-  if (partials_xe)
-    metrics_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset,
-                                                          partials, partials_xe);
-  else
-    metrics_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset,
-                                                           partials, nullptr);
+#define QV2_LAUNCH_METRICS(COS, A16) \
+  metrics_kernel<COS, A16><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset, partials, partials_xe)
+  if (partials_xe) { if (any16) QV2_LAUNCH_METRICS(true, true); else QV2_LAUNCH_METRICS(true, false); }
+  else { if (any16) QV2_LAUNCH_METRICS(false, true); else QV2_LAUNCH_METRICS(false, false); }
+#undef QV2_LAUNCH_METRICS
   return cudaGetLastError();
 }
 

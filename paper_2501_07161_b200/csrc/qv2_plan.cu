@@ -26,7 +26,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
   if (!descs || !out) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   out->tensors.clear(); out->tiles.clear(); out->hist_tiles.clear();
-  out->total_groups = 0; out->total_slots = 0; out->any_percentile = false;
+  out->total_groups = 0; out->total_slots = 0; out->any_percentile = false; out->any_16bit = false;
   out->tensors.reserve(n);
   uint64_t groups = 0;
   for (uint32_t t = 0; t < n; ++t) {
@@ -67,6 +67,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     r.percentile = d.percentile;
     r.bits = bits;
     r.dtype = dtype;
+    if (dtype != kF32) out->any_16bit = true;
 
     size_t first_tile = out->tiles.size();
     if (d.range == QV2_PERCENTILE) out->any_percentile = true;

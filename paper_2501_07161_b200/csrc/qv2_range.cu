@@ -46,11 +46,11 @@ __device__ __forceinline__ void range_flat(const T* __restrict__ x, uint32_t cou
   for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
     float4 v[U];
 #pragma unroll
-    for (uint32_t u = 0; u < U; ++u) v[u] = Ld<T>::vec(xv + 4u * (j + u * kThreads));
+    for (uint32_t u = 0; u < U; ++u) v[u] = ld_vec_at(xv, j + u * kThreads);
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) range_acc4<CAREFUL>(a, v[u]);
   }
-  for (; j < s.nvec; j += kThreads) range_acc4<CAREFUL>(a, Ld<T>::vec(xv + 4u * j));
+  for (; j < s.nvec; j += kThreads) range_acc4<CAREFUL>(a, ld_vec_at(xv, j));
   if (threadIdx.x < s.head) range_acc<CAREFUL>(a, Ld<T>::one(x + threadIdx.x));
   if (threadIdx.x < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(x + s.head + 4u * s.nvec + threadIdx.x));
 }
@@ -145,6 +145,9 @@ __device__ __forceinline__ void publish_slot(RangeAcc& a, uint32_t lane, uint32_
   __syncthreads();
 }
 
+// ANY16 = false is the build for models whose tensors are all binary32: the element-type dispatch
+// is compiled out, so that common case pays nothing for the 16-bit paths.
+template <bool ANY16>
 __global__ void __launch_bounds__(kThreads, 4)
 range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
              uint32_t* kmin, uint32_t* kmax, uint2* rslots, unsigned long long* nonfinite) {
@@ -169,11 +172,11 @@ range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ til
         reset(a);
         cur_group = G; cur_tensor = tl.tensor; cur_slot = tr->per_channel == 0;
       }
-      if (tr->dtype == kF32) range_flat_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, a);
+      if (!ANY16 || tr->dtype == kF32) range_flat_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, a);
       else if (tr->dtype == kF16) range_flat_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, a);
       else range_flat_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, a);
     } else {
-      if (tr->dtype == kF32)
+      if (!ANY16 || tr->dtype == kF32)
         range_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
       else if (tr->dtype == kF16)
         range_rows_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
@@ -246,14 +249,15 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __rest
 
 uint32_t range_grid_cap(int sm_count) {
   static int per_sm = 0;
-  return (uint32_t)persistent_grid((const void*)range_kernel, &per_sm, sm_count, 0x7fffffffu);
+  return (uint32_t)persistent_grid((const void*)range_kernel<false>, &per_sm, sm_count, 0x7fffffffu);
 }
 
-cudaError_t launch_range(const Launch& l, uint32_t grid, const TensorRec* tensors, const Tile* tiles,
+cudaError_t launch_range(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors, const Tile* tiles,
                          uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax, uint2* rslots,
                          unsigned long long* nonfinite) {
   if (n_tiles == 0) return cudaSuccess;
-  range_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, rslots, nonfinite);
+  if (any16) range_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, rslots, nonfinite);
+  else range_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, rslots, nonfinite);
   return cudaGetLastError();
 }
 
