@@ -75,6 +75,10 @@ def _load():
     lib.qv2o_kl_bits.restype = C.c_double
     lib.qv2o_fold_batchnorm.argtypes = [f32p] * 6 + [C.c_uint64, C.c_uint64, f32p, f32p]
     lib.qv2o_fold_batchnorm.restype = None
+    lib.qv2o_group_histograms.argtypes = [f32p, C.c_uint64, C.c_uint64, C.c_uint64, f32p, C.c_double, u64p, f32p]
+    lib.qv2o_group_histograms.restype = None
+    lib.qv2o_qparams_gclip.argtypes = [C.c_int, C.c_int, C.c_uint64, f32p, f32p, f32p, f32p, f32p, f32p, f32p]
+    lib.qv2o_qparams_gclip.restype = None
     lib.qv2o_rank_fused.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p, u32p,
                                     C.c_double, C.c_double, C.c_double, C.c_double,
                                     C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
@@ -128,6 +132,33 @@ def qparams(asym_u8: bool, gmin, gmax, gabsmax, clip: Optional[float] = None, bi
     lib.qv2o_qparams_bits(int(bits), int(asym_u8), int(clip is not None), C.c_float(0.0 if clip is None else clip),
                      g, _p(gmin, C.c_float), _p(gmax, C.c_float), _p(gabsmax, C.c_float),
                      _p(step, C.c_float), _p(inv, C.c_float), _p(off, C.c_float))
+    return step, inv, off
+
+
+def group_histograms(x, outer: int, channels: int, inner: int, gabsmax, p: float):
+    """One |x| histogram and one percentile clip per channel of a [outer][channels][inner] tensor."""
+    lib = _load()
+    x = _f32(x).reshape(-1)
+    assert x.size == outer * channels * inner
+    gabsmax = _f32(gabsmax)
+    assert gabsmax.size == channels
+    hist = np.zeros((channels, BINS), np.uint64)
+    clip = np.zeros(channels, np.float32)
+    lib.qv2o_group_histograms(_p(x, C.c_float), outer, channels, inner, _p(gabsmax, C.c_float), float(p),
+                              _p(hist, C.c_uint64), _p(clip, C.c_float))
+    return hist, clip
+
+
+def qparams_gclip(scheme, gmin, gmax, gabsmax, gclip, bits: int = 8):
+    """qparams with one clip value per group."""
+    lib = _load()
+    gmin, gmax, gabsmax, gclip = _f32(gmin), _f32(gmax), _f32(gabsmax), _f32(gclip)
+    g = gmin.size
+    assert gclip.size == g
+    step = np.zeros(g, np.float32); inv = np.zeros(g, np.float32); off = np.zeros(g, np.float32)
+    lib.qv2o_qparams_gclip(int(bits), int(scheme), g, _p(gclip, C.c_float), _p(gmin, C.c_float),
+                           _p(gmax, C.c_float), _p(gabsmax, C.c_float),
+                           _p(step, C.c_float), _p(inv, C.c_float), _p(off, C.c_float))
     return step, inv, off
 
 
@@ -256,31 +287,40 @@ class TensorResult:
     mse: float
     sqnr_db: float
     codes: Optional[np.ndarray] = None
+    ghist: Optional[np.ndarray] = None     # [groups][2048], per-group percentile calibration only
+    gclip: Optional[np.ndarray] = None     # clip bound applied to each group
 
 
-def calibrate_tensor(x, outer, channels, inner, per_channel, asym_u8, percentile=None, bits=8):
-    """Ranges, optional |x| histogram + percentile clip, then the quantization parameters."""
+def calibrate_tensor(x, outer, channels, inner, per_channel, asym_u8, percentile=None, bits=8,
+                     group_percentile=False):
+    """Ranges, optional |x| histogram + percentile clip, then the quantization parameters.
+    ``group_percentile`` (per-channel tensors only) takes one histogram and one clip per channel
+    instead of one per tensor; the tensor-level clip is then the plain absmax and hist is None."""
     gmin, gmax, gabs, bad = ranges(x, outer, channels, inner, per_channel)
     A = np.float32(gabs.max()) if gabs.size else np.float32(0.0)
-    hist, clip = None, A
+    hist, clip, ghist = None, A, None
+    if percentile is not None and group_percentile and per_channel:
+        ghist, gclip = group_histograms(x, outer, channels, inner, gabs, percentile)
+        step, inv, off = qparams_gclip(asym_u8, gmin, gmax, gabs, gclip, bits)
+        return gmin, gmax, gabs, bad, hist, clip, step, inv, off, ghist, gclip
     if percentile is not None:
         hist = histogram(x, float(A))
         clip = percentile_clip(hist, percentile, float(A))
     step, inv, off = qparams(asym_u8, gmin, gmax, gabs, None if percentile is None else float(clip), bits)
-    return gmin, gmax, gabs, bad, hist, clip, step, inv, off
+    return gmin, gmax, gabs, bad, hist, clip, step, inv, off, ghist, np.full(gabs.size, clip, np.float32)
 
 
 def sweep_tensor(x, y, outer, channels, inner, per_channel, asym_u8, percentile=None,
-                 pair_mode=None, want_codes=False, bits=8) -> TensorResult:
+                 pair_mode=None, want_codes=False, bits=8, group_percentile=False) -> TensorResult:
     """Calibrate on x, then measure: self mode when y is None, else the paired mode."""
-    gmin, gmax, gabs, bad, hist, clip, step, inv, off = calibrate_tensor(
-        x, outer, channels, inner, per_channel, asym_u8, percentile, bits)
+    gmin, gmax, gabs, bad, hist, clip, step, inv, off, ghist, gclip = calibrate_tensor(
+        x, outer, channels, inner, per_channel, asym_u8, percentile, bits, group_percentile)
     if pair_mode is None:
         pair_mode = PAIR_SELF if y is None else PAIR_REQUANT
     m = quant_metrics(x, y, outer, channels, inner, per_channel, asym_u8, pair_mode,
                       step, inv, off, want_codes, bits)
     return TensorResult(gmin, gmax, gabs, bad, hist, clip, step, inv, off,
-                        m["sse"], m["sig"], m["mse"], m["sqnr_db"], m.get("codes"))
+                        m["sse"], m["sig"], m["mse"], m["sqnr_db"], m.get("codes"), ghist, gclip)
 
 
 def sweep_tensors(jobs: Sequence[dict], threads: int = 1) -> List[TensorResult]:

@@ -112,6 +112,32 @@ float qv2o_percentile_clip(const uint64_t *hist, double p, float A)
     return fl_mul((float)(kstar + 1), fl_div(A, (float)QV2O_BINS));
 }
 
+/* Per-channel variant of the calibration histogram: one 2048-bin |x| histogram for EVERY
+ * quantization group c of a tensor laid out [outer][channels][inner], on [0, A_c] with A_c the
+ * group's own absmax, and from it one clip value per group (same percentile rule as above).
+ * hist: channels * 2048 counts; clip: channels values.  The paper's calibration keeps one
+ * histogram per layer; this is the finer-grained reading for per-channel quantizers. */
+void qv2o_group_histograms(const float *x, uint64_t outer, uint64_t channels, uint64_t inner,
+                           const float *gabsmax, double p, uint64_t *hist, float *clip)
+{
+    memset(hist, 0, channels * QV2O_BINS * sizeof(uint64_t));
+    for (uint64_t c = 0; c < channels; ++c) {
+        const float A = gabsmax[c];
+        float w = (A > 0.0f) ? fl_div((float)QV2O_BINS, A) : 0.0f;
+        if (!finite_f(w)) w = 0.0f;
+        uint64_t *h = hist + c * QV2O_BINS;
+        for (uint64_t o = 0; o < outer; ++o)
+            for (uint64_t i = 0; i < inner; ++i) {
+                float v = x[(o * channels + c) * inner + i];
+                if (!finite_f(v)) continue;
+                float f = fl_mul(fabsf(v), w);
+                uint32_t b = (f >= (float)QV2O_BINS) ? (uint32_t)(QV2O_BINS - 1) : (uint32_t)f;
+                h[b] += 1;
+            }
+        clip[c] = qv2o_percentile_clip(h, p, A);
+    }
+}
+
 /* ---------------------------------------------------------------------------------------------
  * Quantization parameters per group.
  * Symmetric int8 (Eq. 4, read as the multiplier S = 127 / max|W|): R = absmax_g, or
@@ -170,6 +196,16 @@ void qv2o_qparams_bits(int bits, int asym_u8, int use_clip, float clip, uint64_t
         }
         step[g] = s; inv[g] = r; offset[g] = off;
     }
+}
+
+/* The same parameters with one clip value per group (per-channel percentile calibration). */
+void qv2o_qparams_gclip(int bits, int scheme, uint64_t groups, const float *gclip,
+                        const float *gmin, const float *gmax, const float *gabsmax,
+                        float *step, float *inv, float *offset)
+{
+    for (uint64_t g = 0; g < groups; ++g)
+        qv2o_qparams_bits(bits, scheme, 1, gclip[g], 1, gmin + g, gmax + g, gabsmax + g,
+                          step + g, inv + g, offset + g);
 }
 
 void qv2o_qparams(int asym_u8, int use_clip, float clip, uint64_t groups,

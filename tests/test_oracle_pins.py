@@ -695,3 +695,52 @@ def test_fold_batchnorm_identity_equivalence_and_float32_ops():
     assert np.array_equal(cc, s * (b - mean) + beta)
     a0, c0 = oracle.fold_batchnorm(w, None, gamma, beta, mean, var)        # no conv bias
     assert np.array_equal(a0, a) and np.array_equal(c0, s * (zero - mean) + beta)
+
+
+# ------------------------------------------------------------------- per-channel percentile clip
+def test_group_histograms_equal_per_tensor_histograms_of_each_channel_slice():
+    """Channel c of an [O][C][I] tensor, cut out with numpy indexing, calibrated on its own as a
+    per-tensor tensor, must give channel c's histogram, clip and parameters: this catches a wrong
+    stride, a wrong group's absmax and a clip applied to the wrong channel."""
+    rng = np.random.default_rng(77)
+    O, Cn, I = 3, 5, 257
+    x = (rng.standard_normal((O, Cn, I)) * (10.0 ** np.arange(-2, 3))[None, :, None]).astype(np.float32)
+    x[1, 2, 7] = np.inf                                     # skipped in channel 2 only
+    x[:, 4, :] = np.maximum(x[:, 4, :], 0)                  # a post-ReLU channel
+    for asym in (0, 1, 2):
+        gmin, gmax, gabs, bad, hist, clip, step, inv, off, ghist, gclip = oracle.calibrate_tensor(
+            x, O, Cn, I, True, asym, 0.97, group_percentile=True)
+        assert hist is None and bad == 1 and clip == gabs.max()
+        for c in range(Cn):
+            xc = np.ascontiguousarray(x[:, c, :])
+            r = oracle.calibrate_tensor(xc, 1, 1, O * I, False, asym, 0.97)
+            assert np.array_equal(ghist[c], r[4]), c
+            assert gclip[c] == r[5], c
+            assert step[c] == r[6][0] and inv[c] == r[7][0] and off[c] == r[8][0], c
+            assert int(ghist[c].sum()) == O * I - (1 if c == 2 else 0)
+
+
+def test_group_percentile_closed_form_and_difference_from_the_tensor_level_clip():
+    """Two channels with known staircases: channel 0 holds k/1000 for k = 1..1000, channel 1 holds
+    100x that.  With p = 0.9 each channel's clip is the upper edge of the bin that holds its 900th
+    value, i.e. ~0.9 of ITS absmax, while a tensor-level histogram would put all of channel 0 in
+    the lowest bins and leave it unclipped."""
+    k = np.arange(1, 1001, dtype=np.float64)
+    x = np.stack([k / 1000.0, k / 10.0]).astype(np.float32).reshape(1, 2, 1000)
+    out = oracle.calibrate_tensor(x, 1, 2, 1000, True, 0, 0.9, group_percentile=True)
+    gabs, step, gclip = out[2], out[6], out[10]
+    for c in range(2):
+        A = float(gabs[c])
+        kstar = int(np.floor(np.float32(np.float32(x[0, c, 899]) * np.float32(np.float32(2048.0) / np.float32(A)))))
+        assert abs(float(gclip[c]) - (kstar + 1) * A / 2048.0) <= 1e-6 * A
+        assert 0.9 * A <= float(gclip[c]) <= 0.9 * A + A / 2048.0 * 1.001
+        assert step[c] == np.float32(gclip[c]) / np.float32(127.0)
+    t = oracle.calibrate_tensor(x, 1, 2, 1000, True, 0, 0.9)           # one clip for the tensor
+    assert float(t[5]) > float(gabs[0])                                 # channel 0 is not clipped by it
+    assert t[6][0] == np.float32(gabs[0]) / np.float32(127.0)
+    # p = 1 clips nothing; a per-tensor tensor ignores the flag
+    full = oracle.calibrate_tensor(x, 1, 2, 1000, True, 0, 1.0, group_percentile=True)
+    assert np.array_equal(full[10], gabs)
+    a = oracle.calibrate_tensor(x, 1, 2, 1000, False, 1, 0.9, group_percentile=True)
+    b = oracle.calibrate_tensor(x, 1, 2, 1000, False, 1, 0.9)
+    assert a[5] == b[5] and np.array_equal(a[4], b[4]) and np.array_equal(a[6], b[6])
