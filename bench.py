@@ -49,6 +49,9 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--input-dtype", default="f32", choices=["f32", "f16", "bf16"],
                     help="element type the tensors are stored in (the default workload is f32)")
+    ap.add_argument("--act-granularity", default="tensor", choices=["tensor", "channel"],
+                    help="channel: activations quantized per channel, each channel with its own percentile clip "
+                         "(a variant; the paper's set-ups and the headline number are per tensor)")
     ap.add_argument("--graph", action="store_true",
                     help="capture one pass in a CUDA graph and time its replays (per-phase times are then not available)")
     return ap.parse_args()
@@ -128,7 +131,7 @@ class ClockSampler:
 
 
 # -------------------------------------------------------------------------------- reference arm
-def oracle_sample_jobs(model, act_images: int, max_weight_elems: int):
+def oracle_sample_jobs(model, act_images: int, max_weight_elems: int, act_per_channel: bool = False):
     """Oracle jobs for a bounded sample: every layer's activations restricted to the first
     `act_images` images, and the weight tensors (in layer order) that fit the element budget (a
     tensor larger than a quarter of the budget is left out so that no single job dominates)."""
@@ -148,7 +151,8 @@ def oracle_sample_jobs(model, act_images: int, max_weight_elems: int):
         x = l.x[:b].detach().cpu().float().numpy().reshape(-1)
         y = l.y[:b].detach().cpu().float().numpy().reshape(-1)
         jobs.append(dict(x=x, y=y, outer=b, channels=l.x.shape[1], inner=l.x.shape[2],
-                         per_channel=False, asym_u8=True, percentile=pct))
+                         per_channel=act_per_channel, asym_u8=True, percentile=pct,
+                         group_percentile=act_per_channel))
         swept += (16 if pct is not None else 12) * x.size
     return jobs, swept, w_used
 
@@ -260,7 +264,7 @@ def ours_main(args):
     stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
     torch.cuda.set_stream(stream)
     ctx = q.Context(local, stream=stream)
-    md = q.model_descs(model)
+    md = q.model_descs(model, act_granularity=args.act_granularity)
     n, L = md.n_tensors, md.n_layers
     rcfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
     sb, t = ctx.alloc_sweep_buffers(md.descs, L)
@@ -354,7 +358,7 @@ def ours_main(args):
             o = _L(); o.w, o.x, o.y, o.macs = w, x, y, l.macs
             hl.append(o)
         hm = _L(); hm.layers = hl; hm.config = model.config
-        hd = q.model_descs(hm, host=True)
+        hd = q.model_descs(hm, host=True, act_granularity=args.act_granularity)
         staging = torch.empty(q.binding.staging_bytes(hd.descs, L), dtype=torch.uint8, device="cuda")
         out = dict(mse=np.zeros(n), sqnr_db=np.zeros(n), nonfinite=np.zeros(n, np.uint64),
                    order=np.zeros(L, np.uint32), keep_fp32=np.zeros(L, np.uint8), n_keep=np.zeros(1, np.uint32))
@@ -384,7 +388,7 @@ def ours_main(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
         images, wbudget = size_sample(args.workload, batch, 2.0, threads)
-        jobs, s_swept, w_used = oracle_sample_jobs(model, images, wbudget)
+        jobs, s_swept, w_used = oracle_sample_jobs(model, images, wbudget, args.act_granularity == "channel")
         threads = min(threads, len(jobs))
         sec, _ = run_oracle_steps(jobs, threads, 1, 0)
         cpu = {"value": s_swept / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
@@ -396,14 +400,15 @@ def ours_main(args):
         peak, peak_src = measured_peak()
         achieved = metrics_bytes / (met_ms * 1e-3) / 1e9
         # the capture was taken on the default workload; DRAM traffic is reported for it only
-        ratio = recorded_traffic() if (args.workload == "vgg16" and batch == cfgw.batch and esz == 4) else None
+        ratio = recorded_traffic() if (args.workload == "vgg16" and batch == cfgw.batch and esz == 4
+                                         and args.act_granularity == "tensor") else None
         traffic = None if ratio is None else ratio * metrics_bytes
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "batch": batch, "layers": L, "tensors": n,
-                       "stored_as": args.input_dtype,
+                       "stored_as": args.input_dtype, "act_granularity": args.act_granularity,
                        "weight_elems": w_elems, "act_elems": a_elems, "swept_bytes_per_step": swept,
                        "resident_bytes": esz * (w_elems + 2 * a_elems),
                        "l2": "inputs larger than L2 (no flush needed)" if 4 * (w_elems + 2 * a_elems) > 4 * 126e6

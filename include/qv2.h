@@ -52,7 +52,7 @@ enum {
 
 enum { QV2_PER_TENSOR = 0, QV2_PER_CHANNEL = 1 };            /* granularity */
 enum { QV2_SYM_I8 = 0, QV2_ASYM_U8 = 1, QV2_ASYM_U8_ZP = 2 }; /* scheme */
-enum { QV2_ABSMAX = 0, QV2_MINMAX = 1, QV2_PERCENTILE = 2 }; /* range */
+enum { QV2_ABSMAX = 0, QV2_MINMAX = 1, QV2_PERCENTILE = 2, QV2_PERCENTILE_GROUP = 3 }; /* range */
 enum { QV2_PAIR_REQUANT = 0, QV2_PAIR_RAW = 1, QV2_STORE_CODES = 2 }; /* flags (bit 0: pair mode) */
 enum { QV2_BY_COUNT = 0, QV2_BY_BOPS_RATE = 1 };             /* select_mode */
 /* Code width other than 8 bits, OR-ed into qv2_tensor_desc.flags: QV2_BITS(b), 2 <= b <= 16.  The
@@ -91,11 +91,13 @@ typedef struct {
                             v^ = (q - z)*step; the offset[] slot of the group then holds z */
   uint32_t range;        /* QV2_ABSMAX and QV2_MINMAX take the group's observed range (|.| max for
                             the symmetric scheme, [min,max] for the asymmetric one);
-                            QV2_PERCENTILE additionally clips it to the tensor's |x| percentile */
+                            QV2_PERCENTILE additionally clips it to the tensor's |x| percentile;
+                            QV2_PERCENTILE_GROUP clips every group to the percentile of its own
+                            |x| histogram (the same as QV2_PERCENTILE for QV2_PER_TENSOR) */
   uint32_t flags;        /* pair mode: QV2_PAIR_REQUANT (default) re-quantizes y on x's grid and
                             measures x - dequant(q(y)); QV2_PAIR_RAW measures x - y.
                             QV2_STORE_CODES writes the 8-bit codes (see qv2_quant_metrics). */
-  double percentile;     /* in [0,1], e.g. 0.9999; read only when range == QV2_PERCENTILE */
+  double percentile;     /* in [0,1], e.g. 0.9999; read only by the two percentile range modes */
 } qv2_tensor_desc;
 
 /* Ranking parameters (Algorithm 2, RankLayersBySensitivity; Eq. 16; Eq. 17). */
@@ -171,6 +173,30 @@ int qv2_calibrate(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
                   uint64_t* hist, float* clip,
                   float* step, float* inv, float* offset,
                   uint64_t* nonfinite);
+
+/*
+ * qv2_calibrate with the per-channel form of the percentile clip (range QV2_PERCENTILE_GROUP on a
+ * QV2_PER_CHANNEL tensor).  The paper's calibration keeps one histogram per layer; a per-channel
+ * quantizer whose channels differ in scale by orders of magnitude gets nothing from a clip taken
+ * over the whole tensor, so this mode repeats the construction per group: group g gets its own
+ * 2048-bin histogram of |x| on [0, absmax_g], bin = min(2047, trunc(|x| * fl(2048/absmax_g))), and
+ * its own clip_g (same cumulative-count rule as clip[t]); its parameters are those of
+ * QV2_PERCENTILE with clip_g in place of the tensor's clip.  For such a tensor clip[t] is the
+ * tensor's absmax and its row of hist stays zero.  Both calls accept the mode; this one can also
+ * return the per-group data:
+ * group_hist: device or NULL (context scratch): one 2048-entry uint64 histogram per group of every
+ *   QV2_PERCENTILE_GROUP per-channel tensor, those tensors in descriptor order, their groups in
+ *   channel order; qv2_group_hist_count gives the number of histograms.
+ * group_clip: device or NULL: qv2_group_count floats, the clip bound applied to each group
+ *   (clip_g in this mode, the tensor's clip[t] otherwise).
+ */
+int qv2_calibrate_ex(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
+                     float* gmin, float* gmax, float* gabsmax,
+                     uint64_t* hist, float* clip,
+                     float* step, float* inv, float* offset,
+                     uint64_t* nonfinite, uint64_t* group_hist, float* group_clip);
+/* Number of per-group histograms qv2_calibrate_ex keeps for these descriptors.  Host only. */
+uint64_t qv2_group_hist_count(const qv2_tensor_desc* descs, uint32_t n);
 
 /*
  * Turns the device-side non-finite counters of qv2_calibrate into a status: synchronises the

@@ -15,7 +15,7 @@ from . import build as _build
 
 PER_TENSOR, PER_CHANNEL = 0, 1
 SYM_I8, ASYM_U8, ASYM_U8_ZP = 0, 1, 2
-ABSMAX, MINMAX, PERCENTILE = 0, 1, 2
+ABSMAX, MINMAX, PERCENTILE, PERCENTILE_GROUP = 0, 1, 2, 3
 PAIR_REQUANT, PAIR_RAW, STORE_CODES = 0, 1, 2
 BY_COUNT, BY_BOPS_RATE = 0, 1
 IN_F32, IN_F16, IN_BF16 = 0, 1 << 16, 2 << 16
@@ -27,7 +27,7 @@ EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_erro
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
            "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm", "qv2_sweep_graph_create", "qv2_sweep_graph_launch",
-           "qv2_sweep_graph_destroy", "qv2_check_nonfinite"]
+           "qv2_sweep_graph_destroy", "qv2_check_nonfinite", "qv2_calibrate_ex", "qv2_group_hist_count"]
 KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
@@ -77,6 +77,8 @@ def lib() -> C.CDLL:
     L.qv2_launch_count.argtypes = [vp]; L.qv2_launch_count.restype = u64
     L.qv2_group_count.argtypes = [dp, u32]; L.qv2_group_count.restype = u64
     L.qv2_calibrate.argtypes = [vp, dp, u32] + [vp] * 9; L.qv2_calibrate.restype = i32
+    L.qv2_calibrate_ex.argtypes = [vp, dp, u32] + [vp] * 11; L.qv2_calibrate_ex.restype = i32
+    L.qv2_group_hist_count.argtypes = [dp, u32]; L.qv2_group_hist_count.restype = C.c_uint64
     L.qv2_quant_metrics.argtypes = [vp, dp, u32, vp, vp, vp, C.POINTER(vp), vp, vp, vp, vp]
     L.qv2_quant_metrics.restype = i32
     L.qv2_quant_metrics_ex.argtypes = [vp, dp, u32, vp, vp, vp, C.POINTER(vp), vp, vp, vp, vp, vp]
@@ -165,6 +167,8 @@ class CalibOut:
     inv: torch.Tensor
     offset: torch.Tensor
     nonfinite: torch.Tensor
+    group_hist: Optional[torch.Tensor] = None     # [qv2_group_hist_count][2048]
+    group_clip: Optional[torch.Tensor] = None     # per group
 
 
 @dataclass
@@ -229,12 +233,22 @@ class Context:
         return sb, t
 
     # -- the three calls of the contract ---------------------------------------------------
-    def calibrate(self, descs, want_hist: bool = True) -> CalibOut:
+    def calibrate(self, descs, want_hist: bool = True, want_group: bool = False) -> CalibOut:
+        """qv2_calibrate; with want_group, qv2_calibrate_ex returning the per-group histograms and clips."""
         n = len(descs)
         g = int(lib().qv2_group_count(descs, n))
         f = lambda k: self._empty(k, torch.float32)
         out = CalibOut(f(g), f(g), f(g), self._empty(n * HIST_BINS, torch.int64) if want_hist else None,
                        f(n), f(g), f(g), f(g), self._empty(n, torch.int64))
+        if want_group:
+            gh = int(lib().qv2_group_hist_count(descs, n))
+            out.group_hist = self._empty(gh * HIST_BINS, torch.int64)
+            out.group_clip = f(g)
+            _check(lib().qv2_calibrate_ex(self._h, descs, n, _ptr(out.gmin), _ptr(out.gmax), _ptr(out.gabsmax),
+                                          _ptr(out.hist), _ptr(out.clip), _ptr(out.step), _ptr(out.inv),
+                                          _ptr(out.offset), _ptr(out.nonfinite), _ptr(out.group_hist),
+                                          _ptr(out.group_clip)), "qv2_calibrate_ex")
+            return out
         _check(lib().qv2_calibrate(self._h, descs, n, _ptr(out.gmin), _ptr(out.gmax), _ptr(out.gabsmax),
                                    _ptr(out.hist), _ptr(out.clip), _ptr(out.step), _ptr(out.inv),
                                    _ptr(out.offset), _ptr(out.nonfinite)), "qv2_calibrate")

@@ -26,6 +26,9 @@ struct qv2_ctx {
   TensorRec* d_tensors = nullptr; size_t cap_tensors = 0;
   Tile* d_tiles = nullptr;        size_t cap_tiles = 0;
   Tile* d_hist_tiles = nullptr;   size_t cap_hist_tiles = 0;
+  Tile* d_ghist_tiles = nullptr;  size_t cap_ghist_tiles = 0;   // per-group histogram mode
+  uint32_t* d_ghist_owner = nullptr; size_t cap_ghist_owner = 0;
+  unsigned long long* d_ghist = nullptr; size_t cap_ghist = 0;  // used when the caller passes no group_hist
   double2* d_partials = nullptr;  size_t cap_slots = 0;
   uint2* d_rslots = nullptr;      size_t cap_rslots = 0;
   double* d_partials_xe = nullptr; size_t cap_slots_xe = 0;   // sum x*e slots, cosine only
@@ -103,14 +106,24 @@ int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* cons
   if ((st = grow(c, &c->d_partials, &c->cap_slots, plan.total_slots ? plan.total_slots : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_rslots, &c->cap_rslots, plan.total_rslots ? plan.total_rslots : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_tensor_absmax, &c->cap_absmax, nt)) != QV2_OK) return st;
+  const size_t ngt = plan.ghist_tiles.size(), ngo = plan.ghist_owner.size();
+  if ((st = grow(c, &c->d_ghist_tiles, &c->cap_ghist_tiles, ngt ? ngt : 1)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_ghist_owner, &c->cap_ghist_owner, ngo ? ngo : 1)) != QV2_OK) return st;
   const size_t b0 = nt * sizeof(TensorRec), b1 = ntl * sizeof(Tile), b2 = nh * sizeof(Tile);
-  if ((st = grow_pinned(c, b0 + b1 + b2)) != QV2_OK) return st;
+  const size_t b3 = ngt * sizeof(Tile), b4 = ngo * sizeof(uint32_t);
+  if ((st = grow_pinned(c, b0 + b1 + b2 + b3 + b4)) != QV2_OK) return st;
   std::memcpy(c->h_pinned, plan.tensors.data(), b0);
   if (b1) std::memcpy(c->h_pinned + b0, plan.tiles.data(), b1);
   if (b2) std::memcpy(c->h_pinned + b0 + b1, plan.hist_tiles.data(), b2);
   QV2_CUDA(c, cudaMemcpyAsync(c->d_tensors, c->h_pinned, b0, cudaMemcpyHostToDevice, c->stream));
   if (b1) QV2_CUDA(c, cudaMemcpyAsync(c->d_tiles, c->h_pinned + b0, b1, cudaMemcpyHostToDevice, c->stream));
   if (b2) QV2_CUDA(c, cudaMemcpyAsync(c->d_hist_tiles, c->h_pinned + b0 + b1, b2, cudaMemcpyHostToDevice, c->stream));
+  if (b3) {
+    std::memcpy(c->h_pinned + b0 + b1 + b2, plan.ghist_tiles.data(), b3);
+    std::memcpy(c->h_pinned + b0 + b1 + b2 + b3, plan.ghist_owner.data(), b4);
+    QV2_CUDA(c, cudaMemcpyAsync(c->d_ghist_tiles, c->h_pinned + b0 + b1 + b2, b3, cudaMemcpyHostToDevice, c->stream));
+    QV2_CUDA(c, cudaMemcpyAsync(c->d_ghist_owner, c->h_pinned + b0 + b1 + b2 + b3, b4, cudaMemcpyHostToDevice, c->stream));
+  }
   c->plan = std::move(plan);
   c->plan_key = std::move(key);
   c->plan_valid = true;
@@ -164,7 +177,7 @@ extern "C" int qv2_destroy(qv2_ctx* c) {
   if (!c) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
-  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_partials); cudaFree(c->d_rslots); cudaFree(c->d_partials_xe); cudaFree(c->d_kl_hist);
+  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_ghist_tiles); cudaFree(c->d_ghist_owner); cudaFree(c->d_ghist); cudaFree(c->d_partials); cudaFree(c->d_rslots); cudaFree(c->d_partials_xe); cudaFree(c->d_kl_hist);
   cudaFree(c->d_tensor_absmax); cudaFree(c->d_hist); cudaFree(c->d_rank);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
   delete c;
@@ -174,9 +187,10 @@ extern "C" int qv2_destroy(qv2_ctx* c) {
 extern "C" int qv2_last_cuda_error(const qv2_ctx* c) { return c ? c->last_cuda : 0; }
 extern "C" uint64_t qv2_launch_count(const qv2_ctx* c) { return c ? c->launches : 0; }
 
-extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* gmin,
-                             float* gmax, float* gabsmax, uint64_t* hist, float* clip, float* step,
-                             float* inv, float* offset, uint64_t* nonfinite) {
+extern "C" int qv2_calibrate_ex(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* gmin,
+                                float* gmax, float* gabsmax, uint64_t* hist, float* clip, float* step,
+                                float* inv, float* offset, uint64_t* nonfinite, uint64_t* group_hist,
+                                float* group_clip) {
   if (!c || !descs || !gmin || !gmax || !gabsmax || !clip || !step || !inv || !offset || !nonfinite)
     return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
@@ -188,6 +202,12 @@ extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t 
     if ((st = grow(c, &c->d_hist, &c->cap_hist, (size_t)n * kBins)) != QV2_OK) return st;
     h = c->d_hist;
   }
+  const size_t n_ghist = p.ghist_owner.size();
+  unsigned long long* gh = reinterpret_cast<unsigned long long*>(group_hist);
+  if (!gh && n_ghist) {
+    if ((st = grow(c, &c->d_ghist, &c->cap_ghist, n_ghist * kBins)) != QV2_OK) return st;
+    gh = c->d_ghist;
+  }
   const Launch l = launch_of(c);
   const size_t G = (size_t)p.total_groups;
   if (G) {
@@ -196,6 +216,7 @@ extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t 
   }
   QV2_CUDA(c, cudaMemsetAsync(nonfinite, 0, (size_t)n * sizeof(uint64_t), c->stream));
   if (h) QV2_CUDA(c, cudaMemsetAsync(h, 0, (size_t)n * kBins * sizeof(uint64_t), c->stream));
+  if (n_ghist) QV2_CUDA(c, cudaMemsetAsync(gh, 0, n_ghist * kBins * sizeof(uint64_t), c->stream));
   if (!p.tiles.empty()) {
     QV2_CUDA(c, launch_range(l, p.range_grid, p.any_16bit, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),
                              reinterpret_cast<uint32_t*>(gmin), reinterpret_cast<uint32_t*>(gmax),
@@ -213,7 +234,25 @@ extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t 
   QV2_CUDA(c, launch_clip_finalize(l, c->d_tensors, n, h, c->d_tensor_absmax, gmin, gmax, gabsmax,
                                    clip, step, inv, offset));
   ++c->launches;
+  if (n_ghist) {
+    QV2_CUDA(c, launch_group_hist(l, p.any_16bit, c->d_tensors, c->d_ghist_tiles, (uint32_t)p.ghist_tiles.size(),
+                                  gabsmax, reinterpret_cast<unsigned long long*>(nonfinite), gh));
+    QV2_CUDA(c, launch_group_clip_finalize(l, c->d_tensors, c->d_ghist_owner, (uint32_t)n_ghist, gh, gmin, gmax,
+                                           gabsmax, group_clip, step, inv, offset));
+    c->launches += p.ghist_tiles.empty() ? 1 : 2;
+  }
+  if (group_clip) {
+    QV2_CUDA(c, launch_fill_group_clip(l, c->d_tensors, n, clip, group_clip));
+    ++c->launches;
+  }
   return QV2_OK;
+}
+
+extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* gmin,
+                             float* gmax, float* gabsmax, uint64_t* hist, float* clip, float* step,
+                             float* inv, float* offset, uint64_t* nonfinite) {
+  return qv2_calibrate_ex(c, descs, n, gmin, gmax, gabsmax, hist, clip, step, inv, offset, nonfinite,
+                          nullptr, nullptr);
 }
 
 extern "C" int qv2_quant_metrics_ex(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n,

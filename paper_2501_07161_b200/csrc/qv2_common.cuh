@@ -34,7 +34,7 @@ struct TensorRec {
   uint32_t n_groups;
   uint32_t per_channel;
   uint32_t asym;             // 0: symmetric, 1: affine with real offset, 2: affine with integer zero point
-  uint32_t range_mode;       // QV2_ABSMAX | QV2_MINMAX | QV2_PERCENTILE
+  uint32_t range_mode;       // QV2_ABSMAX | QV2_MINMAX | QV2_PERCENTILE | QV2_PERCENTILE_GROUP (per-channel only)
   uint32_t pair_mode;        // PairMode
   uint32_t slot_first;       // first partial-sum slot of this tensor
   uint32_t slot_count;       // kWarps slots for every CTA of the metrics grid that owns a tile of it
@@ -43,6 +43,7 @@ struct TensorRec {
   uint32_t rslot_count;      //   one per CTA of the range grid that owns a tile of the tensor
   uint32_t bits;             // code width, 2..16 (8 unless the descriptor asks otherwise)
   uint32_t dtype;            // element type of x and y: 0 binary32, 1 binary16, 2 bfloat16
+  uint32_t ghist_first;      // QV2_PERCENTILE_GROUP: index of group 0's histogram among the per-group histograms
   double percentile;
 };
 
@@ -64,6 +65,8 @@ struct HostPlan {
   std::vector<TensorRec> tensors;
   std::vector<Tile> tiles;        // every tensor, in tensor order
   std::vector<Tile> hist_tiles;   // flat tiles of the tensors that need a histogram
+  std::vector<Tile> ghist_tiles;  // tiles (with their groups) of the tensors that need per-group histograms
+  std::vector<uint32_t> ghist_owner;   // per-group histogram -> tensor index
   uint64_t total_groups = 0;
   uint32_t total_slots = 0;
   uint32_t metrics_grid = 1;      // CTAs of the metrics launch; the slot layout depends on it
@@ -101,6 +104,15 @@ cudaError_t launch_clip_finalize(const Launch& l, const TensorRec* tensors, uint
                                  const unsigned long long* hist, const float* tensor_absmax,
                                  const float* gmin, const float* gmax, const float* gabsmax,
                                  float* clip, float* step, float* inv, float* offset);
+cudaError_t launch_group_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
+                              uint32_t n_tiles, const float* gabsmax, const unsigned long long* nonfinite,
+                              unsigned long long* ghist);
+cudaError_t launch_group_clip_finalize(const Launch& l, const TensorRec* tensors, const uint32_t* owner,
+                                       uint32_t n_hists, const unsigned long long* ghist,
+                                       const float* gmin, const float* gmax, const float* gabsmax,
+                                       float* group_clip, float* step, float* inv, float* offset);
+cudaError_t launch_fill_group_clip(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
+                                   const float* clip, float* group_clip);
 cudaError_t launch_metrics(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors,
                            const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
                            const float* offset, double2* partials, double* partials_xe);

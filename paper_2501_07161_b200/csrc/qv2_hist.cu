@@ -120,7 +120,7 @@ clip_finalize_kernel(const TensorRec* __restrict__ tensors, const unsigned long 
   const uint32_t t = blockIdx.x, tid = threadIdx.x;
   const TensorRec tr = tensors[t];
   const float A = tensor_absmax[t];
-  if (tr.range_mode != QV2_PERCENTILE) {
+  if (tr.range_mode != QV2_PERCENTILE) {     // per-group percentile included: its clips are per group
     if (tid == 0) clip[t] = A;
     return;
   }
@@ -165,7 +165,190 @@ clip_finalize_kernel(const TensorRec* __restrict__ tensors, const unsigned long 
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Per-group histograms (range mode QV2_PERCENTILE_GROUP on per-channel tensors): the same binning,
+// on [0, absmax_g] of each group, one 2048-bin histogram per group.
+//
+// One-group tiles go through the CTA's shared-memory histogram, which is merged into the group's
+// global histogram whenever the group changes; CTAs take runs of kGroupChunk consecutive tiles so
+// that the three or four tiles of one long row are merged once.  Tiles of whole short rows are
+// walked one warp per row and counted straight into global memory, lanes that fall into the same
+// bin combined into one atomic.
+constexpr uint32_t kGroupChunk = 8;
+
+__device__ __forceinline__ float bin_scale(float A) {
+  float w = (A > 0.0f) ? __fdiv_rn((float)kBins, A) : 0.0f;
+  return isfinite(w) ? w : 0.0f;
+}
+
+template <class T>
+__device__ __forceinline__ void group_hist_rows(const T* x, const Tile& tl, const TensorRec* tr,
+                                                const float* __restrict__ gabsmax, unsigned long long* ghist,
+                                                uint32_t lane, uint32_t warp) {
+  const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+  for (uint32_t r = warp; r < tl.rows; r += kWarps) {
+    const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
+    const float w = bin_scale(gabsmax[tr->group_base + g]);
+    unsigned long long* h = ghist + (size_t)(tr->ghist_first + g) * kBins;
+    const T* row = x + (uint64_t)r * inner;
+    for (uint32_t i0 = 0; i0 < inner; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      uint32_t b = 0xffffffffu;                       // lanes past the row's end, NaN and Inf: no bin
+      if (i < inner) {
+        const float v = Ld<T>::one(row + i);
+        if (isfinite(v)) b = bin_of(v, w);
+      }
+      const uint32_t same = __match_any_sync(0xffffffffu, b);
+      if (b != 0xffffffffu && lane == (uint32_t)__ffs(same) - 1u)
+        atomicAdd(h + b, (unsigned long long)__popc(same));
+    }
+  }
+}
+
+template <bool ANY16>
+__global__ void __launch_bounds__(kThreads, 4)
+group_hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
+                  const float* __restrict__ gabsmax, const unsigned long long* __restrict__ nonfinite,
+                  unsigned long long* ghist) {
+  __shared__ uint32_t sh[kBins];
+  for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
+  __syncthreads();
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+
+  bool have = false;                 // sh holds counts of group cur_g of tensor cur_t
+  uint32_t cur_t = 0, cur_g = 0, zeros = 0, since_flush = 0;
+  float w = 0.0f;
+  bool careful = false;
+  auto flush = [&]() {
+    if (zeros) atomicAdd(sh, zeros);
+    zeros = 0;
+    __syncthreads();
+    unsigned long long* h = ghist + (size_t)(tensors[cur_t].ghist_first + cur_g) * kBins;
+    for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {
+      const uint32_t c = sh[b];
+      if (c) { atomicAdd(h + b, (unsigned long long)c); sh[b] = 0; }
+    }
+    __syncthreads();
+    have = false; since_flush = 0;
+  };
+
+  for (uint64_t base = (uint64_t)blockIdx.x * kGroupChunk; base < n_tiles; base += (uint64_t)gridDim.x * kGroupChunk) {
+    for (uint32_t k = 0; k < kGroupChunk && base + k < n_tiles; ++k) {
+      const Tile tl = load_tile(tiles, (uint32_t)(base + k));
+      const TensorRec* tr = tensors + tl.tensor;
+      if (tl.rows == 0) {
+        const uint32_t g = (uint32_t)tl.row0;
+        // 32-bit counts: merge before 2^14 tiles of 2^14 elements have gone into them
+        if (have && (tl.tensor != cur_t || g != cur_g || since_flush >= 16384u)) flush();
+        if (!have) {
+          have = true; cur_t = tl.tensor; cur_g = g;
+          w = bin_scale(gabsmax[tr->group_base + g]);
+          careful = nonfinite[cur_t] != 0ull;
+        }
+        if (!ANY16 || tr->dtype == kF32) hist_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+        else if (tr->dtype == kF16) hist_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+        else hist_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+        ++since_flush;
+      } else {
+        if (!ANY16 || tr->dtype == kF32) group_hist_rows(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, gabsmax, ghist, lane, warp);
+        else if (tr->dtype == kF16) group_hist_rows(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, gabsmax, ghist, lane, warp);
+        else group_hist_rows(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, gabsmax, ghist, lane, warp);
+      }
+    }
+  }
+  if (have) flush();
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// One warp per group histogram: the group's clip by the same cumulative-count rule as
+// clip_finalize_kernel, then the group's quantization parameters.
+__global__ void __launch_bounds__(256)
+group_clip_finalize_kernel(const TensorRec* __restrict__ tensors, const uint32_t* __restrict__ owner,
+                           uint32_t n_hists, const unsigned long long* __restrict__ ghist,
+                           const float* __restrict__ gmin, const float* __restrict__ gmax,
+                           const float* __restrict__ gabsmax, float* group_clip, float* step, float* inv,
+                           float* offset) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t hidx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (hidx >= n_hists) return;
+  const TensorRec* tr = tensors + owner[hidx];
+  const uint32_t G = tr->group_base + (hidx - tr->ghist_first);
+  const unsigned long long* h = ghist + (size_t)hidx * kBins;
+  const float A = gabsmax[G];
+  unsigned long long nf = 0;
+  for (uint32_t i = 0; i < kBins / 32; ++i) nf += h[i * 32 + lane];
+  nf = warp_sum_u64(nf);
+  float c = A;
+  if (nf != 0ull) {
+    const double tt = ceil(__dmul_rn(tr->percentile, (double)nf));
+    unsigned long long T;
+    if (!(tt >= 1.0)) T = 1ull;
+    else if (tt >= (double)nf) T = nf;
+    else T = (unsigned long long)tt;
+    unsigned long long carry = 0;
+    uint32_t kstar = kBins - 1;
+    for (uint32_t i = 0; i < kBins / 32; ++i) {
+      unsigned long long s = h[i * 32 + lane];          // inclusive scan of 32 consecutive bins
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xffffffffu, s, o);
+        if ((int)lane >= o) s += up;
+      }
+      const uint32_t reached = __ballot_sync(0xffffffffu, carry + s >= T);
+      if (reached) { kstar = i * 32 + (uint32_t)__ffs(reached) - 1u; break; }
+      carry += __shfl_sync(0xffffffffu, s, 31);
+    }
+    if (kstar != kBins - 1) c = __fmul_rn((float)(kstar + 1), __fdiv_rn(A, (float)kBins));
+  }
+  if (lane == 0) {
+    if (group_clip) group_clip[G] = c;
+    make_qparams(tr->asym, top_code(tr->asym != 0, tr->bits), true, c, gmin[G], gmax[G], A, step + G, inv + G, offset + G);
+  }
+}
+
+// group_clip for the tensors without per-group histograms: the tensor's clip.
+__global__ void __launch_bounds__(256)
+fill_group_clip_kernel(const TensorRec* __restrict__ tensors, const float* __restrict__ clip, float* group_clip) {
+  const TensorRec* tr = tensors + blockIdx.x;
+  if (tr->range_mode == QV2_PERCENTILE_GROUP) return;
+  const float c = clip[blockIdx.x];
+  for (uint32_t g = threadIdx.x; g < tr->n_groups; g += blockDim.x) group_clip[tr->group_base + g] = c;
+}
+
 }  // namespace
+
+cudaError_t launch_group_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
+                              uint32_t n_tiles, const float* gabsmax, const unsigned long long* nonfinite,
+                              unsigned long long* ghist) {
+  if (n_tiles == 0) return cudaSuccess;
+  static int per_sm = 0;
+  const uint32_t chunks = (n_tiles + kGroupChunk - 1) / kGroupChunk;
+  const int grid = persistent_grid((const void*)group_hist_kernel<false>, &per_sm, l.sm_count, chunks);
+  if (any16) group_hist_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, gabsmax, nonfinite, ghist);
+  else group_hist_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, gabsmax, nonfinite, ghist);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_group_clip_finalize(const Launch& l, const TensorRec* tensors, const uint32_t* owner,
+                                       uint32_t n_hists, const unsigned long long* ghist,
+                                       const float* gmin, const float* gmax, const float* gabsmax,
+                                       float* group_clip, float* step, float* inv, float* offset) {
+  if (n_hists == 0) return cudaSuccess;
+  group_clip_finalize_kernel<<<(n_hists + 7) / 8, 256, 0, l.stream>>>(tensors, owner, n_hists, ghist, gmin, gmax,
+                                                                     gabsmax, group_clip, step, inv, offset);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fill_group_clip(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
+                                   const float* clip, float* group_clip) {
+  fill_group_clip_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, clip, group_clip);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
                         uint32_t n_tiles, const float* tensor_absmax,

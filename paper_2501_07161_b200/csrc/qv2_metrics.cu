@@ -594,7 +594,7 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   if (!desc || !step || !inv || !offset || !result4) return QV2_ERR_NULL;
   if (device < 0 || device >= kMaxDevices) return QV2_ERR_ARG;
   const qv2_tensor_desc& d = *desc;
-  if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE)
+  if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE_GROUP)
     return QV2_ERR_ARG;
   if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_BITS_MASK)) return QV2_ERR_ARG;   // no code output here
   if (QV2_DESC_BITS(d.flags) < 2 || QV2_DESC_BITS(d.flags) > 16) return QV2_ERR_ARG;

@@ -26,12 +26,13 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
   if (!descs || !out) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   out->tensors.clear(); out->tiles.clear(); out->hist_tiles.clear();
+  out->ghist_tiles.clear(); out->ghist_owner.clear();
   out->total_groups = 0; out->total_slots = 0; out->any_percentile = false; out->any_16bit = false;
   out->tensors.reserve(n);
   uint64_t groups = 0;
   for (uint32_t t = 0; t < n; ++t) {
     const qv2_tensor_desc& d = descs[t];
-    if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE)
+    if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE_GROUP)
       return QV2_ERR_ARG;
     if (d.flags & ~(uint32_t)(QV2_PAIR_RAW | QV2_STORE_CODES | QV2_BITS_MASK | QV2_IN_MASK)) return QV2_ERR_ARG;
     const uint32_t dtype = (d.flags & QV2_IN_MASK) >> 16;
@@ -39,7 +40,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     const uint32_t bits = QV2_DESC_BITS(d.flags);
     if (bits < 2 || bits > 16) return QV2_ERR_ARG;
     if ((d.flags & QV2_STORE_CODES) && bits > 8) return QV2_ERR_UNSUPPORTED;   // codes are one byte
-    if (d.range == QV2_PERCENTILE && !(d.percentile >= 0.0 && d.percentile <= 1.0))
+    if (d.range >= QV2_PERCENTILE && !(d.percentile >= 0.0 && d.percentile <= 1.0))
       return QV2_ERR_ARG;
     uint64_t rows, ne;
     if (mul_overflows(d.outer, d.channels, &rows) || rows > (1ull << 62)) return QV2_ERR_SIZE;
@@ -62,7 +63,14 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     r.group_base = (uint32_t)groups;
     groups += r.n_groups;
     r.asym = d.scheme;                  // 0 symmetric, 1 affine with real offset, 2 affine with zero point
-    r.range_mode = d.range;
+    // one group: its histogram is the tensor's, so the per-group mode is the per-tensor one
+    r.range_mode = (d.range == QV2_PERCENTILE_GROUP && !r.per_channel) ? (uint32_t)QV2_PERCENTILE : d.range;
+    r.ghist_first = 0;
+    if (r.range_mode == QV2_PERCENTILE_GROUP) {
+      if (out->ghist_owner.size() + r.n_groups >= (1ull << 32)) return QV2_ERR_SIZE;
+      r.ghist_first = (uint32_t)out->ghist_owner.size();
+      out->ghist_owner.insert(out->ghist_owner.end(), r.n_groups, t);
+    }
     r.pair_mode = !pair ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
     r.percentile = d.percentile;
     r.bits = bits;
@@ -70,7 +78,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     if (dtype != kF32) out->any_16bit = true;
 
     size_t first_tile = out->tiles.size();
-    if (d.range == QV2_PERCENTILE) out->any_percentile = true;
+    if (r.range_mode == QV2_PERCENTILE) out->any_percentile = true;
     if (ne > 0) {
       if (!r.per_channel) {
         cut_flat(t, 0, ne, 0, &out->tiles);
@@ -87,7 +95,9 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
           out->tiles.push_back(tl);
         }
       }
-      if (d.range == QV2_PERCENTILE) cut_flat(t, 0, ne, 0, &out->hist_tiles);
+      if (r.range_mode == QV2_PERCENTILE) cut_flat(t, 0, ne, 0, &out->hist_tiles);
+      if (r.range_mode == QV2_PERCENTILE_GROUP)
+        out->ghist_tiles.insert(out->ghist_tiles.end(), out->tiles.begin() + first_tile, out->tiles.end());
     }
     if (first_tile >= (1ull << 31)) return QV2_ERR_SIZE;
     r.tile_first = (uint32_t)first_tile;
@@ -95,7 +105,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     r.rslot_first = 0; r.rslot_count = 0;
     out->tensors.push_back(r);
   }
-  if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;
+  if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;   // ghist_tiles is a subset of tiles
   // Slots written with plain stores instead of atomics.  In both persistent kernels CTA b walks
   // tiles b, b+grid, ...; a tensor whose tiles are [first, first+count) is therefore touched by
   // min(grid, count) CTAs.  The metrics kernel gives each warp of those CTAs one partial-sum slot;
@@ -138,6 +148,14 @@ extern "C" uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n) {
   if (!descs) return 0;
   for (uint32_t t = 0; t < n; ++t)
     g += descs[t].granularity == QV2_PER_CHANNEL ? descs[t].channels : 1;
+  return g;
+}
+
+extern "C" uint64_t qv2_group_hist_count(const qv2_tensor_desc* descs, uint32_t n) {
+  uint64_t g = 0;
+  if (!descs) return 0;
+  for (uint32_t t = 0; t < n; ++t)
+    if (descs[t].range == QV2_PERCENTILE_GROUP && descs[t].granularity == QV2_PER_CHANNEL) g += descs[t].channels;
   return g;
 }
 

@@ -233,7 +233,7 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __rest
     const float am = fmaxf(fabsf(mn), fabsf(mx));
     gmin[G] = mn; gmax[G] = mx; gabsmax[G] = am;
     amax = fmaxf(amax, am);
-    if (tr.range_mode != QV2_PERCENTILE)
+    if (tr.range_mode < QV2_PERCENTILE)      // the percentile modes set theirs once the clip is known
       make_qparams(tr.asym, top_code(tr.asym != 0, tr.bits), false, 0.0f, mn, mx, am, step + G, inv + G, offset + G);
   }
   red[threadIdx.x] = amax;

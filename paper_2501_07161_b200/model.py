@@ -20,12 +20,16 @@ class ModelDescs:
     rate_permyriad: int
 
 
-def model_descs(model, host: bool = False) -> ModelDescs:
+def model_descs(model, host: bool = False, act_granularity: str = "tensor") -> ModelDescs:
     """`model` is any object with `.layers` (each with w [cout,K], x and y [B,C,HW], macs) and
-    `.config` (w_granularity, a_range, a_percentile, bops_rate_permyriad)."""
+    `.config` (w_granularity, a_range, a_percentile, bops_rate_permyriad).  The paper's set-ups
+    quantize activations per tensor; act_granularity="channel" is the per-channel variant, with
+    one percentile clip per channel where the configuration clips at all."""
     cfg = model.config
     gran = {"tensor": B.PER_TENSOR, "channel": B.PER_CHANNEL}
     a_range = B.PERCENTILE if cfg.a_range == "percentile" else B.MINMAX
+    if a_range == B.PERCENTILE and act_granularity == "channel":
+        a_range = B.PERCENTILE_GROUP
     descs, keep = [], []
     L = model.layers
     for l in L:
@@ -34,8 +38,8 @@ def model_descs(model, host: bool = False) -> ModelDescs:
         keep.append(l.w)
     for l in L:
         b, c, hw = l.x.shape
-        descs.append(B.make_desc(l.x, l.y, b, c, hw, B.PER_TENSOR, B.ASYM_U8, a_range,
-                                 cfg.a_percentile if a_range == B.PERCENTILE else 0.0))
+        descs.append(B.make_desc(l.x, l.y, b, c, hw, gran[act_granularity], B.ASYM_U8, a_range,
+                                 cfg.a_percentile if a_range != B.MINMAX else 0.0))
         keep += [l.x, l.y]
     for g in cfg.w_granularity[1:]:
         for l in L:

@@ -34,6 +34,7 @@ class Spec:
     bits: int = 8
     dtype: torch.dtype = torch.float32  # element type the GPU side stores x and y in
     zp: bool = False                   # affine scheme with an integer zero point (implies asym)
+    group_pct: bool = False            # percentile clip per channel (own histogram per group)
 
 
 def bits(a) -> np.ndarray:
@@ -60,7 +61,7 @@ def make_descs(specs: List[Spec], dev_x, dev_y, store_codes=True):
         descs.append(q.make_desc(dx, dy, s.outer, s.channels, s.inner,
                                  q.PER_CHANNEL if s.per_channel else q.PER_TENSOR,
                                  q.ASYM_U8_ZP if s.zp else (q.ASYM_U8 if s.asym else q.SYM_I8),
-                                 q.PERCENTILE if s.percentile is not None else (q.MINMAX if (s.asym or s.zp) else q.ABSMAX),
+                                 (q.PERCENTILE_GROUP if s.group_pct else q.PERCENTILE) if s.percentile is not None else (q.MINMAX if (s.asym or s.zp) else q.ABSMAX),
                                  s.percentile or 0.0, flags, s.bits))
     return q.desc_array(descs)
 
@@ -73,7 +74,8 @@ def oracle_tensor(s: Spec, want_codes=True):
     if y is not None:
         mode = oracle.PAIR_RAW if s.raw else oracle.PAIR_REQUANT
     return oracle.sweep_tensor(x, y, s.outer, s.channels, s.inner, s.per_channel, 2 if s.zp else s.asym,
-                               s.percentile, pair_mode=mode, want_codes=want_codes and not s.raw, bits=s.bits)
+                               s.percentile, pair_mode=mode, want_codes=want_codes and not s.raw, bits=s.bits,
+                               group_percentile=s.group_pct)
 
 
 def assert_metric_close(got_mse, got_sqnr, ref_mse, ref_sqnr, what=""):
@@ -94,7 +96,8 @@ def check_specs(ctx, specs: List[Spec], misalign_x=0, misalign_y=0, check_codes=
     dev_x = [to_dev(s.x, misalign_x, s.dtype) for s in specs]
     dev_y = [to_dev(s.y, misalign_y, s.dtype) for s in specs]
     descs = make_descs(specs, dev_x, dev_y, store_codes=check_codes)
-    cal = ctx.calibrate(descs)
+    want_group = any(s.group_pct for s in specs)
+    cal = ctx.calibrate(descs, want_group=want_group)
     codes = None
     if check_codes:
         codes = [None if s.raw else torch.full((max(s.x.numel(), 1),), 0x55, dtype=torch.uint8, device="cuda")
@@ -109,7 +112,11 @@ def check_specs(ctx, specs: List[Spec], misalign_x=0, misalign_y=0, check_codes=
             assert np.array_equal(a.cpu().numpy().view(np.uint64), b.cpu().numpy().view(np.uint64)), \
                 "two runs differ"
     g = 0
+    gh = 0                     # running index into the per-group histograms
     hist = cal.hist.cpu().numpy().view(np.uint64).reshape(-1, q.HIST_BINS)
+    if want_group:
+        ghist = cal.group_hist.cpu().numpy().view(np.uint64).reshape(-1, q.HIST_BINS)
+        gclip = cal.group_clip.cpu().numpy()
     for t, s in enumerate(specs):
         ref = oracle_tensor(s, want_codes=check_codes)
         ng = s.channels if s.per_channel else 1
@@ -122,7 +129,15 @@ def check_specs(ctx, specs: List[Spec], misalign_x=0, misalign_y=0, check_codes=
         assert int(cal.nonfinite[t]) == ref.nonfinite, f"{name}: nonfinite"
         assert bits(cal.clip[t:t + 1].cpu().numpy())[0] == bits([ref.clip])[0], \
             f"{name}: clip {float(cal.clip[t])} vs {ref.clip}"
-        if s.percentile is not None:
+        if want_group:
+            assert np.array_equal(bits(gclip[sl]), bits(ref.gclip)), f"{name}: group clips differ"
+        if ref.ghist is not None:
+            got = ghist[gh:gh + ng]
+            assert np.array_equal(got, ref.ghist), \
+                f"{name}: per-group histograms differ in groups {np.nonzero((got != ref.ghist).any(axis=1))[0][:8]}"
+            assert not hist[t].any()
+            gh += ng
+        elif s.percentile is not None:
             assert np.array_equal(hist[t], ref.hist), f"{name}: histogram differs"
             assert int(hist[t].sum()) == s.x.numel() - ref.nonfinite
         else:

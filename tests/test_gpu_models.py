@@ -28,7 +28,7 @@ def _np(t):
     return t.detach().cpu().numpy()
 
 
-def oracle_layer_jobs(model, layer_ids=None):
+def oracle_layer_jobs(model, layer_ids=None, act_per_channel=False):
     """Oracle jobs in the library's descriptor order: weights, activations, extra weight scorings."""
     cfg = model.config
     layers = model.layers if layer_ids is None else [model.layers[i] for i in layer_ids]
@@ -40,7 +40,8 @@ def oracle_layer_jobs(model, layer_ids=None):
     for l in layers:
         b, c, hw = l.x.shape
         jobs.append(dict(x=_np(l.x).reshape(-1), y=_np(l.y).reshape(-1), outer=b, channels=c, inner=hw,
-                         per_channel=False, asym_u8=True, percentile=pct))
+                         per_channel=act_per_channel, asym_u8=True, percentile=pct,
+                         group_percentile=act_per_channel))
     for g in cfg.w_granularity[1:]:
         for l in layers:
             jobs.append(dict(x=_np(l.w).reshape(-1), y=None, outer=1, channels=l.w.shape[0],
@@ -57,8 +58,8 @@ def py_scores(sw, mw, sa, ma, wg=2.0, ag=1.0, cap=200.0):
     return sc, sev
 
 
-def run_sweep(ctx, model):
-    md = q.model_descs(model)
+def run_sweep(ctx, model, act_granularity="tensor"):
+    md = q.model_descs(model, act_granularity=act_granularity)
     cfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
     sb, t = ctx.alloc_sweep_buffers(md.descs, md.n_layers)
     ctx.sweep_model(md.descs, md.n_layers, md.macs, None, cfg, sb)
@@ -79,6 +80,20 @@ def compare_tensor(t, idx, g0, ref, name, check_hist):
     else:
         assert not h.any()
     assert_metric_close(float(t["mse"][idx]), float(t["sqnr_db"][idx]), ref.mse, ref.sqnr_db, name)
+
+
+@pytest.mark.parametrize("name,batch", [("resnet18", 3), ("mobilenetv2", 2), ("squeezenet", 1)])
+def test_model_sweep_with_per_channel_activations_matches_oracle(ctx, name, batch):
+    """The per-channel variant of the activation quantizer over whole models: every channel of every
+    layer its own range and, where the configuration clips, its own histogram and clip."""
+    model = gen.make_model(name, seed=3, device="cuda", batch=batch)
+    md, t = run_sweep(ctx, model, act_granularity="channel")
+    refs = oracle.sweep_tensors(oracle_layer_jobs(model, act_per_channel=True), threads=8)
+    g0 = 0
+    for idx, ref in enumerate(refs):
+        compare_tensor(t, idx, g0, ref, f"{name}[{idx}] per-channel activations", check_hist=ref.hist is not None)
+        g0 += ref.step.size
+    assert g0 == int(q.lib().qv2_group_count(md.descs, md.n_tensors))
 
 
 @pytest.mark.parametrize("name,batch", [("squeezenet", 1), ("resnet18", 2), ("resnet50", 1),

@@ -483,3 +483,95 @@ def test_half_precision_nonfinite_and_mixed_batch(ctx):
     big = torch.tensor([70000.0, 1.0]).repeat(50)            # overflows binary16: stored as Inf
     cal, _ = check_specs(ctx, [Spec(big, 1, 1, 100, dtype=torch.float16)], check_codes=False)
     assert int(cal.nonfinite[0]) == 50
+
+
+# ------------------------------------------------------------ per-channel percentile (own histograms)
+def _scaled_channels(o, c, i, seed, relu=False):
+    """Channels whose scales differ by orders of magnitude, the case the per-group clip is for."""
+    x = torch.randn(o, c, i, generator=_g(seed)) * (10.0 ** torch.linspace(-2, 2, c))[None, :, None]
+    return x.clamp_min(0) if relu else x
+
+
+def test_group_percentile_long_rows_short_rows_and_batches(ctx):
+    specs = []
+    for (o, c, i), seed in (((1, 3, 3 * TILE + 100), 201),        # rows cut into several one-group tiles
+                            ((4, 5, 5000), 202),                  # one tile per row, groups revisited per batch item
+                            ((1, 96, 1153), 203),                 # short ragged rows, several per tile
+                            ((8, 20, 49), 204),                   # 7x7 maps: 334 rows per tile
+                            ((3, 7, 1), 205),                     # one element per row
+                            ((2, 2, 4096), 206)):                 # exactly at the row-tile threshold
+        for asym, zp, p in ((False, False, 0.999), (True, False, 0.99), (False, True, 0.95)):
+            specs.append(Spec(_scaled_channels(o, c, i, seed, relu=asym), o, c, i, per_channel=True, asym=asym, zp=zp,
+                              percentile=p, group_pct=True, name=f"group-pct {o}x{c}x{i} asym={asym} zp={zp}"))
+    check_specs(ctx, specs)
+    check_specs(ctx, specs[:6], misalign_x=3, check_codes=False)
+
+
+def test_group_percentile_mixed_with_other_modes_keeps_the_layouts_apart(ctx):
+    """Per-group histograms exist only for the tensors that ask for them, in descriptor order; the
+    per-tensor histograms, the plain modes and the pair mode around them must be untouched."""
+    n = 2 * TILE + 33
+    a = _scaled_channels(2, 6, 3000, 211, relu=True)
+    specs = [Spec(randn(n, 212), 1, 1, n, asym=True, percentile=0.999),
+             Spec(a, 2, 6, 3000, per_channel=True, asym=True, percentile=0.99, group_pct=True,
+                  y=a + 0.01 * torch.randn(a.shape, generator=_g(213))),
+             Spec(randn(64 * 300, 214), 1, 64, 300, per_channel=True),
+             Spec(randn(n, 215), 1, 1, n, asym=True, percentile=0.9, group_pct=True),     # per tensor: same as PERCENTILE
+             Spec(_scaled_channels(1, 4, 20000, 216), 1, 4, 20000, per_channel=True, percentile=0.9999, group_pct=True),
+             Spec(_scaled_channels(2, 6, 3000, 217), 2, 6, 3000, per_channel=True, percentile=0.99)]  # tensor-level clip
+    cal, _ = check_specs(ctx, specs)
+    assert int(q.lib().qv2_group_hist_count(q.desc_array([]), 0)) == 0
+
+
+def test_group_percentile_nonfinite_constant_and_empty_groups(ctx):
+    o, c, i = 2, 4, 6000
+    x = _scaled_channels(o, c, i, 221)
+    x[0, 1, 17] = float("nan"); x[1, 1, 5999] = float("inf")     # skipped in channel 1's histogram
+    x[:, 2, :] = 0.0                                             # absmax 0: everything in bin 0, degenerate range
+    x[:, 3, :] = -3.5                                            # constant: one bin, clip = absmax
+    specs = [Spec(x, o, c, i, per_channel=True, percentile=0.99, group_pct=True),
+             Spec(x[:, :, :77].contiguous(), o, c, 77, per_channel=True, asym=True, percentile=0.99, group_pct=True),
+             Spec(torch.zeros(0), 1, 5, 0, per_channel=True, percentile=0.5, group_pct=True)]   # no elements at all
+    check_specs(ctx, specs, check_codes=False)
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_group_percentile_sixteen_bit_inputs(ctx, dtype):
+    specs = [Spec(_scaled_channels(2, 5, 9000, 231), 2, 5, 9000, per_channel=True, percentile=0.999, group_pct=True, dtype=dtype),
+             Spec(_scaled_channels(3, 33, 200, 232, relu=True), 3, 33, 200, per_channel=True, asym=True, percentile=0.99,
+                  group_pct=True, dtype=dtype)]
+    check_specs(ctx, specs, check_codes=False)
+    check_specs(ctx, specs, misalign_x=1, check_codes=False)
+
+
+def test_group_percentile_in_the_chained_pass_and_its_graph(ctx):
+    """qv2_sweep_model and the captured pass accept the mode (histograms stay in context scratch)."""
+    w = randn(32 * 500, 241)
+    a = _scaled_channels(4, 32, 400, 242, relu=True)
+    y = a + 0.02 * torch.randn(a.shape, generator=_g(243))
+    dw, da, dy = w.cuda(), a.reshape(-1).cuda(), y.reshape(-1).cuda()
+    descs = q.desc_array([q.make_desc(dw, None, 1, 32, 500, q.PER_CHANNEL, q.SYM_I8),
+                          q.make_desc(da, dy, 4, 32, 400, q.PER_CHANNEL, q.ASYM_U8, q.PERCENTILE_GROUP, 0.99)])
+    cfg = q.default_rank_cfg(select_mode=q.BY_COUNT, keep_count=1)
+    macs = torch.ones(1, dtype=torch.int64, device="cuda")
+    sb, t = ctx.alloc_sweep_buffers(descs, 1)
+    ctx.sweep_model(descs, 1, macs, None, cfg, sb)
+    torch.cuda.synchronize()
+    ref = oracle.sweep_tensor(a.numpy().reshape(-1), y.numpy().reshape(-1), 4, 32, 400, True, True, 0.99,
+                              group_percentile=True)
+    assert np.array_equal(t["step"][32:64].cpu().numpy().view(np.uint32), ref.step.view(np.uint32))
+    assert_metric_close(float(t["mse"][1]), float(t["sqnr_db"][1]), ref.mse, ref.sqnr_db, "chained group-pct")
+    first = [float(t["mse"][1]), float(t["sqnr_db"][1])]
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        gctx = q.Context(0, stream=s)
+        try:
+            sb2, t2 = gctx.alloc_sweep_buffers(descs, 1)
+            graph = gctx.sweep_graph(descs, 1, macs, None, cfg, sb2)
+            t2["mse"].zero_(); t2["step"].zero_()
+            graph.launch()
+            s.synchronize()
+            assert [float(t2["mse"][1]), float(t2["sqnr_db"][1])] == first
+            assert torch.equal(t2["step"], t["step"])
+        finally:
+            gctx.close()
