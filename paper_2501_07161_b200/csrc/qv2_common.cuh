@@ -15,6 +15,8 @@ constexpr int kThreads = 256;            // threads per CTA in the streaming ker
 constexpr int kWarps = kThreads / 32;
 constexpr uint32_t kTileElems = 16384;   // elements per tile (64 KiB of fp32)
 constexpr uint64_t kRowTileMin = 4096;   // rows at least this long are cut into one-group tiles
+constexpr uint64_t kGroupUnitElems = 131072;   // elements per unit of the per-group histogram pass
+constexpr uint64_t kGroupSegMax = 1ull << 22;   // longest contiguous segment of such a unit
 constexpr int kBins = QV2_HIST_BINS;
 constexpr uint32_t kMaxRankLayers = 8192;
 
@@ -65,7 +67,7 @@ struct HostPlan {
   std::vector<TensorRec> tensors;
   std::vector<Tile> tiles;        // every tensor, in tensor order
   std::vector<Tile> hist_tiles;   // flat tiles of the tensors that need a histogram
-  std::vector<Tile> ghist_tiles;  // tiles (with their groups) of the tensors that need per-group histograms
+  std::vector<Tile> ghist_tiles;  // group-major units of the tensors that need per-group histograms (see build_plan)
   std::vector<uint32_t> ghist_owner;   // per-group histogram -> tensor index
   uint64_t total_groups = 0;
   uint32_t total_slots = 0;

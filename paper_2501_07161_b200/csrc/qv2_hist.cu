@@ -169,94 +169,86 @@ clip_finalize_kernel(const TensorRec* __restrict__ tensors, const unsigned long 
 // Per-group histograms (range mode QV2_PERCENTILE_GROUP on per-channel tensors): the same binning,
 // on [0, absmax_g] of each group, one 2048-bin histogram per group.
 //
-// One-group tiles go through the CTA's shared-memory histogram, which is merged into the group's
-// global histogram whenever the group changes; CTAs take runs of kGroupChunk consecutive tiles so
-// that the three or four tiles of one long row are merged once.  Tiles of whole short rows are
-// walked one warp per row and counted straight into global memory, lanes that fall into the same
-// bin combined into one atomic.
-constexpr uint32_t kGroupChunk = 8;
-
+// The pass is group-major: a unit is `rows` segments of `count` contiguous elements of ONE group
+// (the same channel of consecutive batch items), about 128 K elements.  A CTA counts a whole unit
+// into its shared-memory histogram and merges it into the group's global histogram once, at the
+// end of the unit.  Long segments are walked by the whole CTA, short ones by one warp each.
 __device__ __forceinline__ float bin_scale(float A) {
   float w = (A > 0.0f) ? __fdiv_rn((float)kBins, A) : 0.0f;
   return isfinite(w) ? w : 0.0f;
 }
 
+// One segment handled by one warp: 16-byte loads over the aligned body, scalars at the ends.
+template <bool CAREFUL, class T>
+__device__ __forceinline__ void hist_segment_warp(const T* __restrict__ x, uint32_t count, uint32_t lane,
+                                                  float w, uint32_t* sh, uint32_t& zeros) {
+  const FlatSplit s = split_flat(x, count);
+  const T* xv = x + s.head;
+  uint32_t j = lane;
+  for (; j + 96 < s.nvec; j += 128) {
+    float4 v[4];
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u) v[u] = ld_vec_at(xv, j + 32u * u);
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u) {
+      hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
+      hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
+    }
+  }
+  for (; j < s.nvec; j += 32) {
+    const float4 v = ld_vec_at(xv, j);
+    hist_elem<CAREFUL>(v.x, w, sh, zeros); hist_elem<CAREFUL>(v.y, w, sh, zeros);
+    hist_elem<CAREFUL>(v.z, w, sh, zeros); hist_elem<CAREFUL>(v.w, w, sh, zeros);
+  }
+  if (lane < s.head) hist_elem<CAREFUL>(Ld<T>::one(x + lane), w, sh, zeros);
+  if (lane < s.tail) hist_elem<CAREFUL>(Ld<T>::one(x + s.head + 4u * s.nvec + lane), w, sh, zeros);
+}
+
+constexpr uint32_t kWarpSegmentMax = 2048;     // shorter segments go one per warp
+
 template <class T>
-__device__ __forceinline__ void group_hist_rows(const T* x, const Tile& tl, const TensorRec* tr,
-                                                const float* __restrict__ gabsmax, unsigned long long* ghist,
-                                                uint32_t lane, uint32_t warp) {
-  const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
-  for (uint32_t r = warp; r < tl.rows; r += kWarps) {
-    const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
-    const float w = bin_scale(gabsmax[tr->group_base + g]);
-    unsigned long long* h = ghist + (size_t)(tr->ghist_first + g) * kBins;
-    const T* row = x + (uint64_t)r * inner;
-    for (uint32_t i0 = 0; i0 < inner; i0 += 32) {
-      const uint32_t i = i0 + lane;
-      uint32_t b = 0xffffffffu;                       // lanes past the row's end, NaN and Inf: no bin
-      if (i < inner) {
-        const float v = Ld<T>::one(row + i);
-        if (isfinite(v)) b = bin_of(v, w);
-      }
-      const uint32_t same = __match_any_sync(0xffffffffu, b);
-      if (b != 0xffffffffu && lane == (uint32_t)__ffs(same) - 1u)
-        atomicAdd(h + b, (unsigned long long)__popc(same));
+__device__ __forceinline__ void group_hist_unit(const T* x, const Tile& u, uint64_t seg_stride, float w,
+                                                bool careful, uint32_t* sh, uint32_t& zeros) {
+  if (u.count >= kWarpSegmentMax) {
+    for (uint32_t r = 0; r < u.rows; ++r) hist_tile(x + r * seg_stride, u.count, w, careful, sh, zeros);
+  } else {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    for (uint32_t r = warp; r < u.rows; r += kWarps) {
+      if (careful) hist_segment_warp<true>(x + r * seg_stride, u.count, lane, w, sh, zeros);
+      else hist_segment_warp<false>(x + r * seg_stride, u.count, lane, w, sh, zeros);
     }
   }
 }
 
 template <bool ANY16>
 __global__ void __launch_bounds__(kThreads, 4)
-group_hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
+group_hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ units, uint32_t n_units,
                   const float* __restrict__ gabsmax, const unsigned long long* __restrict__ nonfinite,
                   unsigned long long* ghist) {
   __shared__ uint32_t sh[kBins];
   for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
   __syncthreads();
-  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-
-  bool have = false;                 // sh holds counts of group cur_g of tensor cur_t
-  uint32_t cur_t = 0, cur_g = 0, zeros = 0, since_flush = 0;
-  float w = 0.0f;
-  bool careful = false;
-  auto flush = [&]() {
+  for (uint32_t ui = blockIdx.x; ui < n_units; ui += gridDim.x) {
+    const Tile u = load_tile(units, ui);
+    const TensorRec* tr = tensors + u.tensor;
+    const uint32_t g = (uint32_t)u.row0;
+    const float w = bin_scale(gabsmax[tr->group_base + g]);
+    const bool careful = nonfinite[u.tensor] != 0ull;
+    const uint64_t seg_stride = (uint64_t)tr->channels * tr->inner;
+    uint32_t zeros = 0;
+    if (!ANY16 || tr->dtype == kF32) group_hist_unit(reinterpret_cast<const float*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
+    else if (tr->dtype == kF16) group_hist_unit(reinterpret_cast<const __half*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
+    else group_hist_unit(reinterpret_cast<const __nv_bfloat16*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
+    // merge: a unit holds fewer than 2^32 elements, so the 32-bit counts cannot have wrapped
     if (zeros) atomicAdd(sh, zeros);
-    zeros = 0;
     __syncthreads();
-    unsigned long long* h = ghist + (size_t)(tensors[cur_t].ghist_first + cur_g) * kBins;
+    unsigned long long* h = ghist + (size_t)(tr->ghist_first + g) * kBins;
     for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {
       const uint32_t c = sh[b];
       if (c) { atomicAdd(h + b, (unsigned long long)c); sh[b] = 0; }
     }
     __syncthreads();
-    have = false; since_flush = 0;
-  };
-
-  for (uint64_t base = (uint64_t)blockIdx.x * kGroupChunk; base < n_tiles; base += (uint64_t)gridDim.x * kGroupChunk) {
-    for (uint32_t k = 0; k < kGroupChunk && base + k < n_tiles; ++k) {
-      const Tile tl = load_tile(tiles, (uint32_t)(base + k));
-      const TensorRec* tr = tensors + tl.tensor;
-      if (tl.rows == 0) {
-        const uint32_t g = (uint32_t)tl.row0;
-        // 32-bit counts: merge before 2^14 tiles of 2^14 elements have gone into them
-        if (have && (tl.tensor != cur_t || g != cur_g || since_flush >= 16384u)) flush();
-        if (!have) {
-          have = true; cur_t = tl.tensor; cur_g = g;
-          w = bin_scale(gabsmax[tr->group_base + g]);
-          careful = nonfinite[cur_t] != 0ull;
-        }
-        if (!ANY16 || tr->dtype == kF32) hist_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
-        else if (tr->dtype == kF16) hist_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
-        else hist_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
-        ++since_flush;
-      } else {
-        if (!ANY16 || tr->dtype == kF32) group_hist_rows(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, gabsmax, ghist, lane, warp);
-        else if (tr->dtype == kF16) group_hist_rows(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, gabsmax, ghist, lane, warp);
-        else group_hist_rows(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, gabsmax, ghist, lane, warp);
-      }
-    }
   }
-  if (have) flush();
 }
 
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
@@ -327,8 +319,7 @@ cudaError_t launch_group_hist(const Launch& l, bool any16, const TensorRec* tens
                               unsigned long long* ghist) {
   if (n_tiles == 0) return cudaSuccess;
   static int per_sm = 0;
-  const uint32_t chunks = (n_tiles + kGroupChunk - 1) / kGroupChunk;
-  const int grid = persistent_grid((const void*)group_hist_kernel<false>, &per_sm, l.sm_count, chunks);
+  const int grid = persistent_grid((const void*)group_hist_kernel<false>, &per_sm, l.sm_count, n_tiles);
   if (any16) group_hist_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, gabsmax, nonfinite, ghist);
   else group_hist_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, gabsmax, nonfinite, ghist);
   return cudaGetLastError();

@@ -143,12 +143,49 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
   }
 }
 
-// One row handled by one warp.
+// One row handled by one warp: 16-byte loads over the aligned body of the row when x and y sit at
+// the same offset inside their groups of four, scalars at the ends; short rows and rows whose y is
+// shifted against x are read element by element.
 template <uint32_t MODE, bool OFF, bool CODES, class ACC, class T>
 __device__ __forceinline__ void metric_row(const T* __restrict__ x, const T* __restrict__ y,
                                            uint8_t* codes, uint32_t inner, uint32_t lane, const QP& p,
                                            ACC* a) {
   constexpr bool PAIR = MODE != kSelf;
+  if (inner >= 128u) {
+    const FlatSplit s = split_flat(x, inner);
+    const T* xb = x + s.head;
+    const T* yb = PAIR ? y + s.head : nullptr;
+    if (!PAIR || ((((uintptr_t)yb) & (4u * sizeof(T) - 1u)) == 0)) {
+      uint8_t* cb = CODES ? codes + s.head : nullptr;
+      constexpr uint32_t U = PAIR ? 2 : 4;
+      uint32_t j = lane;
+      for (; j + (U - 1) * 32u < s.nvec; j += U * 32u) {
+        float4 vx[U], vy[U];
+#pragma unroll
+        for (uint32_t u = 0; u < U; ++u) {
+          vx[u] = ld_vec_at(xb, j + 32u * u);
+          if (PAIR) vy[u] = ld_vec_at(yb, j + 32u * u); else vy[u] = vx[u];
+        }
+#pragma unroll
+        for (uint32_t u = 0; u < U; ++u)
+          metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + 32u * u) : nullptr);
+      }
+      for (; j < s.nvec; j += 32) {
+        const float4 vx = ld_vec_at(xb, j);
+        const float4 vy = PAIR ? ld_vec_at(yb, j) : vx;
+        metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
+      }
+      if (lane < s.head)
+        metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + lane), PAIR ? Ld<T>::one(y + lane) : 0.0f, p, a[0],
+                                      CODES ? codes + lane : nullptr);
+      if (lane < s.tail) {
+        const uint32_t i = s.head + 4u * s.nvec + lane;
+        metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[1],
+                                      CODES ? codes + i : nullptr);
+      }
+      return;
+    }
+  }
   uint32_t i = lane;
   for (; i + 96 < inner; i += 128) {
     float vx[4], vy[4];

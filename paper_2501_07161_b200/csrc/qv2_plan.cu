@@ -96,8 +96,37 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
         }
       }
       if (r.range_mode == QV2_PERCENTILE) cut_flat(t, 0, ne, 0, &out->hist_tiles);
-      if (r.range_mode == QV2_PERCENTILE_GROUP)
-        out->ghist_tiles.insert(out->ghist_tiles.end(), out->tiles.begin() + first_tile, out->tiles.end());
+      if (r.range_mode == QV2_PERCENTILE_GROUP) {
+        // Group-major units for the per-group histograms: `rows` segments of `count` elements of
+        // ONE group, segment k starting at begin + k * channels * inner (the same channel of the
+        // next batch item).  A unit holds about kGroupUnitElems elements so that a CTA merges its
+        // shared-memory histogram once per unit; rows longer than kGroupSegMax are cut.
+        const uint64_t per = kGroupUnitElems / d.inner ? kGroupUnitElems / d.inner : 1;   // rows per unit
+        const uint64_t per_group = d.inner > kGroupSegMax
+            ? d.outer * ((d.inner + kGroupSegMax - 1) / kGroupSegMax) : (d.outer + per - 1) / per;
+        uint64_t total;
+        if (mul_overflows(per_group, d.channels, &total) || out->ghist_tiles.size() + total > (1ull << 26))
+          return QV2_ERR_SIZE;
+        for (uint64_t c = 0; c < d.channels; ++c) {
+          if (d.inner > kGroupSegMax) {
+            for (uint64_t o = 0; o < d.outer; ++o)
+              for (uint64_t off = 0; off < d.inner; off += kGroupSegMax) {
+                Tile u;
+                u.begin = (o * d.channels + c) * d.inner + off; u.row0 = c;
+                u.count = (uint32_t)(d.inner - off < kGroupSegMax ? d.inner - off : kGroupSegMax);
+                u.tensor = t; u.rows = 1; u.reserved = 0;
+                out->ghist_tiles.push_back(u);
+              }
+          } else {
+            for (uint64_t o = 0; o < d.outer; o += per) {
+              Tile u;
+              u.begin = (o * d.channels + c) * d.inner; u.row0 = c; u.count = (uint32_t)d.inner;
+              u.tensor = t; u.rows = (uint32_t)(d.outer - o < per ? d.outer - o : per); u.reserved = 0;
+              out->ghist_tiles.push_back(u);
+            }
+          }
+        }
+      }
     }
     if (first_tile >= (1ull << 31)) return QV2_ERR_SIZE;
     r.tile_first = (uint32_t)first_tile;
@@ -105,7 +134,7 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     r.rslot_first = 0; r.rslot_count = 0;
     out->tensors.push_back(r);
   }
-  if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;   // ghist_tiles is a subset of tiles
+  if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;
   // Slots written with plain stores instead of atomics.  In both persistent kernels CTA b walks
   // tiles b, b+grid, ...; a tensor whose tiles are [first, first+count) is therefore touched by
   // min(grid, count) CTAs.  The metrics kernel gives each warp of those CTAs one partial-sum slot;

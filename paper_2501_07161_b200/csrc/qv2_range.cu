@@ -55,10 +55,27 @@ __device__ __forceinline__ void range_flat(const T* __restrict__ x, uint32_t cou
   if (threadIdx.x < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(x + s.head + 4u * s.nvec + threadIdx.x));
 }
 
-// One row handled by one warp: lanes stride over the row.
+// One row handled by one warp: 16-byte loads over the aligned body of the row (four in flight per
+// lane), scalars at its ends; rows too short for that are read element by element.
 template <bool CAREFUL, class T>
 __device__ __forceinline__ void range_row(const T* __restrict__ row, uint32_t inner, uint32_t lane,
                                           RangeAcc& a) {
+  if (inner >= 128u) {
+    const FlatSplit s = split_flat(row, inner);
+    const T* xv = row + s.head;
+    uint32_t j = lane;
+    for (; j + 96 < s.nvec; j += 128) {
+      float4 v[4];
+#pragma unroll
+      for (uint32_t u = 0; u < 4; ++u) v[u] = ld_vec_at(xv, j + 32u * u);
+#pragma unroll
+      for (uint32_t u = 0; u < 4; ++u) range_acc4<CAREFUL>(a, v[u]);
+    }
+    for (; j < s.nvec; j += 32) range_acc4<CAREFUL>(a, ld_vec_at(xv, j));
+    if (lane < s.head) range_acc<CAREFUL>(a, Ld<T>::one(row + lane));
+    if (lane < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(row + s.head + 4u * s.nvec + lane));
+    return;
+  }
   uint32_t i = lane;
   for (; i + 96 < inner; i += 128) {
     float v0 = Ld<T>::one(row + i), v1 = Ld<T>::one(row + i + 32), v2 = Ld<T>::one(row + i + 64),

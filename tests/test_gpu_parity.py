@@ -499,7 +499,9 @@ def test_group_percentile_long_rows_short_rows_and_batches(ctx):
                             ((1, 96, 1153), 203),                 # short ragged rows, several per tile
                             ((8, 20, 49), 204),                   # 7x7 maps: 334 rows per tile
                             ((3, 7, 1), 205),                     # one element per row
-                            ((2, 2, 4096), 206)):                 # exactly at the row-tile threshold
+                            ((2, 2, 4096), 206),                  # exactly at the row-tile threshold
+                            ((1, 2, (1 << 22) + 77), 207),        # rows longer than one unit segment
+                            ((70, 3, 2047), 208), ((3, 3, 2048), 209)):   # around the warp / CTA segment switch
         for asym, zp, p in ((False, False, 0.999), (True, False, 0.99), (False, True, 0.95)):
             specs.append(Spec(_scaled_channels(o, c, i, seed, relu=asym), o, c, i, per_channel=True, asym=asym, zp=zp,
                               percentile=p, group_pct=True, name=f"group-pct {o}x{c}x{i} asym={asym} zp={zp}"))
