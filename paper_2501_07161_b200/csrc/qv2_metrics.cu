@@ -91,39 +91,41 @@ __device__ __forceinline__ void metric_vec(const float4& x, const float4& y, con
   metric_elem<MODE, OFF, CODES>(x.w, y.w, p, a[3], code + 3);
 }
 
-// This thread's share of a flat one-group run.  T is the element type of x and y in memory;
-// `vec_y` says y has the same phase as x inside its group of four elements.
-template <uint32_t MODE, bool OFF, bool CODES, class ACC, class T>
+// This thread's share of a flat one-group run walked by STRIDE threads (the whole CTA, or one
+// warp with tid = lane).  T is the element type of x and y in memory; `vec_y` says y has the same
+// phase as x inside its group of four elements.
+template <uint32_t MODE, bool OFF, bool CODES, uint32_t STRIDE = kThreads, class ACC, class T>
 __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __restrict__ y,
-                                            uint8_t* codes, uint32_t count, const QP& p, ACC* a) {
+                                            uint8_t* codes, uint32_t count, const QP& p, ACC* a,
+                                            uint32_t tid = threadIdx.x) {
   constexpr bool PAIR = MODE != kSelf;
   const FlatSplit s = split_flat(x, count);
   const T* xb = x + s.head;
   const T* yb = PAIR ? y + s.head : nullptr;
   uint8_t* cb = CODES ? codes + s.head : nullptr;
   const bool vec_y = !PAIR || ((((uintptr_t)yb) & (4u * sizeof(T) - 1u)) == 0);
-  uint32_t j = threadIdx.x;
+  uint32_t j = tid;
   if (vec_y) {
     constexpr uint32_t U = PAIR ? 4 : 8;
-    for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
+    for (; j + (U - 1) * STRIDE < s.nvec; j += U * STRIDE) {
       float4 vx[U], vy[U];
 #pragma unroll
       for (uint32_t u = 0; u < U; ++u) {
-        vx[u] = ld_vec_at(xb, j + u * kThreads);
-        if (PAIR) vy[u] = ld_vec_at(yb, j + u * kThreads); else vy[u] = vx[u];
+        vx[u] = ld_vec_at(xb, j + u * STRIDE);
+        if (PAIR) vy[u] = ld_vec_at(yb, j + u * STRIDE); else vy[u] = vx[u];
       }
 #pragma unroll
       for (uint32_t u = 0; u < U; ++u)
-        metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * kThreads) : nullptr);
+        metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * STRIDE) : nullptr);
     }
-    for (; j < s.nvec; j += kThreads) {
+    for (; j < s.nvec; j += STRIDE) {
       const float4 vx = ld_vec_at(xb, j);
       const float4 vy = PAIR ? ld_vec_at(yb, j) : vx;
       metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
     }
   } else {
     // x and y sit at different offsets inside their groups of four: vector loads for x, scalar for y
-    for (; j < s.nvec; j += kThreads) {
+    for (; j < s.nvec; j += STRIDE) {
       const float4 vx = ld_vec_at(xb, j);
       float4 vy;
       vy.x = Ld<T>::one(yb + 4u * j); vy.y = Ld<T>::one(yb + 4u * j + 1);
@@ -131,76 +133,15 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
       metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
     }
   }
-  if (threadIdx.x < s.head) {
-    const uint32_t i = threadIdx.x;
-    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[0],
-                                  CODES ? codes + i : nullptr);
+  if (tid < s.head) {
+    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + tid), PAIR ? Ld<T>::one(y + tid) : 0.0f, p, a[0],
+                                  CODES ? codes + tid : nullptr);
   }
-  if (threadIdx.x < s.tail) {
-    const uint32_t i = s.head + 4u * s.nvec + threadIdx.x;
+  if (tid < s.tail) {
+    const uint32_t i = s.head + 4u * s.nvec + tid;
     metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[1],
                                   CODES ? codes + i : nullptr);
   }
-}
-
-// One row handled by one warp: 16-byte loads over the aligned body of the row when x and y sit at
-// the same offset inside their groups of four, scalars at the ends; short rows and rows whose y is
-// shifted against x are read element by element.
-template <uint32_t MODE, bool OFF, bool CODES, class ACC, class T>
-__device__ __forceinline__ void metric_row(const T* __restrict__ x, const T* __restrict__ y,
-                                           uint8_t* codes, uint32_t inner, uint32_t lane, const QP& p,
-                                           ACC* a) {
-  constexpr bool PAIR = MODE != kSelf;
-  if (inner >= 128u) {
-    const FlatSplit s = split_flat(x, inner);
-    const T* xb = x + s.head;
-    const T* yb = PAIR ? y + s.head : nullptr;
-    if (!PAIR || ((((uintptr_t)yb) & (4u * sizeof(T) - 1u)) == 0)) {
-      uint8_t* cb = CODES ? codes + s.head : nullptr;
-      constexpr uint32_t U = PAIR ? 2 : 4;
-      uint32_t j = lane;
-      for (; j + (U - 1) * 32u < s.nvec; j += U * 32u) {
-        float4 vx[U], vy[U];
-#pragma unroll
-        for (uint32_t u = 0; u < U; ++u) {
-          vx[u] = ld_vec_at(xb, j + 32u * u);
-          if (PAIR) vy[u] = ld_vec_at(yb, j + 32u * u); else vy[u] = vx[u];
-        }
-#pragma unroll
-        for (uint32_t u = 0; u < U; ++u)
-          metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + 32u * u) : nullptr);
-      }
-      for (; j < s.nvec; j += 32) {
-        const float4 vx = ld_vec_at(xb, j);
-        const float4 vy = PAIR ? ld_vec_at(yb, j) : vx;
-        metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
-      }
-      if (lane < s.head)
-        metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + lane), PAIR ? Ld<T>::one(y + lane) : 0.0f, p, a[0],
-                                      CODES ? codes + lane : nullptr);
-      if (lane < s.tail) {
-        const uint32_t i = s.head + 4u * s.nvec + lane;
-        metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[1],
-                                      CODES ? codes + i : nullptr);
-      }
-      return;
-    }
-  }
-  uint32_t i = lane;
-  for (; i + 96 < inner; i += 128) {
-    float vx[4], vy[4];
-#pragma unroll
-    for (uint32_t u = 0; u < 4; ++u) {
-      vx[u] = Ld<T>::one(x + i + 32u * u);
-      vy[u] = PAIR ? Ld<T>::one(y + i + 32u * u) : 0.0f;
-    }
-#pragma unroll
-    for (uint32_t u = 0; u < 4; ++u)
-      metric_elem<MODE, OFF, CODES>(vx[u], vy[u], p, a[u], CODES ? codes + i + 32u * u : nullptr);
-  }
-  for (; i < inner; i += 32)
-    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[0],
-                                  CODES ? codes + i : nullptr);
 }
 
 template <uint32_t MODE, bool CODES, class T, class ACC>
@@ -229,15 +170,41 @@ __device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRe
     load_params(tr->group_base + (uint32_t)tl.row0);
     if (MODE == kRaw || p.off == 0.0f) metric_flat<MODE, false, CODES>(x, y, codes, tl.count, p, a);
     else metric_flat<MODE, true, CODES>(x, y, codes, tl.count, p, a);
-  } else {
+  } else if (tr->inner >= kShortRow) {                 // one warp per row
     const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
     for (uint32_t r = warp; r < tl.rows; r += kWarps) {
       load_params(tr->group_base + (uint32_t)((tl.row0 + r) % channels));
       const uint64_t o = (uint64_t)r * inner;
       if (MODE == kRaw || p.off == 0.0f)
-        metric_row<MODE, false, CODES>(x + o, y + o, codes + o, inner, lane, p, a);
+        metric_flat<MODE, false, CODES, 32>(x + o, y + o, codes + o, inner, p, a, lane);
       else
-        metric_row<MODE, true, CODES>(x + o, y + o, codes + o, inner, lane, p, a);
+        metric_flat<MODE, true, CODES, 32>(x + o, y + o, codes + o, inner, p, a, lane);
+    }
+  } else {
+    // Rows shorter than kShortRow (3x3 depthwise filters, 7x7 maps, one element per channel): one
+    // element per thread, each fetching the parameters of its own row's group.  The offset form of
+    // the arithmetic is used throughout; with a zero offset it gives the same value.
+    const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+    const uint32_t row0c = (uint32_t)(tl.row0 % channels);
+    uint32_t e = threadIdx.x;
+    for (; e + 3u * kThreads < tl.count; e += 4u * kThreads) {
+      float vx[4], vy[4];
+#pragma unroll
+      for (uint32_t u = 0; u < 4; ++u) {
+        vx[u] = Ld<T>::one(x + e + u * kThreads);
+        vy[u] = (MODE != kSelf) ? Ld<T>::one(y + e + u * kThreads) : 0.0f;
+      }
+#pragma unroll
+      for (uint32_t u = 0; u < 4; ++u) {
+        const uint32_t i = e + u * kThreads;
+        load_params(tr->group_base + (uint32_t)(((uint64_t)row0c + i / inner) % channels));
+        metric_elem<MODE, MODE != kRaw, CODES>(vx[u], vy[u], p, a[u], CODES ? codes + i : nullptr);
+      }
+    }
+    for (; e < tl.count; e += kThreads) {
+      load_params(tr->group_base + (uint32_t)(((uint64_t)row0c + e / inner) % channels));
+      metric_elem<MODE, MODE != kRaw, CODES>(Ld<T>::one(x + e), (MODE != kSelf) ? Ld<T>::one(y + e) : 0.0f, p, a[0],
+                                             CODES ? codes + e : nullptr);
     }
   }
 }

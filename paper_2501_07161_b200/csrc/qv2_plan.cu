@@ -87,6 +87,9 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
           cut_flat(t, row * d.inner, d.inner, row % d.channels, &out->tiles);
       } else {
         uint64_t per = kTileElems / d.inner;       // inner < kRowTileMin, so per >= 4
+        // rows of kShortRow elements or more go one per warp: keep every warp of the CTA busy
+        // (tiles of such rows then hold between 8 K and 32 K elements)
+        if (d.inner >= kShortRow) per = per < kWarps ? kWarps : per / kWarps * kWarps;
         for (uint64_t row = 0; row < rows; row += per) {
           uint64_t nr = rows - row < per ? rows - row : per;
           Tile tl;

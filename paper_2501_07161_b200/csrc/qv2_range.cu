@@ -35,55 +35,26 @@ __device__ __forceinline__ void range_acc4(RangeAcc& a, const float4& v) {
   range_acc<CAREFUL>(a, v.z); range_acc<CAREFUL>(a, v.w);
 }
 
-// This thread's share of a flat run: group of four number j for j = tid, tid+256, ...; the first
-// `head` and last `tail` scalars go to threads 0..2.  T is the element type in memory.
-template <bool CAREFUL, class T>
-__device__ __forceinline__ void range_flat(const T* __restrict__ x, uint32_t count, RangeAcc& a) {
+// This thread's share of a flat run walked by STRIDE threads (the whole CTA, or one warp with
+// tid = lane): group of four number j for j = tid, tid+STRIDE, ...; the first `head` and last
+// `tail` scalars go to threads 0..2.  T is the element type in memory.
+template <bool CAREFUL, uint32_t STRIDE = kThreads, class T>
+__device__ __forceinline__ void range_flat(const T* __restrict__ x, uint32_t count, RangeAcc& a,
+                                           uint32_t tid = threadIdx.x) {
   const FlatSplit s = split_flat(x, count);
   const T* xv = x + s.head;
   constexpr uint32_t U = sizeof(T) == 4 ? 8 : 16;       // the same bytes in flight for 16-bit types
-  uint32_t j = threadIdx.x;
-  for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
+  uint32_t j = tid;
+  for (; j + (U - 1) * STRIDE < s.nvec; j += U * STRIDE) {
     float4 v[U];
 #pragma unroll
-    for (uint32_t u = 0; u < U; ++u) v[u] = ld_vec_at(xv, j + u * kThreads);
+    for (uint32_t u = 0; u < U; ++u) v[u] = ld_vec_at(xv, j + u * STRIDE);
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) range_acc4<CAREFUL>(a, v[u]);
   }
-  for (; j < s.nvec; j += kThreads) range_acc4<CAREFUL>(a, ld_vec_at(xv, j));
-  if (threadIdx.x < s.head) range_acc<CAREFUL>(a, Ld<T>::one(x + threadIdx.x));
-  if (threadIdx.x < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(x + s.head + 4u * s.nvec + threadIdx.x));
-}
-
-// One row handled by one warp: 16-byte loads over the aligned body of the row (four in flight per
-// lane), scalars at its ends; rows too short for that are read element by element.
-template <bool CAREFUL, class T>
-__device__ __forceinline__ void range_row(const T* __restrict__ row, uint32_t inner, uint32_t lane,
-                                          RangeAcc& a) {
-  if (inner >= 128u) {
-    const FlatSplit s = split_flat(row, inner);
-    const T* xv = row + s.head;
-    uint32_t j = lane;
-    for (; j + 96 < s.nvec; j += 128) {
-      float4 v[4];
-#pragma unroll
-      for (uint32_t u = 0; u < 4; ++u) v[u] = ld_vec_at(xv, j + 32u * u);
-#pragma unroll
-      for (uint32_t u = 0; u < 4; ++u) range_acc4<CAREFUL>(a, v[u]);
-    }
-    for (; j < s.nvec; j += 32) range_acc4<CAREFUL>(a, ld_vec_at(xv, j));
-    if (lane < s.head) range_acc<CAREFUL>(a, Ld<T>::one(row + lane));
-    if (lane < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(row + s.head + 4u * s.nvec + lane));
-    return;
-  }
-  uint32_t i = lane;
-  for (; i + 96 < inner; i += 128) {
-    float v0 = Ld<T>::one(row + i), v1 = Ld<T>::one(row + i + 32), v2 = Ld<T>::one(row + i + 64),
-          v3 = Ld<T>::one(row + i + 96);
-    range_acc<CAREFUL>(a, v0); range_acc<CAREFUL>(a, v1);
-    range_acc<CAREFUL>(a, v2); range_acc<CAREFUL>(a, v3);
-  }
-  for (; i < inner; i += 32) range_acc<CAREFUL>(a, Ld<T>::one(row + i));
+  for (; j < s.nvec; j += STRIDE) range_acc4<CAREFUL>(a, ld_vec_at(xv, j));
+  if (tid < s.head) range_acc<CAREFUL>(a, Ld<T>::one(x + tid));
+  if (tid < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(x + s.head + 4u * s.nvec + tid));
 }
 
 __device__ __forceinline__ void reset(RangeAcc& a) {
@@ -116,7 +87,7 @@ __device__ __forceinline__ void range_flat_tile(const T* x, uint32_t count, Rang
   }
 }
 
-// A tile of whole short rows: one warp per row, one publication per row.
+// A tile of whole rows, each at least kShortRow long: one warp per row, one publication per row.
 template <class T>
 __device__ __forceinline__ void range_rows_tile(const T* x, const Tile& tl, const TensorRec* tr, uint32_t lane,
                                                 uint32_t warp, uint32_t* kmin, uint32_t* kmax,
@@ -126,14 +97,51 @@ __device__ __forceinline__ void range_rows_tile(const T* x, const Tile& tl, cons
   for (uint32_t r = warp; r < tl.rows; r += kWarps) {
     const T* row = x + (uint64_t)r * inner;
     reset(b);
-    range_row<false>(row, inner, lane, b);
+    range_flat<false, 32>(row, inner, b, lane);
     if (__any_sync(0xffffffffu, b.nanflag != b.nanflag)) {
       reset(b);
-      range_row<true>(row, inner, lane, b);
+      range_flat<true, 32>(row, inner, b, lane);
     }
     const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
     publish(b, lane, kmin, kmax, tr->group_base + g, nonfinite + tl.tensor);
   }
+}
+
+// A tile of whole rows shorter than kShortRow (3x3 depthwise filters, 7x7 maps, fully connected
+// activations with one element per channel): one element per thread, so that a row of nine
+// elements does not occupy a warp.  Consecutive lanes hold consecutive elements; the lanes of one
+// row are folded with a segmented shuffle reduction and the first lane of each run publishes.
+template <class T>
+__device__ __forceinline__ void range_short_rows_tile(const T* x, const Tile& tl, const TensorRec* tr,
+                                                      uint32_t lane, uint32_t* kmin, uint32_t* kmax,
+                                                      unsigned long long* nonfinite) {
+  const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+  const uint32_t row0c = (uint32_t)(tl.row0 % channels);
+  uint32_t bad = 0;
+  for (uint32_t e0 = 0; e0 < tl.count; e0 += kThreads) {        // warp-uniform bounds: every lane shuffles
+    const uint32_t e = e0 + threadIdx.x;
+    uint32_t row = 0xffffffffu;
+    float mn = kInf, mx = -kInf;
+    if (e < tl.count) {
+      row = e / inner;
+      const float v = Ld<T>::one(x + e);
+      if (isfinite(v)) { mn = v; mx = v; } else ++bad;
+    }
+#pragma unroll
+    for (uint32_t o = 1; o < 32; o <<= 1) {
+      const float mn2 = __shfl_down_sync(0xffffffffu, mn, o), mx2 = __shfl_down_sync(0xffffffffu, mx, o);
+      const uint32_t row2 = __shfl_down_sync(0xffffffffu, row, o);
+      if (lane + o < 32 && row2 == row) { mn = fminf(mn, mn2); mx = fmaxf(mx, mx2); }
+    }
+    const uint32_t prev = __shfl_up_sync(0xffffffffu, row, 1);
+    if ((lane == 0 || prev != row) && mn <= mx) {
+      const uint32_t G = tr->group_base + (uint32_t)(((uint64_t)row0c + row) % channels);
+      atomicMax(kmax + G, f2key(mx));
+      atomicMax(kmin + G, ~f2key(mn));
+    }
+  }
+  bad = warp_sum_u32(bad);
+  if (lane == 0 && bad) atomicAdd(nonfinite + tl.tensor, (unsigned long long)bad);
 }
 
 // Lanes keep their min/max across consecutive tiles of the same group and merge them only when
@@ -192,6 +200,13 @@ range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ til
       if (!ANY16 || tr->dtype == kF32) range_flat_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, a);
       else if (tr->dtype == kF16) range_flat_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, a);
       else range_flat_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, a);
+    } else if (tr->inner < kShortRow) {
+      if (!ANY16 || tr->dtype == kF32)
+        range_short_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, kmin, kmax, nonfinite);
+      else if (tr->dtype == kF16)
+        range_short_rows_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, lane, kmin, kmax, nonfinite);
+      else
+        range_short_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, kmin, kmax, nonfinite);
     } else {
       if (!ANY16 || tr->dtype == kF32)
         range_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);

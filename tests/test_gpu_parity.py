@@ -577,3 +577,38 @@ def test_group_percentile_in_the_chained_pass_and_its_graph(ctx):
             assert torch.equal(t2["step"], t["step"])
         finally:
             gctx.close()
+
+
+# ------------------------------------------------- rows shorter than a warp's reach (element-parallel path)
+@pytest.mark.parametrize("inner", [1, 9, 27, 49, 127, 128, 196])
+def test_short_rows_per_channel_all_modes(ctx, inner):
+    """Rows below 128 elements are walked one element per thread with per-element parameters; 128
+    and above one warp per row.  Self, re-quantized pair and raw pair, symmetric / affine / zero
+    point, with codes, several batch items so that a channel's rows are far apart."""
+    o, c = 5, 37
+    n = o * c * inner
+    x = _scaled_channels(o, c, inner, 300 + inner)
+    y = x + 0.01 * x.abs().mean() * torch.randn(x.shape, generator=_g(400 + inner))
+    specs = [Spec(x, o, c, inner, per_channel=True, name="self sym"),
+             Spec(x, o, c, inner, per_channel=True, asym=True, name="self affine"),
+             Spec(x, o, c, inner, per_channel=True, zp=True, name="self zero point"),
+             Spec(x, o, c, inner, per_channel=True, asym=True, y=y, name="pair requant"),
+             Spec(x, o, c, inner, per_channel=True, zp=True, y=y, name="pair requant zero point"),
+             Spec(x, o, c, inner, per_channel=True, y=y, raw=True, name="pair raw"),
+             Spec(x, o, c, inner, per_channel=True, bits=4, name="4 bit"),
+             Spec(x.clamp_min(0), o, c, inner, per_channel=True, asym=True, percentile=0.99, group_pct=True,
+                  name="own percentile per channel")]
+    check_specs(ctx, specs)
+    check_specs(ctx, specs[:6], misalign_x=1, misalign_y=2, check_codes=False)
+    half = [Spec(s.x, s.outer, s.channels, s.inner, per_channel=True, asym=s.asym, zp=s.zp, y=s.y, raw=s.raw,
+                 dtype=torch.bfloat16, name=s.name + " bf16") for s in specs[:6]]
+    check_specs(ctx, half, check_codes=False)
+
+
+def test_short_rows_with_nonfinite_elements_and_many_rows_per_tile(ctx):
+    o, c, inner = 3, 2000, 9                      # 6000 rows: four tiles of 1820 rows
+    x = _scaled_channels(o, c, inner, 501)
+    x[0, 5, 3] = float("nan"); x[2, 1999, 8] = float("-inf"); x[1, 0, 0] = float("inf")
+    x[:, 7, :] = 0.0
+    check_specs(ctx, [Spec(x, o, c, inner, per_channel=True), Spec(x, o, c, inner, per_channel=True, asym=True)],
+                check_codes=False)
