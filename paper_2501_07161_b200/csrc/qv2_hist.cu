@@ -44,10 +44,16 @@ __device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t coun
       hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
     }
   }
-  for (; j < s.nvec; j += kThreads) {
-    const float4 v = ld_vec_at(xv, j);
-    hist_elem<CAREFUL>(v.x, w, sh, zeros); hist_elem<CAREFUL>(v.y, w, sh, zeros);
-    hist_elem<CAREFUL>(v.z, w, sh, zeros); hist_elem<CAREFUL>(v.w, w, sh, zeros);
+  if (j < s.nvec) {                 // at most U-1 groups are left for this thread: one predicated round
+    float4 v[U - 1];
+#pragma unroll
+    for (uint32_t u = 0; u < U - 1; ++u) v[u] = ld_vec_at(xv, min(j + u * kThreads, s.nvec - 1u));   // in bounds, maybe unused
+#pragma unroll
+    for (uint32_t u = 0; u < U - 1; ++u)
+      if (j + u * kThreads < s.nvec) {
+        hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
+        hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
+      }
   }
   if (threadIdx.x < s.head) hist_elem<CAREFUL>(Ld<T>::one(x + threadIdx.x), w, sh, zeros);
   if (threadIdx.x < s.tail)
@@ -195,16 +201,22 @@ __device__ __forceinline__ void hist_segment_warp(const T* __restrict__ x, uint3
       hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
     }
   }
-  for (; j < s.nvec; j += 32) {
-    const float4 v = ld_vec_at(xv, j);
-    hist_elem<CAREFUL>(v.x, w, sh, zeros); hist_elem<CAREFUL>(v.y, w, sh, zeros);
-    hist_elem<CAREFUL>(v.z, w, sh, zeros); hist_elem<CAREFUL>(v.w, w, sh, zeros);
+  if (j < s.nvec) {                 // at most three groups are left for this lane: one predicated round
+    float4 v[3];
+#pragma unroll
+    for (uint32_t u = 0; u < 3; ++u) v[u] = ld_vec_at(xv, min(j + 32u * u, s.nvec - 1u));   // in bounds, maybe unused
+#pragma unroll
+    for (uint32_t u = 0; u < 3; ++u)
+      if (j + 32u * u < s.nvec) {
+        hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
+        hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
+      }
   }
   if (lane < s.head) hist_elem<CAREFUL>(Ld<T>::one(x + lane), w, sh, zeros);
   if (lane < s.tail) hist_elem<CAREFUL>(Ld<T>::one(x + s.head + 4u * s.nvec + lane), w, sh, zeros);
 }
 
-constexpr uint32_t kWarpSegmentMax = 2048;     // shorter segments go one per warp
+constexpr uint32_t kWarpSegmentMax = 4096;     // shorter segments go one per warp
 
 template <class T>
 __device__ __forceinline__ void group_hist_unit(const T* x, const Tile& u, uint64_t seg_stride, float w,

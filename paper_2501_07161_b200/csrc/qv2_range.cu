@@ -52,7 +52,14 @@ __device__ __forceinline__ void range_flat(const T* __restrict__ x, uint32_t cou
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) range_acc4<CAREFUL>(a, v[u]);
   }
-  for (; j < s.nvec; j += STRIDE) range_acc4<CAREFUL>(a, ld_vec_at(xv, j));
+  if (j < s.nvec) {                 // at most U-1 groups are left for this thread: one predicated round
+    float4 v[U - 1];
+#pragma unroll
+    for (uint32_t u = 0; u < U - 1; ++u) v[u] = ld_vec_at(xv, min(j + u * STRIDE, s.nvec - 1u));   // in bounds, maybe unused
+#pragma unroll
+    for (uint32_t u = 0; u < U - 1; ++u)
+      if (j + u * STRIDE < s.nvec) range_acc4<CAREFUL>(a, v[u]);
+  }
   if (tid < s.head) range_acc<CAREFUL>(a, Ld<T>::one(x + tid));
   if (tid < s.tail) range_acc<CAREFUL>(a, Ld<T>::one(x + s.head + 4u * s.nvec + tid));
 }
