@@ -612,3 +612,43 @@ def test_short_rows_with_nonfinite_elements_and_many_rows_per_tile(ctx):
     x[:, 7, :] = 0.0
     check_specs(ctx, [Spec(x, o, c, inner, per_channel=True), Spec(x, o, c, inner, per_channel=True, asym=True)],
                 check_codes=False)
+
+
+# ----------------------------------------------------------------------- seeded random descriptor sets
+@pytest.mark.parametrize("seed", [1, 2, 3, 4, 5, 6])
+def test_random_descriptor_sets_in_one_batched_call(ctx, seed):
+    """Forty tensors of random shape, granularity, scheme, range mode, bit width, storage type and
+    pair mode in ONE calibrate and ONE metrics call: every combination of row walker (flat, warp
+    per row, element per thread) and tile kind meets every arithmetic variant, and the planner has
+    to keep their groups, slots and histograms apart."""
+    rng = np.random.default_rng(1000 + seed)
+    inner_pool = [1, 2, 7, 9, 31, 32, 33, 49, 100, 127, 128, 129, 196, 500, 784, 1153, 3136, 4095, 4096, 4097,
+                  12544, 16384, 16385, 40000]
+    specs = []
+    total = 0
+    while len(specs) < 40 and total < 6_000_000:
+        inner = int(rng.choice(inner_pool))
+        per_channel = bool(rng.random() < 0.7)
+        c = int(rng.integers(1, 40 if inner > 1000 else 300))
+        o = int(rng.integers(1, 5))
+        if o * c * inner > 1_500_000:
+            c = max(1, 1_500_000 // (o * inner))
+        n = o * c * inner
+        total += n
+        scheme = int(rng.integers(0, 3))
+        x = _scaled_channels(o, c, inner, int(rng.integers(1 << 30)), relu=bool(rng.random() < 0.4))
+        if rng.random() < 0.1:
+            x = x * 0.0 + 1.25                        # constant tensor
+        pair = rng.random() < 0.5
+        y = x + 0.02 * float(x.abs().mean() + 1e-6) * torch.randn(x.shape, generator=_g(int(rng.integers(1 << 30)))) \
+            if pair else None
+        pct = float(rng.choice([0.9, 0.99, 0.9999, 1.0])) if rng.random() < 0.5 else None
+        specs.append(Spec(x, o, c, inner, per_channel=per_channel, asym=scheme == 1, zp=scheme == 2, percentile=pct,
+                          group_pct=pct is not None and rng.random() < 0.5, y=y, raw=bool(pair and rng.random() < 0.25),
+                          bits=int(rng.choice([8, 8, 8, 4, 2, 12, 16])),
+                          dtype=[torch.float32, torch.float32, torch.float16, torch.bfloat16][int(rng.integers(0, 4))],
+                          name=f"seed {seed} tensor {len(specs)}: {o}x{c}x{inner} pc={per_channel} scheme={scheme}"))
+    order = rng.permutation(len(specs))
+    specs = [specs[i] for i in order]
+    check_specs(ctx, specs, misalign_x=int(rng.integers(0, 4)), misalign_y=int(rng.integers(0, 4)),
+                check_codes=bool(seed % 2))
