@@ -286,14 +286,16 @@ metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ t
 // One CTA per tensor: fixed-order binary64 sum of the tensor's slots, then MSE (Eq. 7), SQNR
 // (Eq. 6) and, when asked for, the cosine similarity (Eq. 8) between the reference tensor A = x
 // and the compared tensor B = x - e:  A.B = sig - xe,  |B|^2 = sig - 2 xe + sse.
-__global__ void __launch_bounds__(256)
+constexpr int kFinalizeThreads = 1024;   // short chains of dependent loads: 3552 slots take 4 rounds
+
+__global__ void __launch_bounds__(kFinalizeThreads)
 metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __restrict__ partials,
                         const double* __restrict__ partials_xe, double* sse_out, double* sig_out,
                         double* mse_out, double* sqnr_out, double* cos_out) {
-  __shared__ double sh_e[256], sh_s[256], sh_x[256];
+  __shared__ double sh_e[kFinalizeThreads], sh_s[kFinalizeThreads], sh_x[kFinalizeThreads];
   const TensorRec tr = tensors[blockIdx.x];
   double e = 0.0, s = 0.0, xe = 0.0;
-  for (uint32_t k = threadIdx.x; k < tr.slot_count; k += 256) {
+  for (uint32_t k = threadIdx.x; k < tr.slot_count; k += kFinalizeThreads) {
     const double2 p = partials[tr.slot_first + k];
     e = __dadd_rn(e, p.x);
     s = __dadd_rn(s, p.y);
@@ -301,7 +303,7 @@ metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __
   }
   sh_e[threadIdx.x] = e; sh_s[threadIdx.x] = s; sh_x[threadIdx.x] = xe;
   __syncthreads();
-  for (uint32_t o = 128; o > 0; o >>= 1) {
+  for (uint32_t o = kFinalizeThreads / 2; o > 0; o >>= 1) {
     if (threadIdx.x < o) {
       sh_e[threadIdx.x] = __dadd_rn(sh_e[threadIdx.x], sh_e[threadIdx.x + o]);
       sh_s[threadIdx.x] = __dadd_rn(sh_s[threadIdx.x], sh_s[threadIdx.x + o]);
@@ -454,7 +456,7 @@ cudaError_t launch_metrics(const Launch& l, uint32_t grid, bool any16, const Ten
 cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                     const double2* partials, const double* partials_xe, double* sse,
                                     double* sig, double* mse, double* sqnr_db, double* cosine) {
-  metrics_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, partials, partials_xe, sse, sig,
+  metrics_finalize_kernel<<<n_tensors, kFinalizeThreads, 0, l.stream>>>(tensors, partials, partials_xe, sse, sig,
                                                            mse, sqnr_db, cosine);
   return cudaGetLastError();
 }

@@ -232,12 +232,16 @@ range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ til
 // One CTA per tensor: fold the CTA slots of a per-tensor tensor, decode the keys in place, write
 // absmax, the tensor-wide absmax and -- for tensors without percentile clipping -- the
 // quantization parameters.
-__global__ void __launch_bounds__(256)
+// The finalize kernels are chains of dependent global loads: many threads keep the chain short
+// (a tensor with 4096 groups takes 4 rounds instead of 16).
+constexpr int kFinalizeThreads = 1024;
+
+__global__ void __launch_bounds__(kFinalizeThreads)
 range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __restrict__ rslots,
                       float* gmin, float* gmax, float* gabsmax, float* step, float* inv, float* offset,
                       float* tensor_absmax) {
-  __shared__ float red[256];
-  __shared__ uint32_t kred[2][256];
+  __shared__ float red[kFinalizeThreads];
+  __shared__ uint32_t kred[2][kFinalizeThreads];
   const TensorRec tr = tensors[blockIdx.x];
   if (!tr.per_channel) {                 // keys of the single group come from the slots
     uint32_t kn = 0, kx = 0;             // both arrays hold "larger is better" keys, 0 = empty
@@ -247,7 +251,7 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __rest
     }
     kred[0][threadIdx.x] = kn; kred[1][threadIdx.x] = kx;
     __syncthreads();
-    for (uint32_t o = 128; o > 0; o >>= 1) {
+    for (uint32_t o = kFinalizeThreads / 2; o > 0; o >>= 1) {
       if (threadIdx.x < o) {
         kred[0][threadIdx.x] = max(kred[0][threadIdx.x], kred[0][threadIdx.x + o]);
         kred[1][threadIdx.x] = max(kred[1][threadIdx.x], kred[1][threadIdx.x + o]);
@@ -277,7 +281,7 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __rest
   }
   red[threadIdx.x] = amax;
   __syncthreads();
-  for (uint32_t o = 128; o > 0; o >>= 1) {
+  for (uint32_t o = kFinalizeThreads / 2; o > 0; o >>= 1) {
     if (threadIdx.x < o) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + o]);
     __syncthreads();
   }
@@ -303,7 +307,7 @@ cudaError_t launch_range(const Launch& l, uint32_t grid, bool any16, const Tenso
 cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                   const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
                                   float* step, float* inv, float* offset, float* tensor_absmax) {
-  range_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, rslots, gmin, gmax, gabsmax, step,
+  range_finalize_kernel<<<n_tensors, kFinalizeThreads, 0, l.stream>>>(tensors, rslots, gmin, gmax, gabsmax, step,
                                                          inv, offset, tensor_absmax);
   return cudaGetLastError();
 }
