@@ -32,6 +32,16 @@ struct Acc {
     sse = __fmaf_rn(e, e, sse);
     sig = __fmaf_rn(x, x, sig);
   }
+  // fresh(): an accumulator that starts from nothing; fold(): four into one, fixed association;
+  // merge(): add another accumulator's sums
+  __device__ __forceinline__ Acc fresh() const { Acc r; r.clear(); return r; }
+  __device__ __forceinline__ static Acc fold(const Acc* a) {
+    Acc r;
+    r.sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
+    r.sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
+    return r;
+  }
+  __device__ __forceinline__ void merge(const Acc& r) { sse = __fadd_rn(sse, r.sse); sig = __fadd_rn(sig, r.sig); }
 };
 struct AccCos {
   static constexpr bool kWantsB = false;
@@ -41,6 +51,17 @@ struct AccCos {
     sse = __fmaf_rn(e, e, sse);
     sig = __fmaf_rn(x, x, sig);
     xe = __fmaf_rn(x, e, xe);
+  }
+  __device__ __forceinline__ AccCos fresh() const { AccCos r; r.clear(); return r; }
+  __device__ __forceinline__ static AccCos fold(const AccCos* a) {
+    AccCos r;
+    r.sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
+    r.sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
+    r.xe = __fadd_rn(__fadd_rn(a[0].xe, a[1].xe), __fadd_rn(a[2].xe, a[3].xe));
+    return r;
+  }
+  __device__ __forceinline__ void merge(const AccCos& r) {
+    sse = __fadd_rn(sse, r.sse); sig = __fadd_rn(sig, r.sig); xe = __fadd_rn(xe, r.xe);
   }
 };
 
@@ -144,36 +165,40 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
   }
 }
 
+// Parameters of group G as the element arithmetic wants them.  Integer zero point z (scheme 2, the
+// offset slot carries z): the arithmetic is the offset-free path on d = q - z -- clamp to
+// [-z, top - z], e = x - d*step -- and only the stored code differs (d + z).  Written without
+// branches: z is 0 for the other schemes.
+__device__ __forceinline__ void load_params(QP& p, const TensorRec* tr, const float* __restrict__ step,
+                                            const float* __restrict__ inv, const float* __restrict__ offset,
+                                            uint32_t G) {
+  const float top = top_code(tr->asym != 0, tr->bits);
+  const float qmin0 = tr->asym ? 0.0f : -top;
+  const bool zp = tr->asym == 2;
+  p.step = __ldg(step + G); p.inv = __ldg(inv + G);
+  const float off = __ldg(offset + G);
+  const float z = zp ? off : 0.0f;
+  p.off = zp ? 0.0f : off;
+  p.bias = z; p.qmin = qmin0 - z; p.qmax = top - z;
+}
+
+// A tile of whole rows.  Kept out of line: these walkers run for a small share of the bytes (weight
+// rows, small feature maps), and inlined into the tile loop they compete with the flat path for
+// its registers.  Returns the tile's sums folded into one accumulator.
 template <uint32_t MODE, bool CODES, class T, class ACC>
-__device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRec* tr,
-                                                  const float* __restrict__ step, const float* __restrict__ inv,
-                                                  const float* __restrict__ offset, ACC* a) {
+__device__ __noinline__ ACC metric_rows(Tile tl, const TensorRec* tr, const float* __restrict__ step,
+                                        const float* __restrict__ inv, const float* __restrict__ offset,
+                                        ACC seed) {
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const T* x = reinterpret_cast<const T*>(tr->x) + tl.begin;
   const T* y = (MODE != kSelf) ? reinterpret_cast<const T*>(tr->y) + tl.begin : nullptr;
   uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
+  const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+  ACC a[4] = {seed, seed, seed, seed};
   QP p;
-  const float top = top_code(tr->asym != 0, tr->bits);
-  const float qmin0 = tr->asym ? 0.0f : -top;
-  // Integer zero point z (tr->asym == 2, the offset slot carries z): the arithmetic is the
-  // offset-free path on d = q - z -- clamp to [-z, top - z], e = x - d*step -- and only the
-  // stored code differs (d + z).  Written without branches: z is 0 for the other schemes.
-  const bool zp = tr->asym == 2;
-  auto load_params = [&](uint32_t G) {
-    p.step = __ldg(step + G); p.inv = __ldg(inv + G);
-    const float off = __ldg(offset + G);
-    const float z = zp ? off : 0.0f;
-    p.off = zp ? 0.0f : off;
-    p.bias = z; p.qmin = qmin0 - z; p.qmax = top - z;
-  };
-  if (tl.rows == 0) {
-    load_params(tr->group_base + (uint32_t)tl.row0);
-    if (MODE == kRaw || p.off == 0.0f) metric_flat<MODE, false, CODES>(x, y, codes, tl.count, p, a);
-    else metric_flat<MODE, true, CODES>(x, y, codes, tl.count, p, a);
-  } else if (tr->inner >= kShortRow) {                 // one warp per row
-    const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+  if (inner >= kShortRow) {                            // one warp per row
     for (uint32_t r = warp; r < tl.rows; r += kWarps) {
-      load_params(tr->group_base + (uint32_t)((tl.row0 + r) % channels));
+      load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)((tl.row0 + r) % channels));
       const uint64_t o = (uint64_t)r * inner;
       if (MODE == kRaw || p.off == 0.0f)
         metric_flat<MODE, false, CODES, 32>(x + o, y + o, codes + o, inner, p, a, lane);
@@ -184,7 +209,6 @@ __device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRe
     // Rows shorter than kShortRow (3x3 depthwise filters, 7x7 maps, one element per channel): one
     // element per thread, each fetching the parameters of its own row's group.  The offset form of
     // the arithmetic is used throughout; with a zero offset it gives the same value.
-    const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
     const uint32_t row0c = (uint32_t)(tl.row0 % channels);
     uint32_t e = threadIdx.x;
     for (; e + 3u * kThreads < tl.count; e += 4u * kThreads) {
@@ -197,15 +221,33 @@ __device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRe
 #pragma unroll
       for (uint32_t u = 0; u < 4; ++u) {
         const uint32_t i = e + u * kThreads;
-        load_params(tr->group_base + (uint32_t)(((uint64_t)row0c + i / inner) % channels));
+        load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)(((uint64_t)row0c + i / inner) % channels));
         metric_elem<MODE, MODE != kRaw, CODES>(vx[u], vy[u], p, a[u], CODES ? codes + i : nullptr);
       }
     }
     for (; e < tl.count; e += kThreads) {
-      load_params(tr->group_base + (uint32_t)(((uint64_t)row0c + e / inner) % channels));
+      load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)(((uint64_t)row0c + e / inner) % channels));
       metric_elem<MODE, MODE != kRaw, CODES>(Ld<T>::one(x + e), (MODE != kSelf) ? Ld<T>::one(y + e) : 0.0f, p, a[0],
                                              CODES ? codes + e : nullptr);
     }
+  }
+  return ACC::fold(a);
+}
+
+template <uint32_t MODE, bool CODES, class T, class ACC>
+__device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRec* tr,
+                                                  const float* __restrict__ step, const float* __restrict__ inv,
+                                                  const float* __restrict__ offset, ACC* a) {
+  if (tl.rows == 0) {
+    const T* x = reinterpret_cast<const T*>(tr->x) + tl.begin;
+    const T* y = (MODE != kSelf) ? reinterpret_cast<const T*>(tr->y) + tl.begin : nullptr;
+    uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
+    QP p;
+    load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)tl.row0);
+    if (MODE == kRaw || p.off == 0.0f) metric_flat<MODE, false, CODES>(x, y, codes, tl.count, p, a);
+    else metric_flat<MODE, true, CODES>(x, y, codes, tl.count, p, a);
+  } else {
+    a[0].merge(metric_rows<MODE, CODES, T>(tl, tr, step, inv, offset, a[0].fresh()));
   }
 }
 
@@ -354,6 +396,10 @@ struct AccKL {
     atomicAdd(hp + bin(x, w), 1u);
     atomicAdd(hq + bin(b, w), 1u);
   }
+  // the counts live in shared memory: a copy counts into the same histograms
+  __device__ __forceinline__ AccKL fresh() const { return *this; }
+  __device__ __forceinline__ static AccKL fold(const AccKL* a) { return a[0]; }
+  __device__ __forceinline__ void merge(const AccKL&) {}
 };
 
 __global__ void __launch_bounds__(kThreads, 2)
