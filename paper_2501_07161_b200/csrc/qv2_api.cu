@@ -81,8 +81,19 @@ int grow_pinned(qv2_ctx* c, size_t need) {
   return QV2_OK;
 }
 
+int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* const* codes);
+
 // Makes ctx->plan describe (descs, codes) and resident on the device.
 int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* const* codes) {
+  try {
+    return ensure_plan_checked(c, descs, n, codes);
+  } catch (const std::bad_alloc&) {          // host tables did not fit: nothing unwinds through the C ABI
+    c->plan_valid = false;
+    return QV2_ERR_NOMEM;
+  }
+}
+
+int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* const* codes) {
   if (!descs) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   const size_t dbytes = (size_t)n * sizeof(qv2_tensor_desc);

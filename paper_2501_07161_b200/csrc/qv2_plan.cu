@@ -1,5 +1,7 @@
 // Host planner: validates tensor descriptors and cuts a whole model's ragged layer list into the
 // tile table that one kernel launch per phase walks (segmented multi-layer batching).
+#include <new>
+
 #include "qv2_common.cuh"
 
 namespace qv2 {
@@ -21,8 +23,12 @@ static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t g
   }
 }
 
-int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
-               uint32_t range_cap, HostPlan* out) {
+// Tables larger than this many tiles (4 GB of records; two trillion elements) are refused before
+// any of them is generated.
+constexpr uint64_t kMaxTiles = 1ull << 27;
+
+static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
+                              uint32_t range_cap, HostPlan* out) {
   if (!descs || !out) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   out->tensors.clear(); out->tiles.clear(); out->hist_tiles.clear();
@@ -78,6 +84,16 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
     if (dtype != kF32) out->any_16bit = true;
 
     size_t first_tile = out->tiles.size();
+    {
+      uint64_t need;
+      if (ne == 0) need = 0;
+      else if (!r.per_channel) need = (ne + kTileElems - 1) / kTileElems;
+      else if (d.inner >= kRowTileMin) need = rows * ((d.inner + kTileElems - 1) / kTileElems);   // <= ne / 16384 + rows: no overflow
+      else need = rows / 4 + 1;                                 // at least four rows per tile
+      if (need > kMaxTiles || out->tiles.size() + need > kMaxTiles) return QV2_ERR_SIZE;
+      if (r.range_mode == QV2_PERCENTILE &&
+          out->hist_tiles.size() + (ne + kTileElems - 1) / kTileElems > kMaxTiles) return QV2_ERR_SIZE;
+    }
     if (r.range_mode == QV2_PERCENTILE) out->any_percentile = true;
     if (ne > 0) {
       if (!r.per_channel) {
@@ -171,6 +187,15 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
   out->total_groups = groups;
   out->total_slots = (uint32_t)slots;
   return QV2_OK;
+}
+
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
+               uint32_t range_cap, HostPlan* out) {
+  try {
+    return build_plan_checked(descs, n, codes, metrics_cap, range_cap, out);
+  } catch (const std::bad_alloc&) {          // nothing may unwind through the C ABI
+    return QV2_ERR_NOMEM;
+  }
 }
 
 }  // namespace qv2

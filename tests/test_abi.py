@@ -85,6 +85,20 @@ def test_group_count_and_plan_errors():
     assert L.qv2_debug_plan_tiles(q.desc_array([_desc(1, 1, 10, False)]), 0, None, 0) == -4
     empty = _desc(0, 4, 10, True); empty.x = None
     assert L.qv2_debug_plan_tiles(q.desc_array([empty]), 1, None, 0) == 0
+    # per-group percentile: same argument checks, histograms only for per-channel tensors that ask
+    g = _desc(2, 5, 100, True, percentile=0.99); g.range = q.PERCENTILE_GROUP
+    t = _desc(2, 5, 100, False, percentile=0.99); t.range = q.PERCENTILE_GROUP
+    p = _desc(2, 7, 100, True, percentile=0.99)
+    assert L.qv2_group_hist_count(q.desc_array([g, t, p, g]), 4) == 10
+    assert L.qv2_debug_plan_tiles(q.desc_array([g, t, p]), 3, None, 0) > 0
+    bad = _desc(2, 5, 100, True, percentile=-0.1); bad.range = q.PERCENTILE_GROUP
+    assert L.qv2_debug_plan_tiles(q.desc_array([bad]), 1, None, 0) == -1
+    bad = _desc(1, 1, 10, False); bad.range = 4
+    assert L.qv2_debug_plan_tiles(q.desc_array([bad]), 1, None, 0) == -1
+    huge = _desc(1 << 24, 1 << 12, 100, True, percentile=0.9); huge.range = q.PERCENTILE_GROUP
+    assert L.qv2_debug_plan_tiles(q.desc_array([huge]), 1, None, 0) == -4      # refused before any table is built
+    assert L.qv2_debug_plan_tiles(q.desc_array([_desc(1, 1, 1 << 50, False)]), 1, None, 0) == -4
+    assert L.qv2_debug_plan_tiles(q.desc_array([_desc(1 << 30, 4, 5000, True)]), 1, None, 0) == -4
 
 
 def test_no_gpu_means_a_loud_failure_not_a_fallback():
