@@ -43,6 +43,9 @@ def cases():
              per_channel=False, asym_u8=True, percentile=0.99),
         dict(name="signed_act_per_channel_asym", x=g, y=None, outer=2, channels=3, inner=200,
              per_channel=True, asym_u8=True, percentile=None),
+        dict(name="signed_act_per_channel_own_percentile", x=g * np.float32([1, 8, 0.125]).repeat(200)[None, :].repeat(2, 0).reshape(-1),
+             y=None, outer=2, channels=3, inner=200, per_channel=True, asym_u8=True, percentile=0.95,
+             group_percentile=True),
     ]
 
 
@@ -55,7 +58,7 @@ def compute():
            "tensors": []}
     for c in cases():
         kw = {k: c[k] for k in ("x", "y", "outer", "channels", "inner", "per_channel", "asym_u8", "percentile")}
-        r = oracle.sweep_tensor(want_codes=True, **kw)
+        r = oracle.sweep_tensor(want_codes=True, group_percentile=c.get("group_percentile", False), **kw)
         mode = oracle.PAIR_SELF if c["y"] is None else oracle.PAIR_REQUANT
         cos = oracle.cosine(c["x"], c["y"], c["outer"], c["channels"], c["inner"], c["per_channel"],
                             c["asym_u8"], mode, r.step, r.inv, r.offset)
@@ -65,7 +68,10 @@ def compute():
             hist_nonzero=[] if r.hist is None else [[int(i), int(v)] for i, v in enumerate(r.hist) if v],
             codes_head=[int(v) for v in r.codes[:40]], codes_sum=int(r.codes.astype(np.int64).sum()),
             sse=float(r.sse).hex(), sig=float(r.sig).hex(), mse=float(r.mse).hex(),
-            sqnr_db=float(r.sqnr_db).hex(), cosine=float(cos).hex()))
+            sqnr_db=float(r.sqnr_db).hex(), cosine=float(cos).hex(),
+            group_clip=hexf(r.gclip),
+            group_hist_nonzero=[] if r.ghist is None else
+            [[int(g), int(i), int(v)] for g in range(r.ghist.shape[0]) for i, v in enumerate(r.ghist[g]) if v]))
     sw = [41.5, 38.25, 39.0, 33.75, 40.5, 36.0, 37.5]
     sa = [30.0, 29.5, 31.25, 27.0, 28.5, 30.75, 26.0]
     mw = [1e-6, 2e-6, 1e-6, 9e-6, 1e-6, 1e-6, 2e-6]

@@ -51,9 +51,10 @@ def test_cuda_path_matches_the_stored_values():
             d = q.make_desc(x, y, c["outer"], c["channels"], c["inner"],
                             q.PER_CHANNEL if c["per_channel"] else q.PER_TENSOR,
                             q.ASYM_U8 if c["asym_u8"] else q.SYM_I8,
-                            q.PERCENTILE if pct is not None else q.MINMAX, pct or 0.0, q.STORE_CODES)
+                            (q.PERCENTILE_GROUP if c.get("group_percentile") else q.PERCENTILE)
+                            if pct is not None else q.MINMAX, pct or 0.0, q.STORE_CODES)
             descs = q.desc_array([d])
-            cal = ctx.calibrate(descs)
+            cal = ctx.calibrate(descs, want_group=True)
             codes = [torch.zeros(x.numel(), dtype=torch.uint8, device="cuda")]
             met = ctx.quant_metrics(descs, cal.step, cal.inv, cal.offset, codes, want_cosine=True)
             torch.cuda.synchronize()
@@ -63,6 +64,11 @@ def test_cuda_path_matches_the_stored_values():
             assert float(cal.clip[0]) == float.fromhex(ref["clip"])
             hist = cal.hist.cpu().numpy().view(np.uint64)[:2048]
             assert [[int(i), int(v)] for i, v in enumerate(hist) if v] == ref["hist_nonzero"]
+            assert np.array_equal(cal.group_clip.cpu().numpy().astype(np.float64), fx(ref["group_clip"])), c["name"]
+            if c.get("group_percentile"):
+                gh = cal.group_hist.cpu().numpy().view(np.uint64).reshape(-1, 2048)
+                got = [[int(g), int(i), int(v)] for g in range(c["channels"]) for i, v in enumerate(gh[g]) if v]
+                assert got == ref["group_hist_nonzero"], c["name"]
             cd = codes[0].cpu().numpy()
             cd = cd if c["asym_u8"] else cd.view(np.int8)
             assert cd[:40].tolist() == ref["codes_head"] and int(cd.astype(np.int64).sum()) == ref["codes_sum"]
