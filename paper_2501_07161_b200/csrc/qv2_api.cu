@@ -221,12 +221,9 @@ extern "C" int qv2_calibrate_ex(qv2_ctx* c, const qv2_tensor_desc* descs, uint32
   }
   const Launch l = launch_of(c);
   const size_t G = (size_t)p.total_groups;
-  if (G) {
-    QV2_CUDA(c, cudaMemsetAsync(gmin, 0, G * sizeof(float), c->stream));   // key 0 = nothing seen
-    QV2_CUDA(c, cudaMemsetAsync(gmax, 0, G * sizeof(float), c->stream));
-  }
-  QV2_CUDA(c, cudaMemsetAsync(nonfinite, 0, (size_t)n * sizeof(uint64_t), c->stream));
-  if (h) QV2_CUDA(c, cudaMemsetAsync(h, 0, (size_t)n * kBins * sizeof(uint64_t), c->stream));
+  QV2_CUDA(c, launch_calib_init(l, reinterpret_cast<uint32_t*>(gmin), reinterpret_cast<uint32_t*>(gmax), G,
+                                reinterpret_cast<unsigned long long*>(nonfinite), n, h, h ? (size_t)n * kBins : 0));
+  ++c->launches;
   if (n_ghist) QV2_CUDA(c, cudaMemsetAsync(gh, 0, n_ghist * kBins * sizeof(uint64_t), c->stream));
   if (!p.tiles.empty()) {
     QV2_CUDA(c, launch_range(l, p.range_grid, p.any_16bit, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),

@@ -96,6 +96,9 @@ struct Launch {
 cudaError_t launch_range(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors, const Tile* tiles,
                          uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax, uint2* rslots,
                          unsigned long long* nonfinite);
+cudaError_t launch_calib_init(const Launch& l, uint32_t* kmin, uint32_t* kmax, size_t groups,
+                              unsigned long long* nonfinite, size_t n_tensors, unsigned long long* hist,
+                              size_t hist_cells);
 uint32_t range_grid_cap(int sm_count);     // resident CTAs per SM x SMs for the range kernel
 cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                   const uint2* rslots, float* gmin, float* gmax, float* gabsmax,

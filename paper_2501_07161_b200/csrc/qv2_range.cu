@@ -288,7 +288,32 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __rest
   if (threadIdx.x == 0) tensor_absmax[blockIdx.x] = red[0];
 }
 
+// Everything a calibration pass accumulates into starts at zero: the min/max keys (0 = nothing
+// seen), the non-finite counters and the per-tensor histograms.  One small kernel instead of four
+// memsets: a pass over a small model is bound by the number of stream operations.
+__global__ void __launch_bounds__(256)
+calib_init_kernel(uint32_t* kmin, uint32_t* kmax, size_t groups, unsigned long long* nonfinite, size_t n_tensors,
+                  unsigned long long* hist, size_t hist_cells) {
+  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = tid; i < groups; i += stride) { kmin[i] = 0u; kmax[i] = 0u; }
+  for (size_t i = tid; i < n_tensors; i += stride) nonfinite[i] = 0ull;
+  for (size_t i = tid; i < hist_cells; i += stride) hist[i] = 0ull;
+}
+
 }  // namespace
+
+cudaError_t launch_calib_init(const Launch& l, uint32_t* kmin, uint32_t* kmax, size_t groups,
+                              unsigned long long* nonfinite, size_t n_tensors, unsigned long long* hist,
+                              size_t hist_cells) {
+  size_t most = groups > hist_cells ? groups : hist_cells;
+  if (n_tensors > most) most = n_tensors;
+  size_t grid = (most + 255) / 256;
+  const size_t cap = (size_t)l.sm_count * 8;
+  if (grid > cap) grid = cap;
+  if (grid < 1) grid = 1;
+  calib_init_kernel<<<(unsigned)grid, 256, 0, l.stream>>>(kmin, kmax, groups, nonfinite, n_tensors, hist, hist_cells);
+  return cudaGetLastError();
+}
 
 uint32_t range_grid_cap(int sm_count) {
   static int per_sm = 0;
