@@ -232,16 +232,18 @@ extern "C" int qv2_calibrate_ex(qv2_ctx* c, const qv2_tensor_desc* descs, uint32
     ++c->launches;
   }
   QV2_CUDA(c, launch_range_finalize(l, c->d_tensors, n, c->d_rslots, gmin, gmax, gabsmax, step, inv, offset,
-                                    c->d_tensor_absmax));
+                                    c->d_tensor_absmax, clip));
   ++c->launches;
   if (!p.hist_tiles.empty()) {
     QV2_CUDA(c, launch_hist(l, p.any_16bit, c->d_tensors, c->d_hist_tiles, (uint32_t)p.hist_tiles.size(),
                             c->d_tensor_absmax, reinterpret_cast<unsigned long long*>(nonfinite), h));
     ++c->launches;
   }
-  QV2_CUDA(c, launch_clip_finalize(l, c->d_tensors, n, h, c->d_tensor_absmax, gmin, gmax, gabsmax,
-                                   clip, step, inv, offset));
-  ++c->launches;
+  if (p.any_percentile) {              // clip[t] of the other tensors is already the absmax
+    QV2_CUDA(c, launch_clip_finalize(l, c->d_tensors, n, h, c->d_tensor_absmax, gmin, gmax, gabsmax,
+                                     clip, step, inv, offset));
+    ++c->launches;
+  }
   if (n_ghist) {
     QV2_CUDA(c, launch_group_hist(l, p.any_16bit, c->d_tensors, c->d_ghist_tiles, (uint32_t)p.ghist_tiles.size(),
                                   gabsmax, reinterpret_cast<unsigned long long*>(nonfinite), gh));

@@ -102,7 +102,7 @@ cudaError_t launch_calib_init(const Launch& l, uint32_t* kmin, uint32_t* kmax, s
 uint32_t range_grid_cap(int sm_count);     // resident CTAs per SM x SMs for the range kernel
 cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                   const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
-                                  float* step, float* inv, float* offset, float* tensor_absmax);
+                                  float* step, float* inv, float* offset, float* tensor_absmax, float* clip);
 cudaError_t launch_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
                         uint32_t n_tiles, const float* tensor_absmax,
                         const unsigned long long* nonfinite, unsigned long long* hist);

@@ -239,7 +239,7 @@ constexpr int kFinalizeThreads = 1024;
 __global__ void __launch_bounds__(kFinalizeThreads)
 range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __restrict__ rslots,
                       float* gmin, float* gmax, float* gabsmax, float* step, float* inv, float* offset,
-                      float* tensor_absmax) {
+                      float* tensor_absmax, float* clip) {
   __shared__ float red[kFinalizeThreads];
   __shared__ uint32_t kred[2][kFinalizeThreads];
   const TensorRec tr = tensors[blockIdx.x];
@@ -285,7 +285,10 @@ range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __rest
     if (threadIdx.x < o) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + o]);
     __syncthreads();
   }
-  if (threadIdx.x == 0) tensor_absmax[blockIdx.x] = red[0];
+  if (threadIdx.x == 0) {
+    tensor_absmax[blockIdx.x] = red[0];
+    clip[blockIdx.x] = red[0];          // the percentile pass replaces it for the tensors it clips
+  }
 }
 
 // Everything a calibration pass accumulates into starts at zero: the min/max keys (0 = nothing
@@ -331,9 +334,9 @@ cudaError_t launch_range(const Launch& l, uint32_t grid, bool any16, const Tenso
 
 cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                   const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
-                                  float* step, float* inv, float* offset, float* tensor_absmax) {
+                                  float* step, float* inv, float* offset, float* tensor_absmax, float* clip) {
   range_finalize_kernel<<<n_tensors, kFinalizeThreads, 0, l.stream>>>(tensors, rslots, gmin, gmax, gabsmax, step,
-                                                         inv, offset, tensor_absmax);
+                                                         inv, offset, tensor_absmax, clip);
   return cudaGetLastError();
 }
 
