@@ -22,131 +22,146 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
             const uint64_t* __restrict__ macs, const double* __restrict__ pos,
             const uint32_t* __restrict__ fuse_group, qv2_rank_cfg cfg, double* score, double* severity,
             uint32_t* place, uint32_t* best, uint32_t* order, uint8_t* keep, uint32_t* n_keep) {
-  // Models have tens of layers: up to kStage layers the serial parts below run out of shared
-  // memory instead of paying a global-memory latency per step.
-  constexpr uint32_t kStage = 1024;
+  // Models have tens of layers: up to kStage layers every input and every intermediate lives in
+  // shared memory, so the phases below cost one trip to global memory at the start and one at the
+  // end instead of one per phase.  Larger n runs the same code on the global arrays.
+  constexpr uint32_t kStage = 512;
   __shared__ double mean_s[2];
-  __shared__ double st_a[kStage], st_b[kStage];
-  __shared__ unsigned long long st_macs[kStage];
-  __shared__ uint32_t st_order[kStage], st_fg[kStage];
+  __shared__ double s_mw[kStage], s_ma[kStage], s_sw[kStage], s_sa[kStage], s_pos[kStage], s_score[kStage],
+      s_sev[kStage];
+  __shared__ unsigned long long s_macs[kStage];
+  __shared__ uint32_t s_fg[kStage], s_place[kStage], s_best[kStage], s_order[kStage];
+  __shared__ uint8_t s_keep[kStage];
   constexpr uint32_t kNoGroup = QV2_NO_GROUP;
   const uint32_t tid = threadIdx.x;
   const bool staged = n <= kStage;
   const double inf = __longlong_as_double(0x7ff0000000000000ll);
+  // the arrays the phases work on: shared copies when staged, the global ones otherwise
+  const double *mw = mse_w, *ma = mse_a, *sw = sqnr_w, *sa = sqnr_a, *ps = pos;
+  const unsigned long long* mc = reinterpret_cast<const unsigned long long*>(macs);
+  const uint32_t* fg = fuse_group;
+  double *sc = score, *sv = severity;
+  uint32_t *pl = place, *bs = best, *od = order;
+  uint8_t* kp = keep;
   if (staged) {
     for (uint32_t i = tid; i < n; i += blockDim.x) {
-      st_a[i] = mse_w[i]; st_b[i] = mse_a[i];
-      st_macs[i] = macs ? macs[i] : 1ull;
-      st_fg[i] = fuse_group ? fuse_group[i] : kNoGroup;
+      s_mw[i] = mse_w[i]; s_ma[i] = mse_a[i]; s_sw[i] = sqnr_w[i]; s_sa[i] = sqnr_a[i];
+      if (pos) s_pos[i] = pos[i];
+      if (macs) s_macs[i] = macs[i];
+      if (fuse_group) s_fg[i] = fuse_group[i];
     }
+    mw = s_mw; ma = s_ma; sw = s_sw; sa = s_sa;
+    if (pos) ps = s_pos;
+    if (macs) mc = s_macs;
+    if (fuse_group) fg = s_fg;
+    sc = s_score; sv = s_sev; pl = s_place; bs = s_best; od = s_order; kp = s_keep;
     __syncthreads();
   }
   if (tid == 0) {                      // means: sums in layer order, as the definition states
-    double sw = 0.0, sa = 0.0;
+    double a = 0.0, b = 0.0;
     for (uint32_t i = 0; i < n; ++i) {
-      sw = __dadd_rn(sw, staged ? st_a[i] : mse_w[i]);
-      sa = __dadd_rn(sa, staged ? st_b[i] : mse_a[i]);
+      a = __dadd_rn(a, mw[i]);
+      b = __dadd_rn(b, ma[i]);
     }
-    mean_s[0] = __ddiv_rn(sw, (double)n);
-    mean_s[1] = __ddiv_rn(sa, (double)n);
+    mean_s[0] = __ddiv_rn(a, (double)n);
+    mean_s[1] = __ddiv_rn(b, (double)n);
   }
   __syncthreads();
   const double mean_w = mean_s[0], mean_a = mean_s[1], cap = cfg.sqnr_cap_db;
   for (uint32_t i = tid; i < n; i += blockDim.x) {
     double dw = 0.0, da = 0.0;
     if (i > 0) {
-      const double den = pos ? __dsub_rn(pos[i], pos[i - 1]) : 1.0;
-      dw = __ddiv_rn(__dsub_rn(clamp_cap(sqnr_w[i], cap), clamp_cap(sqnr_w[i - 1], cap)), den);
-      da = __ddiv_rn(__dsub_rn(clamp_cap(sqnr_a[i], cap), clamp_cap(sqnr_a[i - 1], cap)), den);
+      const double den = ps ? __dsub_rn(ps[i], ps[i - 1]) : 1.0;
+      dw = __ddiv_rn(__dsub_rn(clamp_cap(sw[i], cap), clamp_cap(sw[i - 1], cap)), den);
+      da = __ddiv_rn(__dsub_rn(clamp_cap(sa[i], cap), clamp_cap(sa[i - 1], cap)), den);
     }
-    double sc = __dadd_rn(__dmul_rn(cfg.w_gain, dw), __dmul_rn(cfg.a_gain, da));
-    if (sc != sc) sc = inf;
-    const double rw = mean_w > 0.0 ? __ddiv_rn(mse_w[i], mean_w) : 0.0;
-    const double ra = mean_a > 0.0 ? __ddiv_rn(mse_a[i], mean_a) : 0.0;
-    double sv = rw > ra ? rw : ra;
-    if (sv != sv) sv = 0.0;
-    score[i] = sc; severity[i] = sv; keep[i] = 0;
+    double s = __dadd_rn(__dmul_rn(cfg.w_gain, dw), __dmul_rn(cfg.a_gain, da));
+    if (s != s) s = inf;
+    const double rw = mean_w > 0.0 ? __ddiv_rn(mw[i], mean_w) : 0.0;
+    const double ra = mean_a > 0.0 ? __ddiv_rn(ma[i], mean_a) : 0.0;
+    double v = rw > ra ? rw : ra;
+    if (v != v) v = 0.0;
+    sc[i] = s; sv[i] = v; kp[i] = 0;
   }
   __syncthreads();
   // Position of layer i = number of layers that come before it: all MSE outliers precede the
   // rest; outliers by descending severity, the rest by ascending score, ties by layer index.
   const double fac = cfg.mse_factor;
   for (uint32_t i = tid; i < n; i += blockDim.x) {
-    const double si = score[i], vi = severity[i];
+    const double si = sc[i], vi = sv[i];
     const bool out_i = vi > fac;
     uint32_t rank = 0;
     for (uint32_t j = 0; j < n; ++j) {
-      const double vj = severity[j];
+      const double vj = sv[j];
       const bool out_j = vj > fac;
       if (out_i) {
         if (out_j && (vj > vi || (vj == vi && j < i))) ++rank;
       } else {
         if (out_j) ++rank;
         else {
-          const double sj = score[j];
+          const double sj = sc[j];
           if (sj < si || (sj == si && j < i)) ++rank;
         }
       }
     }
-    order[rank] = i;
-    place[i] = rank;
+    od[rank] = i;
+    pl[i] = rank;
   }
   __syncthreads();
-  if (fuse_group) {
+  if (fg) {
     // Fusion groups: every member moves to the place of the group's best-ranked member and the
     // members stand there in layer order.  Places of different groups differ, so sorting by
     // (best place of my group, layer index) yields exactly that list.
     for (uint32_t i = tid; i < n; i += blockDim.x) {
-      const uint32_t g = fuse_group[i];
-      uint32_t b = place[i];
+      const uint32_t g = fg[i];
+      uint32_t b = pl[i];
       if (g != kNoGroup)
         for (uint32_t j = 0; j < n; ++j)
-          if (fuse_group[j] == g) b = min(b, place[j]);
-      best[i] = b;
+          if (fg[j] == g) b = min(b, pl[j]);
+      bs[i] = b;
     }
     __syncthreads();
     for (uint32_t i = tid; i < n; i += blockDim.x) {
-      const uint32_t bi = best[i];
+      const uint32_t bi = bs[i];
       uint32_t rank = 0;
       for (uint32_t j = 0; j < n; ++j) {
-        const uint32_t bj = best[j];
+        const uint32_t bj = bs[j];
         if (bj < bi || (bj == bi && j < i)) ++rank;
       }
-      order[rank] = i;
+      od[rank] = i;
     }
-    __syncthreads();
-  }
-  if (staged) {
-    for (uint32_t i = tid; i < n; i += blockDim.x) st_order[i] = order[i];
     __syncthreads();
   }
   if (tid == 0) {
     // The FP32-kept prefix grows one whole fusion group at a time (a layer without a group is a
     // group of one): by count while it still fits, by rate while the rate still holds.
-    auto ord = [&](uint32_t j) { return staged ? st_order[j] : order[j]; };
-    auto grp = [&](uint32_t l) { return staged ? st_fg[l] : (fuse_group ? fuse_group[l] : kNoGroup); };
-    auto mac = [&](uint32_t l) { return staged ? st_macs[l] : (macs ? macs[l] : 1ull); };
+    auto grp = [&](uint32_t l) { return fg ? fg[l] : kNoGroup; };
+    auto mac = [&](uint32_t l) { return mc ? mc[l] : 1ull; };
     unsigned __int128 total = 0, kept = 0;
     if (cfg.select_mode != QV2_BY_COUNT)
       for (uint32_t i = 0; i < n; ++i) total += mac(i);
     uint32_t nk = 0, j = 0;
     while (j < n) {
-      const uint32_t g = grp(ord(j));
+      const uint32_t g = grp(od[j]);
       uint32_t e = j + 1;
-      if (g != kNoGroup) while (e < n && grp(ord(e)) == g) ++e;
+      if (g != kNoGroup) while (e < n && grp(od[e]) == g) ++e;
       if (cfg.select_mode == QV2_BY_COUNT) {
         if (e <= cfg.keep_count) nk = e; else break;
       } else {
         unsigned __int128 m = 0;
-        for (uint32_t k = j; k < e; ++k) m += mac(ord(k));
+        for (uint32_t k = j; k < e; ++k) m += mac(od[k]);
         const unsigned __int128 quantized = total - (kept + m);
         if (quantized * 10000u >= (unsigned __int128)cfg.rate_permyriad * total) { kept += m; nk = e; }
         else break;
       }
       j = e;
     }
-    for (uint32_t k = 0; k < nk; ++k) keep[ord(k)] = 1;
+    for (uint32_t k = 0; k < nk; ++k) kp[od[k]] = 1;
     *n_keep = nk;
+  }
+  if (staged) {                        // publish the list and the flags
+    __syncthreads();
+    for (uint32_t i = tid; i < n; i += blockDim.x) { order[i] = s_order[i]; keep[i] = s_keep[i]; }
   }
 }
 
