@@ -15,9 +15,15 @@
  *     demand and released by qv2_destroy.
  *   - Calls enqueue work on the context's stream and return; outputs are valid once the caller has
  *     synchronised that stream.  Argument errors are found on the host before anything is
- *     launched.  Exceptions: a call whose descriptor set differs from the previous call's
- *     synchronises the stream once while it rebuilds its tile table, and qv2_sweep_model_host
- *     synchronises before it returns.
+ *     launched.  Exceptions: a call whose descriptor set (the qv2_tensor_desc bytes) differs from
+ *     the previous call's synchronises the stream once while it rebuilds its tile table -- the
+ *     code pointers of qv2_quant_metrics are not part of that set -- and qv2_sweep_model_host
+ *     and qv2_check_nonfinite synchronise before they return.  qv2_sync_count reports how often
+ *     a context has done so.
+ *   - Accumulators that must start at zero (range keys, counters, histograms, tickets) live in
+ *     context scratch and are put back to zero by the kernel that consumes them, so a pass needs
+ *     no clearing launch.  Partial results of a tensor are folded by whichever thread block
+ *     finishes the tensor last, found with an atomic counter; no block ever waits for another.
  *   - One context serves one stream; use it from one host thread at a time.
  *   - Tensors are fp32, contiguous, viewed as [outer][channels][inner]; element (o,c,i) lives at
  *     index (o*channels + c)*inner + i.  Weights: outer = 1, channels = C_out, inner = C_in/g*k*k.
@@ -55,6 +61,8 @@ enum { QV2_SYM_I8 = 0, QV2_ASYM_U8 = 1, QV2_ASYM_U8_ZP = 2 }; /* scheme */
 enum { QV2_ABSMAX = 0, QV2_MINMAX = 1, QV2_PERCENTILE = 2, QV2_PERCENTILE_GROUP = 3 }; /* range */
 enum { QV2_PAIR_REQUANT = 0, QV2_PAIR_RAW = 1, QV2_STORE_CODES = 2 }; /* flags (bit 0: pair mode) */
 enum { QV2_BY_COUNT = 0, QV2_BY_BOPS_RATE = 1 };             /* select_mode */
+enum { QV2_OUTLIERS_BY_SEVERITY = 0, QV2_OUTLIERS_LITERAL = 1 }; /* outlier_order */
+enum { QV2_SCHEDULE_PHASE_MAJOR = 0, QV2_SCHEDULE_L2_CHUNKED = 1, QV2_SCHEDULE_AUTO = 2 };
 /* Code width other than 8 bits, OR-ed into qv2_tensor_desc.flags: QV2_BITS(b), 2 <= b <= 16.  The
  * largest code is 2^(b-1) - 1 for QV2_SYM_I8 (Eq. 4) and 2^b - 1 for QV2_ASYM_U8 (Eq. 2 with
  * N = 2^b levels); wherever this header says 127 or 255 read that value.  No QV2_BITS means 8.
@@ -112,7 +120,12 @@ typedef struct {
   uint32_t keep_count;     /* QV2_BY_COUNT: how many list entries stay FP32 */
   uint32_t rate_permyriad; /* QV2_BY_BOPS_RATE: requested BOPs-reduction rate, 0..10000
                               (0 = everything FP32, 10000 = everything int8) */
-  uint32_t reserved;
+  uint32_t outlier_order;  /* order among the layers whose MSE exceeds the threshold:
+                              QV2_OUTLIERS_BY_SEVERITY (0): most severe first;
+                              QV2_OUTLIERS_LITERAL: as Algorithm 2's RankLayersBySensitivity is
+                              printed -- it walks the layers in order and puts each outlier at the
+                              head of the list as it meets it, so the outliers end in reverse
+                              layer order (the last one met stands first) */
 } qv2_rank_cfg;
 
 /* Creates a context bound to CUDA device `device` and to `stream` (a cudaStream_t, borrowed, may
@@ -125,6 +138,31 @@ const char* qv2_status_string(int status);
 int qv2_last_cuda_error(const qv2_ctx* ctx);
 /* Number of kernel launches this context has enqueued since it was created. */
 uint64_t qv2_launch_count(const qv2_ctx* ctx);
+/* Number of times this context has synchronised its stream on the host (tile-table rebuilds,
+ * qv2_check_nonfinite, qv2_sweep_model_host, qv2_sweep_graph_create). */
+uint64_t qv2_sync_count(const qv2_ctx* ctx);
+
+/*
+ * Order in which the phases visit the tensors.  The paper's calibration stage and the loop of
+ * Algorithm 2 pass over each tensor three times (range, histogram, error metrics), each pass
+ * needing a result of the one before.
+ *   QV2_SCHEDULE_PHASE_MAJOR (default): one launch per phase over the whole model; every pass
+ *     reads its tensors from HBM.  Right for tensors far larger than L2.
+ *   QV2_SCHEDULE_L2_CHUNKED: consecutive tensors are grouped into stages whose reference tensors
+ *     (x) hold at most chunk_bytes together; the phases run stage by stage, so the second and third
+ *     pass over a stage find x in L2.  Tensors larger than chunk_bytes gather in stages of their
+ *     own.  qv2_calibrate runs range -> histogram per stage; qv2_sweep_model (and its captured
+ *     form) runs range -> histogram -> metrics per stage.  Results are the same bits for integer
+ *     outputs and parameters; sums are added in a stage-dependent order (same tolerances).  Plans
+ *     with QV2_PERCENTILE_GROUP tensors keep one stage.
+ *   QV2_SCHEDULE_AUTO: chunked when the model is larger than two chunks and at least half of its
+ *     reference bytes sit in tensors that fit a chunk, else phase-major.
+ * chunk_bytes: 0 selects the default (48 MiB, well under half of a B200's 126 MB L2).
+ * Takes effect with the next call; QV2_ERR_UNSUPPORTED while a captured pass of this context lives.
+ */
+int qv2_set_schedule(qv2_ctx* ctx, uint32_t schedule, uint64_t chunk_bytes);
+/* Number of stages of the context's current plan (1 for phase-major; 0 before the first call). */
+uint32_t qv2_stage_count(const qv2_ctx* ctx);
 /* Sum over descs of the number of quantization groups (1 or `channels`).  Host only. */
 uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n);
 
@@ -135,7 +173,8 @@ uint64_t qv2_group_count(const qv2_tensor_desc* descs, uint32_t n);
  * each operation rounded once in binary32, in that order.  As printed in the paper there is no
  * epsilon under the root: the caller adds it to var if its framework uses one; var_c <= 0 gives
  * Inf/NaN in that channel.
- * w, w_out: device, [channels][inner] fp32 (w_out may alias w).  bias: device [channels] or NULL
+ * w, w_out: device, [channels][inner] fp32; w_out may be w itself (folding in place), but must not
+ * overlap it otherwise.  bias: device [channels] or NULL
  * (zeros).  gamma, beta, mean, var: device [channels].  bias_out: device [channels] or NULL.
  */
 int qv2_fold_batchnorm(qv2_ctx* ctx, const float* w, const float* bias, const float* gamma,
@@ -143,10 +182,10 @@ int qv2_fold_batchnorm(qv2_ctx* ctx, const float* w, const float* bias, const fl
                        uint64_t channels, uint64_t inner, float* w_out, float* bias_out);
 
 /*
- * Calibration: step 1 of the paper's overview ("collect statistical data on the distribution of
- * weights and activations") together with its calibration stage (a histogram of each layer's
- * value range), followed by the scale computation of step 2 (Eq. 4 for symmetric weights, Eq. 2
- * for the affine form).
+ * Calibration: step 1 of the paper's method overview (range statistics of every layer's weights
+ * and activations) together with its calibration stage (a histogram of each layer's value range),
+ * followed by the scale computation of step 2 (Eq. 4 for symmetric weights, Eq. 2 for the affine
+ * form).
  *
  * For every group g of every tensor: gmin/gmax = min/max over the group's finite elements,
  * gabsmax = max(|gmin|,|gmax|) (a zero is returned as +0).  For every tensor t whose range is
@@ -208,10 +247,10 @@ uint64_t qv2_group_hist_count(const qv2_tensor_desc* descs, uint32_t n);
 int qv2_check_nonfinite(qv2_ctx* ctx, const uint64_t* nonfinite, uint32_t n, uint32_t* first_bad);
 
 /*
- * Fused fake-quantize + error reduction: step 3 of the overview ("measure the SQNR and MSE of each
- * layer by comparing the weights and activations of the original and quantized models"), i.e.
- * CalculateSQNR / CalculateMSE of Algorithm 2 over every element, with the quantizer of Eq. 1 / Eq. 5
- * and the dequantizer of Eq. 3; SQNR is Eq. 6 and MSE is Eq. 7.
+ * Fused fake-quantize + error reduction: step 3 of the method overview (per-layer SQNR and MSE
+ * between the original and the quantized model's weights and activations), i.e. CalculateSQNR /
+ * CalculateMSE of Algorithm 2 over every element, with the quantizer of Eq. 1 / Eq. 5 and the
+ * dequantizer of Eq. 3; SQNR is Eq. 6 and MSE is Eq. 7.
  *
  * Per element of the tensor v being quantized (x in self mode, y in QV2_PAIR_REQUANT):
  *   t = fl(fl(v - offset_g) * inv_g);  q = clamp(round_half_even(t), qmin, qmax);
@@ -279,8 +318,9 @@ int qv2_kl_divergence(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n,
  *   delta_0 = 0, delta_n = (sqnr[n]-sqnr[n-1]) / (pos[n]-pos[n-1]) after clamping sqnr to +-cap;
  *   score_n = w_gain*delta_w_n + a_gain*delta_a_n;
  *   severity_n = max(mse_w[n]/mean(mse_w), mse_a[n]/mean(mse_a)) (a zero mean contributes 0);
- *   order = layers with severity > mse_factor, most severe first, then the others by ascending
- *           score; ties keep layer order.  A NaN score sorts last, a NaN severity counts as 0.
+ *   order = layers with severity > mse_factor, most severe first (or in reverse layer order, see
+ *           qv2_rank_cfg.outlier_order), then the others by ascending score; ties keep layer
+ *           order.  A NaN score sorts last, a NaN severity counts as 0.
  *   QV2_BY_COUNT keeps order[0..keep_count) in FP32; QV2_BY_BOPS_RATE keeps the longest prefix for
  *   which (MACs of the still-quantized layers)/(all MACs) >= rate_permyriad/10000.
  *
@@ -347,8 +387,11 @@ int qv2_sweep_model(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n_tenso
  * it needs a context created on a non-default stream (QV2_ERR_UNSUPPORTED otherwise) and
  * synchronises that stream.  The graph reads the same tensor and buffer ADDRESSES on every
  * replay: refill the tensors in place, do not move or free them while the graph lives, and do not
- * destroy the context before the graph.  qv2_sweep_graph_launch enqueues one replay on the
- * context's stream and returns.
+ * destroy the context before the graph.  It also holds the addresses of the context's tile tables
+ * and scratch: while a graph of a context lives, every other call on that context must use the
+ * descriptor set the graph was captured with (calls with another set, or that would have to move
+ * scratch, return QV2_ERR_UNSUPPORTED and leave the graph intact); use a second context for other
+ * models.  qv2_sweep_graph_launch enqueues one replay on the context's stream and returns.
  */
 typedef struct qv2_graph qv2_graph;
 int qv2_sweep_graph_create(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n_tensors,

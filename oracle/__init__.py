@@ -64,6 +64,10 @@ def _load():
                               C.c_double, C.c_double, C.c_double, C.c_double,
                               C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
     lib.qv2o_rank.restype = None
+    lib.qv2o_rank_ex.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p,
+                                 C.c_double, C.c_double, C.c_double, C.c_double,
+                                 C.c_int, C.c_uint32, C.c_uint32, C.c_int, u32p, u8p, u32p]
+    lib.qv2o_rank_ex.restype = None
     lib.qv2o_qparams_bits.argtypes = [C.c_int] + list(lib.qv2o_qparams.argtypes)
     lib.qv2o_qparams_bits.restype = None
     lib.qv2o_quant_metrics_bits.argtypes = [C.c_int] + list(lib.qv2o_quant_metrics.argtypes)
@@ -83,6 +87,10 @@ def _load():
                                     C.c_double, C.c_double, C.c_double, C.c_double,
                                     C.c_int, C.c_uint32, C.c_uint32, u32p, u8p, u32p]
     lib.qv2o_rank_fused.restype = None
+    lib.qv2o_rank_fused_ex.argtypes = [C.c_uint32, f64p, f64p, f64p, f64p, u64p, f64p, u32p,
+                                       C.c_double, C.c_double, C.c_double, C.c_double,
+                                       C.c_int, C.c_uint32, C.c_uint32, C.c_int, u32p, u8p, u32p]
+    lib.qv2o_rank_fused_ex.restype = None
     _lib = lib
     return lib
 
@@ -231,8 +239,10 @@ def kl_divergence(x, y, outer: int, channels: int, inner: int, per_channel: bool
 
 
 def rank_layers(sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, w_gain=2.0, a_gain=1.0,
-                mse_factor=5.0, cap_db=200.0, select_mode=0, keep_count=0, rate_permyriad=0):
-    """-> (order[n] uint32, keep_fp32[n] uint8, n_keep)."""
+                mse_factor=5.0, cap_db=200.0, select_mode=0, keep_count=0, rate_permyriad=0,
+                outlier_order=0):
+    """-> (order[n] uint32, keep_fp32[n] uint8, n_keep).  outlier_order 1 places the MSE outliers
+    as Algorithm 2's pseudo-code does (each at the head when met: reverse layer order)."""
     lib = _load()
     f = lambda a: np.ascontiguousarray(a, dtype=np.float64)
     sqnr_w, mse_w, sqnr_a, mse_a = f(sqnr_w), f(mse_w), f(sqnr_a), f(mse_a)
@@ -240,10 +250,11 @@ def rank_layers(sqnr_w, mse_w, sqnr_a, mse_a, macs=None, pos=None, w_gain=2.0, a
     m = None if macs is None else np.ascontiguousarray(macs, dtype=np.uint64)
     ps = None if pos is None else f(pos)
     order = np.zeros(n, np.uint32); keep = np.zeros(n, np.uint8); nk = C.c_uint32(0)
-    lib.qv2o_rank(n, _p(sqnr_w, C.c_double), _p(mse_w, C.c_double), _p(sqnr_a, C.c_double),
-                  _p(mse_a, C.c_double), _p(m, C.c_uint64), _p(ps, C.c_double),
-                  w_gain, a_gain, mse_factor, cap_db, int(select_mode), int(keep_count),
-                  int(rate_permyriad), _p(order, C.c_uint32), _p(keep, C.c_uint8), C.byref(nk))
+    lib.qv2o_rank_ex(n, _p(sqnr_w, C.c_double), _p(mse_w, C.c_double), _p(sqnr_a, C.c_double),
+                     _p(mse_a, C.c_double), _p(m, C.c_uint64), _p(ps, C.c_double),
+                     w_gain, a_gain, mse_factor, cap_db, int(select_mode), int(keep_count),
+                     int(rate_permyriad), int(outlier_order), _p(order, C.c_uint32), _p(keep, C.c_uint8),
+                     C.byref(nk))
     return order, keep, int(nk.value)
 
 
@@ -252,7 +263,7 @@ NO_GROUP = 0xFFFFFFFF
 
 def rank_layers_fused(sqnr_w, mse_w, sqnr_a, mse_a, fuse_group, macs=None, pos=None, w_gain=2.0,
                       a_gain=1.0, mse_factor=5.0, cap_db=200.0, select_mode=0, keep_count=0,
-                      rate_permyriad=0):
+                      rate_permyriad=0, outlier_order=0):
     """rank_layers with fusion groups: -> (order, keep_fp32, n_keep).  fuse_group[i] is a group id
     or NO_GROUP; None means no groups at all."""
     lib = _load()
@@ -263,10 +274,11 @@ def rank_layers_fused(sqnr_w, mse_w, sqnr_a, mse_a, fuse_group, macs=None, pos=N
     ps = None if pos is None else f(pos)
     fg = None if fuse_group is None else np.ascontiguousarray(fuse_group, dtype=np.uint32)
     order = np.zeros(n, np.uint32); keep = np.zeros(n, np.uint8); nk = C.c_uint32(0)
-    lib.qv2o_rank_fused(n, _p(sqnr_w, C.c_double), _p(mse_w, C.c_double), _p(sqnr_a, C.c_double),
-                        _p(mse_a, C.c_double), _p(m, C.c_uint64), _p(ps, C.c_double), _p(fg, C.c_uint32),
-                        w_gain, a_gain, mse_factor, cap_db, int(select_mode), int(keep_count),
-                        int(rate_permyriad), _p(order, C.c_uint32), _p(keep, C.c_uint8), C.byref(nk))
+    lib.qv2o_rank_fused_ex(n, _p(sqnr_w, C.c_double), _p(mse_w, C.c_double), _p(sqnr_a, C.c_double),
+                           _p(mse_a, C.c_double), _p(m, C.c_uint64), _p(ps, C.c_double), _p(fg, C.c_uint32),
+                           w_gain, a_gain, mse_factor, cap_db, int(select_mode), int(keep_count),
+                           int(rate_permyriad), int(outlier_order), _p(order, C.c_uint32), _p(keep, C.c_uint8),
+                           C.byref(nk))
     return order, keep, int(nk.value)
 
 

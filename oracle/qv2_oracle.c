@@ -427,7 +427,8 @@ double qv2o_kl_bits(int bits, const float *x, const float *y,
  *  2. delta_0 = 0; delta_n = (sqnr[n] - sqnr[n-1]) / (pos[n] - pos[n-1])  (pos defaults to n).
  *  3. score_n = w_gain * dw_n + a_gain * da_n  (the weighted sum of the two delta lists).
  *  4. r_n = max(mse_w[n] / mean(mse_w), mse_a[n] / mean(mse_a)), a zero mean contributing 0;
- *     layers with r_n > mse_factor (5 in the paper) go to the top, most severe first.
+ *     layers with r_n > mse_factor (5 in the paper) go to the top, most severe first (or, on
+ *     request, in the order the printed pseudo-code produces: see qv2o_rank_ex).
  *  5. the remaining layers follow in ascending score (smaller delta = noise grew = more
  *     sensitive); ties keep layer order.  A NaN score counts as +inf, a NaN severity as 0 (the
  *     paper does not say what an undefined metric does; this keeps the list a permutation).
@@ -443,12 +444,16 @@ static double clampd(double v, double cap)
     return v;
 }
 
-void qv2o_rank(uint32_t n, const double *sqnr_w, const double *mse_w,
-               const double *sqnr_a, const double *mse_a,
-               const uint64_t *macs, const double *pos,
-               double w_gain, double a_gain, double mse_factor, double cap,
-               int select_mode, uint32_t keep_count, uint32_t rate_permyriad,
-               uint32_t *order, uint8_t *keep, uint32_t *n_keep)
+/* outlier_order 0: MSE outliers most severe first (the reading this library takes by default).
+ * outlier_order 1: Algorithm 2's RankLayersBySensitivity as printed: the layers are visited in
+ * order and each outlier is inserted at the head of the list when it is met, so the outliers end
+ * in reverse layer order. */
+void qv2o_rank_ex(uint32_t n, const double *sqnr_w, const double *mse_w,
+                  const double *sqnr_a, const double *mse_a,
+                  const uint64_t *macs, const double *pos,
+                  double w_gain, double a_gain, double mse_factor, double cap,
+                  int select_mode, uint32_t keep_count, uint32_t rate_permyriad, int outlier_order,
+                  uint32_t *order, uint8_t *keep, uint32_t *n_keep)
 {
     if (n == 0) { *n_keep = 0; return; }
     double *score = (double *)malloc(n * sizeof(double));
@@ -475,7 +480,13 @@ void qv2o_rank(uint32_t n, const double *sqnr_w, const double *mse_w,
     }
     /* selection sort, written for clarity: repeatedly take the best remaining layer */
     uint32_t filled = 0;
-    for (;;) {                                   /* MSE outliers, most severe first */
+    if (outlier_order == 1) {                    /* each outlier goes to the head as it is met */
+        for (uint32_t i = 0; i < n; ++i) {
+            if (!(sev[i] > mse_factor)) continue;
+            for (uint32_t k = filled; k > 0; --k) order[k] = order[k - 1];
+            order[0] = i; taken[i] = 1; ++filled;
+        }
+    } else for (;;) {                            /* MSE outliers, most severe first */
         int best = -1;
         for (uint32_t i = 0; i < n; ++i)
             if (!taken[i] && sev[i] > mse_factor && (best < 0 || sev[i] > sev[best])) best = (int)i;
@@ -509,6 +520,17 @@ void qv2o_rank(uint32_t n, const double *sqnr_w, const double *mse_w,
     free(score); free(sev); free(taken);
 }
 
+void qv2o_rank(uint32_t n, const double *sqnr_w, const double *mse_w,
+               const double *sqnr_a, const double *mse_a,
+               const uint64_t *macs, const double *pos,
+               double w_gain, double a_gain, double mse_factor, double cap,
+               int select_mode, uint32_t keep_count, uint32_t rate_permyriad,
+               uint32_t *order, uint8_t *keep, uint32_t *n_keep)
+{
+    qv2o_rank_ex(n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, w_gain, a_gain, mse_factor, cap,
+                 select_mode, keep_count, rate_permyriad, 0, order, keep, n_keep);
+}
+
 /* ---------------------------------------------------------------------------------------------
  * Fusion-aware sensitivity list.  The paper says only that fusion-capable operators (convolution,
  * batch normalisation, add, ReLU) may have their positions in the list adjusted so that they can
@@ -521,19 +543,19 @@ void qv2o_rank(uint32_t n, const double *sqnr_w, const double *mse_w,
  * ------------------------------------------------------------------------------------------- */
 #define QV2O_NO_GROUP 0xFFFFFFFFu
 
-void qv2o_rank_fused(uint32_t n, const double *sqnr_w, const double *mse_w,
-                     const double *sqnr_a, const double *mse_a,
-                     const uint64_t *macs, const double *pos, const uint32_t *fuse_group,
-                     double w_gain, double a_gain, double mse_factor, double cap,
-                     int select_mode, uint32_t keep_count, uint32_t rate_permyriad,
-                     uint32_t *order, uint8_t *keep, uint32_t *n_keep)
+void qv2o_rank_fused_ex(uint32_t n, const double *sqnr_w, const double *mse_w,
+                        const double *sqnr_a, const double *mse_a,
+                        const uint64_t *macs, const double *pos, const uint32_t *fuse_group,
+                        double w_gain, double a_gain, double mse_factor, double cap,
+                        int select_mode, uint32_t keep_count, uint32_t rate_permyriad, int outlier_order,
+                        uint32_t *order, uint8_t *keep, uint32_t *n_keep)
 {
     if (n == 0) { *n_keep = 0; return; }
     uint32_t *base = (uint32_t *)malloc(n * sizeof(uint32_t));
     uint8_t *tmp_keep = (uint8_t *)malloc(n);
     uint32_t tmp_nk;
-    qv2o_rank(n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, w_gain, a_gain, mse_factor, cap,
-              0, 0, 0, base, tmp_keep, &tmp_nk);
+    qv2o_rank_ex(n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, w_gain, a_gain, mse_factor, cap,
+                 0, 0, 0, outlier_order, base, tmp_keep, &tmp_nk);
     uint8_t *done = (uint8_t *)calloc(n, 1);
     uint32_t filled = 0;
     for (uint32_t j = 0; j < n; ++j) {
@@ -566,6 +588,17 @@ void qv2o_rank_fused(uint32_t n, const double *sqnr_w, const double *mse_w,
     for (uint32_t k = 0; k < nk; ++k) keep[order[k]] = 1;
     *n_keep = nk;
     free(base); free(tmp_keep); free(done);
+}
+
+void qv2o_rank_fused(uint32_t n, const double *sqnr_w, const double *mse_w,
+                     const double *sqnr_a, const double *mse_a,
+                     const uint64_t *macs, const double *pos, const uint32_t *fuse_group,
+                     double w_gain, double a_gain, double mse_factor, double cap,
+                     int select_mode, uint32_t keep_count, uint32_t rate_permyriad,
+                     uint32_t *order, uint8_t *keep, uint32_t *n_keep)
+{
+    qv2o_rank_fused_ex(n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, fuse_group, w_gain, a_gain, mse_factor,
+                       cap, select_mode, keep_count, rate_permyriad, 0, order, keep, n_keep);
 }
 
 /* ---------------------------------------------------------------------------------------------

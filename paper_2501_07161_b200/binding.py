@@ -18,6 +18,8 @@ SYM_I8, ASYM_U8, ASYM_U8_ZP = 0, 1, 2
 ABSMAX, MINMAX, PERCENTILE, PERCENTILE_GROUP = 0, 1, 2, 3
 PAIR_REQUANT, PAIR_RAW, STORE_CODES = 0, 1, 2
 BY_COUNT, BY_BOPS_RATE = 0, 1
+OUTLIERS_BY_SEVERITY, OUTLIERS_LITERAL = 0, 1
+SCHEDULE_PHASE_MAJOR, SCHEDULE_L2_CHUNKED, SCHEDULE_AUTO = 0, 1, 2
 IN_F32, IN_F16, IN_BF16 = 0, 1 << 16, 2 << 16
 _DTYPE_FLAG = {torch.float32: IN_F32, torch.float16: IN_F16, torch.bfloat16: IN_BF16}
 HIST_BINS = 2048
@@ -27,7 +29,8 @@ EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_erro
            "qv2_launch_count", "qv2_group_count", "qv2_calibrate", "qv2_quant_metrics",
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
            "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm", "qv2_sweep_graph_create", "qv2_sweep_graph_launch",
-           "qv2_sweep_graph_destroy", "qv2_check_nonfinite", "qv2_calibrate_ex", "qv2_group_hist_count"]
+           "qv2_sweep_graph_destroy", "qv2_check_nonfinite", "qv2_calibrate_ex", "qv2_group_hist_count",
+           "qv2_sync_count", "qv2_set_schedule", "qv2_stage_count"]
 KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
@@ -44,7 +47,7 @@ class RankCfg(C.Structure):
     _fields_ = [("w_gain", C.c_double), ("a_gain", C.c_double), ("mse_factor", C.c_double),
                 ("sqnr_cap_db", C.c_double), ("select_mode", C.c_uint32),
                 ("keep_count", C.c_uint32), ("rate_permyriad", C.c_uint32),
-                ("reserved", C.c_uint32)]
+                ("outlier_order", C.c_uint32)]
 
 
 class SweepBuffers(C.Structure):
@@ -75,6 +78,9 @@ def lib() -> C.CDLL:
     L.qv2_status_string.argtypes = [i32]; L.qv2_status_string.restype = C.c_char_p
     L.qv2_last_cuda_error.argtypes = [vp]; L.qv2_last_cuda_error.restype = i32
     L.qv2_launch_count.argtypes = [vp]; L.qv2_launch_count.restype = u64
+    L.qv2_sync_count.argtypes = [vp]; L.qv2_sync_count.restype = u64
+    L.qv2_set_schedule.argtypes = [vp, u32, u64]; L.qv2_set_schedule.restype = i32
+    L.qv2_stage_count.argtypes = [vp]; L.qv2_stage_count.restype = u32
     L.qv2_group_count.argtypes = [dp, u32]; L.qv2_group_count.restype = u64
     L.qv2_calibrate.argtypes = [vp, dp, u32] + [vp] * 9; L.qv2_calibrate.restype = i32
     L.qv2_calibrate_ex.argtypes = [vp, dp, u32] + [vp] * 11; L.qv2_calibrate_ex.restype = i32
@@ -152,8 +158,9 @@ def desc_array(descs: Sequence[TensorDesc]):
 
 
 def default_rank_cfg(select_mode=BY_COUNT, keep_count=0, rate_permyriad=0, w_gain=2.0, a_gain=1.0,
-                     mse_factor=5.0, sqnr_cap_db=200.0) -> RankCfg:
-    return RankCfg(w_gain, a_gain, mse_factor, sqnr_cap_db, select_mode, keep_count, rate_permyriad, 0)
+                     mse_factor=5.0, sqnr_cap_db=200.0, outlier_order=OUTLIERS_BY_SEVERITY) -> RankCfg:
+    return RankCfg(w_gain, a_gain, mse_factor, sqnr_cap_db, select_mode, keep_count, rate_permyriad,
+                   outlier_order)
 
 
 @dataclass
@@ -209,6 +216,17 @@ class Context:
     @property
     def launches(self) -> int:
         return int(lib().qv2_launch_count(self._h))
+
+    @property
+    def syncs(self) -> int:
+        return int(lib().qv2_sync_count(self._h))
+
+    @property
+    def stages(self) -> int:
+        return int(lib().qv2_stage_count(self._h))
+
+    def set_schedule(self, schedule: int, chunk_bytes: int = 0):
+        _check(lib().qv2_set_schedule(self._h, schedule, chunk_bytes), "qv2_set_schedule")
 
     def last_cuda_error(self) -> int:
         return int(lib().qv2_last_cuda_error(self._h))
@@ -281,10 +299,10 @@ class Context:
             raise Qv2Error(st, "qv2_check_nonfinite")
         return st, (int(bad.value) if st == -5 else None)
 
-    def fold_batchnorm(self, w, bias, gamma, beta, mean, var):
-        """Eq. 10-12: -> (folded weights [C, K], folded bias [C])."""
+    def fold_batchnorm(self, w, bias, gamma, beta, mean, var, inplace: bool = False):
+        """Eq. 10-12: -> (folded weights [C, K], folded bias [C]); inplace overwrites w."""
         c, k = w.shape
-        w_out = torch.empty_like(w)
+        w_out = w if inplace else torch.empty_like(w)
         b_out = self._empty(c, torch.float32)
         _check(lib().qv2_fold_batchnorm(self._h, _ptr(w), _ptr(bias), _ptr(gamma), _ptr(beta), _ptr(mean),
                                         _ptr(var), c, k, _ptr(w_out), _ptr(b_out)), "qv2_fold_batchnorm")

@@ -1,23 +1,40 @@
 // C-ABI layer: context, scratch management, plan caching and the call sequences of the public
 // entry points declared in include/qv2.h.
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
+
+#if defined(__has_include)
+#if __has_include(<nvtx3/nvToolsExt.h>)
+#include <nvtx3/nvToolsExt.h>
+#define QV2_HAVE_NVTX 1
+#endif
+#endif
 
 #include "qv2_common.cuh"
 
 using namespace qv2;
 
+namespace {
+constexpr int kCodeRing = 4;     // pinned staging areas for the per-call table of code pointers
+constexpr uint64_t kDefaultChunkBytes = 48ull << 20;
+}
+
 struct qv2_ctx {
   int device = 0;
   cudaStream_t stream = nullptr;
   int sm_count = 1;
-  uint32_t metrics_cap = 1;   // largest useful grid of the metrics kernel on this device
-  uint32_t range_cap = 1;     // the same for the range kernel
+  GridCaps caps;               // largest useful grid of each persistent kernel on this device
   int last_cuda = 0;
   uint64_t launches = 0;
+  uint64_t syncs = 0;          // host-side stream synchronisations this context has performed
+  uint32_t live_graphs = 0;    // captured passes that hold addresses of this context's scratch
+  bool log = false;            // QV2_LOG=1: one line per call on stderr
+  uint32_t schedule = QV2_SCHEDULE_PHASE_MAJOR;
+  uint64_t chunk_bytes = kDefaultChunkBytes;
 
-  // cached plan: rebuilt only when the descriptor bytes (or code pointers) change
+  // cached plan: rebuilt only when the descriptor bytes or the schedule change
   HostPlan plan;
   std::vector<uint8_t> plan_key;
   bool plan_valid = false;
@@ -34,10 +51,21 @@ struct qv2_ctx {
   double* d_partials_xe = nullptr; size_t cap_slots_xe = 0;   // sum x*e slots, cosine only
   unsigned long long* d_kl_hist = nullptr; size_t cap_kl_hist = 0;   // used when the caller passes no hists
   float* d_tensor_absmax = nullptr; size_t cap_absmax = 0;
-  unsigned long long* d_hist = nullptr; size_t cap_hist = 0;   // used when the caller passes no hist
+  // accumulators that are zero between passes (cleared when a plan is made resident, and by the
+  // CTA that consumes them afterwards)
+  uint32_t* d_keys = nullptr;     size_t cap_keys = 0;         // kmin then kmax, total_groups each
+  unsigned long long* d_nf_acc = nullptr; size_t cap_nf = 0;   // per tensor
+  unsigned long long* d_hist_acc = nullptr; size_t cap_hist_acc = 0;   // 2048 per percentile tensor
+  uint32_t* d_tickets = nullptr;  size_t cap_tickets = 0;      // 3 per tensor: range, histogram, metrics
+  uint8_t** d_codes = nullptr;    size_t cap_codes = 0;        // per-tensor code buffers of the current call
   double* d_rank = nullptr;                                    // 2 * kMaxRankLayers doubles
   // pinned host staging for the plan upload
   uint8_t* h_pinned = nullptr;    size_t cap_pinned = 0;
+  // pinned ring for the code-pointer table: a call fills the next area and copies it on the
+  // stream; the area's event tells when it may be refilled
+  uint8_t** h_codes[kCodeRing] = {}; size_t cap_h_codes = 0;
+  cudaEvent_t code_ev[kCodeRing] = {};
+  uint32_t code_next = 0;
 };
 
 namespace {
@@ -51,8 +79,27 @@ struct DeviceGuard {
   ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
 };
 
+// A named range around each entry point for timeline tools; compiled out without the NVTX headers.
+struct TraceRange {
+#ifdef QV2_HAVE_NVTX
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+#else
+  explicit TraceRange(const char*) {}
+#endif
+};
+
+// QV2_LOG=1: one line per call on stderr (host side only; nothing is read back from the device).
+void log_call(const qv2_ctx* c, const char* call, uint32_t n_tensors, uint64_t launches_before, int status) {
+  if (!c->log) return;
+  std::fprintf(stderr, "qv2: %s tensors=%u tiles=%zu stages=%zu launches=%llu status=%d (%s)\n", call, n_tensors,
+               c->plan_valid ? c->plan.tiles.size() : (size_t)0, c->plan_valid ? c->plan.stages.size() : (size_t)0,
+               (unsigned long long)(c->launches - launches_before), status, qv2_status_string(status));
+}
+
 int cuda_fail(qv2_ctx* c, cudaError_t e) {
   c->last_cuda = (int)e;
+  c->plan_valid = false;          // a pass that stopped half-way may leave accumulators dirty: start over
   return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA;
 }
 
@@ -62,9 +109,12 @@ int cuda_fail(qv2_ctx* c, cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail((c), e__);\
   } while (0)
 
+// graph_held: a captured pass may hold the address of this buffer, so it must not move while one
+// is alive.
 template <class T>
-int grow(qv2_ctx* c, T** p, size_t* cap, size_t need) {
+int grow(qv2_ctx* c, T** p, size_t* cap, size_t need, bool graph_held = true) {
   if (need <= *cap) return QV2_OK;
+  if (graph_held && c->live_graphs) return QV2_ERR_UNSUPPORTED;
   size_t want = need + need / 4 + 16;
   if (*p) { QV2_CUDA(c, cudaFree(*p)); *p = nullptr; *cap = 0; }
   QV2_CUDA(c, cudaMalloc((void**)p, want * sizeof(T)));
@@ -81,42 +131,73 @@ int grow_pinned(qv2_ctx* c, size_t need) {
   return QV2_OK;
 }
 
-int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* const* codes);
+int sync_stream(qv2_ctx* c) {
+  ++c->syncs;
+  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  return QV2_OK;
+}
 
-// Makes ctx->plan describe (descs, codes) and resident on the device.
-int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* const* codes) {
+// Chunk size of the plan about to be built: 0 = phase-major (one stage).  QV2_SCHEDULE_AUTO takes
+// the chunked schedule when most of the reference bytes sit in tensors that fit a chunk and the
+// model is large enough for the extra launches to pay.
+uint64_t plan_chunk_bytes(const qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n) {
+  if (c->schedule == QV2_SCHEDULE_PHASE_MAJOR) return 0;
+  if (c->schedule == QV2_SCHEDULE_L2_CHUNKED) return c->chunk_bytes;
+  uint64_t total = 0, fitting = 0;
+  for (uint32_t t = 0; t < n; ++t) {
+    const uint64_t b = descs[t].outer * descs[t].channels * descs[t].inner *
+                       dtype_size((descs[t].flags & QV2_IN_MASK) >> 16);
+    total += b;
+    if (b <= c->chunk_bytes) fitting += b;
+  }
+  // below ~2 chunks everything is L2-resident across phases anyway; above, chunk when at least
+  // half of the bytes can be reused
+  return (total > 2 * c->chunk_bytes && 2 * fitting >= total) ? c->chunk_bytes : 0;
+}
+
+int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n);
+
+// Makes ctx->plan describe descs and resident on the device.
+int ensure_plan(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n) {
   try {
-    return ensure_plan_checked(c, descs, n, codes);
+    return ensure_plan_checked(c, descs, n);
   } catch (const std::bad_alloc&) {          // host tables did not fit: nothing unwinds through the C ABI
     c->plan_valid = false;
     return QV2_ERR_NOMEM;
   }
 }
 
-int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, void* const* codes) {
+int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n) {
   if (!descs) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   const size_t dbytes = (size_t)n * sizeof(qv2_tensor_desc);
-  const size_t cbytes = codes ? (size_t)n * sizeof(void*) : 0;
-  std::vector<uint8_t> key(dbytes + cbytes + 1);
+  const uint64_t chunk = plan_chunk_bytes(c, descs, n);
+  std::vector<uint8_t> key(dbytes + sizeof(chunk));
   std::memcpy(key.data(), descs, dbytes);
-  if (codes) std::memcpy(key.data() + dbytes, codes, cbytes);
-  key[dbytes + cbytes] = codes ? 1 : 0;
+  std::memcpy(key.data() + dbytes, &chunk, sizeof(chunk));
   if (c->plan_valid && key == c->plan_key) return QV2_OK;
+  // A captured pass replays with the tile tables and scratch addresses of the plan it was
+  // captured with; another descriptor set would overwrite them under it.
+  if (c->live_graphs) return QV2_ERR_UNSUPPORTED;
 
   HostPlan plan;
-  int st = build_plan(descs, n, codes, c->metrics_cap, c->range_cap, &plan);
+  int st = build_plan(descs, n, c->caps, chunk, &plan);
   if (st != QV2_OK) return st;
   // The previous upload may still be reading the pinned buffer, and buffers may be reallocated.
-  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  if ((st = sync_stream(c)) != QV2_OK) return st;
   c->plan_valid = false;
   const size_t nt = plan.tensors.size(), ntl = plan.tiles.size(), nh = plan.hist_tiles.size();
+  const size_t G = (size_t)plan.total_groups, nacc = (size_t)plan.n_hist * kBins;
   if ((st = grow(c, &c->d_tensors, &c->cap_tensors, nt)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_tiles, &c->cap_tiles, ntl ? ntl : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_hist_tiles, &c->cap_hist_tiles, nh ? nh : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_partials, &c->cap_slots, plan.total_slots ? plan.total_slots : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_rslots, &c->cap_rslots, plan.total_rslots ? plan.total_rslots : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_tensor_absmax, &c->cap_absmax, nt)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_keys, &c->cap_keys, 2 * G)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_nf_acc, &c->cap_nf, nt)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_hist_acc, &c->cap_hist_acc, nacc ? nacc : 1)) != QV2_OK) return st;
+  if ((st = grow(c, &c->d_tickets, &c->cap_tickets, 3 * nt)) != QV2_OK) return st;
   const size_t ngt = plan.ghist_tiles.size(), ngo = plan.ghist_owner.size();
   if ((st = grow(c, &c->d_ghist_tiles, &c->cap_ghist_tiles, ngt ? ngt : 1)) != QV2_OK) return st;
   if ((st = grow(c, &c->d_ghist_owner, &c->cap_ghist_owner, ngo ? ngo : 1)) != QV2_OK) return st;
@@ -135,6 +216,11 @@ int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, vo
     QV2_CUDA(c, cudaMemcpyAsync(c->d_ghist_tiles, c->h_pinned + b0 + b1 + b2, b3, cudaMemcpyHostToDevice, c->stream));
     QV2_CUDA(c, cudaMemcpyAsync(c->d_ghist_owner, c->h_pinned + b0 + b1 + b2 + b3, b4, cudaMemcpyHostToDevice, c->stream));
   }
+  // every accumulator starts at zero; from here on the kernels keep them so
+  QV2_CUDA(c, cudaMemsetAsync(c->d_keys, 0, 2 * G * sizeof(uint32_t), c->stream));
+  QV2_CUDA(c, cudaMemsetAsync(c->d_nf_acc, 0, nt * sizeof(unsigned long long), c->stream));
+  if (nacc) QV2_CUDA(c, cudaMemsetAsync(c->d_hist_acc, 0, nacc * sizeof(unsigned long long), c->stream));
+  QV2_CUDA(c, cudaMemsetAsync(c->d_tickets, 0, 3 * nt * sizeof(uint32_t), c->stream));
   c->plan = std::move(plan);
   c->plan_key = std::move(key);
   c->plan_valid = true;
@@ -142,8 +228,105 @@ int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, vo
 }
 
 Launch launch_of(qv2_ctx* c) {
-  Launch l; l.stream = c->stream; l.sm_count = c->sm_count;
+  Launch l; l.stream = c->stream; l.sm_count = c->sm_count; l.pdl = false;
   return l;
+}
+
+CalibArgs calib_args(qv2_ctx* c, float* gmin, float* gmax, float* gabsmax, uint64_t* hist, float* clip,
+                     float* step, float* inv, float* offset, uint64_t* nonfinite) {
+  const size_t nt = c->plan.tensors.size();
+  CalibArgs a;
+  a.tensors = c->d_tensors;
+  a.kmin = c->d_keys; a.kmax = c->d_keys + c->plan.total_groups;
+  a.rslots = c->d_rslots; a.nf_acc = c->d_nf_acc; a.hist_acc = c->d_hist_acc;
+  a.tickets = c->d_tickets; a.hist_tickets = c->d_tickets + nt;
+  a.tensor_absmax = c->d_tensor_absmax;
+  a.gmin = gmin; a.gmax = gmax; a.gabsmax = gabsmax; a.step = step; a.inv = inv; a.offset = offset;
+  a.clip = clip;
+  a.nonfinite = reinterpret_cast<unsigned long long*>(nonfinite);
+  a.hist = reinterpret_cast<unsigned long long*>(hist);
+  return a;
+}
+
+MetricsArgs metrics_args(qv2_ctx* c, const float* step, const float* inv, const float* offset, uint8_t* const* codes,
+                         double* xe, double* sse, double* sig, double* mse, double* sqnr_db, double* cosine) {
+  MetricsArgs a;
+  a.tensors = c->d_tensors; a.step = step; a.inv = inv; a.offset = offset; a.codes = codes;
+  a.partials = c->d_partials; a.partials_xe = xe;
+  a.tickets = c->d_tickets + 2 * c->plan.tensors.size();
+  a.sse = sse; a.sig = sig; a.mse = mse; a.sqnr_db = sqnr_db; a.cosine = cosine;
+  return a;
+}
+
+// Range and histogram phases of one stage.
+int run_calib_stage(qv2_ctx* c, const Stage& st, const CalibArgs& a) {
+  const Launch l = launch_of(c);
+  QV2_CUDA(c, launch_range(l, st, c->plan.any_16bit, c->d_tiles, a));
+  ++c->launches;
+  if (st.any_percentile) {
+    QV2_CUDA(c, launch_hist(l, st, c->plan.any_16bit, c->d_hist_tiles, a));
+    ++c->launches;
+  }
+  return QV2_OK;
+}
+
+int run_metrics_stage(qv2_ctx* c, const Stage& st, const MetricsArgs& a) {
+  QV2_CUDA(c, launch_metrics(launch_of(c), st, c->plan.any_16bit, c->d_tiles, a));
+  ++c->launches;
+  return QV2_OK;
+}
+
+// Per-group percentile clips (a separate, group-major pass; plans that have it are single-stage).
+int run_group_percentile(qv2_ctx* c, uint32_t n, const CalibArgs& a, uint64_t* group_hist, float* group_clip) {
+  const HostPlan& p = c->plan;
+  const size_t n_ghist = p.ghist_owner.size();
+  const Launch l = launch_of(c);
+  int st;
+  if (n_ghist) {
+    unsigned long long* gh = reinterpret_cast<unsigned long long*>(group_hist);
+    if (!gh) {
+      if ((st = grow(c, &c->d_ghist, &c->cap_ghist, n_ghist * kBins)) != QV2_OK) return st;
+      gh = c->d_ghist;
+    }
+    QV2_CUDA(c, cudaMemsetAsync(gh, 0, n_ghist * kBins * sizeof(uint64_t), c->stream));
+    QV2_CUDA(c, launch_group_hist(l, c->caps.ghist, p.any_16bit, c->d_tensors, c->d_ghist_tiles,
+                                  (uint32_t)p.ghist_tiles.size(), a.gabsmax, a.nonfinite, gh));
+    QV2_CUDA(c, launch_group_clip_finalize(l, c->d_tensors, c->d_ghist_owner, (uint32_t)n_ghist, gh, a.gmin, a.gmax,
+                                           a.gabsmax, group_clip, a.step, a.inv, a.offset));
+    c->launches += p.ghist_tiles.empty() ? 1 : 2;
+  }
+  if (group_clip) {
+    QV2_CUDA(c, launch_fill_group_clip(l, c->d_tensors, n, a.clip, group_clip));
+    ++c->launches;
+  }
+  return QV2_OK;
+}
+
+// Makes the device table of code pointers current for this call.  The table is refilled from one
+// of a few pinned areas; an area is reused only once the copy that read it has completed, which
+// in steady state is long past, so the call does not wait.
+int upload_codes(qv2_ctx* c, void* const* codes, const qv2_tensor_desc* descs, uint32_t n) {
+  int st;
+  if ((st = grow(c, &c->d_codes, &c->cap_codes, n, false)) != QV2_OK) return st;
+  if (c->cap_h_codes < n) {
+    if ((st = sync_stream(c)) != QV2_OK) return st;
+    for (int i = 0; i < kCodeRing; ++i) {
+      if (c->h_codes[i]) { QV2_CUDA(c, cudaFreeHost(c->h_codes[i])); c->h_codes[i] = nullptr; }
+      if (!c->code_ev[i]) QV2_CUDA(c, cudaEventCreateWithFlags(&c->code_ev[i], cudaEventDisableTiming));
+    }
+    c->cap_h_codes = 0;
+    const size_t want = (size_t)n + n / 4 + 16;
+    for (int i = 0; i < kCodeRing; ++i) QV2_CUDA(c, cudaMallocHost((void**)&c->h_codes[i], want * sizeof(uint8_t*)));
+    c->cap_h_codes = want;
+  }
+  const uint32_t k = c->code_next++ % kCodeRing;
+  QV2_CUDA(c, cudaEventSynchronize(c->code_ev[k]));      // completed long ago unless calls pile up
+  for (uint32_t t = 0; t < n; ++t)
+    c->h_codes[k][t] = (descs[t].flags & QV2_STORE_CODES) ? (uint8_t*)codes[t] : nullptr;
+  QV2_CUDA(c, cudaMemcpyAsync(c->d_codes, c->h_codes[k], (size_t)n * sizeof(uint8_t*), cudaMemcpyHostToDevice,
+                              c->stream));
+  QV2_CUDA(c, cudaEventRecord(c->code_ev[k], c->stream));
+  return QV2_OK;
 }
 
 }  // namespace
@@ -178,8 +361,14 @@ extern "C" int qv2_create(qv2_ctx** out, int device, void* stream) {
   if (e == cudaSuccess) e = cudaMalloc((void**)&c->d_rank, kRankScratchDoubles * sizeof(double));
   if (e != cudaSuccess) { delete c; return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA; }
   c->sm_count = sms > 0 ? sms : 1;
-  c->metrics_cap = metrics_grid_cap(c->sm_count);
-  c->range_cap = range_grid_cap(c->sm_count);
+  // occupancy of each persistent kernel on THIS device (two contexts on different GPUs differ)
+  c->caps.range = range_grid_cap(c->sm_count);
+  c->caps.hist = hist_grid_cap(c->sm_count);
+  c->caps.metrics = metrics_grid_cap(c->sm_count);
+  c->caps.ghist = group_hist_grid_cap(c->sm_count);
+  c->caps.kl = kl_grid_cap(c->sm_count);
+  const char* lg = std::getenv("QV2_LOG");
+  c->log = lg && lg[0] == '1';
   *out = c;
   return QV2_OK;
 }
@@ -188,15 +377,74 @@ extern "C" int qv2_destroy(qv2_ctx* c) {
   if (!c) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
   cudaStreamSynchronize(c->stream);
-  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_ghist_tiles); cudaFree(c->d_ghist_owner); cudaFree(c->d_ghist); cudaFree(c->d_partials); cudaFree(c->d_rslots); cudaFree(c->d_partials_xe); cudaFree(c->d_kl_hist);
-  cudaFree(c->d_tensor_absmax); cudaFree(c->d_hist); cudaFree(c->d_rank);
+  cudaFree(c->d_tensors); cudaFree(c->d_tiles); cudaFree(c->d_hist_tiles); cudaFree(c->d_ghist_tiles);
+  cudaFree(c->d_ghist_owner); cudaFree(c->d_ghist); cudaFree(c->d_partials); cudaFree(c->d_rslots);
+  cudaFree(c->d_partials_xe); cudaFree(c->d_kl_hist); cudaFree(c->d_tensor_absmax); cudaFree(c->d_keys);
+  cudaFree(c->d_nf_acc); cudaFree(c->d_hist_acc); cudaFree(c->d_tickets); cudaFree(c->d_codes);
+  cudaFree(c->d_rank);
   if (c->h_pinned) cudaFreeHost(c->h_pinned);
+  for (int i = 0; i < kCodeRing; ++i) {
+    if (c->h_codes[i]) cudaFreeHost(c->h_codes[i]);
+    if (c->code_ev[i]) cudaEventDestroy(c->code_ev[i]);
+  }
   delete c;
   return QV2_OK;
 }
 
 extern "C" int qv2_last_cuda_error(const qv2_ctx* c) { return c ? c->last_cuda : 0; }
 extern "C" uint64_t qv2_launch_count(const qv2_ctx* c) { return c ? c->launches : 0; }
+extern "C" uint64_t qv2_sync_count(const qv2_ctx* c) { return c ? c->syncs : 0; }
+
+extern "C" int qv2_set_schedule(qv2_ctx* c, uint32_t schedule, uint64_t chunk_bytes) {
+  if (!c) return QV2_ERR_NULL;
+  if (schedule > QV2_SCHEDULE_AUTO) return QV2_ERR_ARG;
+  if (c->live_graphs) return QV2_ERR_UNSUPPORTED;     // a captured pass replays the schedule it was captured with
+  c->schedule = schedule;
+  c->chunk_bytes = chunk_bytes ? chunk_bytes : kDefaultChunkBytes;
+  return QV2_OK;
+}
+
+extern "C" uint32_t qv2_stage_count(const qv2_ctx* c) {
+  return (c && c->plan_valid) ? (uint32_t)c->plan.stages.size() : 0u;
+}
+
+namespace {
+
+int calibrate_impl(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* gmin, float* gmax,
+                   float* gabsmax, uint64_t* hist, float* clip, float* step, float* inv, float* offset,
+                   uint64_t* nonfinite, uint64_t* group_hist, float* group_clip) {
+  int st = ensure_plan(c, descs, n);
+  if (st != QV2_OK) return st;
+  const CalibArgs a = calib_args(c, gmin, gmax, gabsmax, hist, clip, step, inv, offset, nonfinite);
+  for (const Stage& sg : c->plan.stages)
+    if ((st = run_calib_stage(c, sg, a)) != QV2_OK) return st;
+  return run_group_percentile(c, n, a, group_hist, group_clip);
+}
+
+int metrics_impl(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, const float* step, const float* inv,
+                 const float* offset, void* const* codes, double* sse, double* sig, double* mse,
+                 double* sqnr_db, double* cosine) {
+  bool any_codes = false;
+  if (codes)
+    for (uint32_t t = 0; t < n && n <= 65535u; ++t)
+      if ((descs[t].flags & QV2_STORE_CODES) && codes[t]) any_codes = true;
+  int st = ensure_plan(c, descs, n);
+  if (st != QV2_OK) return st;
+  if (any_codes && (st = upload_codes(c, codes, descs, n)) != QV2_OK) return st;
+  double* xe = nullptr;
+  if (cosine) {                        // third slot array, only when the cosine is wanted
+    const size_t need = c->plan.total_slots ? c->plan.total_slots : 1;
+    if ((st = grow(c, &c->d_partials_xe, &c->cap_slots_xe, need, false)) != QV2_OK) return st;
+    xe = c->d_partials_xe;
+  }
+  const MetricsArgs a = metrics_args(c, step, inv, offset, any_codes ? c->d_codes : nullptr, xe, sse, sig, mse,
+                                     sqnr_db, cosine);
+  for (const Stage& sg : c->plan.stages)
+    if ((st = run_metrics_stage(c, sg, a)) != QV2_OK) return st;
+  return QV2_OK;
+}
+
+}  // namespace
 
 extern "C" int qv2_calibrate_ex(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* gmin,
                                 float* gmax, float* gabsmax, uint64_t* hist, float* clip, float* step,
@@ -205,57 +453,12 @@ extern "C" int qv2_calibrate_ex(qv2_ctx* c, const qv2_tensor_desc* descs, uint32
   if (!c || !descs || !gmin || !gmax || !gabsmax || !clip || !step || !inv || !offset || !nonfinite)
     return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
-  int st = ensure_plan(c, descs, n, nullptr);
-  if (st != QV2_OK) return st;
-  const HostPlan& p = c->plan;
-  unsigned long long* h = reinterpret_cast<unsigned long long*>(hist);
-  if (!h && p.any_percentile) {
-    if ((st = grow(c, &c->d_hist, &c->cap_hist, (size_t)n * kBins)) != QV2_OK) return st;
-    h = c->d_hist;
-  }
-  const size_t n_ghist = p.ghist_owner.size();
-  unsigned long long* gh = reinterpret_cast<unsigned long long*>(group_hist);
-  if (!gh && n_ghist) {
-    if ((st = grow(c, &c->d_ghist, &c->cap_ghist, n_ghist * kBins)) != QV2_OK) return st;
-    gh = c->d_ghist;
-  }
-  const Launch l = launch_of(c);
-  const size_t G = (size_t)p.total_groups;
-  QV2_CUDA(c, launch_calib_init(l, reinterpret_cast<uint32_t*>(gmin), reinterpret_cast<uint32_t*>(gmax), G,
-                                reinterpret_cast<unsigned long long*>(nonfinite), n, h, h ? (size_t)n * kBins : 0));
-  ++c->launches;
-  if (n_ghist) QV2_CUDA(c, cudaMemsetAsync(gh, 0, n_ghist * kBins * sizeof(uint64_t), c->stream));
-  if (!p.tiles.empty()) {
-    QV2_CUDA(c, launch_range(l, p.range_grid, p.any_16bit, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(),
-                             reinterpret_cast<uint32_t*>(gmin), reinterpret_cast<uint32_t*>(gmax),
-                             c->d_rslots, reinterpret_cast<unsigned long long*>(nonfinite)));
-    ++c->launches;
-  }
-  QV2_CUDA(c, launch_range_finalize(l, c->d_tensors, n, c->d_rslots, gmin, gmax, gabsmax, step, inv, offset,
-                                    c->d_tensor_absmax, clip));
-  ++c->launches;
-  if (!p.hist_tiles.empty()) {
-    QV2_CUDA(c, launch_hist(l, p.any_16bit, c->d_tensors, c->d_hist_tiles, (uint32_t)p.hist_tiles.size(),
-                            c->d_tensor_absmax, reinterpret_cast<unsigned long long*>(nonfinite), h));
-    ++c->launches;
-  }
-  if (p.any_percentile) {              // clip[t] of the other tensors is already the absmax
-    QV2_CUDA(c, launch_clip_finalize(l, c->d_tensors, n, h, c->d_tensor_absmax, gmin, gmax, gabsmax,
-                                     clip, step, inv, offset));
-    ++c->launches;
-  }
-  if (n_ghist) {
-    QV2_CUDA(c, launch_group_hist(l, p.any_16bit, c->d_tensors, c->d_ghist_tiles, (uint32_t)p.ghist_tiles.size(),
-                                  gabsmax, reinterpret_cast<unsigned long long*>(nonfinite), gh));
-    QV2_CUDA(c, launch_group_clip_finalize(l, c->d_tensors, c->d_ghist_owner, (uint32_t)n_ghist, gh, gmin, gmax,
-                                           gabsmax, group_clip, step, inv, offset));
-    c->launches += p.ghist_tiles.empty() ? 1 : 2;
-  }
-  if (group_clip) {
-    QV2_CUDA(c, launch_fill_group_clip(l, c->d_tensors, n, clip, group_clip));
-    ++c->launches;
-  }
-  return QV2_OK;
+  TraceRange trace("qv2_calibrate");
+  const uint64_t before = c->launches;
+  const int st = calibrate_impl(c, descs, n, gmin, gmax, gabsmax, hist, clip, step, inv, offset, nonfinite,
+                                group_hist, group_clip);
+  log_call(c, "qv2_calibrate", n, before, st);
+  return st;
 }
 
 extern "C" int qv2_calibrate(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* gmin,
@@ -271,28 +474,11 @@ extern "C" int qv2_quant_metrics_ex(qv2_ctx* c, const qv2_tensor_desc* descs, ui
                                     double* sqnr_db, double* cosine) {
   if (!c || !descs || !step || !inv || !offset || !sse || !sig || !mse || !sqnr_db) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
-  bool any_codes = false;
-  if (codes)
-    for (uint32_t t = 0; t < n && n <= 65535u; ++t)
-      if ((descs[t].flags & QV2_STORE_CODES) && codes[t]) any_codes = true;
-  int st = ensure_plan(c, descs, n, any_codes ? codes : nullptr);
-  if (st != QV2_OK) return st;
-  const HostPlan& p = c->plan;
-  double* xe = nullptr;
-  if (cosine) {                        // third slot array, only when the cosine is wanted
-    if ((st = grow(c, &c->d_partials_xe, &c->cap_slots_xe, p.total_slots ? p.total_slots : 1)) != QV2_OK)
-      return st;
-    xe = c->d_partials_xe;
-  }
-  const Launch l = launch_of(c);
-  if (!p.tiles.empty()) {
-    QV2_CUDA(c, launch_metrics(l, p.metrics_grid, p.any_16bit, c->d_tensors, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
-                               offset, c->d_partials, xe));
-    ++c->launches;
-  }
-  QV2_CUDA(c, launch_metrics_finalize(l, c->d_tensors, n, c->d_partials, xe, sse, sig, mse, sqnr_db, cosine));
-  ++c->launches;
-  return QV2_OK;
+  TraceRange trace("qv2_quant_metrics");
+  const uint64_t before = c->launches;
+  const int st = metrics_impl(c, descs, n, step, inv, offset, codes, sse, sig, mse, sqnr_db, cosine);
+  log_call(c, "qv2_quant_metrics", n, before, st);
+  return st;
 }
 
 extern "C" int qv2_quant_metrics(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n,
@@ -307,17 +493,18 @@ extern "C" int qv2_kl_divergence(qv2_ctx* c, const qv2_tensor_desc* descs, uint3
                                  uint64_t* hists) {
   if (!c || !descs || !step || !inv || !offset || !gabsmax || !kl) return QV2_ERR_NULL;
   DeviceGuard guard(c->device);
-  int st = ensure_plan(c, descs, n, nullptr);
+  TraceRange trace("qv2_kl_divergence");
+  int st = ensure_plan(c, descs, n);
   if (st != QV2_OK) return st;
   const HostPlan& p = c->plan;
   unsigned long long* h = reinterpret_cast<unsigned long long*>(hists);
   const size_t cells = (size_t)n * 2 * QV2_KL_BINS;
   if (!h) {
-    if ((st = grow(c, &c->d_kl_hist, &c->cap_kl_hist, cells)) != QV2_OK) return st;
+    if ((st = grow(c, &c->d_kl_hist, &c->cap_kl_hist, cells, false)) != QV2_OK) return st;
     h = c->d_kl_hist;
   }
   QV2_CUDA(c, cudaMemsetAsync(h, 0, cells * sizeof(unsigned long long), c->stream));
-  QV2_CUDA(c, launch_kl(launch_of(c), c->d_tensors, n, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
+  QV2_CUDA(c, launch_kl(launch_of(c), c->caps.kl, c->d_tensors, n, c->d_tiles, (uint32_t)p.tiles.size(), step, inv,
                         offset, gabsmax, c->d_tensor_absmax, h, kl));
   c->launches += p.tiles.empty() ? 2 : 3;
   return QV2_OK;
@@ -330,7 +517,7 @@ extern "C" int qv2_check_nonfinite(qv2_ctx* c, const uint64_t* nonfinite, uint32
   std::vector<uint64_t> host(n);
   QV2_CUDA(c, cudaMemcpyAsync(host.data(), nonfinite, (size_t)n * sizeof(uint64_t), cudaMemcpyDeviceToHost,
                               c->stream));
-  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (int st = sync_stream(c)) return st;
   for (uint32_t t = 0; t < n; ++t)
     if (host[t]) { if (first_bad) *first_bad = t; return QV2_ERR_NONFINITE; }
   return QV2_OK;
@@ -343,6 +530,10 @@ extern "C" int qv2_fold_batchnorm(qv2_ctx* c, const float* w, const float* bias,
   if (channels && inner && (!w || !w_out)) return QV2_ERR_NULL;
   if (channels != 0 && inner > (1ull << 62) / channels) return QV2_ERR_SIZE;
   if ((((uintptr_t)w) | ((uintptr_t)w_out)) & 3u) return QV2_ERR_ALIGN;
+  if (w != w_out && channels && inner) {        // in place is fine, a partial overlap is not
+    const uintptr_t a0 = (uintptr_t)w, b0 = (uintptr_t)w_out, len = (uintptr_t)(channels * inner * sizeof(float));
+    if (a0 < b0 + len && b0 < a0 + len) return QV2_ERR_ARG;
+  }
   DeviceGuard guard(c->device);
   QV2_CUDA(c, launch_fold(launch_of(c), w, bias, gamma, beta, mean, var, channels, inner, w_out, bias_out));
   c->launches += (channels && inner ? (channels + 65534) / 65535 : 0) + (bias_out && channels ? 1 : 0);
@@ -359,10 +550,13 @@ extern "C" int qv2_rank_layers_ex(qv2_ctx* c, uint32_t n_layers, const double* s
   if (n_layers == 0 || n_layers > kMaxRankLayers) return QV2_ERR_SIZE;
   if (cfg->select_mode > QV2_BY_BOPS_RATE) return QV2_ERR_ARG;
   if (cfg->select_mode == QV2_BY_BOPS_RATE && cfg->rate_permyriad > 10000u) return QV2_ERR_ARG;
+  if (cfg->outlier_order > QV2_OUTLIERS_LITERAL) return QV2_ERR_ARG;
   DeviceGuard guard(c->device);
+  TraceRange trace("qv2_rank_layers");
   QV2_CUDA(c, launch_rank(launch_of(c), n_layers, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, fuse_group,
                           *cfg, c->d_rank, order, keep_fp32, n_keep));
   ++c->launches;
+  if (c->log) std::fprintf(stderr, "qv2: qv2_rank_layers layers=%u launches=1 status=0 (QV2_OK)\n", n_layers);
   return QV2_OK;
 }
 
@@ -382,14 +576,36 @@ extern "C" int qv2_sweep_model(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_
   if ((uint64_t)n_tensors < 2ull * n_layers) return QV2_ERR_ARG;
   if (!b->order || !b->keep_fp32 || !b->n_keep || !b->sse || !b->sig || !b->mse || !b->sqnr_db)
     return QV2_ERR_NULL;
+  if (!b->gmin || !b->gmax || !b->gabsmax || !b->clip || !b->step || !b->inv || !b->offset || !b->nonfinite)
+    return QV2_ERR_NULL;
   if (cfg->select_mode > QV2_BY_BOPS_RATE) return QV2_ERR_ARG;
   if (cfg->select_mode == QV2_BY_BOPS_RATE && cfg->rate_permyriad > 10000u) return QV2_ERR_ARG;
-  int st = qv2_calibrate(c, descs, n_tensors, b->gmin, b->gmax, b->gabsmax, b->hist, b->clip, b->step,
-                         b->inv, b->offset, b->nonfinite);
+  DeviceGuard guard(c->device);
+  int st = ensure_plan(c, descs, n_tensors);
   if (st != QV2_OK) return st;
-  st = qv2_quant_metrics(c, descs, n_tensors, b->step, b->inv, b->offset, nullptr, b->sse, b->sig,
-                         b->mse, b->sqnr_db);
-  if (st != QV2_OK) return st;
+  if (c->plan.stages.size() <= 1) {          // phase-major: the three calls of the contract, chained
+    st = qv2_calibrate(c, descs, n_tensors, b->gmin, b->gmax, b->gabsmax, b->hist, b->clip, b->step,
+                       b->inv, b->offset, b->nonfinite);
+    if (st != QV2_OK) return st;
+    st = qv2_quant_metrics(c, descs, n_tensors, b->step, b->inv, b->offset, nullptr, b->sse, b->sig,
+                           b->mse, b->sqnr_db);
+    if (st != QV2_OK) return st;
+  } else {
+    // L2-chunked: range -> histogram -> metrics stage by stage, so that the second and third read
+    // of a stage's reference tensors hit L2
+    TraceRange trace("qv2_sweep_model (L2-chunked)");
+    const uint64_t before = c->launches;
+    const CalibArgs ca = calib_args(c, b->gmin, b->gmax, b->gabsmax, b->hist, b->clip, b->step, b->inv,
+                                    b->offset, b->nonfinite);
+    const MetricsArgs ma = metrics_args(c, b->step, b->inv, b->offset, nullptr, nullptr, b->sse, b->sig,
+                                        b->mse, b->sqnr_db, nullptr);
+    for (const Stage& sg : c->plan.stages) {
+      if ((st = run_calib_stage(c, sg, ca)) != QV2_OK) break;
+      if ((st = run_metrics_stage(c, sg, ma)) != QV2_OK) break;
+    }
+    log_call(c, "qv2_sweep_model (L2-chunked calibrate+metrics)", n_tensors, before, st);
+    if (st != QV2_OK) return st;
+  }
   return qv2_rank_layers(c, n_layers, b->sqnr_db, b->mse, b->sqnr_db + n_layers, b->mse + n_layers,
                          macs, pos, cfg, b->order, b->keep_fp32, b->n_keep);
 }
@@ -460,7 +676,7 @@ extern "C" int qv2_sweep_model_host(qv2_ctx* c, const qv2_tensor_desc* descs, ui
   QV2_CUDA(c, cudaMemcpyAsync(out->order, b->order, (size_t)n_layers * sizeof(uint32_t), d2h, c->stream));
   QV2_CUDA(c, cudaMemcpyAsync(out->keep_fp32, b->keep_fp32, (size_t)n_layers, d2h, c->stream));
   QV2_CUDA(c, cudaMemcpyAsync(out->n_keep, b->n_keep, sizeof(uint32_t), d2h, c->stream));
-  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (int sst = sync_stream(c)) return sst;
   for (uint32_t t = 0; t < n_tensors; ++t)
     if (out->nonfinite[t]) return QV2_ERR_NONFINITE;
   return QV2_OK;
@@ -490,7 +706,7 @@ extern "C" int qv2_sweep_graph_create(qv2_ctx* c, const qv2_tensor_desc* descs, 
   int st = qv2_sweep_model(c, descs, n_tensors, n_layers, macs, pos, cfg, bufs);
   if (st != QV2_OK) return st;
   const uint64_t per_pass = c->launches - before;
-  QV2_CUDA(c, cudaStreamSynchronize(c->stream));
+  if ((st = sync_stream(c)) != QV2_OK) return st;
   qv2_graph* g = new (std::nothrow) qv2_graph();
   if (!g) return QV2_ERR_NOMEM;
   g->ctx = c; g->launches_per_replay = per_pass;
@@ -506,6 +722,7 @@ extern "C" int qv2_sweep_graph_create(qv2_ctx* c, const qv2_tensor_desc* descs, 
   }
   e = cudaGraphInstantiate(&g->exec, g->graph, 0);
   if (e != cudaSuccess) { cudaGraphDestroy(g->graph); delete g; return cuda_fail(c, e); }
+  ++c->live_graphs;                 // from now on the plan and its scratch stay where they are
   *out = g;
   return QV2_OK;
 }
@@ -520,7 +737,11 @@ extern "C" int qv2_sweep_graph_launch(qv2_graph* g) {
 
 extern "C" int qv2_sweep_graph_destroy(qv2_graph* g) {
   if (!g) return QV2_ERR_NULL;
-  if (g->ctx) { DeviceGuard guard(g->ctx->device); cudaStreamSynchronize(g->ctx->stream); }
+  if (g->ctx) {
+    DeviceGuard guard(g->ctx->device);
+    cudaStreamSynchronize(g->ctx->stream);
+    if (g->ctx->live_graphs) --g->ctx->live_graphs;
+  }
   if (g->exec) cudaGraphExecDestroy(g->exec);
   if (g->graph) cudaGraphDestroy(g->graph);
   delete g;

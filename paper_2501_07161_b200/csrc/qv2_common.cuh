@@ -26,10 +26,17 @@ enum DType : uint32_t { kF32 = 0, kF16 = 1, kBF16 = 2 };
 inline uint32_t dtype_size(uint32_t dtype) { return dtype == kF32 ? 4u : 2u; }
 
 // One tensor, as the kernels see it.
+//
+// A pass is cut into stages (see HostPlan); each phase of a stage is one launch that walks the
+// stage's slice of the tile table.  `tile_first` / `hist_tile_first` are relative to that slice,
+// and the *_ctas fields count the CTAs of that launch that own at least one tile of the tensor:
+// CTA b of a grid of g walks tiles b, b+g, ..., so a tensor whose tiles are [first, first+count)
+// is touched by min(g, count) CTAs, numbered rank = (b - first) mod g.  The CTA that is last to
+// finish its share of a tensor (an atomic ticket, never a wait) folds the tensor's partial
+// results; the slot fields say where those partial results live.
 struct TensorRec {
   const float* x;
   const float* y;
-  uint8_t* codes;            // nullable
   uint64_t n_elems;
   uint64_t inner;
   uint32_t channels;
@@ -39,14 +46,18 @@ struct TensorRec {
   uint32_t asym;             // 0: symmetric, 1: affine with real offset, 2: affine with integer zero point
   uint32_t range_mode;       // QV2_ABSMAX | QV2_MINMAX | QV2_PERCENTILE | QV2_PERCENTILE_GROUP (per-channel only)
   uint32_t pair_mode;        // PairMode
-  uint32_t slot_first;       // first partial-sum slot of this tensor
-  uint32_t slot_count;       // kWarps slots for every CTA of the metrics grid that owns a tile of it
-  uint32_t tile_first;       // index of this tensor's first tile in the tile table
-  uint32_t rslot_first;      // per-tensor tensors: first {min,max} key slot written by the range kernel,
-  uint32_t rslot_count;      //   one per CTA of the range grid that owns a tile of the tensor
+  uint32_t tile_first;       // index of this tensor's first tile in its stage's slice of the tile table
+  uint32_t hist_tile_first;  // the same in the slice of the histogram tile table (percentile tensors)
+  uint32_t slot_first;       // first partial-sum slot of this tensor, one per CTA of the metrics launch
+  uint32_t metrics_ctas;     //   that owns a tile of it
+  uint32_t rslot_first;      // per-tensor tensors: first {min,max} key slot written by the range kernel
+  uint32_t range_ctas;       // CTAs of the range launch that own a tile of the tensor
+  uint32_t hist_ctas;        // CTAs of the histogram launch that own a tile of the tensor
+  uint32_t hist_index;       // percentile tensors: index of the tensor's accumulation histogram in scratch
   uint32_t bits;             // code width, 2..16 (8 unless the descriptor asks otherwise)
   uint32_t dtype;            // element type of x and y: 0 binary32, 1 binary16, 2 bfloat16
   uint32_t ghist_first;      // QV2_PERCENTILE_GROUP: index of group 0's histogram among the per-group histograms
+  uint32_t reserved[2];
   double percentile;
 };
 
@@ -64,26 +75,46 @@ struct Tile {
 };
 static_assert(sizeof(Tile) == 32, "Tile is read as two 16-byte words");
 
+// A run of consecutive tensors whose phases are launched together.  The phase-major schedule has
+// one stage (every tensor); the L2-chunked schedule cuts the model into stages whose reference
+// tensors fit in L2 together, and runs range -> histogram -> metrics stage by stage, so that the
+// second and third pass over a tensor are served from L2.
+struct Stage {
+  uint32_t tensor_begin, tensor_end;
+  uint32_t tile_begin, tile_end;          // slice of HostPlan::tiles
+  uint32_t hist_begin, hist_end;          // slice of HostPlan::hist_tiles
+  uint32_t range_grid, hist_grid, metrics_grid;
+  bool any_empty;                         // some tensor of the stage has no element (no CTA owns it)
+  bool any_percentile;                    // some tensor of the stage is clipped at its percentile
+  bool l2_resident;                       // the stage's reference tensors fit the chunk budget
+};
+
+// Largest useful grid of each persistent kernel on the context's device (resident CTAs per SM x SMs).
+struct GridCaps {
+  uint32_t range = 1, hist = 1, metrics = 1, ghist = 1, kl = 1;
+};
+
 struct HostPlan {
   std::vector<TensorRec> tensors;
   std::vector<Tile> tiles;        // every tensor, in tensor order
   std::vector<Tile> hist_tiles;   // flat tiles of the tensors that need a histogram
   std::vector<Tile> ghist_tiles;  // group-major units of the tensors that need per-group histograms (see build_plan)
   std::vector<uint32_t> ghist_owner;   // per-group histogram -> tensor index
+  std::vector<Stage> stages;
   uint64_t total_groups = 0;
   uint32_t total_slots = 0;
-  uint32_t metrics_grid = 1;      // CTAs of the metrics launch; the slot layout depends on it
   uint32_t total_rslots = 0;
-  uint32_t range_grid = 1;        // CTAs of the range launch; the range-slot layout depends on it
+  uint32_t n_hist = 0;            // tensors clipped at a per-tensor percentile (accumulation histograms in scratch)
   bool any_percentile = false;
   bool any_16bit = false;         // some tensor is stored in binary16 / bfloat16
 };
 
-// Validates the descriptors and cuts them into tiles.  `codes` may be NULL.  `metrics_cap` and
-// `range_cap` are the largest useful grids of those kernels (resident CTAs per SM x SMs).
+// Validates the descriptors and cuts them into tiles and stages.  chunk_bytes == 0 gives the
+// phase-major schedule (one stage); otherwise consecutive tensors are grouped into stages whose
+// reference tensors hold at most chunk_bytes (a larger tensor gets a stage of its own kind).
 // Returns a QV2 status.
-int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
-               uint32_t range_cap, HostPlan* out);
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, const GridCaps& caps, uint64_t chunk_bytes,
+               HostPlan* out);
 
 // ------------------------------------------------------------------------------------------------
 // Launch wrappers (defined next to their kernels).  All enqueue on `stream` and return the
@@ -91,44 +122,59 @@ int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uin
 struct Launch {
   cudaStream_t stream;
   int sm_count;
+  bool pdl;            // launch as a programmatic dependent of the previous kernel in the stream
 };
 
-cudaError_t launch_range(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors, const Tile* tiles,
-                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax, uint2* rslots,
-                         unsigned long long* nonfinite);
-cudaError_t launch_calib_init(const Launch& l, uint32_t* kmin, uint32_t* kmax, size_t groups,
-                              unsigned long long* nonfinite, size_t n_tensors, unsigned long long* hist,
-                              size_t hist_cells);
-uint32_t range_grid_cap(int sm_count);     // resident CTAs per SM x SMs for the range kernel
-cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                  const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
-                                  float* step, float* inv, float* offset, float* tensor_absmax, float* clip);
-cudaError_t launch_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
-                        uint32_t n_tiles, const float* tensor_absmax,
-                        const unsigned long long* nonfinite, unsigned long long* hist);
-cudaError_t launch_clip_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                 const unsigned long long* hist, const float* tensor_absmax,
-                                 const float* gmin, const float* gmax, const float* gabsmax,
-                                 float* clip, float* step, float* inv, float* offset);
-cudaError_t launch_group_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
-                              uint32_t n_tiles, const float* gabsmax, const unsigned long long* nonfinite,
-                              unsigned long long* ghist);
+// Scratch and outputs of the calibration phases.  Accumulators (keys, counters, histograms,
+// tickets) are zero between passes: the CTA that folds a tensor clears what it consumed.
+struct CalibArgs {
+  const TensorRec* tensors;
+  uint32_t* kmin; uint32_t* kmax;            // scratch: order-preserving keys per group, 0 = nothing seen
+  uint2* rslots;                             // scratch: {min,max} key pair per CTA of a per-tensor tensor
+  unsigned long long* nf_acc;                // scratch: non-finite counter per tensor
+  unsigned long long* hist_acc;              // scratch: 2048 bins per percentile tensor
+  uint32_t* tickets;                         // scratch: one per tensor, range phase
+  uint32_t* hist_tickets;                    // scratch: one per tensor, histogram phase
+  float* tensor_absmax;                      // scratch: per tensor
+  float *gmin, *gmax, *gabsmax, *step, *inv, *offset;   // outputs, per group
+  float* clip;                               // output, per tensor
+  unsigned long long* nonfinite;             // output, per tensor
+  unsigned long long* hist;                  // output, 2048 per tensor, nullable
+};
+
+cudaError_t launch_range(const Launch& l, const Stage& st, bool any16, const Tile* tiles, const CalibArgs& a);
+cudaError_t launch_hist(const Launch& l, const Stage& st, bool any16, const Tile* hist_tiles, const CalibArgs& a);
+uint32_t range_grid_cap(int sm_count);     // resident CTAs per SM x SMs
+uint32_t hist_grid_cap(int sm_count);
+uint32_t group_hist_grid_cap(int sm_count);
+uint32_t metrics_grid_cap(int sm_count);
+uint32_t kl_grid_cap(int sm_count);
+
+cudaError_t launch_group_hist(const Launch& l, uint32_t grid_cap, bool any16, const TensorRec* tensors,
+                              const Tile* tiles, uint32_t n_tiles, const float* gabsmax,
+                              const unsigned long long* nonfinite, unsigned long long* ghist);
 cudaError_t launch_group_clip_finalize(const Launch& l, const TensorRec* tensors, const uint32_t* owner,
                                        uint32_t n_hists, const unsigned long long* ghist,
                                        const float* gmin, const float* gmax, const float* gabsmax,
                                        float* group_clip, float* step, float* inv, float* offset);
 cudaError_t launch_fill_group_clip(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
                                    const float* clip, float* group_clip);
-cudaError_t launch_metrics(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors,
-                           const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
-                           const float* offset, double2* partials, double* partials_xe);
-uint32_t metrics_grid_cap(int sm_count);   // resident CTAs per SM x SMs for the metrics kernel
-cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                    const double2* partials, const double* partials_xe, double* sse,
-                                    double* sig, double* mse, double* sqnr_db, double* cosine);
-cudaError_t launch_kl(const Launch& l, const TensorRec* tensors, uint32_t n_tensors, const Tile* tiles,
-                      uint32_t n_tiles, const float* step, const float* inv, const float* offset,
-                      const float* gabsmax, float* tensor_absmax, unsigned long long* hists, double* kl);
+
+struct MetricsArgs {
+  const TensorRec* tensors;
+  const float *step, *inv, *offset;          // per group
+  uint8_t* const* codes;                     // device table of per-tensor code buffers, nullable
+  double2* partials;                         // scratch: {sum e^2, sum x^2} per CTA and tensor
+  double* partials_xe;                       // scratch: sum x*e, cosine only (nullable)
+  uint32_t* tickets;                         // scratch: one per tensor, metrics phase
+  double *sse, *sig, *mse, *sqnr_db, *cosine;   // outputs per tensor (cosine nullable)
+};
+cudaError_t launch_metrics(const Launch& l, const Stage& st, bool any16, const Tile* tiles, const MetricsArgs& a);
+
+cudaError_t launch_kl(const Launch& l, uint32_t grid_cap, const TensorRec* tensors, uint32_t n_tensors,
+                      const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
+                      const float* offset, const float* gabsmax, float* tensor_absmax,
+                      unsigned long long* hists, double* kl);
 cudaError_t launch_fold(const Launch& l, const float* w, const float* bias, const float* gamma,
                         const float* beta, const float* mean, const float* var, uint64_t channels,
                         uint64_t inner, float* w_out, float* bias_out);

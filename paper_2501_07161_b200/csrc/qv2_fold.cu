@@ -14,10 +14,13 @@ __device__ __forceinline__ float fold_scale(float gamma, float var) {
 }
 
 // grid.y = channel, grid.x * blockDim.x covers the row; VEC selects 128-bit accesses.
-template <bool VEC>
+// INPLACE: w_out is w itself.  Every element is then read and written by the same thread, which
+// is safe, but the read-only (non-coherent) load path and the no-alias promise are not: the
+// in-place build uses plain loads and unqualified pointers.
+template <bool VEC, bool INPLACE>
 __global__ void __launch_bounds__(256)
-fold_kernel(const float* __restrict__ w, const float* __restrict__ gamma, const float* __restrict__ var,
-            uint64_t inner, float* __restrict__ w_out) {
+fold_kernel(const float* w, const float* __restrict__ gamma, const float* __restrict__ var,
+            uint64_t inner, float* w_out) {
   const uint64_t c = blockIdx.y;
   const float s = fold_scale(__ldg(gamma + c), __ldg(var + c));
   const float* row = w + c * inner;
@@ -25,13 +28,13 @@ fold_kernel(const float* __restrict__ w, const float* __restrict__ gamma, const 
   if (VEC) {
     const uint64_t nvec = inner >> 2;
     for (uint64_t j = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; j < nvec; j += (uint64_t)gridDim.x * blockDim.x) {
-      float4 v = ld_stream4(reinterpret_cast<const float4*>(row) + j);
+      float4 v = INPLACE ? reinterpret_cast<const float4*>(row)[j] : ld_stream4(reinterpret_cast<const float4*>(row) + j);
       v.x = __fmul_rn(s, v.x); v.y = __fmul_rn(s, v.y); v.z = __fmul_rn(s, v.z); v.w = __fmul_rn(s, v.w);
       reinterpret_cast<float4*>(out)[j] = v;
     }
   } else {
     for (uint64_t j = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; j < inner; j += (uint64_t)gridDim.x * blockDim.x)
-      out[j] = __fmul_rn(s, ld_stream1(row + j));
+      out[j] = __fmul_rn(s, INPLACE ? row[j] : ld_stream1(row + j));
   }
 }
 
@@ -60,8 +63,13 @@ cudaError_t launch_fold(const Launch& l, const float* w, const float* bias, cons
       const uint64_t nc = channels - c0 < 65535 ? channels - c0 : 65535;
       dim3 grid((unsigned)gx, (unsigned)nc);
       const float* wp = w + c0 * inner; float* op = w_out + c0 * inner;
-      if (vec) fold_kernel<true><<<grid, 256, 0, l.stream>>>(wp, gamma + c0, var + c0, inner, op);
-      else fold_kernel<false><<<grid, 256, 0, l.stream>>>(wp, gamma + c0, var + c0, inner, op);
+      if (w == w_out) {
+        if (vec) fold_kernel<true, true><<<grid, 256, 0, l.stream>>>(wp, gamma + c0, var + c0, inner, op);
+        else fold_kernel<false, true><<<grid, 256, 0, l.stream>>>(wp, gamma + c0, var + c0, inner, op);
+      } else {
+        if (vec) fold_kernel<true, false><<<grid, 256, 0, l.stream>>>(wp, gamma + c0, var + c0, inner, op);
+        else fold_kernel<false, false><<<grid, 256, 0, l.stream>>>(wp, gamma + c0, var + c0, inner, op);
+      }
     }
   }
   if (bias_out)

@@ -2,8 +2,9 @@
 // layer's value range): 2048 linear bins on [0, absmax] per tensor, counted exactly.
 //
 // Each CTA keeps a private 2048 x u32 histogram in shared memory across all the tiles it walks of
-// one tensor and merges it into the 64-bit global histogram only when it moves to another tensor.
-// Counts are integers, so the result does not depend on the order of the atomics.
+// one tensor and merges it into the tensor's 64-bit accumulation histogram only when it moves to
+// another tensor; the CTA that merges last turns the counts into the clip and the quantization
+// parameters.  Counts are integers, so the result does not depend on the order of the atomics.
 #include "qv2_device.cuh"
 
 namespace qv2 {
@@ -67,84 +68,42 @@ __device__ __forceinline__ void hist_tile(const T* x, uint32_t count, float w, b
   else hist_flat<false>(x, count, w, sh, zeros);
 }
 
-template <bool ANY16>      // false: every tensor is binary32, no element-type dispatch
-__global__ void __launch_bounds__(kThreads, 4)
-hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
-            const float* __restrict__ tensor_absmax, const unsigned long long* __restrict__ nonfinite,
-            unsigned long long* hist) {
-  __shared__ uint32_t sh[kBins];
-  for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
-  __syncthreads();
-
-  uint32_t cur = 0xffffffffu, since_flush = 0, zeros = 0;
-  float w = 0.0f;
-  bool careful = false;
-  for (uint32_t ti = blockIdx.x;; ti += gridDim.x) {
-    const bool more = ti < n_tiles;
-    Tile tl;
-    if (more) tl = load_tile(tiles, ti);
-    // merge into the global histogram when the tensor changes, at the end, and before a
-    // 32-bit count could overflow (2^14 tiles of 2^14 elements)
-    if (cur != 0xffffffffu && (!more || tl.tensor != cur || since_flush >= 16384u)) {
-      if (zeros) atomicAdd(sh, zeros);
-      zeros = 0;
-      __syncthreads();
-      unsigned long long* h = hist + (size_t)cur * kBins;
-      for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {
-        const uint32_t c = sh[b];
-        if (c) { atomicAdd(h + b, (unsigned long long)c); sh[b] = 0; }
-      }
-      __syncthreads();
-      since_flush = 0;
-    }
-    if (!more) break;
-    if (tl.tensor != cur) {
-      cur = tl.tensor;
-      const float A = tensor_absmax[cur];
-      w = (A > 0.0f) ? __fdiv_rn((float)kBins, A) : 0.0f;
-      if (!isfinite(w)) w = 0.0f;
-      careful = nonfinite[cur] != 0ull;
-    }
-    const TensorRec* tr = tensors + cur;
-    if (!ANY16 || tr->dtype == kF32) hist_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
-    else if (tr->dtype == kF16) hist_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
-    else hist_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
-    ++since_flush;
-  }
-}
-
-// One CTA per tensor: percentile clip from the histogram, then the quantization parameters of the
-// tensor's groups.  T = clamp(ceil(p * Nf), 1, Nf) with Nf the histogram total; k* = first bin
-// whose cumulative count reaches T; clip = upper edge of bin k* (absmax itself for the last bin).
-__global__ void __launch_bounds__(256)
-clip_finalize_kernel(const TensorRec* __restrict__ tensors, const unsigned long long* __restrict__ hist,
-                     const float* __restrict__ tensor_absmax, const float* __restrict__ gmin,
-                     const float* __restrict__ gmax, const float* __restrict__ gabsmax, float* clip,
-                     float* step, float* inv, float* offset) {
-  __shared__ unsigned long long scan[256];
+// Folds the histogram of one tensor once every CTA that owns a tile of it has merged its counts:
+// percentile clip, then the quantization parameters of the tensor's groups.
+// T = clamp(ceil(p * Nf), 1, Nf) with Nf the histogram total; k* = first bin whose cumulative
+// count reaches T; clip = upper edge of bin k* (absmax itself for the last bin).  The counts are
+// copied to the caller's histogram (when it wants one) and the accumulation row is put back to
+// zero for the next pass.  Runs in the CTA that drew the tensor's last ticket; the counts, written
+// by other CTAs, are read through L2.
+__device__ __noinline__ void clip_fold_tensor(const CalibArgs& a, uint32_t t) {
+  __shared__ unsigned long long scan[kThreads];
   __shared__ uint32_t kstar_s;
-  const uint32_t t = blockIdx.x, tid = threadIdx.x;
-  const TensorRec tr = tensors[t];
-  const float A = tensor_absmax[t];
-  if (tr.range_mode != QV2_PERCENTILE) {     // per-group percentile included: its clips are per group
-    if (tid == 0) clip[t] = A;
-    return;
-  }
-  constexpr uint32_t kPer = kBins / 256;
-  const unsigned long long* h = hist + (size_t)t * kBins;
+  const uint32_t tid = threadIdx.x;
+  const TensorRec tr = a.tensors[t];
+  const float A = a.tensor_absmax[t];
+  constexpr uint32_t kPer = kBins / kThreads;
+  unsigned long long* acc = a.hist_acc + (size_t)tr.hist_index * kBins;
   unsigned long long local[kPer], mine = 0;
 #pragma unroll
-  for (uint32_t i = 0; i < kPer; ++i) { local[i] = h[tid * kPer + i]; mine += local[i]; }
+  for (uint32_t i = 0; i < kPer; ++i) {
+    local[i] = __ldcg(acc + tid * kPer + i);
+    acc[tid * kPer + i] = 0ull;
+    mine += local[i];
+  }
+  if (a.hist) {
+#pragma unroll
+    for (uint32_t i = 0; i < kPer; ++i) a.hist[(size_t)t * kBins + tid * kPer + i] = local[i];
+  }
   scan[tid] = mine;
-  if (tid == 0) kstar_s = kBins - 1;
+  if (tid == 0) { kstar_s = kBins - 1; a.hist_tickets[t] = 0u; }
   __syncthreads();
-  for (uint32_t o = 1; o < 256; o <<= 1) {
+  for (uint32_t o = 1; o < kThreads; o <<= 1) {
     const unsigned long long add = tid >= o ? scan[tid - o] : 0ull;
     __syncthreads();
     scan[tid] += add;
     __syncthreads();
   }
-  const unsigned long long nf = scan[255], excl = scan[tid] - mine;
+  const unsigned long long nf = scan[kThreads - 1], excl = scan[tid] - mine;
   float c = A;
   if (nf != 0ull) {
     const double tt = ceil(__dmul_rn(tr.percentile, (double)nf));
@@ -164,10 +123,75 @@ clip_finalize_kernel(const TensorRec* __restrict__ tensors, const unsigned long 
     const uint32_t k = kstar_s;
     if (k != kBins - 1) c = __fmul_rn((float)(k + 1), __fdiv_rn(A, (float)kBins));
   }
-  if (tid == 0) clip[t] = c;
-  for (uint32_t g = tid; g < tr.n_groups; g += blockDim.x) {
+  if (tid == 0) a.clip[t] = c;
+  for (uint32_t g = tid; g < tr.n_groups; g += kThreads) {
     const uint32_t G = tr.group_base + g;
-    make_qparams(tr.asym, top_code(tr.asym != 0, tr.bits), true, c, gmin[G], gmax[G], gabsmax[G], step + G, inv + G, offset + G);
+    make_qparams(tr.asym, top_code(tr.asym != 0, tr.bits), true, c, a.gmin[G], a.gmax[G], a.gabsmax[G],
+                 a.step + G, a.inv + G, a.offset + G);
+  }
+  __syncthreads();                           // the shared arrays may be reused by the next fold
+}
+
+template <bool ANY16>      // false: every tensor is binary32, no element-type dispatch
+__global__ void __launch_bounds__(kThreads, 4)
+hist_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles, uint32_t n_tiles,
+            uint32_t scan_begin, uint32_t scan_end) {
+  __shared__ uint32_t sh[kBins];
+  __shared__ uint32_t s_last;
+  const TensorRec* __restrict__ tensors = a.tensors;
+  for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
+  __syncthreads();
+  // percentile tensors without elements are owned by no CTA: CTA 0 folds them
+  if (blockIdx.x == 0)
+    for (uint32_t t = scan_begin; t < scan_end; ++t)
+      if (tensors[t].range_mode == QV2_PERCENTILE && tensors[t].hist_ctas == 0) clip_fold_tensor(a, t);
+
+  uint32_t cur = 0xffffffffu, since_flush = 0, zeros = 0;
+  float w = 0.0f;
+  bool careful = false;
+  for (uint32_t ti = blockIdx.x;; ti += gridDim.x) {
+    const bool more = ti < n_tiles;
+    Tile tl;
+    if (more) tl = load_tile(tiles, ti);
+    // merge into the accumulation histogram when the tensor changes, at the end, and before a
+    // 32-bit count could overflow (2^14 tiles of 2^14 elements)
+    const bool leaving = cur != 0xffffffffu && (!more || tl.tensor != cur);
+    if (leaving || (cur != 0xffffffffu && since_flush >= 16384u)) {
+      if (zeros) atomicAdd(sh, zeros);
+      zeros = 0;
+      __syncthreads();
+      unsigned long long* h = a.hist_acc + (size_t)tensors[cur].hist_index * kBins;
+      for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {
+        const uint32_t c = sh[b];
+        if (c) { atomicAdd(h + b, (unsigned long long)c); sh[b] = 0; }
+      }
+      since_flush = 0;
+      if (leaving) {                  // the CTA that merges a tensor last folds it; nobody waits
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) s_last = atomicAdd(a.hist_tickets + cur, 1u) == tensors[cur].hist_ctas - 1u;
+        __syncthreads();
+        if (s_last) {
+          __threadfence();
+          clip_fold_tensor(a, cur);
+        }
+      } else {
+        __syncthreads();
+      }
+    }
+    if (!more) break;
+    if (tl.tensor != cur) {
+      cur = tl.tensor;
+      const float A = a.tensor_absmax[cur];
+      w = (A > 0.0f) ? __fdiv_rn((float)kBins, A) : 0.0f;
+      if (!isfinite(w)) w = 0.0f;
+      careful = a.nonfinite[cur] != 0ull;
+    }
+    const TensorRec* tr = tensors + cur;
+    if (!ANY16 || tr->dtype == kF32) hist_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+    else if (tr->dtype == kF16) hist_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+    else hist_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
+    ++since_flush;
   }
 }
 
@@ -270,7 +294,7 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 }
 
 // One warp per group histogram: the group's clip by the same cumulative-count rule as
-// clip_finalize_kernel, then the group's quantization parameters.
+// clip_fold_tensor, then the group's quantization parameters.
 __global__ void __launch_bounds__(256)
 group_clip_finalize_kernel(const TensorRec* __restrict__ tensors, const uint32_t* __restrict__ owner,
                            uint32_t n_hists, const unsigned long long* __restrict__ ghist,
@@ -326,12 +350,20 @@ fill_group_clip_kernel(const TensorRec* __restrict__ tensors, const float* __res
 
 }  // namespace
 
-cudaError_t launch_group_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
-                              uint32_t n_tiles, const float* gabsmax, const unsigned long long* nonfinite,
-                              unsigned long long* ghist) {
+uint32_t hist_grid_cap(int sm_count) {
+  int cache = 0;
+  return (uint32_t)persistent_grid((const void*)hist_kernel<false>, &cache, sm_count, 0x7fffffffu);
+}
+uint32_t group_hist_grid_cap(int sm_count) {
+  int cache = 0;
+  return (uint32_t)persistent_grid((const void*)group_hist_kernel<false>, &cache, sm_count, 0x7fffffffu);
+}
+
+cudaError_t launch_group_hist(const Launch& l, uint32_t grid_cap, bool any16, const TensorRec* tensors,
+                              const Tile* tiles, uint32_t n_tiles, const float* gabsmax,
+                              const unsigned long long* nonfinite, unsigned long long* ghist) {
   if (n_tiles == 0) return cudaSuccess;
-  static int per_sm = 0;
-  const int grid = persistent_grid((const void*)group_hist_kernel<false>, &per_sm, l.sm_count, n_tiles);
+  const uint32_t grid = grid_cap < n_tiles ? (grid_cap ? grid_cap : 1u) : n_tiles;
   if (any16) group_hist_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, gabsmax, nonfinite, ghist);
   else group_hist_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, gabsmax, nonfinite, ghist);
   return cudaGetLastError();
@@ -353,23 +385,14 @@ cudaError_t launch_fill_group_clip(const Launch& l, const TensorRec* tensors, ui
   return cudaGetLastError();
 }
 
-cudaError_t launch_hist(const Launch& l, bool any16, const TensorRec* tensors, const Tile* tiles,
-                        uint32_t n_tiles, const float* tensor_absmax,
-                        const unsigned long long* nonfinite, unsigned long long* hist) {
-  if (n_tiles == 0) return cudaSuccess;
-  static int per_sm = 0;
-  const int grid = persistent_grid((const void*)hist_kernel<false>, &per_sm, l.sm_count, n_tiles);
-  if (any16) hist_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, tensor_absmax, nonfinite, hist);
-  else hist_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, tensor_absmax, nonfinite, hist);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_clip_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                 const unsigned long long* hist, const float* tensor_absmax,
-                                 const float* gmin, const float* gmax, const float* gabsmax,
-                                 float* clip, float* step, float* inv, float* offset) {
-  clip_finalize_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, hist, tensor_absmax, gmin, gmax,
-                                                        gabsmax, clip, step, inv, offset);
+// One launch over the stage's slice of the histogram tile table.  Needed whenever the stage has a
+// percentile tensor: one without elements still gets its (degenerate) clip and parameters.
+cudaError_t launch_hist(const Launch& l, const Stage& st, bool any16, const Tile* hist_tiles, const CalibArgs& a) {
+  if (!st.any_percentile) return cudaSuccess;
+  const uint32_t n_tiles = st.hist_end - st.hist_begin;
+  const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
+  if (any16) hist_kernel<true><<<st.hist_grid, kThreads, 0, l.stream>>>(a, hist_tiles + st.hist_begin, n_tiles, s0, s1);
+  else hist_kernel<false><<<st.hist_grid, kThreads, 0, l.stream>>>(a, hist_tiles + st.hist_begin, n_tiles, s0, s1);
   return cudaGetLastError();
 }
 

@@ -5,10 +5,12 @@
 // One persistent launch walks the tile table of a whole model; CTA b takes tiles b, b+grid, ...
 // Every lane reduces its share of a tile in binary32 (independent accumulators per vector lane),
 // adds the tile's two sums to binary64 running sums that it keeps while the CTA stays on the same
-// tensor, and when the tensor changes the warp folds its lanes with a fixed butterfly and writes
-// one {sum e^2, sum x^2} pair to its own slot.  A second kernel adds each tensor's slots in a
-// fixed order in binary64.  There are no floating-point atomics and no inter-CTA waits: for a
-// given grid size the result is bit-identical from run to run.
+// tensor, and when the tensor changes the CTA folds its lanes and warps in a fixed order and writes
+// one {sum e^2, sum x^2} pair to its own slot.  The CTA that finishes a tensor last (an atomic
+// ticket) adds the tensor's slots in a fixed order in binary64 and writes the metrics.  There are
+// no floating-point atomics and no inter-CTA waits: for a given grid size the result is
+// bit-identical from run to run.
+#include <mutex>
 #include <type_traits>
 
 #include "qv2_device.cuh"
@@ -188,11 +190,11 @@ __device__ __forceinline__ void load_params(QP& p, const TensorRec* tr, const fl
 template <uint32_t MODE, bool CODES, class T, class ACC>
 __device__ __noinline__ ACC metric_rows(Tile tl, const TensorRec* tr, const float* __restrict__ step,
                                         const float* __restrict__ inv, const float* __restrict__ offset,
-                                        ACC seed) {
+                                        uint8_t* codes_base, ACC seed) {
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const T* x = reinterpret_cast<const T*>(tr->x) + tl.begin;
   const T* y = (MODE != kSelf) ? reinterpret_cast<const T*>(tr->y) + tl.begin : nullptr;
-  uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
+  uint8_t* codes = CODES ? codes_base + tl.begin : nullptr;
   const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
   ACC a[4] = {seed, seed, seed, seed};
   QP p;
@@ -237,17 +239,17 @@ __device__ __noinline__ ACC metric_rows(Tile tl, const TensorRec* tr, const floa
 template <uint32_t MODE, bool CODES, class T, class ACC>
 __device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRec* tr,
                                                   const float* __restrict__ step, const float* __restrict__ inv,
-                                                  const float* __restrict__ offset, ACC* a) {
+                                                  const float* __restrict__ offset, uint8_t* codes_base, ACC* a) {
   if (tl.rows == 0) {
     const T* x = reinterpret_cast<const T*>(tr->x) + tl.begin;
     const T* y = (MODE != kSelf) ? reinterpret_cast<const T*>(tr->y) + tl.begin : nullptr;
-    uint8_t* codes = CODES ? tr->codes + tl.begin : nullptr;
+    uint8_t* codes = CODES ? codes_base + tl.begin : nullptr;
     QP p;
     load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)tl.row0);
     if (MODE == kRaw || p.off == 0.0f) metric_flat<MODE, false, CODES>(x, y, codes, tl.count, p, a);
     else metric_flat<MODE, true, CODES>(x, y, codes, tl.count, p, a);
   } else {
-    a[0].merge(metric_rows<MODE, CODES, T>(tl, tr, step, inv, offset, a[0].fresh()));
+    a[0].merge(metric_rows<MODE, CODES, T>(tl, tr, step, inv, offset, codes_base, a[0].fresh()));
   }
 }
 
@@ -255,122 +257,152 @@ __device__ __forceinline__ void metric_tile_typed(const Tile& tl, const TensorRe
 template <uint32_t MODE, bool CODES, bool ANY16 = true, class ACC>
 __device__ __forceinline__ void metric_tile(const Tile& tl, const TensorRec* tr,
                                             const float* __restrict__ step, const float* __restrict__ inv,
-                                            const float* __restrict__ offset, ACC* a) {
-  if (!ANY16 || tr->dtype == kF32) metric_tile_typed<MODE, CODES, float>(tl, tr, step, inv, offset, a);
-  else if (tr->dtype == kF16) metric_tile_typed<MODE, CODES, __half>(tl, tr, step, inv, offset, a);
-  else metric_tile_typed<MODE, CODES, __nv_bfloat16>(tl, tr, step, inv, offset, a);
+                                            const float* __restrict__ offset, uint8_t* codes_base, ACC* a) {
+  if (!ANY16 || tr->dtype == kF32) metric_tile_typed<MODE, CODES, float>(tl, tr, step, inv, offset, codes_base, a);
+  else if (tr->dtype == kF16) metric_tile_typed<MODE, CODES, __half>(tl, tr, step, inv, offset, codes_base, a);
+  else metric_tile_typed<MODE, CODES, __nv_bfloat16>(tl, tr, step, inv, offset, codes_base, a);
 }
 
-// Slot of (tensor, CTA, warp): the CTAs that own tiles of a tensor are numbered in the order of
-// the tensor's first tiles, rank = (b - tile_first) mod grid < min(grid, tiles of the tensor).
-__device__ __forceinline__ uint32_t slot_of(const TensorRec* tr, uint32_t warp) {
+// Slot of (tensor, CTA): the CTAs that own tiles of a tensor are numbered in the order of the
+// tensor's first tiles, rank = (b - tile_first) mod grid < min(grid, tiles of the tensor).
+__device__ __forceinline__ uint32_t slot_of(const TensorRec* tr) {
   const uint32_t g = gridDim.x;
   const uint32_t rank = (blockIdx.x + g - tr->tile_first % g) % g;
-  return tr->slot_first + rank * kWarps + warp;
+  return tr->slot_first + rank;
+}
+
+// Folds one tensor once every CTA that owns a tile of it has written its slot: fixed-order
+// binary64 sum of the tensor's slots, then MSE (Eq. 7), SQNR (Eq. 6) and, when asked for, the
+// cosine similarity (Eq. 8) between the reference tensor A = x and the compared tensor B = x - e:
+// A.B = sig - xe, |B|^2 = sig - 2 xe + sse.  Runs in the CTA that drew the tensor's last ticket
+// (CTA 0 for a tensor without elements); the slots, written by other CTAs, are read through L2.
+template <bool COS>
+__device__ __noinline__ void metrics_fold_tensor(const MetricsArgs& a, uint32_t t) {
+  __shared__ double sh_e[kThreads], sh_s[kThreads], sh_x[COS ? kThreads : 1];
+  const TensorRec tr = a.tensors[t];
+  const uint32_t tid = threadIdx.x;
+  double e = 0.0, s = 0.0, xe = 0.0;
+  for (uint32_t k = tid; k < tr.metrics_ctas; k += kThreads) {
+    const double2 p = __ldcg(a.partials + tr.slot_first + k);
+    e = __dadd_rn(e, p.x);
+    s = __dadd_rn(s, p.y);
+    if (COS) xe = __dadd_rn(xe, __ldcg(a.partials_xe + tr.slot_first + k));
+  }
+  sh_e[tid] = e; sh_s[tid] = s;
+  if (COS) sh_x[tid] = xe;
+  __syncthreads();
+  for (uint32_t o = kThreads / 2; o > 0; o >>= 1) {
+    if (tid < o) {
+      sh_e[tid] = __dadd_rn(sh_e[tid], sh_e[tid + o]);
+      sh_s[tid] = __dadd_rn(sh_s[tid], sh_s[tid + o]);
+      if (COS) sh_x[tid] = __dadd_rn(sh_x[tid], sh_x[tid + o]);
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const double sse = sh_e[0], sig = sh_s[0];
+    const double inf = __longlong_as_double(0x7ff0000000000000ll);
+    a.sse[t] = sse;
+    a.sig[t] = sig;
+    a.mse[t] = tr.n_elems ? __ddiv_rn(sse, (double)tr.n_elems) : 0.0;
+    double q;
+    if (sse == 0.0) q = inf;
+    else if (sig == 0.0) q = -inf;
+    else q = __dmul_rn(10.0, log10(__ddiv_rn(sig, sse)));
+    a.sqnr_db[t] = q;
+    if (COS) {
+      const double ab = sig - sh_x[0];
+      const double bb = sig - 2.0 * sh_x[0] + sse;
+      const double den = sqrt(sig) * sqrt(bb > 0.0 ? bb : 0.0);
+      a.cosine[t] = den > 0.0 ? ab / den : 0.0;       // a zero vector has no direction
+    }
+    a.tickets[t] = 0u;                                // ready for the next pass
+  }
+  __syncthreads();                                    // the shared arrays may be reused by the next fold
 }
 
 // COS adds the sum x*e (third slot array) needed for the cosine similarity.
 template <bool COS, bool ANY16>
-__global__ void __launch_bounds__(kThreads, 3)       // 85 registers: nothing spills; 4 CTAs per SM did not run faster
-metrics_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
-               const float* __restrict__ step, const float* __restrict__ inv,
-               const float* __restrict__ offset, double2* __restrict__ partials,
-               double* __restrict__ partials_xe) {
+__global__ void __launch_bounds__(kThreads, 3)       // 4 CTAs per SM did not run faster
+metrics_kernel(const __grid_constant__ MetricsArgs a, const Tile* __restrict__ tiles, uint32_t n_tiles,
+               uint32_t scan_begin, uint32_t scan_end) {
   using ACC = typename std::conditional<COS, AccCos, Acc>::type;
   constexpr uint32_t kNone = 0xffffffffu;
+  __shared__ double sh_w[3][kWarps];
+  __shared__ uint32_t s_last;
+  const TensorRec* __restrict__ tensors = a.tensors;
+  const float* __restrict__ step = a.step;
+  const float* __restrict__ inv = a.inv;
+  const float* __restrict__ offset = a.offset;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  // tensors without elements are owned by no CTA: CTA 0 folds them
+  if (blockIdx.x == 0)
+    for (uint32_t t = scan_begin; t < scan_end; ++t)
+      if (tensors[t].metrics_ctas == 0) metrics_fold_tensor<COS>(a, t);
   uint32_t cur = kNone;
   double run_sse = 0.0, run_sig = 0.0, run_xe = 0.0;
-  auto flush = [&](const TensorRec* tr) {
+  // The CTA is done with tensor t: lanes fold by a fixed butterfly, warps in warp order, one
+  // {sum e^2, sum x^2} pair goes to the CTA's own slot; the CTA that draws the tensor's last
+  // ticket folds the slots.  Nobody waits.
+  auto flush = [&](uint32_t t) {
+    const TensorRec* tr = tensors + t;
     const double sse = warp_sum_f64(run_sse), sig = warp_sum_f64(run_sig);
     double xe = 0.0;
     if (COS) xe = warp_sum_f64(run_xe);
-    if (lane == 0) {
-      const uint32_t slot = slot_of(tr, warp);
-      partials[slot] = make_double2(sse, sig);
-      if (COS) partials_xe[slot] = xe;
+    if (lane == 0) { sh_w[0][warp] = sse; sh_w[1][warp] = sig; if (COS) sh_w[2][warp] = xe; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double e = sh_w[0][0], s = sh_w[1][0], x = COS ? sh_w[2][0] : 0.0;
+#pragma unroll
+      for (int w = 1; w < kWarps; ++w) {
+        e = __dadd_rn(e, sh_w[0][w]); s = __dadd_rn(s, sh_w[1][w]);
+        if (COS) x = __dadd_rn(x, sh_w[2][w]);
+      }
+      const uint32_t slot = slot_of(tr);
+      a.partials[slot] = make_double2(e, s);
+      if (COS) a.partials_xe[slot] = x;
+      __threadfence();                                 // the slot is visible before the ticket is
+      s_last = atomicAdd(a.tickets + t, 1u) == tr->metrics_ctas - 1u;
+    }
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      metrics_fold_tensor<COS>(a, t);
     }
   };
   for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile tl = load_tile(tiles, ti);
     const TensorRec* tr = tensors + tl.tensor;
     if (tl.tensor != cur) {
-      if (cur != kNone) flush(tensors + cur);
+      if (cur != kNone) flush(cur);
       cur = tl.tensor; run_sse = 0.0; run_sig = 0.0; run_xe = 0.0;
     }
-    ACC a[4];
+    ACC acc[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) a[k].clear();
+    for (int k = 0; k < 4; ++k) acc[k].clear();
     const uint32_t mode = tr->pair_mode;
-    const bool codes = tr->codes != nullptr && mode != kRaw;
+    uint8_t* cbase = a.codes ? a.codes[tl.tensor] : nullptr;
+    const bool codes = cbase != nullptr && mode != kRaw;
     if (mode == kSelf) {
-      if (codes) metric_tile<kSelf, true, ANY16>(tl, tr, step, inv, offset, a);
-      else metric_tile<kSelf, false, ANY16>(tl, tr, step, inv, offset, a);
+      if (codes) metric_tile<kSelf, true, ANY16>(tl, tr, step, inv, offset, cbase, acc);
+      else metric_tile<kSelf, false, ANY16>(tl, tr, step, inv, offset, nullptr, acc);
     } else if (mode == kRequant) {
-      if (codes) metric_tile<kRequant, true, ANY16>(tl, tr, step, inv, offset, a);
-      else metric_tile<kRequant, false, ANY16>(tl, tr, step, inv, offset, a);
+      if (codes) metric_tile<kRequant, true, ANY16>(tl, tr, step, inv, offset, cbase, acc);
+      else metric_tile<kRequant, false, ANY16>(tl, tr, step, inv, offset, nullptr, acc);
     } else {
-      metric_tile<kRaw, false, ANY16>(tl, tr, step, inv, offset, a);
+      metric_tile<kRaw, false, ANY16>(tl, tr, step, inv, offset, nullptr, acc);
     }
     // this lane's tile sums in binary32 with a fixed association, then into the binary64 totals
-    const float sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
-    const float sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
+    const float sse = __fadd_rn(__fadd_rn(acc[0].sse, acc[1].sse), __fadd_rn(acc[2].sse, acc[3].sse));
+    const float sig = __fadd_rn(__fadd_rn(acc[0].sig, acc[1].sig), __fadd_rn(acc[2].sig, acc[3].sig));
     run_sse = __dadd_rn(run_sse, (double)sse);
     run_sig = __dadd_rn(run_sig, (double)sig);
     if constexpr (COS) {
-      const float xe = __fadd_rn(__fadd_rn(a[0].xe, a[1].xe), __fadd_rn(a[2].xe, a[3].xe));
+      const float xe = __fadd_rn(__fadd_rn(acc[0].xe, acc[1].xe), __fadd_rn(acc[2].xe, acc[3].xe));
       run_xe = __dadd_rn(run_xe, (double)xe);
     }
   }
-  if (cur != kNone) flush(tensors + cur);
-}
-
-// One CTA per tensor: fixed-order binary64 sum of the tensor's slots, then MSE (Eq. 7), SQNR
-// (Eq. 6) and, when asked for, the cosine similarity (Eq. 8) between the reference tensor A = x
-// and the compared tensor B = x - e:  A.B = sig - xe,  |B|^2 = sig - 2 xe + sse.
-constexpr int kFinalizeThreads = 1024;   // short chains of dependent loads: 3552 slots take 4 rounds
-
-__global__ void __launch_bounds__(kFinalizeThreads)
-metrics_finalize_kernel(const TensorRec* __restrict__ tensors, const double2* __restrict__ partials,
-                        const double* __restrict__ partials_xe, double* sse_out, double* sig_out,
-                        double* mse_out, double* sqnr_out, double* cos_out) {
-  __shared__ double sh_e[kFinalizeThreads], sh_s[kFinalizeThreads], sh_x[kFinalizeThreads];
-  const TensorRec tr = tensors[blockIdx.x];
-  double e = 0.0, s = 0.0, xe = 0.0;
-  for (uint32_t k = threadIdx.x; k < tr.slot_count; k += kFinalizeThreads) {
-    const double2 p = partials[tr.slot_first + k];
-    e = __dadd_rn(e, p.x);
-    s = __dadd_rn(s, p.y);
-    if (cos_out) xe = __dadd_rn(xe, partials_xe[tr.slot_first + k]);
-  }
-  sh_e[threadIdx.x] = e; sh_s[threadIdx.x] = s; sh_x[threadIdx.x] = xe;
-  __syncthreads();
-  for (uint32_t o = kFinalizeThreads / 2; o > 0; o >>= 1) {
-    if (threadIdx.x < o) {
-      sh_e[threadIdx.x] = __dadd_rn(sh_e[threadIdx.x], sh_e[threadIdx.x + o]);
-      sh_s[threadIdx.x] = __dadd_rn(sh_s[threadIdx.x], sh_s[threadIdx.x + o]);
-      sh_x[threadIdx.x] = __dadd_rn(sh_x[threadIdx.x], sh_x[threadIdx.x + o]);
-    }
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) {
-    const double sse = sh_e[0], sig = sh_s[0];
-    const double inf = __longlong_as_double(0x7ff0000000000000ll);
-    sse_out[blockIdx.x] = sse;
-    sig_out[blockIdx.x] = sig;
-    mse_out[blockIdx.x] = tr.n_elems ? __ddiv_rn(sse, (double)tr.n_elems) : 0.0;
-    double q;
-    if (sse == 0.0) q = inf;
-    else if (sig == 0.0) q = -inf;
-    else q = __dmul_rn(10.0, log10(__ddiv_rn(sig, sse)));
-    sqnr_out[blockIdx.x] = q;
-    if (cos_out) {
-      const double ab = sig - sh_x[0];
-      const double bb = sig - 2.0 * sh_x[0] + sse;
-      const double den = sqrt(sig) * sqrt(bb > 0.0 ? bb : 0.0);
-      cos_out[blockIdx.x] = den > 0.0 ? ab / den : 0.0;       // a zero vector has no direction
-    }
-  }
+  if (cur != kNone) flush(cur);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -439,9 +471,9 @@ kl_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles,
 #pragma unroll
     for (int k = 0; k < 4; ++k) { a[k].hp = sh + warp * 2 * kKlBins; a[k].hq = a[k].hp + kKlBins; a[k].w = w; }
     const uint32_t mode = tr->pair_mode;
-    if (mode == kSelf) metric_tile<kSelf, false>(tl, tr, step, inv, offset, a);
-    else if (mode == kRequant) metric_tile<kRequant, false>(tl, tr, step, inv, offset, a);
-    else metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
+    if (mode == kSelf) metric_tile<kSelf, false>(tl, tr, step, inv, offset, nullptr, a);
+    else if (mode == kRequant) metric_tile<kRequant, false>(tl, tr, step, inv, offset, nullptr, a);
+    else metric_tile<kRaw, false>(tl, tr, step, inv, offset, nullptr, a);
     ++since_flush;
   }
 }
@@ -483,45 +515,38 @@ __global__ void kl_finalize_kernel(uint32_t n, const unsigned long long* __restr
 }  // namespace
 
 uint32_t metrics_grid_cap(int sm_count) {
-  static int per_sm = 0;
-  return (uint32_t)persistent_grid((const void*)metrics_kernel<false, false>, &per_sm, sm_count, 0x7fffffffu);
+  int cache = 0;
+  return (uint32_t)persistent_grid((const void*)metrics_kernel<false, false>, &cache, sm_count, 0x7fffffffu);
+}
+uint32_t kl_grid_cap(int sm_count) {
+  int cache = 0;
+  return (uint32_t)persistent_grid((const void*)kl_kernel, &cache, sm_count, 0x7fffffffu);
 }
 
-cudaError_t launch_metrics(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors,
-                           const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
-                           const float* offset, double2* partials, double* partials_xe) {
-  if (n_tiles == 0) return cudaSuccess;
+cudaError_t launch_metrics(const Launch& l, const Stage& st, bool any16, const Tile* tiles, const MetricsArgs& a) {
+  const uint32_t n_tiles = st.tile_end - st.tile_begin;
+  const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
 #define QV2_LAUNCH_METRICS(COS, A16) \
-  metrics_kernel<COS, A16><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset, partials, partials_xe)
-  if (partials_xe) { if (any16) QV2_LAUNCH_METRICS(true, true); else QV2_LAUNCH_METRICS(true, false); }
+  metrics_kernel<COS, A16><<<st.metrics_grid, kThreads, 0, l.stream>>>(a, tiles + st.tile_begin, n_tiles, s0, s1)
+  if (a.cosine) { if (any16) QV2_LAUNCH_METRICS(true, true); else QV2_LAUNCH_METRICS(true, false); }
   else { if (any16) QV2_LAUNCH_METRICS(false, true); else QV2_LAUNCH_METRICS(false, false); }
 #undef QV2_LAUNCH_METRICS
   return cudaGetLastError();
 }
 
-cudaError_t launch_metrics_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                    const double2* partials, const double* partials_xe, double* sse,
-                                    double* sig, double* mse, double* sqnr_db, double* cosine) {
-  metrics_finalize_kernel<<<n_tensors, kFinalizeThreads, 0, l.stream>>>(tensors, partials, partials_xe, sse, sig,
-                                                           mse, sqnr_db, cosine);
-  return cudaGetLastError();
-}
-
-}  // namespace qv2
-
-namespace qv2 {
-cudaError_t launch_kl(const Launch& l, const TensorRec* tensors, uint32_t n_tensors, const Tile* tiles,
-                      uint32_t n_tiles, const float* step, const float* inv, const float* offset,
-                      const float* gabsmax, float* tensor_absmax, unsigned long long* hists, double* kl) {
+cudaError_t launch_kl(const Launch& l, uint32_t grid_cap, const TensorRec* tensors, uint32_t n_tensors,
+                      const Tile* tiles, uint32_t n_tiles, const float* step, const float* inv,
+                      const float* offset, const float* gabsmax, float* tensor_absmax,
+                      unsigned long long* hists, double* kl) {
   tensor_absmax_kernel<<<n_tensors, 256, 0, l.stream>>>(tensors, gabsmax, tensor_absmax);
   if (n_tiles) {
-    static int per_sm = 0;
-    const int grid = persistent_grid((const void*)kl_kernel, &per_sm, l.sm_count, n_tiles);
+    const uint32_t grid = grid_cap < n_tiles ? (grid_cap ? grid_cap : 1u) : n_tiles;
     kl_kernel<<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, step, inv, offset, tensor_absmax, hists);
   }
   kl_finalize_kernel<<<(n_tensors + 63) / 64, 64, 0, l.stream>>>(n_tensors, hists, kl);
   return cudaGetLastError();
 }
+
 }  // namespace qv2
 
 // ================================================================================================
@@ -585,9 +610,9 @@ metrics_noalloc_kernel(const __grid_constant__ NoAllocJob job, const float* __re
     Acc a[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) a[k].clear();
-    if (tr->pair_mode == kSelf) metric_tile<kSelf, false>(tl, tr, step, inv, offset, a);
-    else if (tr->pair_mode == kRequant) metric_tile<kRequant, false>(tl, tr, step, inv, offset, a);
-    else metric_tile<kRaw, false>(tl, tr, step, inv, offset, a);
+    if (tr->pair_mode == kSelf) metric_tile<kSelf, false>(tl, tr, step, inv, offset, nullptr, a);
+    else if (tr->pair_mode == kRequant) metric_tile<kRequant, false>(tl, tr, step, inv, offset, nullptr, a);
+    else metric_tile<kRaw, false>(tl, tr, step, inv, offset, nullptr, a);
     float sse = __fadd_rn(__fadd_rn(a[0].sse, a[1].sse), __fadd_rn(a[2].sse, a[3].sse));
     float sig = __fadd_rn(__fadd_rn(a[0].sig, a[1].sig), __fadd_rn(a[2].sig, a[3].sig));
     sse = warp_sum(sse);
@@ -630,8 +655,8 @@ metrics_noalloc_finalize_kernel(uint32_t n_slots, uint64_t n_elems, const double
 // has to be asked for, once per device, with that device current.
 constexpr int kMaxDevices = 64;
 struct NoAllocDevice {
-  bool ready = false;
-  double2* slots = nullptr;
+  std::once_flag once;
+  double2* slots = nullptr;     // null until the set-up has succeeded
   int grid_cap = 1;
 };
 NoAllocDevice g_noalloc_dev[kMaxDevices];
@@ -660,18 +685,15 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   if (ne > 0 && !d.x) return QV2_ERR_NULL;
   if (((uintptr_t)d.x & 3u) || ((uintptr_t)d.y & 3u)) return QV2_ERR_ALIGN;
 
-  NoAllocJob job;
-  job.tr.x = d.x; job.tr.y = d.y; job.tr.codes = nullptr;
+  NoAllocJob job{};                      // every field the kernel does not use reads zero
+  job.tr.x = d.x; job.tr.y = d.y;
   job.tr.n_elems = ne; job.tr.inner = d.inner; job.tr.channels = (uint32_t)d.channels;
-  job.tr.group_base = 0;
   job.tr.per_channel = d.granularity == QV2_PER_CHANNEL;
   job.tr.n_groups = job.tr.per_channel ? (uint32_t)d.channels : 1u;
   job.tr.asym = d.scheme;
   job.tr.range_mode = d.range;
   job.tr.pair_mode = !d.y ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
-  job.tr.slot_first = 0; job.tr.slot_count = 0; job.tr.tile_first = 0;
   job.tr.percentile = d.percentile;
-  job.tr.rslot_first = 0; job.tr.rslot_count = 0;
   job.tr.bits = QV2_DESC_BITS(d.flags);
   job.tr.dtype = kF32;                  // this entry point takes binary32 tensors only
   job.rows = rows; job.tiles_per_row = 1; job.rows_per_tile = 1;
@@ -696,27 +718,34 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   if (prev != device && cudaSetDevice(device) != cudaSuccess) return QV2_ERR_CUDA;
   int status = QV2_OK;
   NoAllocDevice& nd = g_noalloc_dev[device];
-  if (!nd.ready) {                        // first call on this device: resolve the array's address
+  // first call on this device: resolve the array's address; host threads racing here run it once
+  std::call_once(nd.once, [&]() {
     double2* p = nullptr;
     int sms = 0, per_sm = 0;
     if (cudaGetSymbolAddress((void**)&p, g_noalloc_slots) != cudaSuccess || !p ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
-      status = QV2_ERR_CUDA;
-    } else {
-      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)metrics_noalloc_kernel,
-                                                        kThreads, 0) != cudaSuccess || per_sm < 1)
-        per_sm = 1;
-      nd.slots = p; nd.grid_cap = per_sm * (sms > 0 ? sms : 1); nd.ready = true;
-    }
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+      return;                                   // nd.slots stays null: every call reports QV2_ERR_CUDA
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)metrics_noalloc_kernel,
+                                                      kThreads, 0) != cudaSuccess || per_sm < 1)
+      per_sm = 1;
+    nd.grid_cap = per_sm * (sms > 0 ? sms : 1);
+    nd.slots = p;
+  });
+  if (!nd.slots) {
+    (void)cudaGetLastError();                   // the failed set-up call must not poison later launches
+    status = QV2_ERR_CUDA;
   }
   if (status == QV2_OK) {
     cudaStream_t s = (cudaStream_t)stream;
     if (job.n_tiles) {
       const uint32_t grid = job.n_tiles < (uint32_t)nd.grid_cap ? job.n_tiles : (uint32_t)nd.grid_cap;
       metrics_noalloc_kernel<<<grid, kThreads, 0, s>>>(job, step, inv, offset, nd.slots);
+      if (cudaPeekAtLastError() != cudaSuccess) { (void)cudaGetLastError(); status = QV2_ERR_CUDA; }
     }
-    metrics_noalloc_finalize_kernel<<<1, 1024, 0, s>>>(job.n_tiles * kWarps, ne, nd.slots, result4);
-    if (cudaGetLastError() != cudaSuccess) status = QV2_ERR_CUDA;
+    if (status == QV2_OK) {
+      metrics_noalloc_finalize_kernel<<<1, 1024, 0, s>>>(job.n_tiles * kWarps, ne, nd.slots, result4);
+      if (cudaPeekAtLastError() != cudaSuccess) { (void)cudaGetLastError(); status = QV2_ERR_CUDA; }
+    }
   }
   if (prev != device) cudaSetDevice(prev);
   return status;

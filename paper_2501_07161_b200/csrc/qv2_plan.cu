@@ -27,15 +27,15 @@ static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t g
 // any of them is generated.
 constexpr uint64_t kMaxTiles = 1ull << 27;
 
-static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
-                              uint32_t range_cap, HostPlan* out) {
+static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const GridCaps& caps,
+                              uint64_t chunk_bytes, HostPlan* out) {
   if (!descs || !out) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
-  out->tensors.clear(); out->tiles.clear(); out->hist_tiles.clear();
-  out->ghist_tiles.clear(); out->ghist_owner.clear();
-  out->total_groups = 0; out->total_slots = 0; out->any_percentile = false; out->any_16bit = false;
+  *out = HostPlan();
   out->tensors.reserve(n);
+  std::vector<uint32_t> tile_cnt(n, 0), hist_cnt(n, 0);
   uint64_t groups = 0;
+  bool any_group_pct = false;
   for (uint32_t t = 0; t < n; ++t) {
     const qv2_tensor_desc& d = descs[t];
     if (d.granularity > QV2_PER_CHANNEL || d.scheme > QV2_ASYM_U8_ZP || d.range > QV2_PERCENTILE_GROUP)
@@ -58,9 +58,8 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, void* co
     bool pair = d.y != nullptr;
     if ((d.flags & QV2_PAIR_RAW) && !pair) return QV2_ERR_ARG;
 
-    TensorRec r;
+    TensorRec r = TensorRec();
     r.x = d.x; r.y = d.y;
-    r.codes = (codes && (d.flags & QV2_STORE_CODES)) ? (uint8_t*)codes[t] : nullptr;
     r.n_elems = ne; r.inner = d.inner;
     r.channels = (uint32_t)d.channels;
     r.per_channel = d.granularity == QV2_PER_CHANNEL;
@@ -71,11 +70,11 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, void* co
     r.asym = d.scheme;                  // 0 symmetric, 1 affine with real offset, 2 affine with zero point
     // one group: its histogram is the tensor's, so the per-group mode is the per-tensor one
     r.range_mode = (d.range == QV2_PERCENTILE_GROUP && !r.per_channel) ? (uint32_t)QV2_PERCENTILE : d.range;
-    r.ghist_first = 0;
     if (r.range_mode == QV2_PERCENTILE_GROUP) {
       if (out->ghist_owner.size() + r.n_groups >= (1ull << 32)) return QV2_ERR_SIZE;
       r.ghist_first = (uint32_t)out->ghist_owner.size();
       out->ghist_owner.insert(out->ghist_owner.end(), r.n_groups, t);
+      any_group_pct = true;
     }
     r.pair_mode = !pair ? kSelf : ((d.flags & QV2_PAIR_RAW) ? kRaw : kRequant);
     r.percentile = d.percentile;
@@ -83,7 +82,7 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, void* co
     r.dtype = dtype;
     if (dtype != kF32) out->any_16bit = true;
 
-    size_t first_tile = out->tiles.size();
+    const size_t first_tile = out->tiles.size(), first_hist = out->hist_tiles.size();
     {
       uint64_t need;
       if (ne == 0) need = 0;
@@ -94,7 +93,10 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, void* co
       if (r.range_mode == QV2_PERCENTILE &&
           out->hist_tiles.size() + (ne + kTileElems - 1) / kTileElems > kMaxTiles) return QV2_ERR_SIZE;
     }
-    if (r.range_mode == QV2_PERCENTILE) out->any_percentile = true;
+    if (r.range_mode == QV2_PERCENTILE) {
+      out->any_percentile = true;
+      r.hist_index = out->n_hist++;
+    }
     if (ne > 0) {
       if (!r.per_channel) {
         cut_flat(t, 0, ne, 0, &out->tiles);
@@ -147,52 +149,85 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, void* co
         }
       }
     }
-    if (first_tile >= (1ull << 31)) return QV2_ERR_SIZE;
-    r.tile_first = (uint32_t)first_tile;
-    r.slot_first = 0; r.slot_count = 0;             // filled in below, once the grids are known
-    r.rslot_first = 0; r.rslot_count = 0;
+    if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;
+    tile_cnt[t] = (uint32_t)(out->tiles.size() - first_tile);
+    hist_cnt[t] = (uint32_t)(out->hist_tiles.size() - first_hist);
     out->tensors.push_back(r);
   }
-  if (out->tiles.size() >= (1ull << 31) || out->hist_tiles.size() >= (1ull << 31)) return QV2_ERR_SIZE;
-  // Slots written with plain stores instead of atomics.  In both persistent kernels CTA b walks
-  // tiles b, b+grid, ...; a tensor whose tiles are [first, first+count) is therefore touched by
-  // min(grid, count) CTAs.  The metrics kernel gives each warp of those CTAs one partial-sum slot;
-  // the range kernel gives each of those CTAs one {min,max} slot for per-tensor tensors (a single
-  // group shared by thousands of tiles; per-channel groups are merged with atomics).
-  const uint64_t n_tiles = out->tiles.size();
-  uint64_t mgrid = metrics_cap < 1 ? 1 : metrics_cap, rgrid = range_cap < 1 ? 1 : range_cap;
-  if (mgrid > n_tiles) mgrid = n_tiles ? n_tiles : 1;
-  if (rgrid > n_tiles) rgrid = n_tiles ? n_tiles : 1;
-  uint64_t slots = 0, rslots = 0;
-  for (uint32_t t = 0; t < n; ++t) {
-    TensorRec& r = out->tensors[t];
-    const uint64_t next = (t + 1 < n) ? out->tensors[t + 1].tile_first : n_tiles;
-    const uint64_t cnt = next - r.tile_first;
-    const uint64_t ctas = cnt < mgrid ? cnt : mgrid;
-    if (slots + ctas * kWarps >= (1ull << 32)) return QV2_ERR_SIZE;
-    r.slot_first = (uint32_t)slots;
-    r.slot_count = (uint32_t)(ctas * kWarps);
-    slots += ctas * kWarps;
-    if (!r.per_channel) {
-      const uint64_t rc = cnt < rgrid ? cnt : rgrid;
-      if (rslots + rc >= (1ull << 32)) return QV2_ERR_SIZE;
-      r.rslot_first = (uint32_t)rslots;
-      r.rslot_count = (uint32_t)rc;
-      rslots += rc;
+
+  // Stages: runs of consecutive tensors.  A "resident" stage holds reference tensors of at most
+  // chunk_bytes together; tensors larger than that gather in stages of their own, where a second
+  // pass cannot hit L2 anyway.  Per-group histograms are walked by a separate table that is not
+  // cut into stages, so a plan that has them keeps the single-stage schedule.
+  {
+    const bool chunked = chunk_bytes != 0 && !any_group_pct;
+    Stage st = Stage();
+    uint64_t held = 0;
+    bool open = false, open_big = false;
+    auto close = [&](uint32_t end) { st.tensor_end = end; out->stages.push_back(st); };
+    for (uint32_t t = 0; t < n; ++t) {
+      const TensorRec& r = out->tensors[t];
+      const uint64_t bytes = r.n_elems * dtype_size(r.dtype);
+      const bool big = chunked && bytes > chunk_bytes;
+      const bool fits = open && (!chunked || (big && open_big) || (!big && !open_big && held + bytes <= chunk_bytes));
+      if (open && !fits) { close(t); open = false; }
+      if (!open) { st = Stage(); st.tensor_begin = t; st.l2_resident = chunked && !big; held = 0; open = true; open_big = big; }
+      held += bytes;
     }
+    close(n);
   }
-  out->metrics_grid = (uint32_t)mgrid;
-  out->range_grid = (uint32_t)rgrid;
+
+  // Slots written with plain stores instead of atomics.  In every persistent kernel CTA b walks
+  // tiles b, b+grid, ... of its stage's slice; a tensor whose tiles are [first, first+count) is
+  // therefore touched by min(grid, count) CTAs.  The metrics kernel gives each of those CTAs one
+  // partial-sum slot; the range kernel gives each of them one {min,max} slot for per-tensor
+  // tensors (a single group shared by thousands of tiles; per-channel groups are merged with
+  // atomics).
+  uint64_t slots = 0, rslots = 0, tile_at = 0, hist_at = 0;
+  for (Stage& st : out->stages) {
+    st.tile_begin = (uint32_t)tile_at; st.hist_begin = (uint32_t)hist_at;
+    uint64_t nt = 0, nh = 0;
+    for (uint32_t t = st.tensor_begin; t < st.tensor_end; ++t) { nt += tile_cnt[t]; nh += hist_cnt[t]; }
+    st.tile_end = (uint32_t)(tile_at + nt); st.hist_end = (uint32_t)(hist_at + nh);
+    auto grid_of = [](uint32_t cap, uint64_t tiles) -> uint32_t {
+      uint64_t g = cap < 1 ? 1 : cap;
+      if (g > tiles) g = tiles;
+      return g < 1 ? 1u : (uint32_t)g;
+    };
+    st.range_grid = grid_of(caps.range, nt);
+    st.metrics_grid = grid_of(caps.metrics, nt);
+    st.hist_grid = grid_of(caps.hist, nh);
+    uint64_t rel = 0, hrel = 0;
+    for (uint32_t t = st.tensor_begin; t < st.tensor_end; ++t) {
+      TensorRec& r = out->tensors[t];
+      r.tile_first = (uint32_t)rel; r.hist_tile_first = (uint32_t)hrel;
+      rel += tile_cnt[t]; hrel += hist_cnt[t];
+      r.metrics_ctas = tile_cnt[t] < st.metrics_grid ? tile_cnt[t] : st.metrics_grid;
+      r.range_ctas = tile_cnt[t] < st.range_grid ? tile_cnt[t] : st.range_grid;
+      r.hist_ctas = hist_cnt[t] < st.hist_grid ? hist_cnt[t] : st.hist_grid;
+      if (slots + r.metrics_ctas >= (1ull << 32)) return QV2_ERR_SIZE;
+      r.slot_first = (uint32_t)slots;
+      slots += r.metrics_ctas;
+      if (!r.per_channel) {
+        if (rslots + r.range_ctas >= (1ull << 32)) return QV2_ERR_SIZE;
+        r.rslot_first = (uint32_t)rslots;
+        rslots += r.range_ctas;
+      }
+      if (tile_cnt[t] == 0) st.any_empty = true;
+      if (r.range_mode == QV2_PERCENTILE) st.any_percentile = true;
+    }
+    tile_at += nt; hist_at += nh;
+  }
   out->total_rslots = (uint32_t)rslots;
   out->total_groups = groups;
   out->total_slots = (uint32_t)slots;
   return QV2_OK;
 }
 
-int build_plan(const qv2_tensor_desc* descs, uint32_t n, void* const* codes, uint32_t metrics_cap,
-               uint32_t range_cap, HostPlan* out) {
+int build_plan(const qv2_tensor_desc* descs, uint32_t n, const GridCaps& caps, uint64_t chunk_bytes,
+               HostPlan* out) {
   try {
-    return build_plan_checked(descs, n, codes, metrics_cap, range_cap, out);
+    return build_plan_checked(descs, n, caps, chunk_bytes, out);
   } catch (const std::bad_alloc&) {          // nothing may unwind through the C ABI
     return QV2_ERR_NOMEM;
   }
@@ -219,7 +254,7 @@ extern "C" uint64_t qv2_group_hist_count(const qv2_tensor_desc* descs, uint32_t 
 extern "C" int64_t qv2_debug_plan_tiles(const qv2_tensor_desc* descs, uint32_t n, uint64_t* out,
                                         uint64_t max_tiles) {
   qv2::HostPlan plan;
-  int st = qv2::build_plan(descs, n, nullptr, 1, 1, &plan);
+  int st = qv2::build_plan(descs, n, qv2::GridCaps(), 0, &plan);
   if (st != QV2_OK) return st;
   uint64_t w = 0;
   for (const qv2::Tile& t : plan.tiles) {

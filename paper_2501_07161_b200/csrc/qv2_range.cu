@@ -1,6 +1,6 @@
-// Range calibration: one persistent launch sweeps every tile of every tensor and records the
-// per-group minimum and maximum; a small second kernel turns them into absmax and quantization
-// parameters (step 1 and step 2 of the paper's overview, Eq. 2 and Eq. 4).
+// Range calibration: one persistent launch sweeps every tile of a stage's tensors and records the
+// per-group minimum and maximum; the CTA that finishes a tensor last turns them into absmax and
+// quantization parameters (step 1 and step 2 of the paper's overview, Eq. 2 and Eq. 4).
 //
 // min/max are exact and order-independent, so the per-warp results are merged with integer
 // atomicMax on an order-preserving key; no floating-point atomics are used anywhere.
@@ -157,12 +157,12 @@ __device__ __forceinline__ void range_short_rows_tile(const T* x, const Tile& tl
 // slot (atomics from every warp of every CTA on that single address would serialise).  Per-channel
 // groups are touched by one or two CTAs each and are merged with atomics.
 __device__ __forceinline__ void publish_slot(RangeAcc& a, uint32_t lane, uint32_t warp, const TensorRec* tr,
-                                             uint2* rslots, unsigned long long* nonfinite_t, float* sh) {
+                                             uint2* rslots, unsigned long long* nf_acc_t, float* sh) {
   const float mn = warp_min(a.mn), mx = warp_max(a.mx);
   const uint32_t bad = warp_sum_u32(a.bad);
   if (lane == 0) {
     sh[warp] = mn; sh[kWarps + warp] = mx;
-    if (bad) atomicAdd(nonfinite_t, (unsigned long long)bad);
+    if (bad) atomicAdd(nf_acc_t, (unsigned long long)bad);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -177,166 +177,166 @@ __device__ __forceinline__ void publish_slot(RangeAcc& a, uint32_t lane, uint32_
   __syncthreads();
 }
 
-// ANY16 = false is the build for models whose tensors are all binary32: the element-type dispatch
-// is compiled out, so that common case pays nothing for the 16-bit paths.
-template <bool ANY16>
-__global__ void __launch_bounds__(kThreads, 4)
-range_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ tiles, uint32_t n_tiles,
-             uint32_t* kmin, uint32_t* kmax, uint2* rslots, unsigned long long* nonfinite) {
-  constexpr uint32_t kNone = 0xffffffffu;
-  __shared__ float sh[2 * kWarps];
-  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-  RangeAcc a;
-  reset(a);
-  uint32_t cur_group = kNone, cur_tensor = 0;
-  bool cur_slot = false;           // the pending group belongs to a per-tensor tensor
-  for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
-    const Tile tl = load_tile(tiles, ti);
-    const TensorRec* tr = tensors + tl.tensor;
-    const uint32_t gbase = tr->group_base;
-    if (tl.rows == 0) {
-      const uint32_t G = gbase + (uint32_t)tl.row0;
-      if (G != cur_group) {        // block-uniform: every warp of the CTA takes this branch together
-        if (cur_group != kNone) {
-          if (cur_slot) publish_slot(a, lane, warp, tensors + cur_tensor, rslots, nonfinite + cur_tensor, sh);
-          else publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
-        }
-        reset(a);
-        cur_group = G; cur_tensor = tl.tensor; cur_slot = tr->per_channel == 0;
-      }
-      if (!ANY16 || tr->dtype == kF32) range_flat_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, a);
-      else if (tr->dtype == kF16) range_flat_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, a);
-      else range_flat_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, a);
-    } else if (tr->inner < kShortRow) {
-      if (!ANY16 || tr->dtype == kF32)
-        range_short_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, kmin, kmax, nonfinite);
-      else if (tr->dtype == kF16)
-        range_short_rows_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, lane, kmin, kmax, nonfinite);
-      else
-        range_short_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, kmin, kmax, nonfinite);
-    } else {
-      if (!ANY16 || tr->dtype == kF32)
-        range_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
-      else if (tr->dtype == kF16)
-        range_rows_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
-      else
-        range_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, warp, kmin, kmax, nonfinite);
-    }
-  }
-  if (cur_group != kNone) {
-    if (cur_slot) publish_slot(a, lane, warp, tensors + cur_tensor, rslots, nonfinite + cur_tensor, sh);
-    else publish(a, lane, kmin, kmax, cur_group, nonfinite + cur_tensor);
-  }
-}
-
-// One CTA per tensor: fold the CTA slots of a per-tensor tensor, decode the keys in place, write
-// absmax, the tensor-wide absmax and -- for tensors without percentile clipping -- the
-// quantization parameters.
-// The finalize kernels are chains of dependent global loads: many threads keep the chain short
-// (a tensor with 4096 groups takes 4 rounds instead of 16).
-constexpr int kFinalizeThreads = 1024;
-
-__global__ void __launch_bounds__(kFinalizeThreads)
-range_finalize_kernel(const TensorRec* __restrict__ tensors, const uint2* __restrict__ rslots,
-                      float* gmin, float* gmax, float* gabsmax, float* step, float* inv, float* offset,
-                      float* tensor_absmax, float* clip) {
-  __shared__ float red[kFinalizeThreads];
-  __shared__ uint32_t kred[2][kFinalizeThreads];
-  const TensorRec tr = tensors[blockIdx.x];
-  if (!tr.per_channel) {                 // keys of the single group come from the slots
-    uint32_t kn = 0, kx = 0;             // both arrays hold "larger is better" keys, 0 = empty
-    for (uint32_t k = threadIdx.x; k < tr.rslot_count; k += blockDim.x) {
-      const uint2 v = rslots[tr.rslot_first + k];
+// Folds one tensor once every CTA that owns a tile of it has published: decodes the keys, writes
+// min / max / absmax per group, the tensor-wide absmax, the default clip, the non-finite count
+// and -- for tensors without percentile clipping -- the quantization parameters; then puts every
+// accumulator it consumed back to zero, so that the next pass needs no clearing launch.  Runs in
+// the CTA that drew the tensor's last ticket (or in CTA 0 for a tensor without elements); values
+// written by other CTAs are read through L2.
+__device__ __noinline__ void range_fold_tensor(const CalibArgs& a, uint32_t t) {
+  __shared__ float red[kThreads];
+  __shared__ uint32_t kred[2][kThreads];
+  const TensorRec tr = a.tensors[t];
+  const uint32_t tid = threadIdx.x;
+  if (!tr.per_channel) {                 // keys of the single group come from the CTA slots
+    uint32_t kn = 0, kx = 0;             // both hold "larger is better" keys, 0 = empty
+    for (uint32_t k = tid; k < tr.range_ctas; k += kThreads) {
+      const uint2 v = __ldcg(a.rslots + tr.rslot_first + k);
       kn = max(kn, v.x); kx = max(kx, v.y);
     }
-    kred[0][threadIdx.x] = kn; kred[1][threadIdx.x] = kx;
+    kred[0][tid] = kn; kred[1][tid] = kx;
     __syncthreads();
-    for (uint32_t o = kFinalizeThreads / 2; o > 0; o >>= 1) {
-      if (threadIdx.x < o) {
-        kred[0][threadIdx.x] = max(kred[0][threadIdx.x], kred[0][threadIdx.x + o]);
-        kred[1][threadIdx.x] = max(kred[1][threadIdx.x], kred[1][threadIdx.x + o]);
+    for (uint32_t o = kThreads / 2; o > 0; o >>= 1) {
+      if (tid < o) {
+        kred[0][tid] = max(kred[0][tid], kred[0][tid + o]);
+        kred[1][tid] = max(kred[1][tid], kred[1][tid + o]);
       }
       __syncthreads();
     }
-    if (threadIdx.x == 0) {
-      reinterpret_cast<uint32_t*>(gmin)[tr.group_base] = kred[0][0];
-      reinterpret_cast<uint32_t*>(gmax)[tr.group_base] = kred[1][0];
-    }
-    __syncthreads();
   }
   float amax = 0.0f;
-  for (uint32_t g = threadIdx.x; g < tr.n_groups; g += blockDim.x) {
+  for (uint32_t g = tid; g < tr.n_groups; g += kThreads) {
     const uint32_t G = tr.group_base + g;
-    const uint32_t kn = reinterpret_cast<uint32_t*>(gmin)[G];
-    const uint32_t kx = reinterpret_cast<uint32_t*>(gmax)[G];
+    uint32_t kn, kx;
+    if (tr.per_channel) {
+      kn = __ldcg(a.kmin + G); kx = __ldcg(a.kmax + G);
+      a.kmin[G] = 0u; a.kmax[G] = 0u;                  // ready for the next pass
+    } else {
+      kn = kred[0][0]; kx = kred[1][0];
+    }
     float mn = kn ? key2f(~kn) : 0.0f;
     float mx = kx ? key2f(kx) : 0.0f;
     mn = __fadd_rn(mn, 0.0f);           // -0 -> +0, every other value unchanged
     mx = __fadd_rn(mx, 0.0f);
     const float am = fmaxf(fabsf(mn), fabsf(mx));
-    gmin[G] = mn; gmax[G] = mx; gabsmax[G] = am;
+    a.gmin[G] = mn; a.gmax[G] = mx; a.gabsmax[G] = am;
     amax = fmaxf(amax, am);
     if (tr.range_mode < QV2_PERCENTILE)      // the percentile modes set theirs once the clip is known
-      make_qparams(tr.asym, top_code(tr.asym != 0, tr.bits), false, 0.0f, mn, mx, am, step + G, inv + G, offset + G);
+      make_qparams(tr.asym, top_code(tr.asym != 0, tr.bits), false, 0.0f, mn, mx, am, a.step + G, a.inv + G,
+                   a.offset + G);
   }
-  red[threadIdx.x] = amax;
+  red[tid] = amax;
   __syncthreads();
-  for (uint32_t o = kFinalizeThreads / 2; o > 0; o >>= 1) {
-    if (threadIdx.x < o) red[threadIdx.x] = fmaxf(red[threadIdx.x], red[threadIdx.x + o]);
+  for (uint32_t o = kThreads / 2; o > 0; o >>= 1) {
+    if (tid < o) red[tid] = fmaxf(red[tid], red[tid + o]);
     __syncthreads();
   }
+  if (tid == 0) {
+    a.tensor_absmax[t] = red[0];
+    a.clip[t] = red[0];                 // the percentile pass replaces it for the tensors it clips
+    a.nonfinite[t] = __ldcg(a.nf_acc + t);
+    a.nf_acc[t] = 0ull;
+    a.tickets[t] = 0u;
+  }
+  // the histogram row of a tensor that is not clipped at a per-tensor percentile reads zero
+  if (a.hist && tr.range_mode != QV2_PERCENTILE) {
+    unsigned long long* row = a.hist + (size_t)t * kBins;
+    for (uint32_t b = tid; b < kBins; b += kThreads) row[b] = 0ull;
+  }
+  __syncthreads();                      // the shared arrays may be reused by the next fold
+}
+
+// Called by every CTA when it has published its share of tensor t: the one that draws the last
+// ticket folds the tensor.  Nobody waits.
+__device__ __forceinline__ void range_tensor_done(const CalibArgs& a, uint32_t t, uint32_t* s_last) {
+  __threadfence();                       // this thread's atomics and slot stores are visible ...
+  __syncthreads();
   if (threadIdx.x == 0) {
-    tensor_absmax[blockIdx.x] = red[0];
-    clip[blockIdx.x] = red[0];          // the percentile pass replaces it for the tensors it clips
+    const uint32_t n = a.tensors[t].range_ctas;
+    *s_last = atomicAdd(a.tickets + t, 1u) == n - 1u;     // ... before the ticket is
+  }
+  __syncthreads();
+  if (*s_last) {
+    __threadfence();
+    range_fold_tensor(a, t);
   }
 }
 
-// Everything a calibration pass accumulates into starts at zero: the min/max keys (0 = nothing
-// seen), the non-finite counters and the per-tensor histograms.  One small kernel instead of four
-// memsets: a pass over a small model is bound by the number of stream operations.
-__global__ void __launch_bounds__(256)
-calib_init_kernel(uint32_t* kmin, uint32_t* kmax, size_t groups, unsigned long long* nonfinite, size_t n_tensors,
-                  unsigned long long* hist, size_t hist_cells) {
-  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
-  for (size_t i = tid; i < groups; i += stride) { kmin[i] = 0u; kmax[i] = 0u; }
-  for (size_t i = tid; i < n_tensors; i += stride) nonfinite[i] = 0ull;
-  for (size_t i = tid; i < hist_cells; i += stride) hist[i] = 0ull;
+// ANY16 = false is the build for models whose tensors are all binary32: the element-type dispatch
+// is compiled out, so that common case pays nothing for the 16-bit paths.
+template <bool ANY16>
+__global__ void __launch_bounds__(kThreads, 4)
+range_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles, uint32_t n_tiles,
+             uint32_t scan_begin, uint32_t scan_end) {
+  constexpr uint32_t kNone = 0xffffffffu;
+  __shared__ float sh[2 * kWarps];
+  __shared__ uint32_t s_last;
+  const TensorRec* __restrict__ tensors = a.tensors;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  // tensors without elements are owned by no CTA: CTA 0 folds them (the planner asks for the
+  // scan only when the stage has one)
+  if (blockIdx.x == 0)
+    for (uint32_t t = scan_begin; t < scan_end; ++t)
+      if (tensors[t].range_ctas == 0) range_fold_tensor(a, t);
+  RangeAcc acc;
+  reset(acc);
+  uint32_t cur_group = kNone, cur_tensor = kNone;
+  bool cur_slot = false;           // the pending group belongs to a per-tensor tensor
+  auto flush_group = [&]() {
+    if (cur_group == kNone) return;
+    if (cur_slot) publish_slot(acc, lane, warp, tensors + cur_tensor, a.rslots, a.nf_acc + cur_tensor, sh);
+    else publish(acc, lane, a.kmin, a.kmax, cur_group, a.nf_acc + cur_tensor);
+    cur_group = kNone;
+  };
+  for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+    const Tile tl = load_tile(tiles, ti);
+    const TensorRec* tr = tensors + tl.tensor;
+    if (tl.tensor != cur_tensor) {   // block-uniform: every warp of the CTA takes these branches together
+      if (cur_tensor != kNone) { flush_group(); range_tensor_done(a, cur_tensor, &s_last); }
+      cur_tensor = tl.tensor;
+    }
+    const uint32_t gbase = tr->group_base;
+    if (tl.rows == 0) {
+      const uint32_t G = gbase + (uint32_t)tl.row0;
+      if (G != cur_group) {
+        flush_group();
+        reset(acc);
+        cur_group = G; cur_slot = tr->per_channel == 0;
+      }
+      if (!ANY16 || tr->dtype == kF32) range_flat_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl.count, acc);
+      else if (tr->dtype == kF16) range_flat_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl.count, acc);
+      else range_flat_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, acc);
+    } else if (tr->inner < kShortRow) {
+      if (!ANY16 || tr->dtype == kF32)
+        range_short_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, a.kmin, a.kmax, a.nf_acc);
+      else if (tr->dtype == kF16)
+        range_short_rows_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, lane, a.kmin, a.kmax, a.nf_acc);
+      else
+        range_short_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, a.kmin, a.kmax, a.nf_acc);
+    } else {
+      if (!ANY16 || tr->dtype == kF32)
+        range_rows_tile(reinterpret_cast<const float*>(tr->x) + tl.begin, tl, tr, lane, warp, a.kmin, a.kmax, a.nf_acc);
+      else if (tr->dtype == kF16)
+        range_rows_tile(reinterpret_cast<const __half*>(tr->x) + tl.begin, tl, tr, lane, warp, a.kmin, a.kmax, a.nf_acc);
+      else
+        range_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, warp, a.kmin, a.kmax, a.nf_acc);
+    }
+  }
+  if (cur_tensor != kNone) { flush_group(); range_tensor_done(a, cur_tensor, &s_last); }
 }
 
 }  // namespace
 
-cudaError_t launch_calib_init(const Launch& l, uint32_t* kmin, uint32_t* kmax, size_t groups,
-                              unsigned long long* nonfinite, size_t n_tensors, unsigned long long* hist,
-                              size_t hist_cells) {
-  size_t most = groups > hist_cells ? groups : hist_cells;
-  if (n_tensors > most) most = n_tensors;
-  size_t grid = (most + 255) / 256;
-  const size_t cap = (size_t)l.sm_count * 8;
-  if (grid > cap) grid = cap;
-  if (grid < 1) grid = 1;
-  calib_init_kernel<<<(unsigned)grid, 256, 0, l.stream>>>(kmin, kmax, groups, nonfinite, n_tensors, hist, hist_cells);
-  return cudaGetLastError();
-}
-
 uint32_t range_grid_cap(int sm_count) {
-  static int per_sm = 0;
-  return (uint32_t)persistent_grid((const void*)range_kernel<false>, &per_sm, sm_count, 0x7fffffffu);
+  int cache = 0;
+  return (uint32_t)persistent_grid((const void*)range_kernel<false>, &cache, sm_count, 0x7fffffffu);
 }
 
-cudaError_t launch_range(const Launch& l, uint32_t grid, bool any16, const TensorRec* tensors, const Tile* tiles,
-                         uint32_t n_tiles, uint32_t* kmin, uint32_t* kmax, uint2* rslots,
-                         unsigned long long* nonfinite) {
-  if (n_tiles == 0) return cudaSuccess;
-  if (any16) range_kernel<true><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, rslots, nonfinite);
-  else range_kernel<false><<<grid, kThreads, 0, l.stream>>>(tensors, tiles, n_tiles, kmin, kmax, rslots, nonfinite);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_range_finalize(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,
-                                  const uint2* rslots, float* gmin, float* gmax, float* gabsmax,
-                                  float* step, float* inv, float* offset, float* tensor_absmax, float* clip) {
-  range_finalize_kernel<<<n_tensors, kFinalizeThreads, 0, l.stream>>>(tensors, rslots, gmin, gmax, gabsmax, step,
-                                                         inv, offset, tensor_absmax, clip);
+cudaError_t launch_range(const Launch& l, const Stage& st, bool any16, const Tile* tiles, const CalibArgs& a) {
+  const uint32_t n_tiles = st.tile_end - st.tile_begin;
+  const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
+  if (any16) range_kernel<true><<<st.range_grid, kThreads, 0, l.stream>>>(a, tiles + st.tile_begin, n_tiles, s0, s1);
+  else range_kernel<false><<<st.range_grid, kThreads, 0, l.stream>>>(a, tiles + st.tile_begin, n_tiles, s0, s1);
   return cudaGetLastError();
 }
 

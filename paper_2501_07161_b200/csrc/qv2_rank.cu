@@ -85,8 +85,11 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
   }
   __syncthreads();
   // Position of layer i = number of layers that come before it: all MSE outliers precede the
-  // rest; outliers by descending severity, the rest by ascending score, ties by layer index.
+  // rest; outliers by descending severity (or, in the literal reading of the pseudo-code, where
+  // each outlier is put at the head of the list when the layer loop meets it, in reverse layer
+  // order), the rest by ascending score, ties by layer index.
   const double fac = cfg.mse_factor;
+  const bool literal = cfg.outlier_order == QV2_OUTLIERS_LITERAL;
   for (uint32_t i = tid; i < n; i += blockDim.x) {
     const double si = sc[i], vi = sv[i];
     const bool out_i = vi > fac;
@@ -95,7 +98,7 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
       const double vj = sv[j];
       const bool out_j = vj > fac;
       if (out_i) {
-        if (out_j && (vj > vi || (vj == vi && j < i))) ++rank;
+        if (out_j && (literal ? j > i : (vj > vi || (vj == vi && j < i)))) ++rank;
       } else {
         if (out_j) ++rank;
         else {

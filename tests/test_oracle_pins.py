@@ -352,6 +352,51 @@ def test_rank_hand_worked_six_layers():
     assert order.tolist()[:2] == [2, 3]
 
 
+def test_rank_literal_outlier_order_of_algorithm_2():
+    """Algorithm 2, RankLayersBySensitivity, as printed: the layer loop inserts every layer whose
+    MSE exceeds 5x the mean at the HEAD of the list when it meets it, so among the outliers the
+    one met last stands first (reverse layer order), whatever their severities."""
+    sw = [40.0, 35.0, 37.0, 36.0, 42.0, 34.0, 33.0, 39.0]
+    sa = [30.0, 31.0, 27.0, 30.0, 28.0, 29.0, 30.0, 31.0]
+    # three large weight MSEs among eight layers, none above 5x the mean
+    mw = [1.0, 80.0, 1.0, 1.0, 100.0, 1.0, 90.0, 1.0]    # mean 34.375; ratios 2.33, 2.91, 2.62: none > 5
+    ma = [1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0]
+    o_sev, _, _ = oracle.rank_layers(sw, mw, sa, ma)
+    o_lit, _, _ = oracle.rank_layers(sw, mw, sa, ma, outlier_order=1)
+    assert o_sev.tolist() == o_lit.tolist()              # no outlier: the two readings coincide
+    # 20 layers so that three large MSEs exceed 5x the mean: mean = (17 + 300 + 500 + 400)/20 = 60.85
+    n = 20
+    sw = [40.0 - 0.5 * i for i in range(n)]              # all deltas equal: the rest keeps layer order
+    sa = [30.0] * n
+    mw = [1.0] * n
+    mw[3], mw[9], mw[14] = 400.0, 500.0, 310.0           # ratios 6.57, 8.22, 5.09
+    ma = [1.0] * n
+    o_sev, _, _ = oracle.rank_layers(sw, mw, sa, ma)
+    o_lit, k_lit, nk = oracle.rank_layers(sw, mw, sa, ma, outlier_order=1, keep_count=2)
+    rest = [i for i in range(n) if i not in (3, 9, 14)]
+    # layer 0 has delta 0, the others -0.5*2 = -1: they precede it
+    rest_sorted = [i for i in rest if i != 0] + [0]
+    assert o_sev.tolist() == [9, 3, 14] + rest_sorted    # by severity
+    assert o_lit.tolist() == [14, 9, 3] + rest_sorted    # as printed: last met, first in the list
+    assert nk == 2 and k_lit[14] == 1 and k_lit[9] == 1 and k_lit.sum() == 2
+    # brute force: simulate the printed loop with a Python list on random inputs
+    for _ in range(200):
+        n = int(RNG.integers(1, 12))
+        sw = RNG.uniform(-10, 60, n).round(1); sa = RNG.uniform(-10, 60, n).round(1)
+        mw = RNG.choice([1e-6, 1e-6, 1e-6, 5e-4], n); ma = RNG.choice([1e-3, 1e-3, 1e-3, 1e-3, 9e-2], n)
+        base = _py_rank(list(sw), list(mw), list(sa), list(ma))
+        mean_w, mean_a = sum(mw) / n, sum(ma) / n
+        sev = [max(mw[i] / mean_w, ma[i] / mean_a) for i in range(n)]
+        lst = [i for i in base if not sev[i] > 5.0]      # L_sqnr: the non-outliers by ascending score
+        for i in range(n):                               # the printed loop
+            if sev[i] > 5.0:
+                lst.insert(0, i)
+        got, _, _ = oracle.rank_layers(sw, mw, sa, ma, outlier_order=1)
+        assert got.tolist() == lst
+        gf, _, _ = oracle.rank_layers_fused(sw, mw, sa, ma, None, outlier_order=1)
+        assert gf.tolist() == lst
+
+
 def test_rank_degenerate_variants_of_the_ablation():
     n = 12
     sw = RNG.uniform(20, 50, n); sa = RNG.uniform(20, 50, n)
