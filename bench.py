@@ -52,6 +52,15 @@ def parse():
     ap.add_argument("--act-granularity", default="tensor", choices=["tensor", "channel"],
                     help="channel: activations quantized per channel, each channel with its own percentile clip "
                          "(a variant; the paper's set-ups and the headline number are per tensor)")
+    ap.add_argument("--schedule", default="phase", choices=["phase", "chunked", "auto"],
+                    help="phase: one launch per phase over the whole model (default); chunked: stage by stage so that "
+                         "re-reads hit L2 (qv2_set_schedule); auto: the library decides by size")
+    ap.add_argument("--chunk-mb", type=float, default=0.0, help="chunk size of the chunked schedule (0: library default)")
+    ap.add_argument("--fold", default="auto", choices=["auto", "fused", "separate"],
+                    help="where per-tensor partial results are folded (qv2_set_fold_mode)")
+    ap.add_argument("--api", default=None, choices=["calls", "sweep"],
+                    help="calls: qv2_calibrate + qv2_quant_metrics + qv2_rank_layers (default for the phase-major "
+                         "schedule); sweep: the chained qv2_sweep_model (default otherwise; per-phase times are then not available)")
     ap.add_argument("--graph", action="store_true",
                     help="capture one pass in a CUDA graph and time its replays (per-phase times are then not available)")
     return ap.parse_args()
@@ -264,6 +273,10 @@ def ours_main(args):
     stream = torch.cuda.Stream() if args.graph else torch.cuda.current_stream()
     torch.cuda.set_stream(stream)
     ctx = q.Context(local, stream=stream)
+    sched = {"phase": q.SCHEDULE_PHASE_MAJOR, "chunked": q.SCHEDULE_L2_CHUNKED, "auto": q.SCHEDULE_AUTO}[args.schedule]
+    ctx.set_schedule(sched, int(args.chunk_mb * (1 << 20)))
+    ctx.set_fold_mode({"auto": q.FOLD_AUTO, "fused": q.FOLD_FUSED, "separate": q.FOLD_SEPARATE}[args.fold])
+    api = args.api or ("calls" if args.schedule == "phase" else "sweep")
     md = q.model_descs(model, act_granularity=args.act_granularity)
     n, L = md.n_tensors, md.n_layers
     rcfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
@@ -277,7 +290,13 @@ def ours_main(args):
     h = ctx._h
 
     def one_step(ev=None):
-        """The three calls of the contract, back to back on the context's stream."""
+        """The three calls of the contract, back to back on the context's stream (or the chained call)."""
+        if api == "sweep":
+            if ev: ev[0].record()
+            ctx.sweep_model(md.descs, L, md.macs, None, rcfg, sb)
+            if ev:
+                for e in ev[1:]: e.record()
+            return
         if ev: ev[0].record()
         st = lib.qv2_calibrate(h, md.descs, n, *[t[k].data_ptr() for k in
                                ("gmin", "gmax", "gabsmax", "hist", "clip", "step", "inv", "offset", "nonfinite")])
@@ -319,7 +338,7 @@ def ours_main(args):
     step_ms = sorted(e[0].elapsed_time(e[3]) for e in evs)
     clocks = sampler.summary(t_wall0, t_wall1)
 
-    launch_mode = "one C-ABI call per phase"
+    launch_mode = "one C-ABI call per phase" if api == "calls" else "qv2_sweep_model"
     if args.graph:       # headline from replays of one captured pass; phase times stay from the loop above
         g = ctx.sweep_graph(md.descs, L, md.macs, None, rcfg, sb)     # qv2_sweep_graph_create
         for _ in range(3):
@@ -398,7 +417,7 @@ def ours_main(args):
 
     if rank == 0:
         peak, peak_src = measured_peak()
-        achieved = metrics_bytes / (met_ms * 1e-3) / 1e9
+        achieved = metrics_bytes / (met_ms * 1e-3) / 1e9 if met_ms > 1e-6 else None   # no per-phase time with --api sweep
         # the capture was taken on the default workload; DRAM traffic is reported for it only
         ratio = recorded_traffic() if (args.workload == "vgg16" and batch == cfgw.batch and esz == 4
                                          and args.act_granularity == "tensor") else None
@@ -414,14 +433,14 @@ def ours_main(args):
                        "l2": "inputs larger than L2 (no flush needed)" if 4 * (w_elems + 2 * a_elems) > 4 * 126e6
                              else "inputs fit in L2: this is an L2 number, not an HBM one",
                        "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
-                       "launch": launch_mode,
+                       "launch": launch_mode, "schedule": args.schedule, "stages": ctx.stages, "api": api, "fold": args.fold,
                        "seed": 0},
             "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_min": step_ms[0],
             "phases_ms": {"calibrate": cal_ms, "quant_metrics": met_ms, "rank": rank_ms},
             "frac_of_measured_copy_peak": value / world / peak,
             "frac_of_8000_nominal": value / world / 8000.0,
             "roofline": {"kernel": "metrics_kernel (qv2_quant_metrics)", "bound": "hbm",
-                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak if achieved else None,
                          "traffic": traffic, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": metrics_bytes,
                          "duration_ms": met_ms,

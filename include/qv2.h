@@ -21,9 +21,10 @@
  *     and qv2_check_nonfinite synchronise before they return.  qv2_sync_count reports how often
  *     a context has done so.
  *   - Accumulators that must start at zero (range keys, counters, histograms, tickets) live in
- *     context scratch and are put back to zero by the kernel that consumes them, so a pass needs
- *     no clearing launch.  Partial results of a tensor are folded by whichever thread block
- *     finishes the tensor last, found with an atomic counter; no block ever waits for another.
+ *     context scratch and are put back to zero by the code that consumes them, so a pass needs
+ *     no clearing launch.  Partial results of a tensor are folded either by whichever thread
+ *     block finishes the tensor last, found with an atomic counter, or by a small follow-up
+ *     kernel (qv2_set_fold_mode); no block ever waits for another.
  *   - One context serves one stream; use it from one host thread at a time.
  *   - Tensors are fp32, contiguous, viewed as [outer][channels][inner]; element (o,c,i) lives at
  *     index (o*channels + c)*inner + i.  Weights: outer = 1, channels = C_out, inner = C_in/g*k*k.
@@ -63,6 +64,7 @@ enum { QV2_PAIR_REQUANT = 0, QV2_PAIR_RAW = 1, QV2_STORE_CODES = 2 }; /* flags (
 enum { QV2_BY_COUNT = 0, QV2_BY_BOPS_RATE = 1 };             /* select_mode */
 enum { QV2_OUTLIERS_BY_SEVERITY = 0, QV2_OUTLIERS_LITERAL = 1 }; /* outlier_order */
 enum { QV2_SCHEDULE_PHASE_MAJOR = 0, QV2_SCHEDULE_L2_CHUNKED = 1, QV2_SCHEDULE_AUTO = 2 };
+enum { QV2_FOLD_AUTO = 0, QV2_FOLD_FUSED = 1, QV2_FOLD_SEPARATE = 2 };
 /* Code width other than 8 bits, OR-ed into qv2_tensor_desc.flags: QV2_BITS(b), 2 <= b <= 16.  The
  * largest code is 2^(b-1) - 1 for QV2_SYM_I8 (Eq. 4) and 2^b - 1 for QV2_ASYM_U8 (Eq. 2 with
  * N = 2^b levels); wherever this header says 127 or 255 read that value.  No QV2_BITS means 8.
@@ -161,6 +163,18 @@ uint64_t qv2_sync_count(const qv2_ctx* ctx);
  * Takes effect with the next call; QV2_ERR_UNSUPPORTED while a captured pass of this context lives.
  */
 int qv2_set_schedule(qv2_ctx* ctx, uint32_t schedule, uint64_t chunk_bytes);
+/*
+ * Where a tensor's partial results (per-block ranges, histogram counts, partial sums) are folded
+ * into its outputs.  QV2_FOLD_SEPARATE: by a small kernel after each streaming kernel (one block
+ * per tensor); the streaming kernels then carry no fold code, no fences and no per-tensor
+ * barriers.  QV2_FOLD_FUSED: inside the streaming kernel, by the block that finishes the tensor
+ * last (found with an atomic ticket; nobody waits) -- one launch per phase instead of two, paid
+ * for with a barrier per tensor and block.  QV2_FOLD_AUTO (default) currently always takes the
+ * separate form, which measured faster on every workload from 62 MB to 15 GB; the fused form is
+ * kept for callers to whom the number of launches matters more.  The outputs do not depend on
+ * the choice.  QV2_ERR_UNSUPPORTED while a captured pass of this context lives.
+ */
+int qv2_set_fold_mode(qv2_ctx* ctx, uint32_t mode);
 /* Number of stages of the context's current plan (1 for phase-major; 0 before the first call). */
 uint32_t qv2_stage_count(const qv2_ctx* ctx);
 /* Sum over descs of the number of quantization groups (1 or `channels`).  Host only. */

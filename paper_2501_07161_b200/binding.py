@@ -20,6 +20,7 @@ PAIR_REQUANT, PAIR_RAW, STORE_CODES = 0, 1, 2
 BY_COUNT, BY_BOPS_RATE = 0, 1
 OUTLIERS_BY_SEVERITY, OUTLIERS_LITERAL = 0, 1
 SCHEDULE_PHASE_MAJOR, SCHEDULE_L2_CHUNKED, SCHEDULE_AUTO = 0, 1, 2
+FOLD_AUTO, FOLD_FUSED, FOLD_SEPARATE = 0, 1, 2
 IN_F32, IN_F16, IN_BF16 = 0, 1 << 16, 2 << 16
 _DTYPE_FLAG = {torch.float32: IN_F32, torch.float16: IN_F16, torch.bfloat16: IN_BF16}
 HIST_BINS = 2048
@@ -30,7 +31,7 @@ EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_erro
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
            "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm", "qv2_sweep_graph_create", "qv2_sweep_graph_launch",
            "qv2_sweep_graph_destroy", "qv2_check_nonfinite", "qv2_calibrate_ex", "qv2_group_hist_count",
-           "qv2_sync_count", "qv2_set_schedule", "qv2_stage_count"]
+           "qv2_sync_count", "qv2_set_schedule", "qv2_stage_count", "qv2_set_fold_mode"]
 KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
@@ -81,6 +82,7 @@ def lib() -> C.CDLL:
     L.qv2_sync_count.argtypes = [vp]; L.qv2_sync_count.restype = u64
     L.qv2_set_schedule.argtypes = [vp, u32, u64]; L.qv2_set_schedule.restype = i32
     L.qv2_stage_count.argtypes = [vp]; L.qv2_stage_count.restype = u32
+    L.qv2_set_fold_mode.argtypes = [vp, u32]; L.qv2_set_fold_mode.restype = i32
     L.qv2_group_count.argtypes = [dp, u32]; L.qv2_group_count.restype = u64
     L.qv2_calibrate.argtypes = [vp, dp, u32] + [vp] * 9; L.qv2_calibrate.restype = i32
     L.qv2_calibrate_ex.argtypes = [vp, dp, u32] + [vp] * 11; L.qv2_calibrate_ex.restype = i32
@@ -227,6 +229,9 @@ class Context:
 
     def set_schedule(self, schedule: int, chunk_bytes: int = 0):
         _check(lib().qv2_set_schedule(self._h, schedule, chunk_bytes), "qv2_set_schedule")
+
+    def set_fold_mode(self, mode: int):
+        _check(lib().qv2_set_fold_mode(self._h, mode), "qv2_set_fold_mode")
 
     def last_cuda_error(self) -> int:
         return int(lib().qv2_last_cuda_error(self._h))

@@ -33,6 +33,7 @@ struct qv2_ctx {
   bool log = false;            // QV2_LOG=1: one line per call on stderr
   uint32_t schedule = QV2_SCHEDULE_PHASE_MAJOR;
   uint64_t chunk_bytes = kDefaultChunkBytes;
+  uint32_t fold_mode = QV2_FOLD_AUTO;
 
   // cached plan: rebuilt only when the descriptor bytes or the schedule change
   HostPlan plan;
@@ -172,16 +173,17 @@ int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n) {
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   const size_t dbytes = (size_t)n * sizeof(qv2_tensor_desc);
   const uint64_t chunk = plan_chunk_bytes(c, descs, n);
-  std::vector<uint8_t> key(dbytes + sizeof(chunk));
+  std::vector<uint8_t> key(dbytes + sizeof(chunk) + sizeof(c->fold_mode));
   std::memcpy(key.data(), descs, dbytes);
   std::memcpy(key.data() + dbytes, &chunk, sizeof(chunk));
+  std::memcpy(key.data() + dbytes + sizeof(chunk), &c->fold_mode, sizeof(c->fold_mode));
   if (c->plan_valid && key == c->plan_key) return QV2_OK;
   // A captured pass replays with the tile tables and scratch addresses of the plan it was
   // captured with; another descriptor set would overwrite them under it.
   if (c->live_graphs) return QV2_ERR_UNSUPPORTED;
 
   HostPlan plan;
-  int st = build_plan(descs, n, c->caps, chunk, &plan);
+  int st = build_plan(descs, n, c->caps, chunk, c->fold_mode, &plan);
   if (st != QV2_OK) return st;
   // The previous upload may still be reading the pinned buffer, and buffers may be reallocated.
   if ((st = sync_stream(c)) != QV2_OK) return st;
@@ -261,18 +263,22 @@ MetricsArgs metrics_args(qv2_ctx* c, const float* step, const float* inv, const 
 // Range and histogram phases of one stage.
 int run_calib_stage(qv2_ctx* c, const Stage& st, const CalibArgs& a) {
   const Launch l = launch_of(c);
+  // a stage that folds in its streaming kernels is one launch per phase; otherwise the streaming
+  // kernel (when the stage has tiles) and a fold kernel
+  const uint64_t per_range = st.fused_fold ? 1 : (st.tile_end > st.tile_begin ? 2 : 1);
+  const uint64_t per_hist = st.fused_fold ? 1 : (st.hist_end > st.hist_begin ? 2 : 1);
   QV2_CUDA(c, launch_range(l, st, c->plan.any_16bit, c->d_tiles, a));
-  ++c->launches;
+  c->launches += per_range;
   if (st.any_percentile) {
     QV2_CUDA(c, launch_hist(l, st, c->plan.any_16bit, c->d_hist_tiles, a));
-    ++c->launches;
+    c->launches += per_hist;
   }
   return QV2_OK;
 }
 
 int run_metrics_stage(qv2_ctx* c, const Stage& st, const MetricsArgs& a) {
   QV2_CUDA(c, launch_metrics(launch_of(c), st, c->plan.any_16bit, c->d_tiles, a));
-  ++c->launches;
+  c->launches += st.fused_fold ? 1 : (st.tile_end > st.tile_begin ? 2 : 1);
   return QV2_OK;
 }
 
@@ -362,9 +368,12 @@ extern "C" int qv2_create(qv2_ctx** out, int device, void* stream) {
   if (e != cudaSuccess) { delete c; return e == cudaErrorMemoryAllocation ? QV2_ERR_NOMEM : QV2_ERR_CUDA; }
   c->sm_count = sms > 0 ? sms : 1;
   // occupancy of each persistent kernel on THIS device (two contexts on different GPUs differ)
-  c->caps.range = range_grid_cap(c->sm_count);
-  c->caps.hist = hist_grid_cap(c->sm_count);
-  c->caps.metrics = metrics_grid_cap(c->sm_count);
+  c->caps.range = range_grid_cap(c->sm_count, false);
+  c->caps.hist = hist_grid_cap(c->sm_count, false);
+  c->caps.metrics = metrics_grid_cap(c->sm_count, false);
+  c->caps.range_fused = range_grid_cap(c->sm_count, true);
+  c->caps.hist_fused = hist_grid_cap(c->sm_count, true);
+  c->caps.metrics_fused = metrics_grid_cap(c->sm_count, true);
   c->caps.ghist = group_hist_grid_cap(c->sm_count);
   c->caps.kl = kl_grid_cap(c->sm_count);
   const char* lg = std::getenv("QV2_LOG");
@@ -401,6 +410,14 @@ extern "C" int qv2_set_schedule(qv2_ctx* c, uint32_t schedule, uint64_t chunk_by
   if (c->live_graphs) return QV2_ERR_UNSUPPORTED;     // a captured pass replays the schedule it was captured with
   c->schedule = schedule;
   c->chunk_bytes = chunk_bytes ? chunk_bytes : kDefaultChunkBytes;
+  return QV2_OK;
+}
+
+extern "C" int qv2_set_fold_mode(qv2_ctx* c, uint32_t mode) {
+  if (!c) return QV2_ERR_NULL;
+  if (mode > QV2_FOLD_SEPARATE) return QV2_ERR_ARG;
+  if (c->live_graphs) return QV2_ERR_UNSUPPORTED;
+  c->fold_mode = mode;
   return QV2_OK;
 }
 

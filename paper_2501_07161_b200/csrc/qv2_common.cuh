@@ -87,11 +87,22 @@ struct Stage {
   bool any_empty;                         // some tensor of the stage has no element (no CTA owns it)
   bool any_percentile;                    // some tensor of the stage is clipped at its percentile
   bool l2_resident;                       // the stage's reference tensors fit the chunk budget
+  bool fused_fold;                        // small stage: the streaming kernels fold each tensor themselves (the CTA
+                                          // that finishes it last); large stage: lean streaming kernels, each
+                                          // followed by a small fold kernel with one CTA per tensor
 };
+// QV2_FOLD_AUTO takes the fused fold for stages that sweep at most this many bytes per phase.
+// Zero: never.  Measured on a B200, the fused kernels lose more at their per-tensor barriers (every
+// warp of a CTA drains its loads before the CTA publishes, 560 against 86 barrier-stall samples in
+// the range kernel on ResNet-18 shapes) than the saved launches return, even for a 62 MB model
+// replayed from a CUDA graph (30.8 against 28.7 us); the mode stays available on request.
+constexpr uint64_t kFusedFoldMaxBytes = 0;
 
 // Largest useful grid of each persistent kernel on the context's device (resident CTAs per SM x SMs).
+// The streaming kernels come in two builds with different register counts (fold inside or not).
 struct GridCaps {
   uint32_t range = 1, hist = 1, metrics = 1, ghist = 1, kl = 1;
+  uint32_t range_fused = 1, hist_fused = 1, metrics_fused = 1;
 };
 
 struct HostPlan {
@@ -113,8 +124,9 @@ struct HostPlan {
 // phase-major schedule (one stage); otherwise consecutive tensors are grouped into stages whose
 // reference tensors hold at most chunk_bytes (a larger tensor gets a stage of its own kind).
 // Returns a QV2 status.
+// fold_mode: QV2_FOLD_AUTO decides per stage by its size, QV2_FOLD_FUSED / QV2_FOLD_SEPARATE force it.
 int build_plan(const qv2_tensor_desc* descs, uint32_t n, const GridCaps& caps, uint64_t chunk_bytes,
-               HostPlan* out);
+               uint32_t fold_mode, HostPlan* out);
 
 // ------------------------------------------------------------------------------------------------
 // Launch wrappers (defined next to their kernels).  All enqueue on `stream` and return the
@@ -144,10 +156,10 @@ struct CalibArgs {
 
 cudaError_t launch_range(const Launch& l, const Stage& st, bool any16, const Tile* tiles, const CalibArgs& a);
 cudaError_t launch_hist(const Launch& l, const Stage& st, bool any16, const Tile* hist_tiles, const CalibArgs& a);
-uint32_t range_grid_cap(int sm_count);     // resident CTAs per SM x SMs
-uint32_t hist_grid_cap(int sm_count);
+uint32_t range_grid_cap(int sm_count, bool fused);     // resident CTAs per SM x SMs
+uint32_t hist_grid_cap(int sm_count, bool fused);
 uint32_t group_hist_grid_cap(int sm_count);
-uint32_t metrics_grid_cap(int sm_count);
+uint32_t metrics_grid_cap(int sm_count, bool fused);
 uint32_t kl_grid_cap(int sm_count);
 
 cudaError_t launch_group_hist(const Launch& l, uint32_t grid_cap, bool any16, const TensorRec* tensors,

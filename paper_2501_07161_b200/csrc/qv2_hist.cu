@@ -132,31 +132,47 @@ __device__ __noinline__ void clip_fold_tensor(const CalibArgs& a, uint32_t t) {
   __syncthreads();                           // the shared arrays may be reused by the next fold
 }
 
-template <bool ANY16>      // false: every tensor is binary32, no element-type dispatch
+// ANY16 = false: every tensor is binary32, no element-type dispatch.  FOLD as in range_kernel:
+// true folds in the CTA that merges a tensor last, false leaves it to clip_fold_kernel.
+template <bool ANY16, bool FOLD>
 __global__ void __launch_bounds__(kThreads, 4)
-hist_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles, uint32_t n_tiles,
-            uint32_t scan_begin, uint32_t scan_end) {
+hist_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ tensors,
+            const Tile* __restrict__ tiles, uint32_t n_tiles, uint32_t scan_begin, uint32_t scan_end) {
   __shared__ uint32_t sh[kBins];
   __shared__ uint32_t s_last;
-  const TensorRec* __restrict__ tensors = a.tensors;
   for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
   __syncthreads();
   // percentile tensors without elements are owned by no CTA: CTA 0 folds them
-  if (blockIdx.x == 0)
+  if (FOLD && blockIdx.x == 0)
     for (uint32_t t = scan_begin; t < scan_end; ++t)
       if (tensors[t].range_mode == QV2_PERCENTILE && tensors[t].hist_ctas == 0) clip_fold_tensor(a, t);
 
-  uint32_t cur = 0xffffffffu, since_flush = 0, zeros = 0;
+  constexpr uint32_t kNone = 0xffffffffu;
+  uint32_t cur = kNone, since_flush = 0, zeros = 0;
+  uint32_t owed = kNone, drawn = 0;   // FOLD: the tensor before cur and the ticket thread 0 drew for it
   float w = 0.0f;
   bool careful = false;
+  // Ticket protocol of the fused fold: after a tensor's merge (and a barrier), thread 0 fences and
+  // draws the tensor's ticket without looking at the result; the CTA looks at it at its next
+  // tensor boundary and folds the tensor if the ticket was the last one.  The atomic's round
+  // trip hides behind the next tensor's stream; nobody waits for another CTA.
+  auto settle = [&](uint32_t t) {
+    if (threadIdx.x == 0) {
+      const bool last = drawn == tensors[t].hist_ctas - 1u;
+      if (last) __threadfence();
+      s_last = last;
+    }
+    __syncthreads();
+    if (s_last) clip_fold_tensor(a, t);
+  };
   for (uint32_t ti = blockIdx.x;; ti += gridDim.x) {
     const bool more = ti < n_tiles;
     Tile tl;
     if (more) tl = load_tile(tiles, ti);
     // merge into the accumulation histogram when the tensor changes, at the end, and before a
     // 32-bit count could overflow (2^14 tiles of 2^14 elements)
-    const bool leaving = cur != 0xffffffffu && (!more || tl.tensor != cur);
-    if (leaving || (cur != 0xffffffffu && since_flush >= 16384u)) {
+    const bool leaving = cur != kNone && (!more || tl.tensor != cur);
+    if (leaving || (cur != kNone && since_flush >= 16384u)) {
       if (zeros) atomicAdd(sh, zeros);
       zeros = 0;
       __syncthreads();
@@ -165,21 +181,18 @@ hist_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles,
         const uint32_t c = sh[b];
         if (c) { atomicAdd(h + b, (unsigned long long)c); sh[b] = 0; }
       }
+      __syncthreads();
       since_flush = 0;
-      if (leaving) {                  // the CTA that merges a tensor last folds it; nobody waits
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) s_last = atomicAdd(a.hist_tickets + cur, 1u) == tensors[cur].hist_ctas - 1u;
-        __syncthreads();
-        if (s_last) {
-          __threadfence();
-          clip_fold_tensor(a, cur);
-        }
-      } else {
-        __syncthreads();
+      if (FOLD && leaving) {
+        if (owed != kNone) settle(owed);
+        if (threadIdx.x == 0) { __threadfence(); drawn = atomicAdd(a.hist_tickets + cur, 1u); }
+        owed = cur;
       }
     }
-    if (!more) break;
+    if (!more) {
+      if (FOLD && owed != kNone) settle(owed);
+      break;
+    }
     if (tl.tensor != cur) {
       cur = tl.tensor;
       const float A = a.tensor_absmax[cur];
@@ -193,6 +206,13 @@ hist_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles,
     else hist_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl.count, w, careful, sh, zeros);
     ++since_flush;
   }
+}
+
+// One CTA per tensor of the stage: the fold, for stages whose streaming kernel does not fold.
+__global__ void __launch_bounds__(kThreads)
+clip_fold_kernel(const __grid_constant__ CalibArgs a, uint32_t tensor_begin) {
+  const uint32_t t = tensor_begin + blockIdx.x;
+  if (a.tensors[t].range_mode == QV2_PERCENTILE) clip_fold_tensor(a, t);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -350,9 +370,10 @@ fill_group_clip_kernel(const TensorRec* __restrict__ tensors, const float* __res
 
 }  // namespace
 
-uint32_t hist_grid_cap(int sm_count) {
+uint32_t hist_grid_cap(int sm_count, bool fused) {
   int cache = 0;
-  return (uint32_t)persistent_grid((const void*)hist_kernel<false>, &cache, sm_count, 0x7fffffffu);
+  const void* k = fused ? (const void*)hist_kernel<false, true> : (const void*)hist_kernel<false, false>;
+  return (uint32_t)persistent_grid(k, &cache, sm_count, 0x7fffffffu);
 }
 uint32_t group_hist_grid_cap(int sm_count) {
   int cache = 0;
@@ -390,9 +411,18 @@ cudaError_t launch_fill_group_clip(const Launch& l, const TensorRec* tensors, ui
 cudaError_t launch_hist(const Launch& l, const Stage& st, bool any16, const Tile* hist_tiles, const CalibArgs& a) {
   if (!st.any_percentile) return cudaSuccess;
   const uint32_t n_tiles = st.hist_end - st.hist_begin;
-  const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
-  if (any16) hist_kernel<true><<<st.hist_grid, kThreads, 0, l.stream>>>(a, hist_tiles + st.hist_begin, n_tiles, s0, s1);
-  else hist_kernel<false><<<st.hist_grid, kThreads, 0, l.stream>>>(a, hist_tiles + st.hist_begin, n_tiles, s0, s1);
+  const Tile* tp = hist_tiles + st.hist_begin;
+  if (st.fused_fold) {
+    const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
+    if (any16) hist_kernel<true, true><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
+    else hist_kernel<false, true><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
+    return cudaGetLastError();
+  }
+  if (n_tiles) {
+    if (any16) hist_kernel<true, false><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
+    else hist_kernel<false, false><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
+  }
+  clip_fold_kernel<<<st.tensor_end - st.tensor_begin, kThreads, 0, l.stream>>>(a, st.tensor_begin);
   return cudaGetLastError();
 }
 

@@ -321,30 +321,45 @@ __device__ __noinline__ void metrics_fold_tensor(const MetricsArgs& a, uint32_t 
   __syncthreads();                                    // the shared arrays may be reused by the next fold
 }
 
-// COS adds the sum x*e (third slot array) needed for the cosine similarity.
-template <bool COS, bool ANY16>
+// COS adds the sum x*e (third slot array) needed for the cosine similarity.  FOLD = true: the CTA
+// that finishes a tensor last folds its slots; FOLD = false: metrics_fold_kernel follows, and the
+// main loop carries neither the fold code nor a fence.
+template <bool COS, bool ANY16, bool FOLD>
 __global__ void __launch_bounds__(kThreads, 3)       // 4 CTAs per SM did not run faster
-metrics_kernel(const __grid_constant__ MetricsArgs a, const Tile* __restrict__ tiles, uint32_t n_tiles,
-               uint32_t scan_begin, uint32_t scan_end) {
+metrics_kernel(const __grid_constant__ MetricsArgs a, const TensorRec* __restrict__ tensors,
+               const Tile* __restrict__ tiles, uint32_t n_tiles, uint32_t scan_begin, uint32_t scan_end) {
   using ACC = typename std::conditional<COS, AccCos, Acc>::type;
   constexpr uint32_t kNone = 0xffffffffu;
   __shared__ double sh_w[3][kWarps];
   __shared__ uint32_t s_last;
-  const TensorRec* __restrict__ tensors = a.tensors;
   const float* __restrict__ step = a.step;
   const float* __restrict__ inv = a.inv;
   const float* __restrict__ offset = a.offset;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   // tensors without elements are owned by no CTA: CTA 0 folds them
-  if (blockIdx.x == 0)
+  if (FOLD && blockIdx.x == 0)
     for (uint32_t t = scan_begin; t < scan_end; ++t)
       if (tensors[t].metrics_ctas == 0) metrics_fold_tensor<COS>(a, t);
   uint32_t cur = kNone;
+  uint32_t owed = kNone, drawn = 0; // FOLD: the tensor before cur and the ticket thread 0 drew for it
   double run_sse = 0.0, run_sig = 0.0, run_xe = 0.0;
+  // Ticket protocol of the fused fold: right after its slot store thread 0 fences and draws the
+  // tensor's ticket without looking at the result; the CTA looks at it at its next tensor
+  // boundary and folds the tensor if the ticket was the last one.  The atomic's round trip hides
+  // behind the next tensor's stream; nobody waits for another CTA.
+  auto settle = [&](uint32_t t) {
+    if (threadIdx.x == 0) {
+      const bool last = drawn == tensors[t].metrics_ctas - 1u;
+      if (last) __threadfence();
+      s_last = last;
+    }
+    __syncthreads();
+    if (s_last) metrics_fold_tensor<COS>(a, t);
+  };
   // The CTA is done with tensor t: lanes fold by a fixed butterfly, warps in warp order, one
-  // {sum e^2, sum x^2} pair goes to the CTA's own slot; the CTA that draws the tensor's last
-  // ticket folds the slots.  Nobody waits.
+  // {sum e^2, sum x^2} pair goes to the CTA's own slot.
   auto flush = [&](uint32_t t) {
+    if (FOLD && owed != kNone) settle(owed);
     const TensorRec* tr = tensors + t;
     const double sse = warp_sum_f64(run_sse), sig = warp_sum_f64(run_sig);
     double xe = 0.0;
@@ -361,14 +376,13 @@ metrics_kernel(const __grid_constant__ MetricsArgs a, const Tile* __restrict__ t
       const uint32_t slot = slot_of(tr);
       a.partials[slot] = make_double2(e, s);
       if (COS) a.partials_xe[slot] = x;
-      __threadfence();                                 // the slot is visible before the ticket is
-      s_last = atomicAdd(a.tickets + t, 1u) == tr->metrics_ctas - 1u;
+      if (FOLD) {
+        __threadfence();                               // the slot is visible before the ticket is
+        drawn = atomicAdd(a.tickets + t, 1u);
+      }
     }
-    __syncthreads();
-    if (s_last) {
-      __threadfence();
-      metrics_fold_tensor<COS>(a, t);
-    }
+    __syncthreads();                                   // sh_w may be rewritten by the next flush
+    owed = t;
   };
   for (uint32_t ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile tl = load_tile(tiles, ti);
@@ -402,7 +416,17 @@ metrics_kernel(const __grid_constant__ MetricsArgs a, const Tile* __restrict__ t
       run_xe = __dadd_rn(run_xe, (double)xe);
     }
   }
-  if (cur != kNone) flush(cur);
+  if (cur != kNone) {
+    flush(cur);
+    if (FOLD) settle(cur);
+  }
+}
+
+// One CTA per tensor of the stage: the fold, for stages whose streaming kernel does not fold.
+template <bool COS>
+__global__ void __launch_bounds__(kThreads)
+metrics_fold_kernel(const __grid_constant__ MetricsArgs a, uint32_t tensor_begin) {
+  metrics_fold_tensor<COS>(a, tensor_begin + blockIdx.x);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -514,9 +538,10 @@ __global__ void kl_finalize_kernel(uint32_t n, const unsigned long long* __restr
 
 }  // namespace
 
-uint32_t metrics_grid_cap(int sm_count) {
+uint32_t metrics_grid_cap(int sm_count, bool fused) {
   int cache = 0;
-  return (uint32_t)persistent_grid((const void*)metrics_kernel<false, false>, &cache, sm_count, 0x7fffffffu);
+  const void* k = fused ? (const void*)metrics_kernel<false, false, true> : (const void*)metrics_kernel<false, false, false>;
+  return (uint32_t)persistent_grid(k, &cache, sm_count, 0x7fffffffu);
 }
 uint32_t kl_grid_cap(int sm_count) {
   int cache = 0;
@@ -525,12 +550,21 @@ uint32_t kl_grid_cap(int sm_count) {
 
 cudaError_t launch_metrics(const Launch& l, const Stage& st, bool any16, const Tile* tiles, const MetricsArgs& a) {
   const uint32_t n_tiles = st.tile_end - st.tile_begin;
-  const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
-#define QV2_LAUNCH_METRICS(COS, A16) \
-  metrics_kernel<COS, A16><<<st.metrics_grid, kThreads, 0, l.stream>>>(a, tiles + st.tile_begin, n_tiles, s0, s1)
-  if (a.cosine) { if (any16) QV2_LAUNCH_METRICS(true, true); else QV2_LAUNCH_METRICS(true, false); }
-  else { if (any16) QV2_LAUNCH_METRICS(false, true); else QV2_LAUNCH_METRICS(false, false); }
+  const Tile* tp = tiles + st.tile_begin;
+  const bool fold = st.fused_fold;
+  const uint32_t s0 = fold && st.any_empty ? st.tensor_begin : 0u, s1 = fold && st.any_empty ? st.tensor_end : 0u;
+#define QV2_LAUNCH_METRICS(COS, A16, FOLD) \
+  metrics_kernel<COS, A16, FOLD><<<st.metrics_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1)
+#define QV2_LAUNCH_METRICS_F(COS, A16) do { if (fold) QV2_LAUNCH_METRICS(COS, A16, true); else if (n_tiles) QV2_LAUNCH_METRICS(COS, A16, false); } while (0)
+  if (a.cosine) { if (any16) QV2_LAUNCH_METRICS_F(true, true); else QV2_LAUNCH_METRICS_F(true, false); }
+  else { if (any16) QV2_LAUNCH_METRICS_F(false, true); else QV2_LAUNCH_METRICS_F(false, false); }
+#undef QV2_LAUNCH_METRICS_F
 #undef QV2_LAUNCH_METRICS
+  if (!fold) {
+    const uint32_t nt = st.tensor_end - st.tensor_begin;
+    if (a.cosine) metrics_fold_kernel<true><<<nt, kThreads, 0, l.stream>>>(a, st.tensor_begin);
+    else metrics_fold_kernel<false><<<nt, kThreads, 0, l.stream>>>(a, st.tensor_begin);
+  }
   return cudaGetLastError();
 }
 

@@ -28,7 +28,7 @@ static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t g
 constexpr uint64_t kMaxTiles = 1ull << 27;
 
 static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const GridCaps& caps,
-                              uint64_t chunk_bytes, HostPlan* out) {
+                              uint64_t chunk_bytes, uint32_t fold_mode, HostPlan* out) {
   if (!descs || !out) return QV2_ERR_NULL;
   if (n == 0 || n > 65535u) return QV2_ERR_SIZE;
   *out = HostPlan();
@@ -194,9 +194,15 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
       if (g > tiles) g = tiles;
       return g < 1 ? 1u : (uint32_t)g;
     };
-    st.range_grid = grid_of(caps.range, nt);
-    st.metrics_grid = grid_of(caps.metrics, nt);
-    st.hist_grid = grid_of(caps.hist, nh);
+    uint64_t swept = 0;                    // bytes one metrics launch of the stage reads
+    for (uint32_t t = st.tensor_begin; t < st.tensor_end; ++t) {
+      const TensorRec& r = out->tensors[t];
+      swept += r.n_elems * dtype_size(r.dtype) * (r.y ? 2u : 1u);
+    }
+    st.fused_fold = fold_mode == QV2_FOLD_AUTO ? swept <= kFusedFoldMaxBytes : fold_mode == QV2_FOLD_FUSED;
+    st.range_grid = grid_of(st.fused_fold ? caps.range_fused : caps.range, nt);
+    st.metrics_grid = grid_of(st.fused_fold ? caps.metrics_fused : caps.metrics, nt);
+    st.hist_grid = grid_of(st.fused_fold ? caps.hist_fused : caps.hist, nh);
     uint64_t rel = 0, hrel = 0;
     for (uint32_t t = st.tensor_begin; t < st.tensor_end; ++t) {
       TensorRec& r = out->tensors[t];
@@ -225,9 +231,9 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
 }
 
 int build_plan(const qv2_tensor_desc* descs, uint32_t n, const GridCaps& caps, uint64_t chunk_bytes,
-               HostPlan* out) {
+               uint32_t fold_mode, HostPlan* out) {
   try {
-    return build_plan_checked(descs, n, caps, chunk_bytes, out);
+    return build_plan_checked(descs, n, caps, chunk_bytes, fold_mode, out);
   } catch (const std::bad_alloc&) {          // nothing may unwind through the C ABI
     return QV2_ERR_NOMEM;
   }
@@ -254,7 +260,7 @@ extern "C" uint64_t qv2_group_hist_count(const qv2_tensor_desc* descs, uint32_t 
 extern "C" int64_t qv2_debug_plan_tiles(const qv2_tensor_desc* descs, uint32_t n, uint64_t* out,
                                         uint64_t max_tiles) {
   qv2::HostPlan plan;
-  int st = qv2::build_plan(descs, n, qv2::GridCaps(), 0, &plan);
+  int st = qv2::build_plan(descs, n, qv2::GridCaps(), 0, QV2_FOLD_AUTO, &plan);
   if (st != QV2_OK) return st;
   uint64_t w = 0;
   for (const qv2::Tile& t : plan.tiles) {

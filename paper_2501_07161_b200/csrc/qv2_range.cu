@@ -246,41 +246,49 @@ __device__ __noinline__ void range_fold_tensor(const CalibArgs& a, uint32_t t) {
   __syncthreads();                      // the shared arrays may be reused by the next fold
 }
 
-// Called by every CTA when it has published its share of tensor t: the one that draws the last
-// ticket folds the tensor.  Nobody waits.
-__device__ __forceinline__ void range_tensor_done(const CalibArgs& a, uint32_t t, uint32_t* s_last) {
-  __threadfence();                       // this thread's atomics and slot stores are visible ...
-  __syncthreads();
+// Ticket protocol of the fused fold.  When a CTA has published its share of tensor t (and a
+// barrier has ordered every thread's publication before thread 0), thread 0 fences and draws the
+// tensor's ticket WITHOUT looking at the result; the CTA goes on with its next tensor.  At its
+// next tensor boundary (or when it runs out of tiles) the CTA looks at the ticket it drew: if it
+// was the last one, every other owner had published before, and this CTA folds the tensor.  The
+// atomic's round trip is thus hidden behind the next tensor's stream; nobody ever waits for
+// another CTA.
+__device__ __forceinline__ uint32_t draw_ticket(uint32_t* ticket) {    // thread 0 only
+  __threadfence();                       // the CTA's publications are visible before the ticket is
+  return atomicAdd(ticket, 1u);
+}
+__device__ __forceinline__ void range_settle(const CalibArgs& a, uint32_t t, uint32_t drawn, uint32_t* s_last) {
   if (threadIdx.x == 0) {
-    const uint32_t n = a.tensors[t].range_ctas;
-    *s_last = atomicAdd(a.tickets + t, 1u) == n - 1u;     // ... before the ticket is
+    const bool last = drawn == a.tensors[t].range_ctas - 1u;
+    if (last) __threadfence();
+    *s_last = last;
   }
   __syncthreads();
-  if (*s_last) {
-    __threadfence();
-    range_fold_tensor(a, t);
-  }
+  if (*s_last) range_fold_tensor(a, t);
 }
 
 // ANY16 = false is the build for models whose tensors are all binary32: the element-type dispatch
 // is compiled out, so that common case pays nothing for the 16-bit paths.
-template <bool ANY16>
+// FOLD = true: the CTA that finishes a tensor last folds it (small stages, where a separate fold
+// launch would be a visible share of the pass).  FOLD = false: the kernel only publishes, and
+// range_fold_kernel follows; the main loop is then free of the fold code and of its fences.
+template <bool ANY16, bool FOLD>
 __global__ void __launch_bounds__(kThreads, 4)
-range_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles, uint32_t n_tiles,
-             uint32_t scan_begin, uint32_t scan_end) {
+range_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ tensors,
+             const Tile* __restrict__ tiles, uint32_t n_tiles, uint32_t scan_begin, uint32_t scan_end) {
   constexpr uint32_t kNone = 0xffffffffu;
   __shared__ float sh[2 * kWarps];
   __shared__ uint32_t s_last;
-  const TensorRec* __restrict__ tensors = a.tensors;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   // tensors without elements are owned by no CTA: CTA 0 folds them (the planner asks for the
   // scan only when the stage has one)
-  if (blockIdx.x == 0)
+  if (FOLD && blockIdx.x == 0)
     for (uint32_t t = scan_begin; t < scan_end; ++t)
       if (tensors[t].range_ctas == 0) range_fold_tensor(a, t);
   RangeAcc acc;
   reset(acc);
   uint32_t cur_group = kNone, cur_tensor = kNone;
+  uint32_t owed = kNone, drawn = 0; // FOLD: the tensor before cur_tensor and the ticket thread 0 drew for it
   bool cur_slot = false;           // the pending group belongs to a per-tensor tensor
   auto flush_group = [&]() {
     if (cur_group == kNone) return;
@@ -292,7 +300,15 @@ range_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles
     const Tile tl = load_tile(tiles, ti);
     const TensorRec* tr = tensors + tl.tensor;
     if (tl.tensor != cur_tensor) {   // block-uniform: every warp of the CTA takes these branches together
-      if (cur_tensor != kNone) { flush_group(); range_tensor_done(a, cur_tensor, &s_last); }
+      if (cur_tensor != kNone) {
+        flush_group();
+        if (FOLD) {
+          if (owed != kNone) range_settle(a, owed, drawn, &s_last);
+          __syncthreads();                    // every thread's publication of cur_tensor precedes the fence
+          if (threadIdx.x == 0) drawn = draw_ticket(a.tickets + cur_tensor);
+          owed = cur_tensor;
+        }
+      }
       cur_tensor = tl.tensor;
     }
     const uint32_t gbase = tr->group_base;
@@ -322,21 +338,45 @@ range_kernel(const __grid_constant__ CalibArgs a, const Tile* __restrict__ tiles
         range_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, warp, a.kmin, a.kmax, a.nf_acc);
     }
   }
-  if (cur_tensor != kNone) { flush_group(); range_tensor_done(a, cur_tensor, &s_last); }
+  if (cur_tensor != kNone) {
+    flush_group();
+    if (FOLD) {
+      if (owed != kNone) range_settle(a, owed, drawn, &s_last);
+      __syncthreads();
+      if (threadIdx.x == 0) drawn = draw_ticket(a.tickets + cur_tensor);
+      range_settle(a, cur_tensor, drawn, &s_last);
+    }
+  }
+}
+
+// One CTA per tensor of the stage: the fold, for stages whose streaming kernel does not fold.
+__global__ void __launch_bounds__(kThreads)
+range_fold_kernel(const __grid_constant__ CalibArgs a, uint32_t tensor_begin) {
+  range_fold_tensor(a, tensor_begin + blockIdx.x);
 }
 
 }  // namespace
 
-uint32_t range_grid_cap(int sm_count) {
+uint32_t range_grid_cap(int sm_count, bool fused) {
   int cache = 0;
-  return (uint32_t)persistent_grid((const void*)range_kernel<false>, &cache, sm_count, 0x7fffffffu);
+  const void* k = fused ? (const void*)range_kernel<false, true> : (const void*)range_kernel<false, false>;
+  return (uint32_t)persistent_grid(k, &cache, sm_count, 0x7fffffffu);
 }
 
 cudaError_t launch_range(const Launch& l, const Stage& st, bool any16, const Tile* tiles, const CalibArgs& a) {
   const uint32_t n_tiles = st.tile_end - st.tile_begin;
-  const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
-  if (any16) range_kernel<true><<<st.range_grid, kThreads, 0, l.stream>>>(a, tiles + st.tile_begin, n_tiles, s0, s1);
-  else range_kernel<false><<<st.range_grid, kThreads, 0, l.stream>>>(a, tiles + st.tile_begin, n_tiles, s0, s1);
+  const Tile* tp = tiles + st.tile_begin;
+  if (st.fused_fold) {
+    const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
+    if (any16) range_kernel<true, true><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
+    else range_kernel<false, true><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
+    return cudaGetLastError();
+  }
+  if (n_tiles) {
+    if (any16) range_kernel<true, false><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
+    else range_kernel<false, false><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
+  }
+  range_fold_kernel<<<st.tensor_end - st.tensor_begin, kThreads, 0, l.stream>>>(a, st.tensor_begin);
   return cudaGetLastError();
 }
 

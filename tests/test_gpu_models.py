@@ -294,14 +294,14 @@ def test_library_sweep_graph_replays_the_pass():
             sb_ref, t_ref = gctx.alloc_sweep_buffers(md.descs, md.n_layers)
             m0 = gctx.launches
             gctx.sweep_model(md.descs, md.n_layers, md.macs, None, cfg, sb_ref)
-            per_pass = gctx.launches - m0                  # 3 kernels here: range, metrics, rank (no histogram pass)
+            per_pass = gctx.launches - m0                  # range + fold, metrics + fold, rank: no clearing launch, no histogram pass
             g = gctx.sweep_graph(md.descs, md.n_layers, md.macs, None, cfg, sb)
             n0 = gctx.launches
             for k in ("mse", "sqnr_db", "order", "hist"):
                 t[k].zero_()
             g.launch()
             s.synchronize()
-            assert gctx.launches - n0 == per_pass == 3
+            assert gctx.launches - n0 == per_pass == 5
             for k in ("mse", "sqnr_db", "order", "keep_fp32", "n_keep", "step", "hist", "clip"):
                 assert torch.equal(t[k].view(torch.uint8), t_ref[k].view(torch.uint8)), k
             model.layers[5].x.mul_(0.5)                   # refill a tensor in place

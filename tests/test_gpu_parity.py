@@ -17,9 +17,13 @@ pytestmark = pytest.mark.gpu
 TILE = 16384
 
 
-@pytest.fixture(scope="module")
-def ctx():
+@pytest.fixture(scope="module", params=["fold-separate", "fold-fused"])
+def ctx(request):
+    """Every test runs twice: with the separate fold kernels (the default) and with the fold inside
+    the streaming kernels."""
     c = q.Context(0)
+    if request.param == "fold-fused":
+        c.set_fold_mode(q.FOLD_FUSED)
     yield c
     c.close()
 

@@ -31,9 +31,10 @@ def _sweep(ctx, model):
     return md, t
 
 
+@pytest.mark.parametrize("fold", [q.FOLD_SEPARATE, q.FOLD_FUSED])
 @pytest.mark.parametrize("name,batch,chunk", [("resnet18", 2, 4 << 20), ("mobilenetv2", 1, 2 << 20),
                                               ("squeezenet", 1, 1 << 20), ("vgg16", 1, 8 << 20)])
-def test_l2_chunked_schedule_matches_oracle_and_phase_major(name, batch, chunk):
+def test_l2_chunked_schedule_matches_oracle_and_phase_major(name, batch, chunk, fold):
     """The chunked schedule (range -> histogram -> metrics stage by stage) gives the oracle's
     results, the same bits as the phase-major schedule for everything that is integer-decided,
     and sums within the metric tolerance; the ranking is a bit-exact function of its metrics."""
@@ -41,6 +42,7 @@ def test_l2_chunked_schedule_matches_oracle_and_phase_major(name, batch, chunk):
     a, b = q.Context(0), q.Context(0)
     try:
         b.set_schedule(q.SCHEDULE_L2_CHUNKED, chunk)
+        b.set_fold_mode(fold)
         md, ta = _sweep(a, model)
         _, tb = _sweep(b, model)
         assert a.stages == 1 and b.stages > 3, (a.stages, b.stages)
@@ -114,12 +116,15 @@ def test_chunked_schedule_with_empty_tensors_mixed_modes_and_codes():
         ctx.close()
 
 
-def test_steady_state_passes_never_synchronise_and_launch_four_kernels():
+@pytest.mark.parametrize("fold,per_phase", [(q.FOLD_FUSED, 1), (q.FOLD_SEPARATE, 2), (q.FOLD_AUTO, 2)])
+def test_steady_state_passes_never_synchronise_and_need_no_clearing_launch(fold, per_phase):
     """After the first call of a descriptor set nothing synchronises the stream: not a calibrate
-    after a code-storing metrics call, not new code buffers.  A percentile pass is range +
-    histogram + metrics (+ rank): no clearing and no finalize launches."""
+    after a code-storing metrics call, not new code buffers.  A percentile pass is range,
+    histogram and metrics, each one launch (fused fold) or two (separate fold kernel): there is
+    no clearing launch."""
     ctx = q.Context(0)
     try:
+        ctx.set_fold_mode(fold)
         g = torch.Generator(device="cuda"); g.manual_seed(0)
         x = torch.randn(70000, generator=g, device="cuda")
         w = torch.randn(32 * 300, generator=g, device="cuda")
@@ -137,7 +142,7 @@ def test_steady_state_passes_never_synchronise_and_launch_four_kernels():
             met = ctx.quant_metrics(descs, cal.step, cal.inv, cal.offset, other if it % 2 else codes)
             met_plain = ctx.quant_metrics(descs, cal.step, cal.inv, cal.offset)
         assert ctx.syncs == s0, "a steady-state call synchronised the stream"
-        assert ctx.launches - l0 == 6 * (2 + 1 + 1)
+        assert ctx.launches - l0 == 6 * (2 + 1 + 1) * per_phase
         torch.cuda.synchronize()
         assert torch.equal(other[0], codes[0]) and torch.equal(other[1], codes[1]) and int(codes[0].max()) > 0
         assert torch.equal(met.sse.view(torch.int64), met0.sse.view(torch.int64))
