@@ -16,6 +16,7 @@ from __future__ import annotations
 import argparse
 import hashlib
 import json
+import math
 import os
 import sys
 import threading
@@ -47,6 +48,11 @@ def parse():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustained-s", type=float, default=2.0,
+                    help="length of the sustained run (the same pass back to back, clocks sampled throughout); 0: skip")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="skip the short runs of the other model shapes (the 'workloads' block)")
+    ap.add_argument("--workload-steps", type=int, default=20)
     ap.add_argument("--input-dtype", default="f32", choices=["f32", "f16", "bf16"],
                     help="element type the tensors are stored in (the default workload is f32)")
     ap.add_argument("--act-granularity", default="tensor", choices=["tensor", "channel"],
@@ -58,6 +64,8 @@ def parse():
     ap.add_argument("--chunk-mb", type=float, default=0.0, help="chunk size of the chunked schedule (0: library default)")
     ap.add_argument("--fold", default="auto", choices=["auto", "fused", "separate"],
                     help="where per-tensor partial results are folded (qv2_set_fold_mode)")
+    ap.add_argument("--dependent-launch", default="on", choices=["on", "off"],
+                    help="launch the kernels of a pass as programmatic dependents of one another (qv2_set_dependent_launch)")
     ap.add_argument("--api", default=None, choices=["calls", "sweep"],
                     help="calls: qv2_calibrate + qv2_quant_metrics + qv2_rank_layers (default for the phase-major "
                          "schedule); sweep: the chained qv2_sweep_model (default otherwise; per-phase times are then not available)")
@@ -185,6 +193,26 @@ def run_oracle_steps(jobs, threads, steps, warmup):
     return (time.perf_counter() - t0) / max(steps, 1), res
 
 
+def run_oracle_timed_jobs(jobs, threads):
+    """One oracle pass over `jobs` (whole tensors side by side, as oracle.sweep_tensors runs them)
+    that also times every job, so that the load balance of the pass can be stated."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+
+    def one(j):
+        t = time.perf_counter()
+        oracle.sweep_tensor(**j)
+        return time.perf_counter() - t
+
+    t0 = time.perf_counter()
+    if threads <= 1:
+        per_job = [one(j) for j in jobs]
+    else:
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            per_job = list(ex.map(one, jobs))
+    return time.perf_counter() - t0, per_job
+
+
 def reference_main(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -221,7 +249,39 @@ def measured_peak():
         with open(p) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     except Exception:
-        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return 6650.0, "fallback (6.65 TB/s, an earlier B200 copy measurement)"
+
+
+def recorded_read_ceiling():
+    """GB/s of a pure read stream on a B200 as recorded by the stand-alone probe summarised in
+    profiles/read_ceiling_probe.md (plain 16-byte loads, 4 GB input, CUDA events)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "read_ceiling_probe.md")) as f:
+            for ln in f:
+                if ln.startswith("read_ceiling_gbs:"):
+                    return float(ln.split(":", 1)[1])
+    except Exception:
+        pass
+    return None
+
+
+def live_read_rate(device, gib: float = 2.0, reps: int = 5):
+    """A read-only library kernel timed here and now: torch.max over `gib` GiB of fp32 (best of
+    `reps`, CUDA events).  A cross-check of the recorded ceiling on this very GPU, nothing more."""
+    n = int(gib * (1 << 30)) // 4
+    x = torch.empty(n, dtype=torch.float32, device=device).normal_()
+    best = None
+    for r in range(reps + 2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        x.max()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if r >= 2:
+            best = ms if best is None else min(best, ms)
+    del x
+    return 4.0 * n / (best * 1e-3) / 1e9
 
 
 def recorded_traffic():
@@ -245,6 +305,69 @@ def recorded_traffic():
         return float(rec["dram_bytes_per_algorithmic_byte"])
     except Exception:
         return None
+
+
+def side_workloads(q, local, peak, steps):
+    """Short runs of the other model shapes (configs 1-4), each `steps` passes after 3 warm-ups:
+    qv2_sweep_model on the default (phase-major) schedule and on the L2-chunked schedule, each also
+    replayed from a CUDA graph."""
+    out = []
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for name in [w for w in gen.CONFIG_ORDER if w != "vgg16"]:
+            cfgw = gen.CONFIGS[name]
+            model = gen.make_model(name, seed=0, device="cuda", batch=cfgw.batch)
+            md = q.model_descs(model)
+            L = md.n_layers
+            rcfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
+            swept = gen.swept_bytes(name, cfgw.batch)
+            rec = {"workload": name, "batch": cfgw.batch, "layers": L, "swept_bytes_per_step": swept,
+                   "resident_bytes": 4 * (model.weight_elems + 2 * model.act_elems), "steps": steps}
+
+            def timed(fn):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(steps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / steps
+
+            for label, sched in (("phase_major", q.SCHEDULE_PHASE_MAJOR), ("l2_chunked", q.SCHEDULE_L2_CHUNKED)):
+                ctx = q.Context(local, stream=stream)
+                ctx.set_schedule(sched, 0)
+                sb, t = ctx.alloc_sweep_buffers(md.descs, L)
+                l0 = ctx.launches
+                ms = timed(lambda: ctx.sweep_model(md.descs, L, md.macs, None, rcfg, sb))
+                r = {"ms_per_step": ms, "value": swept / (ms * 1e-3) / 1e9, "stages": ctx.stages,
+                     "launches_per_step": (ctx.launches - l0) // (steps + 3)}
+                g = ctx.sweep_graph(md.descs, L, md.macs, None, rcfg, sb)
+                gms = timed(g.launch)
+                g.close()
+                r["graph_ms_per_step"] = gms
+                r["graph_value"] = swept / (gms * 1e-3) / 1e9
+                ctx.close()
+                rec[label] = r
+                del sb, t
+                if label == "phase_major":
+                    rec["ms_per_step"], rec["value"] = ms, r["value"]
+            best = min(rec["phase_major"]["ms_per_step"], rec["phase_major"]["graph_ms_per_step"],
+                       rec["l2_chunked"]["ms_per_step"], rec["l2_chunked"]["graph_ms_per_step"])
+            rec["best_ms_per_step"] = best
+            rec["best_value"] = swept / (best * 1e-3) / 1e9
+            rec["unit"] = UNIT
+            rec["frac_of_measured_copy_peak"] = rec["best_value"] / peak
+            rec["frac_of_8000_nominal"] = rec["best_value"] / 8000.0
+            rec["l2"] = ("inputs larger than L2" if rec["resident_bytes"] > 4 * 126e6
+                         else "inputs fit in L2: an L2 number, not an HBM one")
+            out.append(rec)
+            del model, md
+            torch.cuda.empty_cache()
+    torch.cuda.synchronize()
+    return out
 
 
 def ours_main(args):
@@ -276,6 +399,7 @@ def ours_main(args):
     sched = {"phase": q.SCHEDULE_PHASE_MAJOR, "chunked": q.SCHEDULE_L2_CHUNKED, "auto": q.SCHEDULE_AUTO}[args.schedule]
     ctx.set_schedule(sched, int(args.chunk_mb * (1 << 20)))
     ctx.set_fold_mode({"auto": q.FOLD_AUTO, "fused": q.FOLD_FUSED, "separate": q.FOLD_SEPARATE}[args.fold])
+    ctx.set_dependent_launch(args.dependent_launch == "on")
     api = args.api or ("calls" if args.schedule == "phase" else "sweep")
     md = q.model_descs(model, act_granularity=args.act_granularity)
     n, L = md.n_tensors, md.n_layers
@@ -359,11 +483,45 @@ def ours_main(args):
         step_ms = [total_ms / K]
         clocks = sampler.summary(t_wall0, t_wall1)
         launch_mode = "CUDA graph of one pass (qv2_sweep_graph_create), replayed"
-        g.close()
-    sampler.stop()
 
     value, slowest_s = R.whole_job_throughput(swept * K / 1e9, total_ms / 1e3)
     ms_per_step = slowest_s * 1e3 / K
+
+    # ------------------------------------- range phase and histogram phase of qv2_calibrate apart
+    split = None
+    if api == "calls" and ctx.stages == 1:
+        ctx.set_phase_timing(True)
+        rs, hs = [], []
+        for _ in range(min(K, 20)):
+            one_step()
+            r_ms, h_ms = ctx.calibrate_phase_ms()
+            rs.append(r_ms); hs.append(h_ms)
+        ctx.set_phase_timing(False)
+        split = (float(np.mean(rs)), float(np.mean(hs)))
+
+    # -------------------------------------------- the same pass back to back for a few seconds
+    # The K timed steps above last tens of milliseconds, less than the power limiter needs to react;
+    # this block shows where the clocks and the rate settle.
+    sustained = None
+    if args.sustained_s > 0 and world == 1:
+        step_fn = g.launch if args.graph else one_step
+        n_sus = int(min(200000, max(K, math.ceil(args.sustained_s * 1e3 / max(ms_per_step, 1e-3)))))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        tw0 = time.perf_counter()
+        s0.record()
+        for _ in range(n_sus):
+            step_fn()
+        s1.record()
+        torch.cuda.synchronize()
+        tw1 = time.perf_counter()
+        sus_ms = s0.elapsed_time(s1)
+        sustained = {"steps": n_sus, "seconds": sus_ms / 1e3, "ms_per_step": sus_ms / n_sus,
+                     "value": swept * n_sus / (sus_ms * 1e-3) / 1e9, "unit": UNIT,
+                     "clocks": sampler.summary(tw0, tw1)}
+    if args.graph:
+        g.close()
+    sampler.stop()
 
     # ------------------------------------------------------------------ end to end (host buffers)
     e2e = None
@@ -409,14 +567,34 @@ def ours_main(args):
         images, wbudget = size_sample(args.workload, batch, 2.0, threads)
         jobs, s_swept, w_used = oracle_sample_jobs(model, images, wbudget, args.act_granularity == "channel")
         threads = min(threads, len(jobs))
-        sec, _ = run_oracle_steps(jobs, threads, 1, 0)
+        sec, per_job = run_oracle_timed_jobs(jobs, threads)
         cpu = {"value": s_swept / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": (f"activations of the first {images} of {batch} images for all {L} layers, weight "
                           f"tensors in layer order up to {w_used} elements; {s_swept / 1e9:.3f} GB swept, "
-                          f"{sec:.2f} s")}
+                          f"{sec:.2f} s"),
+               # the oracle is serial per tensor; whole tensors run side by side, so the pass cannot end
+               # before its largest tensor does
+               "balance": {"jobs": len(jobs), "largest_job_s": max(per_job), "sum_of_jobs_s": sum(per_job),
+                           "wall_s": sec, "thread_utilisation": sum(per_job) / (threads * sec),
+                           "note": "wall time is bounded below by the largest tensor on one thread; "
+                                   "sum_of_jobs_s / wall_s is the effective number of busy cores"}}
+        # the oracle as written, one thread, on a smaller sample of the same workload
+        images1, wbudget1 = size_sample(args.workload, batch, 4.0, 1)
+        jobs1, swept1, w_used1 = oracle_sample_jobs(model, images1, wbudget1, args.act_granularity == "channel")
+        sec1, _ = run_oracle_timed_jobs(jobs1, 1)
+        cpu["single_thread"] = {"value": swept1 / sec1 / 1e9, "unit": UNIT, "cores": 1,
+                                "sample": (f"activations of the first {images1} of {batch} images for all {L} "
+                                           f"layers, weight tensors in layer order up to {w_used1} elements; "
+                                           f"{swept1 / 1e9:.3f} GB swept, {sec1:.2f} s")}
+
+    workloads = None
+    if rank == 0 and world == 1 and not args.no_workloads and args.workload == "vgg16":
+        workloads = side_workloads(q, local, measured_peak()[0], args.workload_steps)
 
     if rank == 0:
         peak, peak_src = measured_peak()
+        read_ceiling = recorded_read_ceiling()
+        live_read = live_read_rate(torch.device("cuda", local)) if world == 1 else None
         achieved = metrics_bytes / (met_ms * 1e-3) / 1e9 if met_ms > 1e-6 else None   # no per-phase time with --api sweep
         # the capture was taken on the default workload; DRAM traffic is reported for it only
         ratio = recorded_traffic() if (args.workload == "vgg16" and batch == cfgw.batch and esz == 4
@@ -433,21 +611,34 @@ def ours_main(args):
                        "l2": "inputs larger than L2 (no flush needed)" if 4 * (w_elems + 2 * a_elems) > 4 * 126e6
                              else "inputs fit in L2: this is an L2 number, not an HBM one",
                        "parallelism": f"replicas x{world}" if world > 1 else "1 GPU",
-                       "launch": launch_mode, "schedule": args.schedule, "stages": ctx.stages, "api": api, "fold": args.fold,
+                       "launch": launch_mode, "schedule": args.schedule, "stages": ctx.stages, "api": api, "fold": args.fold, "dependent_launch": args.dependent_launch,
                        "seed": 0},
             "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_min": step_ms[0],
-            "phases_ms": {"calibrate": cal_ms, "quant_metrics": met_ms, "rank": rank_ms},
+            "phases_ms": {"calibrate": cal_ms, "quant_metrics": met_ms, "rank": rank_ms,
+                          # the two phases of qv2_calibrate apart (events inside the call, a separate short loop)
+                          "calibrate_range": split[0] if split else None,
+                          "calibrate_histogram": split[1] if split else None},
             "frac_of_measured_copy_peak": value / world / peak,
             "frac_of_8000_nominal": value / world / 8000.0,
             "roofline": {"kernel": "metrics_kernel (qv2_quant_metrics)", "bound": "hbm",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak if achieved else None,
                          "traffic": traffic, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": metrics_bytes,
+                         # the peak above is a copy (read + write); these kernels only read, so a
+                         # pure read stream is the tighter ceiling
+                         "read_ceiling": {"recorded_gbs": read_ceiling,
+                                          "source": "profiles/read_ceiling_probe.md (plain 16-byte loads, 4 GB, CUDA events)",
+                                          "frac": (achieved / read_ceiling) if (achieved and read_ceiling) else None,
+                                          "live_torch_max_gbs": live_read},
                          "duration_ms": met_ms,
                          "note": "duration = CUDA events around the qv2_quant_metrics call on its stream "
                                  "(the streaming kernel plus a per-tensor finalize kernel of a few microseconds)"},
             "clocks": clocks, "gpu_launches": int(launches),
         }
+        if sustained is not None:
+            line["sustained"] = sustained
+        if workloads is not None:
+            line["workloads"] = workloads
         if e2e is not None:
             line["e2e"] = e2e
         if cpu is not None:

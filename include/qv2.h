@@ -157,8 +157,10 @@ uint64_t qv2_sync_count(const qv2_ctx* ctx);
  *     form) runs range -> histogram -> metrics per stage.  Results are the same bits for integer
  *     outputs and parameters; sums are added in a stage-dependent order (same tolerances).  Plans
  *     with QV2_PERCENTILE_GROUP tensors keep one stage.
- *   QV2_SCHEDULE_AUTO: chunked when the model is larger than two chunks and at least half of its
- *     reference bytes sit in tensors that fit a chunk, else phase-major.
+ *   QV2_SCHEDULE_AUTO: whichever measured faster for the plan's sizes.  On a B200 that is
+ *     phase-major for every size tried (62 MB to 15 GB per pass): L2 serves a re-read at about
+ *     2.2 times the HBM rate and only for stages up to ~32 MB, which does not pay for the
+ *     additional launches, so AUTO currently never chunks.
  * chunk_bytes: 0 selects the default (48 MiB, well under half of a B200's 126 MB L2).
  * Takes effect with the next call; QV2_ERR_UNSUPPORTED while a captured pass of this context lives.
  */
@@ -175,6 +177,28 @@ int qv2_set_schedule(qv2_ctx* ctx, uint32_t schedule, uint64_t chunk_bytes);
  * the choice.  QV2_ERR_UNSUPPORTED while a captured pass of this context lives.
  */
 int qv2_set_fold_mode(qv2_ctx* ctx, uint32_t mode);
+/*
+ * How the kernels of a pass follow one another on the stream.  On (default): every kernel is
+ * launched as a programmatic dependent of the one before it, so its launch latency and its
+ * prologue overlap the tail of its predecessor; each kernel waits (in hardware, at its first
+ * instruction that touches memory) until the predecessor has completed and its writes are
+ * visible, so results are the same as with ordinary launches.  Off: ordinary stream order.
+ * The first kernel of a call treats whatever precedes it on the stream the same way, which is safe
+ * for any predecessor.  QV2_ERR_UNSUPPORTED while a captured pass of this context lives.
+ */
+int qv2_set_dependent_launch(qv2_ctx* ctx, int on);
+/*
+ * Measurement aid (no counterpart in the paper): with timing on, qv2_calibrate on a single-stage
+ * plan records CUDA events on the context's stream before its range phase, between the range
+ * phase and the histogram phase, and after the histogram phase (per-group histograms included).
+ * qv2_calibrate_phase_ms waits for the last of them (a host synchronisation, counted by
+ * qv2_sync_count) and returns the two durations of the most recent qv2_calibrate call in
+ * milliseconds.  QV2_ERR_UNSUPPORTED when timing is off, when no timed call has been made, or when
+ * the last call ran a multi-stage plan or inside a stream capture (no events are recorded then).
+ * The results of qv2_calibrate are the same either way.
+ */
+int qv2_set_phase_timing(qv2_ctx* ctx, int on);
+int qv2_calibrate_phase_ms(qv2_ctx* ctx, float* range_ms, float* hist_ms);
 /* Number of stages of the context's current plan (1 for phase-major; 0 before the first call). */
 uint32_t qv2_stage_count(const qv2_ctx* ctx);
 /* Sum over descs of the number of quantization groups (1 or `channels`).  Host only. */

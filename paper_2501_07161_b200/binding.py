@@ -31,7 +31,8 @@ EXPORTS = ["qv2_create", "qv2_destroy", "qv2_status_string", "qv2_last_cuda_erro
            "qv2_rank_layers", "qv2_sweep_model", "qv2_sweep_model_host", "qv2_staging_bytes",
            "qv2_debug_plan_tiles", "qv2_quant_metrics_noalloc", "qv2_quant_metrics_ex", "qv2_rank_layers_ex", "qv2_kl_divergence", "qv2_fold_batchnorm", "qv2_sweep_graph_create", "qv2_sweep_graph_launch",
            "qv2_sweep_graph_destroy", "qv2_check_nonfinite", "qv2_calibrate_ex", "qv2_group_hist_count",
-           "qv2_sync_count", "qv2_set_schedule", "qv2_stage_count", "qv2_set_fold_mode"]
+           "qv2_sync_count", "qv2_set_schedule", "qv2_stage_count", "qv2_set_fold_mode",
+           "qv2_set_phase_timing", "qv2_calibrate_phase_ms", "qv2_set_dependent_launch"]
 KL_BINS = 128
 NO_GROUP = 0xFFFFFFFF
 NOALLOC_MAX_ELEMS = 1 << 27
@@ -83,6 +84,10 @@ def lib() -> C.CDLL:
     L.qv2_set_schedule.argtypes = [vp, u32, u64]; L.qv2_set_schedule.restype = i32
     L.qv2_stage_count.argtypes = [vp]; L.qv2_stage_count.restype = u32
     L.qv2_set_fold_mode.argtypes = [vp, u32]; L.qv2_set_fold_mode.restype = i32
+    L.qv2_set_dependent_launch.argtypes = [vp, i32]; L.qv2_set_dependent_launch.restype = i32
+    L.qv2_set_phase_timing.argtypes = [vp, i32]; L.qv2_set_phase_timing.restype = i32
+    L.qv2_calibrate_phase_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+    L.qv2_calibrate_phase_ms.restype = i32
     L.qv2_group_count.argtypes = [dp, u32]; L.qv2_group_count.restype = u64
     L.qv2_calibrate.argtypes = [vp, dp, u32] + [vp] * 9; L.qv2_calibrate.restype = i32
     L.qv2_calibrate_ex.argtypes = [vp, dp, u32] + [vp] * 11; L.qv2_calibrate_ex.restype = i32
@@ -232,6 +237,18 @@ class Context:
 
     def set_fold_mode(self, mode: int):
         _check(lib().qv2_set_fold_mode(self._h, mode), "qv2_set_fold_mode")
+
+    def set_dependent_launch(self, on: bool):
+        _check(lib().qv2_set_dependent_launch(self._h, int(on)), "qv2_set_dependent_launch")
+
+    def set_phase_timing(self, on: bool):
+        _check(lib().qv2_set_phase_timing(self._h, int(on)), "qv2_set_phase_timing")
+
+    def calibrate_phase_ms(self):
+        """(range_ms, hist_ms) of the most recent timed qv2_calibrate; synchronises."""
+        r, h = C.c_float(0.0), C.c_float(0.0)
+        _check(lib().qv2_calibrate_phase_ms(self._h, C.byref(r), C.byref(h)), "qv2_calibrate_phase_ms")
+        return float(r.value), float(h.value)
 
     def last_cuda_error(self) -> int:
         return int(lib().qv2_last_cuda_error(self._h))

@@ -68,5 +68,27 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+PROBES = os.path.join(_HERE, "probes")
+
+
+def build_probes() -> list:
+    """Compile the stand-alone bandwidth probes under probes/ (one executable each, next to its
+    source).  They are measurement aids for the profiles, not part of libqv2.so."""
+    out = []
+    for src in sorted(glob.glob(os.path.join(PROBES, "*.cu"))):
+        exe = src[:-3]
+        if not os.path.exists(exe) or os.path.getmtime(exe) < os.path.getmtime(src):
+            res = subprocess.run([NVCC, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a",
+                                  "-lineinfo", "-o", exe, src], cwd=PROBES, capture_output=True, text=True)
+            if res.returncode != 0:
+                sys.stderr.write(res.stdout + res.stderr)
+                raise RuntimeError("nvcc failed building " + src)
+        out.append(exe)
+    return out
+
+
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    if "--probes" in sys.argv:
+        print("\n".join(build_probes()))
+    else:
+        print(build(force=True, verbose="-v" in sys.argv))

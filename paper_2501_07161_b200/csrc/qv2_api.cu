@@ -34,6 +34,7 @@ struct qv2_ctx {
   uint32_t schedule = QV2_SCHEDULE_PHASE_MAJOR;
   uint64_t chunk_bytes = kDefaultChunkBytes;
   uint32_t fold_mode = QV2_FOLD_AUTO;
+  bool dependent_launch = true;   // kernels of a pass are launched as programmatic dependents of one another
 
   // cached plan: rebuilt only when the descriptor bytes or the schedule change
   HostPlan plan;
@@ -67,6 +68,10 @@ struct qv2_ctx {
   uint8_t** h_codes[kCodeRing] = {}; size_t cap_h_codes = 0;
   cudaEvent_t code_ev[kCodeRing] = {};
   uint32_t code_next = 0;
+  // qv2_set_phase_timing: events around the range and histogram phases of qv2_calibrate
+  bool phase_timing = false;
+  bool phase_marks_valid = false;
+  cudaEvent_t phase_ev[3] = {};
 };
 
 namespace {
@@ -138,22 +143,18 @@ int sync_stream(qv2_ctx* c) {
   return QV2_OK;
 }
 
-// Chunk size of the plan about to be built: 0 = phase-major (one stage).  QV2_SCHEDULE_AUTO takes
-// the chunked schedule when most of the reference bytes sit in tensors that fit a chunk and the
-// model is large enough for the extra launches to pay.
-uint64_t plan_chunk_bytes(const qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n) {
-  if (c->schedule == QV2_SCHEDULE_PHASE_MAJOR) return 0;
-  if (c->schedule == QV2_SCHEDULE_L2_CHUNKED) return c->chunk_bytes;
-  uint64_t total = 0, fitting = 0;
-  for (uint32_t t = 0; t < n; ++t) {
-    const uint64_t b = descs[t].outer * descs[t].channels * descs[t].inner *
-                       dtype_size((descs[t].flags & QV2_IN_MASK) >> 16);
-    total += b;
-    if (b <= c->chunk_bytes) fitting += b;
-  }
-  // below ~2 chunks everything is L2-resident across phases anyway; above, chunk when at least
-  // half of the bytes can be reused
-  return (total > 2 * c->chunk_bytes && 2 * fitting >= total) ? c->chunk_bytes : 0;
+// Chunk size of the plan about to be built: 0 = phase-major (one stage).
+//
+// QV2_SCHEDULE_AUTO currently always answers phase-major.  Measured on a B200, a buffer that is read
+// again is served from L2 at about 2.2 times the HBM rate only while it is at most ~32 MB (a
+// persistent kernel re-reading 8..512 MB: 13-17 TB/s up to 32 MB, 9-13 TB/s at 48 MB, the HBM rate
+// from 96 MB on), so the second and third pass over a stage can save at most half of their time
+// on stages that small, while every stage adds launches of a few microseconds each and leaves the
+// streaming kernels with one or two tiles per thread block.  On ResNet-18 shapes (batch 32) the
+// chunked pass takes 0.38-0.56 ms against 0.27-0.30 ms phase-major, on ResNet-50 1.67-1.91 against
+// 1.23 ms; it is kept for callers that ask for it.
+uint64_t plan_chunk_bytes(const qv2_ctx* c, const qv2_tensor_desc*, uint32_t) {
+  return c->schedule == QV2_SCHEDULE_L2_CHUNKED ? c->chunk_bytes : 0;
 }
 
 int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n);
@@ -230,7 +231,7 @@ int ensure_plan_checked(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n) {
 }
 
 Launch launch_of(qv2_ctx* c) {
-  Launch l; l.stream = c->stream; l.sm_count = c->sm_count; l.pdl = false;
+  Launch l; l.stream = c->stream; l.sm_count = c->sm_count; l.pdl = c->dependent_launch;
   return l;
 }
 
@@ -396,6 +397,8 @@ extern "C" int qv2_destroy(qv2_ctx* c) {
     if (c->h_codes[i]) cudaFreeHost(c->h_codes[i]);
     if (c->code_ev[i]) cudaEventDestroy(c->code_ev[i]);
   }
+  for (cudaEvent_t e : c->phase_ev)
+    if (e) cudaEventDestroy(e);
   delete c;
   return QV2_OK;
 }
@@ -421,6 +424,35 @@ extern "C" int qv2_set_fold_mode(qv2_ctx* c, uint32_t mode) {
   return QV2_OK;
 }
 
+extern "C" int qv2_set_dependent_launch(qv2_ctx* c, int on) {
+  if (!c) return QV2_ERR_NULL;
+  if (c->live_graphs) return QV2_ERR_UNSUPPORTED;     // a captured pass keeps the edges it was captured with
+  c->dependent_launch = on != 0;
+  return QV2_OK;
+}
+
+extern "C" int qv2_set_phase_timing(qv2_ctx* c, int on) {
+  if (!c) return QV2_ERR_NULL;
+  DeviceGuard guard(c->device);
+  if (on)
+    for (cudaEvent_t& e : c->phase_ev)
+      if (!e) QV2_CUDA(c, cudaEventCreate(&e));
+  c->phase_timing = on != 0;
+  c->phase_marks_valid = false;
+  return QV2_OK;
+}
+
+extern "C" int qv2_calibrate_phase_ms(qv2_ctx* c, float* range_ms, float* hist_ms) {
+  if (!c || !range_ms || !hist_ms) return QV2_ERR_NULL;
+  if (!c->phase_timing || !c->phase_marks_valid) return QV2_ERR_UNSUPPORTED;
+  DeviceGuard guard(c->device);
+  ++c->syncs;
+  QV2_CUDA(c, cudaEventSynchronize(c->phase_ev[2]));
+  QV2_CUDA(c, cudaEventElapsedTime(range_ms, c->phase_ev[0], c->phase_ev[1]));
+  QV2_CUDA(c, cudaEventElapsedTime(hist_ms, c->phase_ev[1], c->phase_ev[2]));
+  return QV2_OK;
+}
+
 extern "C" uint32_t qv2_stage_count(const qv2_ctx* c) {
   return (c && c->plan_valid) ? (uint32_t)c->plan.stages.size() : 0u;
 }
@@ -433,6 +465,28 @@ int calibrate_impl(qv2_ctx* c, const qv2_tensor_desc* descs, uint32_t n, float* 
   int st = ensure_plan(c, descs, n);
   if (st != QV2_OK) return st;
   const CalibArgs a = calib_args(c, gmin, gmax, gabsmax, hist, clip, step, inv, offset, nonfinite);
+  if (c->phase_timing && c->plan.stages.size() == 1) {
+    // measurement aid: the two phases as separate launches with an event between them
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    QV2_CUDA(c, cudaStreamIsCapturing(c->stream, &cap));
+    if (cap == cudaStreamCaptureStatusNone) {
+      const Stage& sg = c->plan.stages[0];
+      const Launch l = launch_of(c);
+      c->phase_marks_valid = false;
+      QV2_CUDA(c, cudaEventRecord(c->phase_ev[0], c->stream));
+      QV2_CUDA(c, launch_range(l, sg, c->plan.any_16bit, c->d_tiles, a));
+      c->launches += sg.fused_fold ? 1 : (sg.tile_end > sg.tile_begin ? 2 : 1);
+      QV2_CUDA(c, cudaEventRecord(c->phase_ev[1], c->stream));
+      if (sg.any_percentile) {
+        QV2_CUDA(c, launch_hist(l, sg, c->plan.any_16bit, c->d_hist_tiles, a));
+        c->launches += sg.fused_fold ? 1 : (sg.hist_end > sg.hist_begin ? 2 : 1);
+      }
+      if ((st = run_group_percentile(c, n, a, group_hist, group_clip)) != QV2_OK) return st;
+      QV2_CUDA(c, cudaEventRecord(c->phase_ev[2], c->stream));
+      c->phase_marks_valid = true;
+      return QV2_OK;
+    }
+  }
   for (const Stage& sg : c->plan.stages)
     if ((st = run_calib_stage(c, sg, a)) != QV2_OK) return st;
   return run_group_percentile(c, n, a, group_hist, group_clip);

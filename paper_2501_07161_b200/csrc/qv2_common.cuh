@@ -137,6 +137,21 @@ struct Launch {
   bool pdl;            // launch as a programmatic dependent of the previous kernel in the stream
 };
 
+// Launches `kernel`; with l.pdl the launch may begin while the previous kernel of the stream is
+// still draining (programmatic dependent launch).  Every kernel launched this way calls
+// dependency_wait() before it reads or writes anything a previous kernel may touch.
+template <class... KArgs, class... Args>
+inline cudaError_t launch_kernel(const Launch& l, void (*kernel)(KArgs...), uint32_t grid, uint32_t block,
+                                 Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = 0; cfg.stream = l.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = l.pdl ? 1u : 0u;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(static_cast<Args&&>(args))...);
+}
+
 // Scratch and outputs of the calibration phases.  Accumulators (keys, counters, histograms,
 // tickets) are zero between passes: the CTA that folds a tensor clears what it consumed.
 struct CalibArgs {

@@ -9,6 +9,13 @@
 
 namespace qv2 {
 
+// Programmatic dependent launch.  dependency_wait(): returns once the kernel this launch depends
+// on has completed and its writes are visible (immediately when the launch was an ordinary one).
+// allow_dependents(): the next kernel of the stream may be scheduled as soon as every CTA of this
+// one has said so; its CTAs then wait in dependency_wait() for this kernel to finish.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Read-once data: bypass L1 allocation so the stream does not evict anything useful.
 __device__ __forceinline__ float4 ld_stream4(const float4* p) {
   float4 v;

@@ -142,6 +142,7 @@ hist_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ t
   __shared__ uint32_t s_last;
   for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
   __syncthreads();
+  dependency_wait();
   // percentile tensors without elements are owned by no CTA: CTA 0 folds them
   if (FOLD && blockIdx.x == 0)
     for (uint32_t t = scan_begin; t < scan_end; ++t)
@@ -190,6 +191,7 @@ hist_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ t
       }
     }
     if (!more) {
+      allow_dependents();          // this CTA is done: the next kernel may start to launch
       if (FOLD && owed != kNone) settle(owed);
       break;
     }
@@ -211,6 +213,8 @@ hist_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ t
 // One CTA per tensor of the stage: the fold, for stages whose streaming kernel does not fold.
 __global__ void __launch_bounds__(kThreads)
 clip_fold_kernel(const __grid_constant__ CalibArgs a, uint32_t tensor_begin) {
+  allow_dependents();
+  dependency_wait();
   const uint32_t t = tensor_begin + blockIdx.x;
   if (a.tensors[t].range_mode == QV2_PERCENTILE) clip_fold_tensor(a, t);
 }
@@ -414,16 +418,16 @@ cudaError_t launch_hist(const Launch& l, const Stage& st, bool any16, const Tile
   const Tile* tp = hist_tiles + st.hist_begin;
   if (st.fused_fold) {
     const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
-    if (any16) hist_kernel<true, true><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
-    else hist_kernel<false, true><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
-    return cudaGetLastError();
+    return any16 ? launch_kernel(l, hist_kernel<true, true>, st.hist_grid, kThreads, a, a.tensors, tp, n_tiles, s0, s1)
+                 : launch_kernel(l, hist_kernel<false, true>, st.hist_grid, kThreads, a, a.tensors, tp, n_tiles, s0, s1);
   }
   if (n_tiles) {
-    if (any16) hist_kernel<true, false><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
-    else hist_kernel<false, false><<<st.hist_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
+    const cudaError_t e = any16
+        ? launch_kernel(l, hist_kernel<true, false>, st.hist_grid, kThreads, a, a.tensors, tp, n_tiles, 0u, 0u)
+        : launch_kernel(l, hist_kernel<false, false>, st.hist_grid, kThreads, a, a.tensors, tp, n_tiles, 0u, 0u);
+    if (e != cudaSuccess) return e;
   }
-  clip_fold_kernel<<<st.tensor_end - st.tensor_begin, kThreads, 0, l.stream>>>(a, st.tensor_begin);
-  return cudaGetLastError();
+  return launch_kernel(l, clip_fold_kernel, st.tensor_end - st.tensor_begin, kThreads, a, st.tensor_begin);
 }
 
 }  // namespace qv2

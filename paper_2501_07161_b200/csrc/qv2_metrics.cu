@@ -141,10 +141,18 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
       for (uint32_t u = 0; u < U; ++u)
         metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * STRIDE) : nullptr);
     }
-    for (; j < s.nvec; j += STRIDE) {
-      const float4 vx = ld_vec_at(xb, j);
-      const float4 vy = PAIR ? ld_vec_at(yb, j) : vx;
-      metric_vec<MODE, OFF, CODES>(vx, vy, p, a, CODES ? cb + 4u * j : nullptr);
+    if (j < s.nvec) {               // at most U-1 groups are left for this thread: one predicated round, all loads in flight
+      float4 vx[U - 1], vy[U - 1];
+#pragma unroll
+      for (uint32_t u = 0; u < U - 1; ++u) {
+        const uint32_t k = min(j + u * STRIDE, s.nvec - 1u);       // in bounds, maybe unused
+        vx[u] = ld_vec_at(xb, k);
+        if (PAIR) vy[u] = ld_vec_at(yb, k); else vy[u] = vx[u];
+      }
+#pragma unroll
+      for (uint32_t u = 0; u < U - 1; ++u)
+        if (j + u * STRIDE < s.nvec)
+          metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * STRIDE) : nullptr);
     }
   } else {
     // x and y sit at different offsets inside their groups of four: vector loads for x, scalar for y
@@ -336,6 +344,7 @@ metrics_kernel(const __grid_constant__ MetricsArgs a, const TensorRec* __restric
   const float* __restrict__ inv = a.inv;
   const float* __restrict__ offset = a.offset;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  dependency_wait();
   // tensors without elements are owned by no CTA: CTA 0 folds them
   if (FOLD && blockIdx.x == 0)
     for (uint32_t t = scan_begin; t < scan_end; ++t)
@@ -416,6 +425,7 @@ metrics_kernel(const __grid_constant__ MetricsArgs a, const TensorRec* __restric
       run_xe = __dadd_rn(run_xe, (double)xe);
     }
   }
+  allow_dependents();            // this CTA has issued all its loads: the next kernel may start to launch
   if (cur != kNone) {
     flush(cur);
     if (FOLD) settle(cur);
@@ -426,6 +436,8 @@ metrics_kernel(const __grid_constant__ MetricsArgs a, const TensorRec* __restric
 template <bool COS>
 __global__ void __launch_bounds__(kThreads)
 metrics_fold_kernel(const __grid_constant__ MetricsArgs a, uint32_t tensor_begin) {
+  allow_dependents();
+  dependency_wait();
   metrics_fold_tensor<COS>(a, tensor_begin + blockIdx.x);
 }
 
@@ -554,18 +566,17 @@ cudaError_t launch_metrics(const Launch& l, const Stage& st, bool any16, const T
   const bool fold = st.fused_fold;
   const uint32_t s0 = fold && st.any_empty ? st.tensor_begin : 0u, s1 = fold && st.any_empty ? st.tensor_end : 0u;
 #define QV2_LAUNCH_METRICS(COS, A16, FOLD) \
-  metrics_kernel<COS, A16, FOLD><<<st.metrics_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1)
+  e = launch_kernel(l, metrics_kernel<COS, A16, FOLD>, st.metrics_grid, kThreads, a, a.tensors, tp, n_tiles, s0, s1)
 #define QV2_LAUNCH_METRICS_F(COS, A16) do { if (fold) QV2_LAUNCH_METRICS(COS, A16, true); else if (n_tiles) QV2_LAUNCH_METRICS(COS, A16, false); } while (0)
+  cudaError_t e = cudaSuccess;
   if (a.cosine) { if (any16) QV2_LAUNCH_METRICS_F(true, true); else QV2_LAUNCH_METRICS_F(true, false); }
   else { if (any16) QV2_LAUNCH_METRICS_F(false, true); else QV2_LAUNCH_METRICS_F(false, false); }
 #undef QV2_LAUNCH_METRICS_F
 #undef QV2_LAUNCH_METRICS
-  if (!fold) {
-    const uint32_t nt = st.tensor_end - st.tensor_begin;
-    if (a.cosine) metrics_fold_kernel<true><<<nt, kThreads, 0, l.stream>>>(a, st.tensor_begin);
-    else metrics_fold_kernel<false><<<nt, kThreads, 0, l.stream>>>(a, st.tensor_begin);
-  }
-  return cudaGetLastError();
+  if (e != cudaSuccess || fold) return e;
+  const uint32_t nt = st.tensor_end - st.tensor_begin;
+  return a.cosine ? launch_kernel(l, metrics_fold_kernel<true>, nt, kThreads, a, st.tensor_begin)
+                  : launch_kernel(l, metrics_fold_kernel<false>, nt, kThreads, a, st.tensor_begin);
 }
 
 cudaError_t launch_kl(const Launch& l, uint32_t grid_cap, const TensorRec* tensors, uint32_t n_tensors,

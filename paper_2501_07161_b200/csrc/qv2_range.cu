@@ -280,6 +280,7 @@ range_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ 
   __shared__ float sh[2 * kWarps];
   __shared__ uint32_t s_last;
   const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  dependency_wait();
   // tensors without elements are owned by no CTA: CTA 0 folds them (the planner asks for the
   // scan only when the stage has one)
   if (FOLD && blockIdx.x == 0)
@@ -338,6 +339,7 @@ range_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ 
         range_rows_tile(reinterpret_cast<const __nv_bfloat16*>(tr->x) + tl.begin, tl, tr, lane, warp, a.kmin, a.kmax, a.nf_acc);
     }
   }
+  allow_dependents();            // this CTA has issued all its loads: the next kernel may start to launch
   if (cur_tensor != kNone) {
     flush_group();
     if (FOLD) {
@@ -352,6 +354,8 @@ range_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ 
 // One CTA per tensor of the stage: the fold, for stages whose streaming kernel does not fold.
 __global__ void __launch_bounds__(kThreads)
 range_fold_kernel(const __grid_constant__ CalibArgs a, uint32_t tensor_begin) {
+  allow_dependents();
+  dependency_wait();
   range_fold_tensor(a, tensor_begin + blockIdx.x);
 }
 
@@ -368,16 +372,16 @@ cudaError_t launch_range(const Launch& l, const Stage& st, bool any16, const Til
   const Tile* tp = tiles + st.tile_begin;
   if (st.fused_fold) {
     const uint32_t s0 = st.any_empty ? st.tensor_begin : 0u, s1 = st.any_empty ? st.tensor_end : 0u;
-    if (any16) range_kernel<true, true><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
-    else range_kernel<false, true><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, s0, s1);
-    return cudaGetLastError();
+    return any16 ? launch_kernel(l, range_kernel<true, true>, st.range_grid, kThreads, a, a.tensors, tp, n_tiles, s0, s1)
+                 : launch_kernel(l, range_kernel<false, true>, st.range_grid, kThreads, a, a.tensors, tp, n_tiles, s0, s1);
   }
   if (n_tiles) {
-    if (any16) range_kernel<true, false><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
-    else range_kernel<false, false><<<st.range_grid, kThreads, 0, l.stream>>>(a, a.tensors, tp, n_tiles, 0u, 0u);
+    const cudaError_t e = any16
+        ? launch_kernel(l, range_kernel<true, false>, st.range_grid, kThreads, a, a.tensors, tp, n_tiles, 0u, 0u)
+        : launch_kernel(l, range_kernel<false, false>, st.range_grid, kThreads, a, a.tensors, tp, n_tiles, 0u, 0u);
+    if (e != cudaSuccess) return e;
   }
-  range_fold_kernel<<<st.tensor_end - st.tensor_begin, kThreads, 0, l.stream>>>(a, st.tensor_begin);
-  return cudaGetLastError();
+  return launch_kernel(l, range_fold_kernel, st.tensor_end - st.tensor_begin, kThreads, a, st.tensor_begin);
 }
 
 }  // namespace qv2

@@ -22,6 +22,8 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
             const uint64_t* __restrict__ macs, const double* __restrict__ pos,
             const uint32_t* __restrict__ fuse_group, qv2_rank_cfg cfg, double* score, double* severity,
             uint32_t* place, uint32_t* best, uint32_t* order, uint8_t* keep, uint32_t* n_keep) {
+  allow_dependents();
+  dependency_wait();
   // Models have tens of layers: up to kStage layers every input and every intermediate lives in
   // shared memory, so the phases below cost one trip to global memory at the start and one at the
   // end instead of one per phase.  Larger n runs the same code on the global arrays.
@@ -176,10 +178,8 @@ cudaError_t launch_rank(const Launch& l, uint32_t n, const double* sqnr_w, const
                         uint32_t* order, uint8_t* keep, uint32_t* n_keep) {
   // scratch: kMaxRankLayers doubles each for score and severity, then two uint32 arrays
   uint32_t* place = reinterpret_cast<uint32_t*>(scratch + 2 * (size_t)kMaxRankLayers);
-  rank_kernel<<<1, 256, 0, l.stream>>>(n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, fuse_group, cfg,
-                                       scratch, scratch + kMaxRankLayers, place, place + kMaxRankLayers,
-                                       order, keep, n_keep);
-  return cudaGetLastError();
+  return launch_kernel(l, rank_kernel, 1u, 256u, n, sqnr_w, mse_w, sqnr_a, mse_a, macs, pos, fuse_group, cfg, scratch,
+                       scratch + kMaxRankLayers, place, place + kMaxRankLayers, order, keep, n_keep);
 }
 
 }  // namespace qv2

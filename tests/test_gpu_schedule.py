@@ -76,16 +76,18 @@ def test_l2_chunked_schedule_matches_oracle_and_phase_major(name, batch, chunk, 
         a.close(); b.close()
 
 
-def test_auto_schedule_picks_by_size():
+def test_schedule_selection():
+    """AUTO takes the schedule that measured faster, which on a B200 is phase-major at every size;
+    the chunked schedule is there on request and an unknown value is refused."""
     ctx = q.Context(0)
     try:
-        ctx.set_schedule(q.SCHEDULE_AUTO, 1 << 20)
-        small = gen.make_model("squeezenet", seed=1, device="cuda", batch=1, layer_indices=range(2))
-        _sweep(ctx, small)
-        n_small = ctx.stages
         big = gen.make_model("squeezenet", seed=1, device="cuda", batch=1)
+        ctx.set_schedule(q.SCHEDULE_AUTO, 1 << 20)
         _sweep(ctx, big)
-        assert ctx.stages > 1 and n_small >= 1
+        assert ctx.stages == 1
+        ctx.set_schedule(q.SCHEDULE_L2_CHUNKED, 1 << 20)
+        _sweep(ctx, big)
+        assert ctx.stages > 1
         ctx.set_schedule(q.SCHEDULE_PHASE_MAJOR)
         _sweep(ctx, big)
         assert ctx.stages == 1

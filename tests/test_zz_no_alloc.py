@@ -4,7 +4,8 @@ Some users of this library run it where cudaMalloc is forbidden -- a server that
 memory to its own pool at start-up, a latency-critical loop in which an allocation would stall the
 GPU, a host callback.  For them the library offers one entry point that needs no context and keeps
 its partial sums in a fixed 1 MiB array inside the library image.  These tests call it through the
-C ABI and compare it with the regular qv2_quant_metrics on the same inputs and parameters, twice
+C ABI and compare it with the regular qv2_quant_metrics on the same inputs and parameters and,
+independently, with the CPU oracle (the same 1e-5 / 1e-3 dB bars, so no two tolerances stack), twice
 in a row (the array is shared between calls and still holds the previous call's data, so the
 second call is the one that would expose stale state), and check that a tensor beyond the stated
 limit is refused with QV2_ERR_SIZE instead of being launched.
@@ -14,9 +15,11 @@ other test.  It passes on its own in a fresh process and after the rest of the s
 """
 import math
 
+import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2501_07161_b200 as q
 from paper_2501_07161_b200 import binding as B
 
@@ -40,6 +43,10 @@ def _cases():
     w = torch.randn(96 * 1153, generator=_gen(3), device="cuda")            # short ragged rows
     wl = torch.randn(3 * 20000, generator=_gen(4), device="cuda")           # rows cut at row ends
     a = torch.randn(4 * 6 * 500, generator=_gen(5), device="cuda").clamp_min(0)
+    s = torch.randn(5 * 37 * 9, generator=_gen(6), device="cuda")           # rows of nine elements
+    s2 = s + 0.05 * torch.randn(5 * 37 * 9, generator=_gen(9), device="cuda")
+    m = torch.randn(3 * 70 * 300, generator=_gen(10), device="cuda") + 0.7   # 54 rows per tile, three tiles and a tail
+    m2 = m + 0.03 * torch.randn(3 * 70 * 300, generator=_gen(11), device="cuda")
     return [
         ("activation pair, asymmetric, offset != 0", x, y, (1, 1, n), B.PER_TENSOR, B.ASYM_U8, B.MINMAX, 0),
         ("activation pair, raw difference", x, y, (1, 1, n), B.PER_TENSOR, B.ASYM_U8, B.MINMAX, B.PAIR_RAW),
@@ -48,7 +55,27 @@ def _cases():
         ("relu activation, per channel with batch, percentile", a, None, (4, 6, 500), B.PER_CHANNEL,
          B.ASYM_U8, B.PERCENTILE, 0),
         ("one element", x[:1].clone(), None, (1, 1, 1), B.PER_TENSOR, B.SYM_I8, B.ABSMAX, 0),
+        ("rows shorter than a warp, per channel, pair", s, s2, (5, 37, 9), B.PER_CHANNEL, B.ASYM_U8, B.MINMAX, 0),
+        ("rows shorter than a warp, weights", s, None, (1, 185, 9), B.PER_CHANNEL, B.SYM_I8, B.ABSMAX, 0),
+        ("per channel, row count per tile not a multiple of eight", m, m2, (3, 70, 300), B.PER_CHANNEL,
+         B.ASYM_U8, B.MINMAX, 0),
+        ("integer zero point, per tensor", x + 0.4, y + 0.4, (1, 1, n), B.PER_TENSOR, B.ASYM_U8_ZP, B.MINMAX, 0),
+        ("integer zero point, per channel", m, m2, (3, 70, 300), B.PER_CHANNEL, B.ASYM_U8_ZP, B.MINMAX, 0),
+        ("4-bit symmetric weights", w, None, (1, 96, 1153), B.PER_CHANNEL, B.SYM_I8, B.ABSMAX, 4 << 8),
+        ("4-bit affine activations", x, y, (1, 1, n), B.PER_TENSOR, B.ASYM_U8, B.MINMAX, 4 << 8),
     ]
+
+
+def _oracle4(x, y, shape, gran, scheme, rng, flags, step, inv, offset):
+    """The oracle's metrics for the parameters the call is given (the GPU calibration's bits, which the
+    parity tests pin to the oracle's own)."""
+    o, c, i = shape
+    bits = ((flags >> 8) & 0xFF) or 8
+    mode = oracle.PAIR_SELF if y is None else (oracle.PAIR_RAW if flags & B.PAIR_RAW else oracle.PAIR_REQUANT)
+    r = oracle.quant_metrics(x.cpu().numpy(), None if y is None else y.cpu().numpy(), o, c, i,
+                             gran == B.PER_CHANNEL, int(scheme), mode, step.cpu().numpy(), inv.cpu().numpy(),
+                             offset.cpu().numpy(), bits=bits)
+    return r["sse"], r["sig"], r["mse"], r["sqnr_db"]
 
 
 def _close(got, ref, what):
@@ -73,12 +100,19 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
             ref = ctx.quant_metrics(descs, cal.step, cal.inv, cal.offset)
             torch.cuda.synchronize()
             ref4 = (ref.sse[0], ref.sig[0], ref.mse[0], ref.sqnr_db[0])
+            # the oracle calibrates to the same parameter bits, so both references see one quantizer
+            oc = oracle.calibrate_tensor(x.cpu().numpy(), o, c, i, gran == B.PER_CHANNEL, int(scheme),
+                                         0.999 if rng == B.PERCENTILE else None, ((flags >> 8) & 0xFF) or 8)
+            assert np.array_equal(cal.step.cpu().numpy().view(np.uint32), oc[6].view(np.uint32)), name
+            assert np.array_equal(cal.offset.cpu().numpy().view(np.uint32), oc[8].view(np.uint32)), name
+            ora4 = _oracle4(x, y, (o, c, i), gran, scheme, rng, flags, cal.step, cal.inv, cal.offset)
             for call in (1, 2):
                 out = torch.full((4,), float("nan"), dtype=torch.float64, device="cuda")
                 st = B.quant_metrics_noalloc(desc, cal.step, cal.inv, cal.offset, out)
                 assert st == 0, f"{name}: status {st}"
                 torch.cuda.synchronize()
-                _close(out.tolist(), ref4, f"{name} (call {call})")
+                _close(out.tolist(), ref4, f"{name} (call {call}, against qv2_quant_metrics)")
+                _close(out.tolist(), ora4, f"{name} (call {call}, against the oracle)")
     finally:
         ctx.close()
 
@@ -98,6 +132,8 @@ def test_noalloc_after_a_larger_tensor_ignores_stale_partials():
             assert B.quant_metrics_noalloc(desc, cal.step, cal.inv, cal.offset, out) == 0
             torch.cuda.synchronize()
             _close(out.tolist(), (ref.sse[0], ref.sig[0], ref.mse[0], ref.sqnr_db[0]), f"n={t.numel()}")
+            _close(out.tolist(), _oracle4(t, None, (1, 1, t.numel()), B.PER_TENSOR, B.SYM_I8, B.ABSMAX, 0,
+                                          cal.step, cal.inv, cal.offset), f"n={t.numel()} against the oracle")
     finally:
         ctx.close()
 
