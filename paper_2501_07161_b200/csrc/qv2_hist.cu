@@ -20,17 +20,29 @@ __device__ __forceinline__ uint32_t bin_of(float v, float w) {
   return min(b, (uint32_t)(kBins - 1));
 }
 
+// Two bins are counted in registers instead of shared memory: bin 0 (half of a post-ReLU tensor
+// sits there) and the top bin (every element that a ReLU6 or another saturating layer clipped sits
+// at absmax).  Both would otherwise be many lanes of a warp adding to one shared-memory word.
+struct EdgeCount {
+  uint32_t lo, hi;
+};
 template <bool CAREFUL>
-__device__ __forceinline__ void hist_elem(float v, float w, uint32_t* sh, uint32_t& zeros) {
+__device__ __forceinline__ void hist_elem(float v, float w, uint32_t* sh, EdgeCount& edge) {
   if (CAREFUL && !isfinite(v)) return;
   const uint32_t b = bin_of(v, w);
-  if (b == 0) ++zeros;                 // bin 0 (half of a post-ReLU tensor) stays in a register
+  if (b == 0) ++edge.lo;
+  else if (b == (uint32_t)(kBins - 1)) ++edge.hi;
   else atomicAdd(sh + b, 1u);
+}
+__device__ __forceinline__ void flush_edges(uint32_t* sh, EdgeCount& edge) {
+  if (edge.lo) atomicAdd(sh, edge.lo);
+  if (edge.hi) atomicAdd(sh + (kBins - 1), edge.hi);
+  edge.lo = 0; edge.hi = 0;
 }
 
 template <bool CAREFUL, class T>
 __device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t count, float w,
-                                          uint32_t* sh, uint32_t& zeros) {
+                                          uint32_t* sh, EdgeCount& zeros) {
   const FlatSplit s = split_flat(x, count);
   const T* xv = x + s.head;
   constexpr uint32_t U = 4;
@@ -63,7 +75,7 @@ __device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t coun
 
 template <class T>
 __device__ __forceinline__ void hist_tile(const T* x, uint32_t count, float w, bool careful, uint32_t* sh,
-                                          uint32_t& zeros) {
+                                          EdgeCount& zeros) {
   if (careful) hist_flat<true>(x, count, w, sh, zeros);
   else hist_flat<false>(x, count, w, sh, zeros);
 }
@@ -149,7 +161,8 @@ hist_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ t
       if (tensors[t].range_mode == QV2_PERCENTILE && tensors[t].hist_ctas == 0) clip_fold_tensor(a, t);
 
   constexpr uint32_t kNone = 0xffffffffu;
-  uint32_t cur = kNone, since_flush = 0, zeros = 0;
+  uint32_t cur = kNone, since_flush = 0;
+  EdgeCount zeros = {0u, 0u};
   uint32_t owed = kNone, drawn = 0;   // FOLD: the tensor before cur and the ticket thread 0 drew for it
   float w = 0.0f;
   bool careful = false;
@@ -174,8 +187,7 @@ hist_kernel(const __grid_constant__ CalibArgs a, const TensorRec* __restrict__ t
     // 32-bit count could overflow (2^14 tiles of 2^14 elements)
     const bool leaving = cur != kNone && (!more || tl.tensor != cur);
     if (leaving || (cur != kNone && since_flush >= 16384u)) {
-      if (zeros) atomicAdd(sh, zeros);
-      zeros = 0;
+      flush_edges(sh, zeros);
       __syncthreads();
       unsigned long long* h = a.hist_acc + (size_t)tensors[cur].hist_index * kBins;
       for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {
@@ -235,7 +247,7 @@ __device__ __forceinline__ float bin_scale(float A) {
 // One segment handled by one warp: 16-byte loads over the aligned body, scalars at the ends.
 template <bool CAREFUL, class T>
 __device__ __forceinline__ void hist_segment_warp(const T* __restrict__ x, uint32_t count, uint32_t lane,
-                                                  float w, uint32_t* sh, uint32_t& zeros) {
+                                                  float w, uint32_t* sh, EdgeCount& zeros) {
   const FlatSplit s = split_flat(x, count);
   const T* xv = x + s.head;
   uint32_t j = lane;
@@ -268,7 +280,7 @@ constexpr uint32_t kWarpSegmentMax = 4096;     // shorter segments go one per wa
 
 template <class T>
 __device__ __forceinline__ void group_hist_unit(const T* x, const Tile& u, uint64_t seg_stride, float w,
-                                                bool careful, uint32_t* sh, uint32_t& zeros) {
+                                                bool careful, uint32_t* sh, EdgeCount& zeros) {
   if (u.count >= kWarpSegmentMax) {
     for (uint32_t r = 0; r < u.rows; ++r) hist_tile(x + r * seg_stride, u.count, w, careful, sh, zeros);
   } else {
@@ -295,12 +307,12 @@ group_hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict_
     const float w = bin_scale(gabsmax[tr->group_base + g]);
     const bool careful = nonfinite[u.tensor] != 0ull;
     const uint64_t seg_stride = (uint64_t)tr->channels * tr->inner;
-    uint32_t zeros = 0;
+    EdgeCount zeros = {0u, 0u};
     if (!ANY16 || tr->dtype == kF32) group_hist_unit(reinterpret_cast<const float*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
     else if (tr->dtype == kF16) group_hist_unit(reinterpret_cast<const __half*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
     else group_hist_unit(reinterpret_cast<const __nv_bfloat16*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
     // merge: a unit holds fewer than 2^32 elements, so the 32-bit counts cannot have wrapped
-    if (zeros) atomicAdd(sh, zeros);
+    flush_edges(sh, zeros);
     __syncthreads();
     unsigned long long* h = ghist + (size_t)(tr->ghist_first + g) * kBins;
     for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {

@@ -195,51 +195,145 @@ __device__ __forceinline__ void load_params(QP& p, const TensorRec* tr, const fl
 // A tile of whole rows.  Kept out of line: these walkers run for a small share of the bytes (weight
 // rows, small feature maps), and inlined into the tile loop they compete with the flat path for
 // its registers.  Returns the tile's sums folded into one accumulator.
+//
+// The metrics are sums over the whole tensor; only the quantization parameters change from row to
+// row.  A tile of rows shorter than kPieceRow is therefore streamed like a flat run by the whole CTA
+// (16-byte loads, several in flight per thread) and every vector fetches the parameters of the row
+// it lies in; these loads hit L1, since neighbouring vectors share a row.  That needs rows of a
+// multiple of four elements and a 16-byte aligned tile; otherwise the tile is walked one element
+// per thread.  (For long rows the index arithmetic per vector costs more than it saves.)
+struct RowParams {
+  const TensorRec* tr;
+  const float* __restrict__ step;
+  const float* __restrict__ inv;
+  const float* __restrict__ offset;
+  uint32_t inner, channels, row0c, gbase;
+  float top, qmin0;
+  bool zp;
+  __device__ __forceinline__ RowParams(const Tile& tl, const TensorRec* t, const float* s, const float* i, const float* o)
+      : tr(t), step(s), inv(i), offset(o), inner((uint32_t)t->inner), channels(t->channels),
+        row0c((uint32_t)(tl.row0 % t->channels)), gbase(t->group_base), top(top_code(t->asym != 0, t->bits)),
+        qmin0(t->asym ? 0.0f : -top_code(false, t->bits)), zp(t->asym == 2) {}
+  // parameters of the row that holds element e of the tile (same values as load_params)
+  __device__ __forceinline__ QP of_elem(uint32_t e) const {
+    const uint32_t G = gbase + (row0c + e / inner) % channels;
+    QP p;
+    p.step = __ldg(step + G); p.inv = __ldg(inv + G);
+    const float off = __ldg(offset + G);
+    const float z = zp ? off : 0.0f;
+    p.off = zp ? 0.0f : off;
+    p.bias = z; p.qmin = qmin0 - z; p.qmax = top - z;
+    return p;
+  }
+};
+
+template <uint32_t MODE, bool OFF, bool CODES, class T, class ACC>
+__device__ __forceinline__ void metric_rows_vec(const T* __restrict__ x, const T* __restrict__ y, uint8_t* codes,
+                                                uint32_t count, const RowParams& rp, ACC* a) {
+  constexpr bool PAIR = MODE != kSelf;
+  constexpr uint32_t U = 4;
+  const uint32_t nvec = count >> 2;
+  uint32_t j = threadIdx.x;
+  for (; j < nvec; j += U * kThreads) {          // the last round is clamped: loads in bounds, maybe unused
+    float4 vx[U], vy[U];
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) {
+      const uint32_t k = min(j + u * kThreads, nvec - 1u);
+      vx[u] = ld_vec_at(x, k);
+      if (PAIR) vy[u] = ld_vec_at(y, k); else vy[u] = vx[u];
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) {
+      const uint32_t k = j + u * kThreads;
+      if (k < nvec) {
+        const QP p = rp.of_elem(4u * k);
+        metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? codes + 4u * k : nullptr);
+      }
+    }
+  }
+}
+
+template <uint32_t MODE, bool OFF, bool CODES, class T, class ACC>
+__device__ __forceinline__ void metric_rows_scalar(const T* __restrict__ x, const T* __restrict__ y, uint8_t* codes,
+                                                   uint32_t count, const RowParams& rp, ACC* a) {
+  uint32_t e = threadIdx.x;
+  for (; e + 3u * kThreads < count; e += 4u * kThreads) {
+    float vx[4], vy[4];
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u) {
+      vx[u] = Ld<T>::one(x + e + u * kThreads);
+      vy[u] = (MODE != kSelf) ? Ld<T>::one(y + e + u * kThreads) : 0.0f;
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u) {
+      const uint32_t i = e + u * kThreads;
+      const QP p = rp.of_elem(i);
+      metric_elem<MODE, OFF, CODES>(vx[u], vy[u], p, a[u], CODES ? codes + i : nullptr);
+    }
+  }
+  for (; e < count; e += kThreads) {
+    const QP p = rp.of_elem(e);
+    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + e), (MODE != kSelf) ? Ld<T>::one(y + e) : 0.0f, p, a[0],
+                                  CODES ? codes + e : nullptr);
+  }
+}
+
+// Rows of kPieceRow elements or more: the tile is cut into one contiguous chunk per warp (a multiple
+// of four elements); a warp walks its chunk row piece by row piece with the flat walker, fetching
+// the row's parameters once per piece.  Eight independent streams whatever the row length.
+constexpr uint32_t kPieceRow = 512;
+
+template <uint32_t MODE, bool CODES, class T, class ACC>
+__device__ __forceinline__ void metric_rows_pieces(const T* __restrict__ x, const T* __restrict__ y, uint8_t* codes,
+                                                   const Tile& tl, const TensorRec* tr,
+                                                   const float* __restrict__ step, const float* __restrict__ inv,
+                                                   const float* __restrict__ offset, ACC* a) {
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+  const uint32_t chunk = (tl.count + 4u * kWarps - 1u) / (4u * kWarps) * 4u;
+  uint32_t c0 = min(warp * chunk, tl.count);
+  const uint32_t c1 = min(c0 + chunk, tl.count);
+  uint32_t row = c0 / inner;
+  uint32_t row_end = (row + 1u) * inner;
+  uint32_t g = (uint32_t)((tl.row0 + row) % channels);
+  QP p;
+  while (c0 < c1) {
+    const uint32_t p1 = min(c1, row_end);
+    load_params(p, tr, step, inv, offset, tr->group_base + g);
+    if (MODE == kRaw || p.off == 0.0f)
+      metric_flat<MODE, false, CODES, 32>(x + c0, y + c0, codes + c0, p1 - c0, p, a, lane);
+    else
+      metric_flat<MODE, true, CODES, 32>(x + c0, y + c0, codes + c0, p1 - c0, p, a, lane);
+    c0 = p1; row_end += inner;
+    if (++g == channels) g = 0;
+  }
+}
+
 template <uint32_t MODE, bool CODES, class T, class ACC>
 __device__ __noinline__ ACC metric_rows(Tile tl, const TensorRec* tr, const float* __restrict__ step,
                                         const float* __restrict__ inv, const float* __restrict__ offset,
                                         uint8_t* codes_base, ACC seed) {
-  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
   const T* x = reinterpret_cast<const T*>(tr->x) + tl.begin;
   const T* y = (MODE != kSelf) ? reinterpret_cast<const T*>(tr->y) + tl.begin : nullptr;
   uint8_t* codes = CODES ? codes_base + tl.begin : nullptr;
-  const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
   ACC a[4] = {seed, seed, seed, seed};
-  QP p;
-  if (inner >= kShortRow) {                            // one warp per row
-    for (uint32_t r = warp; r < tl.rows; r += kWarps) {
-      load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)((tl.row0 + r) % channels));
-      const uint64_t o = (uint64_t)r * inner;
-      if (MODE == kRaw || p.off == 0.0f)
-        metric_flat<MODE, false, CODES, 32>(x + o, y + o, codes + o, inner, p, a, lane);
-      else
-        metric_flat<MODE, true, CODES, 32>(x + o, y + o, codes + o, inner, p, a, lane);
-    }
+  if (tr->inner >= kPieceRow) {
+    metric_rows_pieces<MODE, CODES>(x, y, codes, tl, tr, step, inv, offset, a);
+    return ACC::fold(a);
+  }
+  const RowParams rp(tl, tr, step, inv, offset);
+  constexpr uintptr_t kVecMask = 4u * sizeof(T) - 1u;
+  const bool vec = (rp.inner & 3u) == 0 && (((uintptr_t)x) & kVecMask) == 0 &&
+                   (MODE == kSelf || (((uintptr_t)y) & kVecMask) == 0);
+  // a real-valued offset needs the form of the arithmetic that splits x - offset exactly; with a
+  // zero offset both forms give the same value
+  const bool off = MODE != kRaw && tr->asym == 1;
+  if (vec) {
+    if (off) metric_rows_vec<MODE, MODE != kRaw, CODES>(x, y, codes, tl.count, rp, a);
+    else metric_rows_vec<MODE, false, CODES>(x, y, codes, tl.count, rp, a);
   } else {
-    // Rows shorter than kShortRow (3x3 depthwise filters, 7x7 maps, one element per channel): one
-    // element per thread, each fetching the parameters of its own row's group.  The offset form of
-    // the arithmetic is used throughout; with a zero offset it gives the same value.
-    const uint32_t row0c = (uint32_t)(tl.row0 % channels);
-    uint32_t e = threadIdx.x;
-    for (; e + 3u * kThreads < tl.count; e += 4u * kThreads) {
-      float vx[4], vy[4];
-#pragma unroll
-      for (uint32_t u = 0; u < 4; ++u) {
-        vx[u] = Ld<T>::one(x + e + u * kThreads);
-        vy[u] = (MODE != kSelf) ? Ld<T>::one(y + e + u * kThreads) : 0.0f;
-      }
-#pragma unroll
-      for (uint32_t u = 0; u < 4; ++u) {
-        const uint32_t i = e + u * kThreads;
-        load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)(((uint64_t)row0c + i / inner) % channels));
-        metric_elem<MODE, MODE != kRaw, CODES>(vx[u], vy[u], p, a[u], CODES ? codes + i : nullptr);
-      }
-    }
-    for (; e < tl.count; e += kThreads) {
-      load_params(p, tr, step, inv, offset, tr->group_base + (uint32_t)(((uint64_t)row0c + e / inner) % channels));
-      metric_elem<MODE, MODE != kRaw, CODES>(Ld<T>::one(x + e), (MODE != kSelf) ? Ld<T>::one(y + e) : 0.0f, p, a[0],
-                                             CODES ? codes + e : nullptr);
-    }
+    if (off) metric_rows_scalar<MODE, MODE != kRaw, CODES>(x, y, codes, tl.count, rp, a);
+    else metric_rows_scalar<MODE, false, CODES>(x, y, codes, tl.count, rp, a);
   }
   return ACC::fold(a);
 }
@@ -746,7 +840,7 @@ extern "C" int qv2_quant_metrics_noalloc(int device, void* stream, const qv2_ten
   if (!job.tr.per_channel || ne == 0) {
     job.cut = 0;
     n_tiles = (ne + kTileElems - 1) / kTileElems;
-  } else if (d.inner >= kRowTileMin) {
+  } else if (d.inner >= 4096) {          // this entry point keeps its own cut: long rows at row boundaries
     job.cut = 1;
     job.tiles_per_row = (uint32_t)((d.inner + kTileElems - 1) / kTileElems);
     n_tiles = rows * job.tiles_per_row;

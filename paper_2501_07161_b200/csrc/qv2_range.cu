@@ -94,23 +94,34 @@ __device__ __forceinline__ void range_flat_tile(const T* x, uint32_t count, Rang
   }
 }
 
-// A tile of whole rows, each at least kShortRow long: one warp per row, one publication per row.
+// A tile of whole rows, each at least kShortRow long.  The tile's elements are cut into one
+// contiguous chunk per warp (a multiple of four elements, so a 16-byte aligned tile stays
+// aligned); a warp walks its chunk row piece by row piece and publishes each piece's range to the
+// row's group.  Eight independent streams per CTA whatever the row length: a tile of two rows of
+// 8000 elements keeps every warp as busy as a tile of sixty rows of 270.
 template <class T>
 __device__ __forceinline__ void range_rows_tile(const T* x, const Tile& tl, const TensorRec* tr, uint32_t lane,
                                                 uint32_t warp, uint32_t* kmin, uint32_t* kmax,
                                                 unsigned long long* nonfinite) {
   const uint32_t inner = (uint32_t)tr->inner, channels = tr->channels;
+  const uint32_t chunk = (tl.count + 4u * kWarps - 1u) / (4u * kWarps) * 4u;
+  uint32_t c0 = min(warp * chunk, tl.count);
+  const uint32_t c1 = min(c0 + chunk, tl.count);
+  uint32_t row = c0 / inner;
+  uint32_t row_end = (row + 1u) * inner;
+  uint32_t g = (uint32_t)((tl.row0 + row) % channels);
   RangeAcc b;
-  for (uint32_t r = warp; r < tl.rows; r += kWarps) {
-    const T* row = x + (uint64_t)r * inner;
+  while (c0 < c1) {
+    const uint32_t p1 = min(c1, row_end);
     reset(b);
-    range_flat<false, 32>(row, inner, b, lane);
+    range_flat<false, 32>(x + c0, p1 - c0, b, lane);
     if (__any_sync(0xffffffffu, b.nanflag != b.nanflag)) {
       reset(b);
-      range_flat<true, 32>(row, inner, b, lane);
+      range_flat<true, 32>(x + c0, p1 - c0, b, lane);
     }
-    const uint32_t g = (uint32_t)((tl.row0 + r) % channels);
     publish(b, lane, kmin, kmax, tr->group_base + g, nonfinite + tl.tensor);
+    c0 = p1; row_end += inner;
+    if (++g == channels) g = 0;
   }
 }
 

@@ -47,7 +47,7 @@ def _desc(outer, ch, inner, per_channel, ptr=4096, percentile=None):
 
 
 @pytest.mark.parametrize("outer,ch,inner,pc", [(1, 1, 1, False), (1, 1, 5 * TILE + 3, False),
-                                               (1, 960, 9, True), (1, 64, 576, True), (64, 256, 3136, True), (2, 9, 127, True), (2, 9, 128, True), (1, 7, 4096, True),
+                                               (1, 960, 9, True), (1, 64, 576, True), (64, 256, 3136, True), (2, 9, 127, True), (2, 9, 128, True), (1, 7, 4096, True), (5, 3, 9000, True), (1, 4, TILE - 1, True),
                                                (1, 3, 25088, True), (3, 5, 4095, True), (2, 3, 40000, True),
                                                (1, 1, TILE, True), (4, 1, 1, True)])
 def test_tiles_cover_every_element_once(outer, ch, inner, pc):
@@ -57,10 +57,10 @@ def test_tiles_cover_every_element_once(outer, ch, inner, pc):
     mine = [t for t in tiles if t[0] == 0]
     pos = 0
     for tensor, begin, count, kind in mine:
-        assert begin == pos and 0 < count <= (2 * TILE if kind == 1 else TILE)
-        if kind == 1:                       # whole rows only; rows walked one per warp come in eights
-            assert begin % inner == 0 and count % inner == 0
-            assert inner < 128 or (count // inner) % 8 == 0 or begin + count == n
+        assert begin == pos and 0 < count <= TILE
+        if kind == 1:                       # whole rows only, as many as fit a tile
+            assert begin % inner == 0 and count % inner == 0 and inner < TILE
+            assert count // inner == max(1, TILE // inner) or begin + count == n
         elif pc:                            # one-group tile never crosses a row
             assert begin // inner == (begin + count - 1) // inner
         pos += count
