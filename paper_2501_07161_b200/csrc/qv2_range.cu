@@ -35,15 +35,72 @@ __device__ __forceinline__ void range_acc4(RangeAcc& a, const float4& v) {
   range_acc<CAREFUL>(a, v.z); range_acc<CAREFUL>(a, v.w);
 }
 
+// 16-bit elements, fast path: minimum, maximum and the non-finite detector are taken two elements
+// per instruction in the storage format itself (minimum and maximum are exact in any format, and
+// v*0 is NaN for a NaN or an infinity in any format), and widened to binary32 once per run.
+template <class T> struct Packed2;
+template <> struct Packed2<__half> {
+  using type = __half2;
+  static __device__ __forceinline__ type both(unsigned short bits) { return __half2half2(__ushort_as_half(bits)); }
+  static constexpr unsigned short kPosInf = 0x7c00u, kNegInf = 0xfc00u;
+};
+template <> struct Packed2<__nv_bfloat16> {
+  using type = __nv_bfloat162;
+  static __device__ __forceinline__ type both(unsigned short bits) {
+    return __bfloat162bfloat162(__ushort_as_bfloat16(bits));
+  }
+  static constexpr unsigned short kPosInf = 0x7f80u, kNegInf = 0xff80u;
+};
+
+template <uint32_t STRIDE, class T>
+__device__ __forceinline__ void range_flat_packed(const T* __restrict__ x, uint32_t count, RangeAcc& a, uint32_t tid) {
+  using P = Packed2<T>;
+  using V = typename P::type;
+  const FlatSplit s = split_flat(x, count);
+  const T* xv = x + s.head;
+  constexpr uint32_t U = 16;                             // 8-byte loads: the same bytes in flight as 8 x 16
+  V mn = P::both(P::kPosInf), mx = P::both(P::kNegInf), flag = P::both(0), zero = P::both(0);
+  auto take = [&](const uint2& r) {
+    const V v0 = *reinterpret_cast<const V*>(&r.x), v1 = *reinterpret_cast<const V*>(&r.y);
+    mn = __hmin2(mn, v0); mx = __hmax2(mx, v0); flag = __hfma2(v0, zero, flag);
+    mn = __hmin2(mn, v1); mx = __hmax2(mx, v1); flag = __hfma2(v1, zero, flag);
+  };
+  uint32_t j = tid;
+  for (; j + (U - 1) * STRIDE < s.nvec; j += U * STRIDE) {
+    uint2 r[U];
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) r[u] = ld_stream_u2(xv + 4 * (size_t)(j + u * STRIDE));
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) take(r[u]);
+  }
+  if (j < s.nvec) {                 // at most U-1 groups are left for this thread: one predicated round
+    uint2 r[U - 1];
+#pragma unroll
+    for (uint32_t u = 0; u < U - 1; ++u) r[u] = ld_stream_u2(xv + 4 * (size_t)min(j + u * STRIDE, s.nvec - 1u));
+#pragma unroll
+    for (uint32_t u = 0; u < U - 1; ++u)
+      if (j + u * STRIDE < s.nvec) take(r[u]);
+  }
+  a.mn = fminf(a.mn, fminf((float)mn.x, (float)mn.y));
+  a.mx = fmaxf(a.mx, fmaxf((float)mx.x, (float)mx.y));
+  a.nanflag = __fadd_rn(a.nanflag, __fadd_rn((float)flag.x, (float)flag.y));     // NaN if any element was not finite
+  if (tid < s.head) range_acc<false>(a, Ld<T>::one(x + tid));
+  if (tid < s.tail) range_acc<false>(a, Ld<T>::one(x + s.head + 4u * s.nvec + tid));
+}
+
 // This thread's share of a flat run walked by STRIDE threads (the whole CTA, or one warp with
 // tid = lane): group of four number j for j = tid, tid+STRIDE, ...; the first `head` and last
 // `tail` scalars go to threads 0..2.  T is the element type in memory.
 template <bool CAREFUL, uint32_t STRIDE = kThreads, class T>
 __device__ __forceinline__ void range_flat(const T* __restrict__ x, uint32_t count, RangeAcc& a,
                                            uint32_t tid = threadIdx.x) {
+  if constexpr (sizeof(T) == 2 && !CAREFUL) {
+    range_flat_packed<STRIDE>(x, count, a, tid);
+    return;
+  }
   const FlatSplit s = split_flat(x, count);
   const T* xv = x + s.head;
-  constexpr uint32_t U = sizeof(T) == 4 ? 8 : 16;       // the same bytes in flight for 16-bit types
+  constexpr uint32_t U = 8;
   uint32_t j = tid;
   for (; j + (U - 1) * STRIDE < s.nvec; j += U * STRIDE) {
     float4 v[U];
