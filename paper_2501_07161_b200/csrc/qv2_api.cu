@@ -298,7 +298,7 @@ int run_group_percentile(qv2_ctx* c, uint32_t n, const CalibArgs& a, uint64_t* g
     QV2_CUDA(c, cudaMemsetAsync(gh, 0, n_ghist * kBins * sizeof(uint64_t), c->stream));
     QV2_CUDA(c, launch_group_hist(l, c->caps.ghist, p.any_16bit, c->d_tensors, c->d_ghist_tiles,
                                   (uint32_t)p.ghist_tiles.size(), a.gabsmax, a.nonfinite, gh));
-    QV2_CUDA(c, launch_group_clip_finalize(l, c->d_tensors, c->d_ghist_owner, (uint32_t)n_ghist, gh, a.gmin, a.gmax,
+    QV2_CUDA(c, launch_group_clip_finalize(l, c->d_tensors, c->d_ghist_owner, (uint32_t)n_ghist, gh, a.nonfinite, a.gmin, a.gmax,
                                            a.gabsmax, group_clip, a.step, a.inv, a.offset));
     c->launches += p.ghist_tiles.empty() ? 1 : 2;
   }

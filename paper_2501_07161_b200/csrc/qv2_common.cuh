@@ -185,6 +185,7 @@ cudaError_t launch_group_hist(const Launch& l, uint32_t grid_cap, bool any16, co
                               const unsigned long long* nonfinite, unsigned long long* ghist);
 cudaError_t launch_group_clip_finalize(const Launch& l, const TensorRec* tensors, const uint32_t* owner,
                                        uint32_t n_hists, const unsigned long long* ghist,
+                                       const unsigned long long* nonfinite,
                                        const float* gmin, const float* gmax, const float* gabsmax,
                                        float* group_clip, float* step, float* inv, float* offset);
 cudaError_t launch_fill_group_clip(const Launch& l, const TensorRec* tensors, uint32_t n_tensors,

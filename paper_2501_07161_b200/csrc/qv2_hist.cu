@@ -331,22 +331,36 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 
 // One warp per group histogram: the group's clip by the same cumulative-count rule as
 // clip_fold_tensor, then the group's quantization parameters.
+//
+// The rule asks for k* = first bin whose cumulative count reaches T.  With A(k) = number of
+// elements above bin k that is the same as k* = first k with A(k) <= N - T, and for the usual
+// percentiles (close to 1) that bin is near the top; so the warp scans the histogram from the top
+// down, 32 bins at a time, and stops at the highest bin b whose count-from-b-upwards exceeds
+// N - T: k* = b.  Thousands of 16 KB histograms are then read a few hundred bytes each.  N is the
+// group's element count when the tensor holds no NaN or Inf; otherwise the histogram is summed.
 __global__ void __launch_bounds__(256)
 group_clip_finalize_kernel(const TensorRec* __restrict__ tensors, const uint32_t* __restrict__ owner,
                            uint32_t n_hists, const unsigned long long* __restrict__ ghist,
+                           const unsigned long long* __restrict__ nonfinite,
                            const float* __restrict__ gmin, const float* __restrict__ gmax,
                            const float* __restrict__ gabsmax, float* group_clip, float* step, float* inv,
                            float* offset) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t hidx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (hidx >= n_hists) return;
-  const TensorRec* tr = tensors + owner[hidx];
+  const uint32_t t = owner[hidx];
+  const TensorRec* tr = tensors + t;
   const uint32_t G = tr->group_base + (hidx - tr->ghist_first);
   const unsigned long long* h = ghist + (size_t)hidx * kBins;
   const float A = gabsmax[G];
-  unsigned long long nf = 0;
-  for (uint32_t i = 0; i < kBins / 32; ++i) nf += h[i * 32 + lane];
-  nf = warp_sum_u64(nf);
+  unsigned long long nf;
+  if (nonfinite[t] == 0ull) {
+    nf = tr->n_elems / tr->n_groups;              // every element of the group was counted
+  } else {
+    nf = 0;
+    for (uint32_t i = 0; i < kBins / 32; ++i) nf += h[i * 32 + lane];
+    nf = warp_sum_u64(nf);
+  }
   float c = A;
   if (nf != 0ull) {
     const double tt = ceil(__dmul_rn(tr->percentile, (double)nf));
@@ -354,18 +368,19 @@ group_clip_finalize_kernel(const TensorRec* __restrict__ tensors, const uint32_t
     if (!(tt >= 1.0)) T = 1ull;
     else if (tt >= (double)nf) T = nf;
     else T = (unsigned long long)tt;
-    unsigned long long carry = 0;
-    uint32_t kstar = kBins - 1;
-    for (uint32_t i = 0; i < kBins / 32; ++i) {
-      unsigned long long s = h[i * 32 + lane];          // inclusive scan of 32 consecutive bins
+    const unsigned long long rem = nf - T;        // elements allowed above bin k*
+    unsigned long long carry = 0;                 // count of the bins above the current 32
+    uint32_t kstar = 0;
+    for (int i = kBins / 32 - 1; i >= 0; --i) {
+      unsigned long long sfx = h[i * 32 + lane];  // inclusive suffix sum over the 32 bins, upwards from this lane
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const unsigned long long up = __shfl_up_sync(0xffffffffu, s, o);
-        if ((int)lane >= o) s += up;
+        const unsigned long long up = __shfl_down_sync(0xffffffffu, sfx, o);
+        if ((int)lane + o < 32) sfx += up;
       }
-      const uint32_t reached = __ballot_sync(0xffffffffu, carry + s >= T);
-      if (reached) { kstar = i * 32 + (uint32_t)__ffs(reached) - 1u; break; }
-      carry += __shfl_sync(0xffffffffu, s, 31);
+      const uint32_t over = __ballot_sync(0xffffffffu, carry + sfx > rem);
+      if (over) { kstar = (uint32_t)i * 32u + (31u - (uint32_t)__clz(over)); break; }
+      carry += __shfl_sync(0xffffffffu, sfx, 0);
     }
     if (kstar != kBins - 1) c = __fmul_rn((float)(kstar + 1), __fdiv_rn(A, (float)kBins));
   }
@@ -408,11 +423,12 @@ cudaError_t launch_group_hist(const Launch& l, uint32_t grid_cap, bool any16, co
 
 cudaError_t launch_group_clip_finalize(const Launch& l, const TensorRec* tensors, const uint32_t* owner,
                                        uint32_t n_hists, const unsigned long long* ghist,
+                                       const unsigned long long* nonfinite,
                                        const float* gmin, const float* gmax, const float* gabsmax,
                                        float* group_clip, float* step, float* inv, float* offset) {
   if (n_hists == 0) return cudaSuccess;
-  group_clip_finalize_kernel<<<(n_hists + 7) / 8, 256, 0, l.stream>>>(tensors, owner, n_hists, ghist, gmin, gmax,
-                                                                     gabsmax, group_clip, step, inv, offset);
+  group_clip_finalize_kernel<<<(n_hists + 7) / 8, 256, 0, l.stream>>>(tensors, owner, n_hists, ghist, nonfinite, gmin,
+                                                                     gmax, gabsmax, group_clip, step, inv, offset);
   return cudaGetLastError();
 }
 
