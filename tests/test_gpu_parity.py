@@ -541,6 +541,19 @@ def test_group_percentile_nonfinite_constant_and_empty_groups(ctx):
     check_specs(ctx, specs, check_codes=False)
 
 
+@pytest.mark.parametrize("p", [0.0, 1e-9, 0.1, 0.5, 0.731, 1.0 - 1e-12, 1.0])
+def test_group_percentile_any_percentile(ctx, p):
+    """The per-group clip is found by a scan from the top bin down; the bin must be the one the
+    cumulative-count rule names for percentiles anywhere in [0, 1], with and without skipped
+    (non-finite) elements, where the group's count is no longer its size."""
+    x = _scaled_channels(3, 9, 2500, 251, relu=True)
+    xn = x.clone(); xn[1, 4, 100] = float("nan"); xn[2, 0, 7] = float("-inf")
+    specs = [Spec(x, 3, 9, 2500, per_channel=True, asym=True, percentile=p, group_pct=True),
+             Spec(xn, 3, 9, 2500, per_channel=True, percentile=p, group_pct=True),
+             Spec(randn(5 * 40, 252), 1, 5, 40, per_channel=True, percentile=p, group_pct=True)]
+    check_specs(ctx, specs, check_codes=False)
+
+
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
 def test_group_percentile_sixteen_bit_inputs(ctx, dtype):
     specs = [Spec(_scaled_channels(2, 5, 9000, 231), 2, 5, 9000, per_channel=True, percentile=0.999, group_pct=True, dtype=dtype),

@@ -97,6 +97,50 @@ def test_schedule_selection():
         ctx.close()
 
 
+def test_dependent_launch_and_phase_timing_do_not_change_results():
+    """Programmatic dependent launch only changes when a kernel may start, and the phase events only
+    add markers: every output of a pass is the same bits with either switched on or off, also when
+    the pass is replayed from a graph captured with dependent launch on."""
+    model = gen.make_model("resnet18", seed=3, device="cuda", batch=1)
+    outs = []
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()             # a captured pass needs a non-default stream; torch's fills run on it too
+    for dependent in (True, False):
+        ctx = q.Context(0, stream=stream)
+        try:
+          with torch.cuda.stream(stream):
+            ctx.set_dependent_launch(dependent)
+            md, t = _sweep(ctx, model)
+            outs.append({k: v.clone() for k, v in t.items()})
+            if dependent:
+                cfg = q.default_rank_cfg(select_mode=q.BY_BOPS_RATE, rate_permyriad=md.rate_permyriad)
+                g = ctx.sweep_graph(md.descs, md.n_layers, md.macs, None, cfg,
+                                    q.binding.SweepBuffers(**{k: v.data_ptr() for k, v in t.items()}))
+                for v in t.values():
+                    v.view(torch.uint8).fill_(0x5A)
+                g.launch(); g.launch()
+                torch.cuda.synchronize()
+                for k in t:
+                    assert torch.equal(t[k].view(torch.uint8), outs[0][k].view(torch.uint8)), ("graph", k)
+                with pytest.raises(q.binding.Qv2Error):
+                    ctx.set_dependent_launch(False)          # a live captured pass keeps its edges
+                g.close()
+            # the phase events: same bits, and two positive durations
+            ctx.set_phase_timing(True)
+            cal = ctx.calibrate(md.descs)
+            r_ms, h_ms = ctx.calibrate_phase_ms()
+            assert r_ms > 0.0 and h_ms > 0.0
+            assert torch.equal(cal.step.view(torch.int32), t["step"].view(torch.int32)[: cal.step.numel()])
+            assert torch.equal(cal.hist.view(torch.int64), t["hist"].view(torch.int64)[: cal.hist.numel()])
+            ctx.set_phase_timing(False)
+            with pytest.raises(q.binding.Qv2Error):
+                ctx.calibrate_phase_ms()
+        finally:
+            ctx.close()
+    for k in outs[0]:
+        assert torch.equal(outs[0][k].view(torch.uint8), outs[1][k].view(torch.uint8)), k
+
+
 def test_chunked_schedule_with_empty_tensors_mixed_modes_and_codes():
     """Stage boundaries fall between tensors of every kind; empty tensors are folded by block 0."""
     g = torch.Generator(); g.manual_seed(3)
