@@ -198,10 +198,10 @@ __device__ __forceinline__ void load_params(QP& p, const TensorRec* tr, const fl
 //
 // The metrics are sums over the whole tensor; only the quantization parameters change from row to
 // row.  A tile of rows shorter than kPieceRow is therefore streamed like a flat run by the whole CTA
-// (16-byte loads, several in flight per thread) and every vector fetches the parameters of the row
-// it lies in; these loads hit L1, since neighbouring vectors share a row.  That needs rows of a
-// multiple of four elements and a 16-byte aligned tile; otherwise the tile is walked one element
-// per thread.  (For long rows the index arithmetic per vector costs more than it saves.)
+// (16-byte loads, several in flight per thread) and every 16-byte group fetches the parameters of
+// the row(s) it lies in; these loads hit L1, since neighbouring groups share a row.  Rows shorter
+// than four elements, and pairs whose x and y sit at different offsets inside a 16-byte group,
+// are walked one element per thread.
 struct RowParams {
   const TensorRec* tr;
   const float* __restrict__ step;
@@ -215,8 +215,9 @@ struct RowParams {
         row0c((uint32_t)(tl.row0 % t->channels)), gbase(t->group_base), top(top_code(t->asym != 0, t->bits)),
         qmin0(t->asym ? 0.0f : -top_code(false, t->bits)), zp(t->asym == 2) {}
   // parameters of the row that holds element e of the tile (same values as load_params)
-  __device__ __forceinline__ QP of_elem(uint32_t e) const {
-    const uint32_t G = gbase + (row0c + e / inner) % channels;
+  __device__ __forceinline__ QP of_elem(uint32_t e) const { return of_group((row0c + e / inner) % channels); }
+  __device__ __forceinline__ QP of_group(uint32_t g) const {
+    const uint32_t G = gbase + g;
     QP p;
     p.step = __ldg(step + G); p.inv = __ldg(inv + G);
     const float off = __ldg(offset + G);
@@ -227,29 +228,63 @@ struct RowParams {
   }
 };
 
+// Rows of 4..kPieceRow-1 elements, x (and y) 16-byte aligned after the same `head` elements: the
+// aligned body is walked like a flat run (thread t takes 16-byte groups t, t+256, ...), and every
+// thread tracks the row its current group starts in incrementally -- a step of 1024 elements
+// advances the row by 1024 / inner and the position in the row by 1024 % inner -- so that no
+// division is needed per group.  A group that straddles a row end takes the parameters of both
+// rows and picks per element.
 template <uint32_t MODE, bool OFF, bool CODES, class T, class ACC>
 __device__ __forceinline__ void metric_rows_vec(const T* __restrict__ x, const T* __restrict__ y, uint8_t* codes,
-                                                uint32_t count, const RowParams& rp, ACC* a) {
+                                                uint32_t count, uint32_t head, const RowParams& rp, ACC* a) {
   constexpr bool PAIR = MODE != kSelf;
-  constexpr uint32_t U = 4;
-  const uint32_t nvec = count >> 2;
-  uint32_t j = threadIdx.x;
-  for (; j < nvec; j += U * kThreads) {          // the last round is clamped: loads in bounds, maybe unused
+  constexpr uint32_t U = PAIR ? 4 : 8;                      // the same bytes in flight as the flat walker
+  const uint32_t inner = rp.inner, channels = rp.channels;
+  const uint32_t nvec = (count - head) >> 2, tail = (count - head) & 3u;
+  const T* xb = x + head;
+  const T* yb = PAIR ? y + head : nullptr;
+  uint8_t* cb = CODES ? codes + head : nullptr;
+  constexpr uint32_t kStep = 4u * kThreads;                    // elements between a thread's consecutive groups
+  const uint32_t q = kStep / inner, r = kStep - q * inner;
+  uint32_t e = head + 4u * threadIdx.x;                       // index in the tile of the group's first element
+  uint32_t rem = e % inner;                                    // its position in its row
+  uint32_t g = (rp.row0c + e / inner) % channels;              // the row's group
+  for (uint32_t j = threadIdx.x; j < nvec; j += U * kThreads) {          // the last round is clamped: loads in bounds, maybe unused
     float4 vx[U], vy[U];
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) {
       const uint32_t k = min(j + u * kThreads, nvec - 1u);
-      vx[u] = ld_vec_at(x, k);
-      if (PAIR) vy[u] = ld_vec_at(y, k); else vy[u] = vx[u];
+      vx[u] = ld_vec_at(xb, k);
+      if (PAIR) vy[u] = ld_vec_at(yb, k); else vy[u] = vx[u];
     }
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) {
       const uint32_t k = j + u * kThreads;
       if (k < nvec) {
-        const QP p = rp.of_elem(4u * k);
-        metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? codes + 4u * k : nullptr);
+        const QP pa = rp.of_group(g);
+        const uint32_t left = inner - rem;                     // elements of this row from the group's first one on
+        uint8_t* c = CODES ? cb + 4u * k : nullptr;
+        if (left >= 4u) {
+          metric_vec<MODE, OFF, CODES>(vx[u], vy[u], pa, a, c);
+        } else {                                               // the group ends in the next row (inner >= 4: at most one row end)
+          const QP pb = rp.of_group(g + 1u == channels ? 0u : g + 1u);
+          metric_elem<MODE, OFF, CODES>(vx[u].x, vy[u].x, pa, a[0], c);
+          metric_elem<MODE, OFF, CODES>(vx[u].y, vy[u].y, left > 1u ? pa : pb, a[1], c + 1);
+          metric_elem<MODE, OFF, CODES>(vx[u].z, vy[u].z, left > 2u ? pa : pb, a[2], c + 2);
+          metric_elem<MODE, OFF, CODES>(vx[u].w, vy[u].w, pb, a[3], c + 3);
+        }
+        // next group of this thread: kStep elements on
+        rem += r; g += q;
+        if (rem >= inner) { rem -= inner; ++g; }
+        if (g >= channels) g %= channels;
       }
     }
+  }
+  // the few elements before and after the aligned body, one per thread
+  if (threadIdx.x < head + tail) {
+    const uint32_t i = threadIdx.x < head ? threadIdx.x : head + 4u * nvec + (threadIdx.x - head);
+    const QP p = rp.of_elem(i);
+    metric_elem<MODE, OFF, CODES>(Ld<T>::one(x + i), PAIR ? Ld<T>::one(y + i) : 0.0f, p, a[0], CODES ? codes + i : nullptr);
   }
 }
 
@@ -322,15 +357,17 @@ __device__ __noinline__ ACC metric_rows(Tile tl, const TensorRec* tr, const floa
     return ACC::fold(a);
   }
   const RowParams rp(tl, tr, step, inv, offset);
+  // elements up to the first 16-byte boundary of x; the vector walker needs y at the same phase
+  const uint32_t head = min((4u - (uint32_t)(((uintptr_t)x / sizeof(T)) & 3u)) & 3u, tl.count);
   constexpr uintptr_t kVecMask = 4u * sizeof(T) - 1u;
-  const bool vec = (rp.inner & 3u) == 0 && (((uintptr_t)x) & kVecMask) == 0 &&
-                   (MODE == kSelf || (((uintptr_t)y) & kVecMask) == 0);
+  const bool vec = rp.inner >= 4u && tl.count - head >= 4u &&
+                   (MODE == kSelf || (((uintptr_t)(y + head)) & kVecMask) == 0);
   // a real-valued offset needs the form of the arithmetic that splits x - offset exactly; with a
   // zero offset both forms give the same value
   const bool off = MODE != kRaw && tr->asym == 1;
   if (vec) {
-    if (off) metric_rows_vec<MODE, MODE != kRaw, CODES>(x, y, codes, tl.count, rp, a);
-    else metric_rows_vec<MODE, false, CODES>(x, y, codes, tl.count, rp, a);
+    if (off) metric_rows_vec<MODE, MODE != kRaw, CODES>(x, y, codes, tl.count, head, rp, a);
+    else metric_rows_vec<MODE, false, CODES>(x, y, codes, tl.count, head, rp, a);
   } else {
     if (off) metric_rows_scalar<MODE, MODE != kRaw, CODES>(x, y, codes, tl.count, rp, a);
     else metric_rows_scalar<MODE, false, CODES>(x, y, codes, tl.count, rp, a);
