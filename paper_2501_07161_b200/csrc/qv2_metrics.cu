@@ -129,7 +129,7 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
   const bool vec_y = !PAIR || ((((uintptr_t)yb) & (4u * sizeof(T) - 1u)) == 0);
   uint32_t j = tid;
   if (vec_y) {
-    constexpr uint32_t U = PAIR ? 4 : 8;
+    constexpr uint32_t U = (PAIR ? 4 : 8) * (sizeof(T) == 2 ? 2 : 1);   // 16-bit elements: the same bytes in flight
     for (; j + (U - 1) * STRIDE < s.nvec; j += U * STRIDE) {
       float4 vx[U], vy[U];
 #pragma unroll
