@@ -31,7 +31,7 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
   __shared__ double mean_s[2];
   __shared__ double s_mw[kStage], s_ma[kStage], s_sw[kStage], s_sa[kStage], s_pos[kStage], s_score[kStage],
       s_sev[kStage];
-  __shared__ unsigned long long s_macs[kStage];
+  __shared__ unsigned long long s_macs[kStage], s_mlist[kStage];
   __shared__ uint32_t s_fg[kStage], s_place[kStage], s_best[kStage], s_order[kStage];
   __shared__ uint8_t s_keep[kStage];
   constexpr uint32_t kNoGroup = QV2_NO_GROUP;
@@ -59,23 +59,25 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
     sc = s_score; sv = s_sev; pl = s_place; bs = s_best; od = s_order; kp = s_keep;
     __syncthreads();
   }
-  if (tid == 0) {                      // means: sums in layer order, as the definition states
-    double a = 0.0, b = 0.0;
-    for (uint32_t i = 0; i < n; ++i) {
-      a = __dadd_rn(a, mw[i]);
-      b = __dadd_rn(b, ma[i]);
-    }
-    mean_s[0] = __ddiv_rn(a, (double)n);
-    mean_s[1] = __ddiv_rn(b, (double)n);
+  if (tid == 0 || tid == 32) {         // means: sums in layer order, as the definition states; one warp per list
+    const double* m = tid == 0 ? mw : ma;
+    double a = 0.0;
+#pragma unroll 8
+    for (uint32_t i = 0; i < n; ++i) a = __dadd_rn(a, m[i]);      // the loads run ahead of the chain of additions
+    mean_s[tid == 0 ? 0 : 1] = __ddiv_rn(a, (double)n);
   }
   __syncthreads();
   const double mean_w = mean_s[0], mean_a = mean_s[1], cap = cfg.sqnr_cap_db;
   for (uint32_t i = tid; i < n; i += blockDim.x) {
     double dw = 0.0, da = 0.0;
     if (i > 0) {
-      const double den = ps ? __dsub_rn(ps[i], ps[i - 1]) : 1.0;
-      dw = __ddiv_rn(__dsub_rn(clamp_cap(sw[i], cap), clamp_cap(sw[i - 1], cap)), den);
-      da = __ddiv_rn(__dsub_rn(clamp_cap(sa[i], cap), clamp_cap(sa[i - 1], cap)), den);
+      dw = __dsub_rn(clamp_cap(sw[i], cap), clamp_cap(sw[i - 1], cap));
+      da = __dsub_rn(clamp_cap(sa[i], cap), clamp_cap(sa[i - 1], cap));
+      if (ps) {                          // default positions 0,1,2,...: a division by 1 changes nothing
+        const double den = __dsub_rn(ps[i], ps[i - 1]);
+        dw = __ddiv_rn(dw, den);
+        da = __ddiv_rn(da, den);
+      }
     }
     double s = __dadd_rn(__dmul_rn(cfg.w_gain, dw), __dmul_rn(cfg.a_gain, da));
     if (s != s) s = inf;
@@ -92,27 +94,40 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
   // order), the rest by ascending score, ties by layer index.
   const double fac = cfg.mse_factor;
   const bool literal = cfg.outlier_order == QV2_OUTLIERS_LITERAL;
-  for (uint32_t i = tid; i < n; i += blockDim.x) {
+  // The n*n comparisons are spread over the whole block: with n <= blockDim/2 several threads share
+  // a layer (thread p of a layer takes every parts-th j) and add their counts in `place`.
+  const uint32_t parts = n <= blockDim.x / 2 ? blockDim.x / n : 1u;
+  if (parts > 1) {
+    for (uint32_t i = tid; i < n; i += blockDim.x) pl[i] = 0;
+    __syncthreads();
+  }
+  for (uint32_t w = tid; w < n * parts; w += blockDim.x) {
+    const uint32_t i = parts > 1 ? w % n : w, part = parts > 1 ? w / n : 0u;
     const double si = sc[i], vi = sv[i];
     const bool out_i = vi > fac;
     uint32_t rank = 0;
-    for (uint32_t j = 0; j < n; ++j) {
-      const double vj = sv[j];
-      const bool out_j = vj > fac;
-      if (out_i) {
-        if (out_j && (literal ? j > i : (vj > vi || (vj == vi && j < i)))) ++rank;
-      } else {
-        if (out_j) ++rank;
-        else {
-          const double sj = sc[j];
-          if (sj < si || (sj == si && j < i)) ++rank;
-        }
+    if (out_i) {
+#pragma unroll 4
+      for (uint32_t j = part; j < n; j += parts) {
+        const double vj = sv[j];
+        const bool before = literal ? j > i : (vj > vi) | ((vj == vi) & (j < i));
+        rank += (uint32_t)((vj > fac) & before);
+      }
+    } else {
+#pragma unroll 4
+      for (uint32_t j = part; j < n; j += parts) {
+        const double vj = sv[j], sj = sc[j];
+        rank += (uint32_t)((vj > fac) | (sj < si) | ((sj == si) & (j < i)));
       }
     }
-    od[rank] = i;
-    pl[i] = rank;
+    if (parts > 1) atomicAdd(pl + i, rank);
+    else { od[rank] = i; pl[i] = rank; }
   }
   __syncthreads();
+  if (parts > 1) {
+    for (uint32_t i = tid; i < n; i += blockDim.x) od[pl[i]] = i;
+    __syncthreads();
+  }
   if (fg) {
     // Fusion groups: every member moves to the place of the group's best-ranked member and the
     // members stand there in layer order.  Places of different groups differ, so sorting by
@@ -137,14 +152,56 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
     }
     __syncthreads();
   }
-  if (tid == 0) {
-    // The FP32-kept prefix grows one whole fusion group at a time (a layer without a group is a
-    // group of one): by count while it still fits, by rate while the rate still holds.
+  // The FP32-kept prefix grows one whole fusion group at a time (a layer without a group is a group
+  // of one): by count while it still fits, by rate while the rate still holds.  With K the MACs
+  // kept so far, "quantized share >= rate" is (total - K) * 10000 >= rate * total, i.e.
+  // K * 10000 <= total * (10000 - rate); 128-bit integers, exact.  Both tests only get harder as
+  // the prefix grows, so the walk "stop at the first group that fails" ends at the LONGEST prefix
+  // that ends on a group boundary and passes.
+  if (staged) {
+    // Every list position is tested by its own thread: MACs and groups gathered in list order, a
+    // 128-bit prefix sum per position (n <= 512 additions each), then the largest passing cut.
+    unsigned long long* p_lo = reinterpret_cast<unsigned long long*>(s_score);   // scores and severities
+    unsigned long long* p_hi = reinterpret_cast<unsigned long long*>(s_sev);     // are no longer needed
+    __shared__ uint32_t s_nk;
+    if (tid == 0) s_nk = 0;
+    for (uint32_t k = tid; k < n; k += blockDim.x) {
+      const uint32_t l = od[k];
+      s_mlist[k] = mc ? mc[l] : 1ull;
+      s_best[k] = fg ? fg[l] : kNoGroup;
+    }
+    __syncthreads();
+    const bool by_count = cfg.select_mode == QV2_BY_COUNT;
+    if (!by_count) {
+      for (uint32_t k = tid; k < n; k += blockDim.x) {
+        unsigned __int128 acc = 0;
+#pragma unroll 4
+        for (uint32_t q = 0; q <= k; ++q) acc += s_mlist[q];
+        p_lo[k] = (unsigned long long)acc; p_hi[k] = (unsigned long long)(acc >> 64);
+      }
+      __syncthreads();
+    }
+    const unsigned __int128 total = by_count ? 0 : (((unsigned __int128)p_hi[n - 1] << 64) | p_lo[n - 1]);
+    const unsigned __int128 limit = total * (unsigned __int128)(10000u - cfg.rate_permyriad);
+    for (uint32_t k = tid; k < n; k += blockDim.x) {
+      const uint32_t e = k + 1, g = s_best[k];
+      const bool boundary = e == n || g == kNoGroup || s_best[e] != g;
+      bool pass;
+      if (by_count) pass = e <= cfg.keep_count;
+      else pass = ((((unsigned __int128)p_hi[k] << 64) | p_lo[k]) * 10000u) <= limit;
+      if (boundary && pass) atomicMax(&s_nk, e);
+    }
+    __syncthreads();
+    const uint32_t nk = s_nk;
+    for (uint32_t k = tid; k < nk; k += blockDim.x) kp[od[k]] = 1;
+    if (tid == 0) *n_keep = nk;
+  } else if (tid == 0) {
     auto grp = [&](uint32_t l) { return fg ? fg[l] : kNoGroup; };
     auto mac = [&](uint32_t l) { return mc ? mc[l] : 1ull; };
     unsigned __int128 total = 0, kept = 0;
     if (cfg.select_mode != QV2_BY_COUNT)
       for (uint32_t i = 0; i < n; ++i) total += mac(i);
+    const unsigned __int128 limit = total * (unsigned __int128)(10000u - cfg.rate_permyriad);
     uint32_t nk = 0, j = 0;
     while (j < n) {
       const uint32_t g = grp(od[j]);
@@ -155,8 +212,7 @@ rank_kernel(uint32_t n, const double* __restrict__ sqnr_w, const double* __restr
       } else {
         unsigned __int128 m = 0;
         for (uint32_t k = j; k < e; ++k) m += mac(od[k]);
-        const unsigned __int128 quantized = total - (kept + m);
-        if (quantized * 10000u >= (unsigned __int128)cfg.rate_permyriad * total) { kept += m; nk = e; }
+        if ((kept + m) * 10000u <= limit) { kept += m; nk = e; }
         else break;
       }
       j = e;
