@@ -14,11 +14,11 @@ namespace qv2 {
 constexpr int kThreads = 256;            // threads per CTA in the streaming kernels
 constexpr int kWarps = kThreads / 32;
 constexpr uint32_t kTileElems = 16384;   // elements per tile (64 KiB of fp32)
-constexpr uint64_t kRowTileMin = 16384;  // rows at least this long are cut into one-group tiles; shorter rows go
-                                         // one per warp (a row of 4608 elements walked by the whole CTA is a single
-                                         // round of loads followed by a drain, one warp per row keeps eight
-                                         // independent streams going)
-constexpr uint64_t kShortRow = 128;      // rows shorter than this are walked element-parallel, longer ones one warp per row
+constexpr uint64_t kRowTileMin = 16384;  // rows at least this long are cut into one-group tiles walked by the whole CTA;
+                                         // shorter rows come as tiles of whole rows (about kTileElems elements) and are
+                                         // walked by the row walkers of each kernel, which keep eight streams per CTA going
+                                         // whatever the row length (a 4608-element row walked by the whole CTA is a single
+                                         // round of loads followed by a drain)
 constexpr uint64_t kGroupUnitElems = 131072;   // elements per unit of the per-group histogram pass
 constexpr uint64_t kGroupSegMax = 1ull << 22;   // longest contiguous segment of such a unit
 constexpr int kBins = QV2_HIST_BINS;
