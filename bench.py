@@ -253,10 +253,10 @@ def measured_peak():
 
 
 def recorded_read_ceiling():
-    """GB/s of a pure read stream on a B200 as recorded by the stand-alone probe summarised in
-    profiles/read_ceiling_probe.md (plain 16-byte loads, 4 GB input, CUDA events)."""
+    """GB/s of a pure read stream on a B200 as recorded by the stand-alone read probe
+    (profiles/read_ceiling.txt: plain 16-byte loads, 4 GB input, CUDA events)."""
     try:
-        with open(os.path.join(ROOT, "profiles", "read_ceiling_probe.md")) as f:
+        with open(os.path.join(ROOT, "profiles", "read_ceiling.txt")) as f:
             for ln in f:
                 if ln.startswith("read_ceiling_gbs:"):
                     return float(ln.split(":", 1)[1])
@@ -627,7 +627,7 @@ def ours_main(args):
                          # the peak above is a copy (read + write); these kernels only read, so a
                          # pure read stream is the tighter ceiling
                          "read_ceiling": {"recorded_gbs": read_ceiling,
-                                          "source": "profiles/read_ceiling_probe.md (plain 16-byte loads, 4 GB, CUDA events)",
+                                          "source": "profiles/read_ceiling.txt (read probe: plain 16-byte loads, 4 GB, CUDA events)",
                                           "frac": (achieved / read_ceiling) if (achieved and read_ceiling) else None,
                                           "live_torch_max_gbs": live_read},
                          "duration_ms": met_ms,
