@@ -419,7 +419,7 @@ int qv2_sweep_model(qv2_ctx* ctx, const qv2_tensor_desc* descs, uint32_t n_tenso
 /*
  * The pass of qv2_sweep_model captured once in a CUDA graph and replayed with a single launch.
  * Algorithm 2 on a small model is a chain of short kernels whose launch overhead exceeds their
- * run time; replaying a captured chain removes it (SqueezeNet shapes: 74 us -> 33 us per pass).
+ * run time; replaying a captured chain removes it (SqueezeNet shapes: about 50 us -> 23 us per pass).
  * qv2_sweep_graph_create runs one ordinary pass first (argument checks, tile tables, scratch
  * sizing -- results are written as usual), then captures an identical pass on the context's stream;
  * it needs a context created on a non-default stream (QV2_ERR_UNSUPPORTED otherwise) and
