@@ -596,12 +596,15 @@ def test_group_percentile_in_the_chained_pass_and_its_graph(ctx):
             gctx.close()
 
 
-# ------------------------------------------------- rows shorter than a warp's reach (element-parallel path)
-@pytest.mark.parametrize("inner", [1, 9, 27, 49, 127, 128, 196])
+# ------------------------------------------------- the row walkers and the row lengths at which they change
+@pytest.mark.parametrize("inner", [1, 2, 3, 4, 5, 9, 27, 49, 127, 128, 196, 319, 320, 321, 510, 511, 512, 513, 1021])
 def test_short_rows_per_channel_all_modes(ctx, inner):
-    """Rows below 128 elements are walked one element per thread with per-element parameters; 128
-    and above one warp per row.  Self, re-quantized pair and raw pair, symmetric / affine / zero
-    point, with codes, several batch items so that a channel's rows are far apart."""
+    """The range kernel walks rows below 320 elements lane-contiguously (32 consecutive elements per
+    thread) and longer ones in per-warp chunks; the metrics kernel fetches parameters per 16-byte
+    group below 512 elements per row (per element below 4) and walks longer rows in per-warp
+    chunks.  Lengths on both sides of every switch, multiples of four and not.  Self, re-quantized
+    pair and raw pair, symmetric / affine / zero point, with codes, several batch items so that a
+    channel's rows are far apart."""
     o, c = 5, 37
     n = o * c * inner
     x = _scaled_channels(o, c, inner, 300 + inner)
@@ -639,8 +642,8 @@ def test_random_descriptor_sets_in_one_batched_call(ctx, seed):
     per row, element per thread) and tile kind meets every arithmetic variant, and the planner has
     to keep their groups, slots and histograms apart."""
     rng = np.random.default_rng(1000 + seed)
-    inner_pool = [1, 2, 7, 9, 31, 32, 33, 49, 100, 127, 128, 129, 196, 500, 784, 1153, 3136, 4095, 4096, 4097,
-                  12544, 16384, 16385, 40000]
+    inner_pool = [1, 2, 3, 7, 9, 31, 32, 33, 49, 100, 127, 128, 129, 196, 318, 322, 500, 514, 784, 1153, 3136, 4095, 4096,
+                  4097, 12544, 16383, 16384, 16385, 40000]
     specs = []
     total = 0
     while len(specs) < 40 and total < 6_000_000:
