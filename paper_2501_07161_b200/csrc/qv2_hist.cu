@@ -47,7 +47,8 @@ __device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t coun
   const T* xv = x + s.head;
   constexpr uint32_t U = 4;
   uint32_t j = threadIdx.x;
-  for (; j + (U - 1) * kThreads < s.nvec; j += U * kThreads) {
+  const uint32_t n_full = s.nvec / (U * kThreads) * (U * kThreads);   // rounds in which every thread has U groups
+  for (; j < n_full; j += U * kThreads) {
     float4 v[U];
 #pragma unroll
     for (uint32_t u = 0; u < U; ++u) v[u] = ld_vec_at(xv, j + u * kThreads);
@@ -57,12 +58,12 @@ __device__ __forceinline__ void hist_flat(const T* __restrict__ x, uint32_t coun
       hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
     }
   }
-  if (j < s.nvec) {                 // at most U-1 groups are left for this thread: one predicated round
-    float4 v[U - 1];
+  if (n_full < s.nvec) {            // what is left: one predicated round
+    float4 v[U];
 #pragma unroll
-    for (uint32_t u = 0; u < U - 1; ++u) v[u] = ld_vec_at(xv, min(j + u * kThreads, s.nvec - 1u));   // in bounds, maybe unused
+    for (uint32_t u = 0; u < U; ++u) v[u] = ld_vec_at(xv, min(j + u * kThreads, s.nvec - 1u));   // in bounds, maybe unused
 #pragma unroll
-    for (uint32_t u = 0; u < U - 1; ++u)
+    for (uint32_t u = 0; u < U; ++u)
       if (j + u * kThreads < s.nvec) {
         hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
         hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
@@ -251,7 +252,8 @@ __device__ __forceinline__ void hist_segment_warp(const T* __restrict__ x, uint3
   const FlatSplit s = split_flat(x, count);
   const T* xv = x + s.head;
   uint32_t j = lane;
-  for (; j + 96 < s.nvec; j += 128) {
+  const uint32_t n_full = s.nvec / 128u * 128u;      // rounds in which every lane has four groups
+  for (; j < n_full; j += 128) {
     float4 v[4];
 #pragma unroll
     for (uint32_t u = 0; u < 4; ++u) v[u] = ld_vec_at(xv, j + 32u * u);
@@ -261,12 +263,12 @@ __device__ __forceinline__ void hist_segment_warp(const T* __restrict__ x, uint3
       hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
     }
   }
-  if (j < s.nvec) {                 // at most three groups are left for this lane: one predicated round
-    float4 v[3];
+  if (n_full < s.nvec) {            // what is left: one predicated round
+    float4 v[4];
 #pragma unroll
-    for (uint32_t u = 0; u < 3; ++u) v[u] = ld_vec_at(xv, min(j + 32u * u, s.nvec - 1u));   // in bounds, maybe unused
+    for (uint32_t u = 0; u < 4; ++u) v[u] = ld_vec_at(xv, min(j + 32u * u, s.nvec - 1u));   // in bounds, maybe unused
 #pragma unroll
-    for (uint32_t u = 0; u < 3; ++u)
+    for (uint32_t u = 0; u < 4; ++u)
       if (j + 32u * u < s.nvec) {
         hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
         hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);

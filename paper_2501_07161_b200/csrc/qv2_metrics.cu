@@ -130,7 +130,11 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
   uint32_t j = tid;
   if (vec_y) {
     constexpr uint32_t U = (PAIR ? 4 : 8) * (sizeof(T) == 2 ? 2 : 1);   // 16-bit elements: the same bytes in flight
-    for (; j + (U - 1) * STRIDE < s.nvec; j += U * STRIDE) {
+    // Full rounds while EVERY thread of the walk still has U groups (the same trip count for all of
+    // them: a warp never runs a round for a few of its lanes), then one predicated round with all
+    // loads in flight for what is left.
+    const uint32_t n_full = s.nvec / (U * STRIDE) * (U * STRIDE);
+    for (; j < n_full; j += U * STRIDE) {
       float4 vx[U], vy[U];
 #pragma unroll
       for (uint32_t u = 0; u < U; ++u) {
@@ -141,16 +145,16 @@ __device__ __forceinline__ void metric_flat(const T* __restrict__ x, const T* __
       for (uint32_t u = 0; u < U; ++u)
         metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * STRIDE) : nullptr);
     }
-    if (j < s.nvec) {               // at most U-1 groups are left for this thread: one predicated round, all loads in flight
-      float4 vx[U - 1], vy[U - 1];
+    if (n_full < s.nvec) {          // fewer than U * STRIDE groups are left for the walk
+      float4 vx[U], vy[U];
 #pragma unroll
-      for (uint32_t u = 0; u < U - 1; ++u) {
+      for (uint32_t u = 0; u < U; ++u) {
         const uint32_t k = min(j + u * STRIDE, s.nvec - 1u);       // in bounds, maybe unused
         vx[u] = ld_vec_at(xb, k);
         if (PAIR) vy[u] = ld_vec_at(yb, k); else vy[u] = vx[u];
       }
 #pragma unroll
-      for (uint32_t u = 0; u < U - 1; ++u)
+      for (uint32_t u = 0; u < U; ++u)
         if (j + u * STRIDE < s.nvec)
           metric_vec<MODE, OFF, CODES>(vx[u], vy[u], p, a, CODES ? cb + 4u * (j + u * STRIDE) : nullptr);
     }
