@@ -324,8 +324,22 @@ def side_workloads(q, local, peak, steps):
             rec = {"workload": name, "batch": cfgw.batch, "layers": L, "swept_bytes_per_step": swept,
                    "resident_bytes": 4 * (model.weight_elems + 2 * model.act_elems), "steps": steps}
 
-            def timed(fn):
+            calls = [0]
+
+            def timed(fn0):
+                def fn():
+                    calls[0] += 1
+                    fn0()
+                # at least 3 passes and ~60 ms of work before the timed ones: the clocks of a GPU that has
+                # just been idle (the model was being generated) take tens of milliseconds to come up
+                w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                w0.record()
                 for _ in range(3):
+                    fn()
+                w1.record()
+                torch.cuda.synchronize()
+                per = max(w0.elapsed_time(w1) / 3.0, 1e-3)
+                for _ in range(int(min(2000, 60.0 / per))):
                     fn()
                 torch.cuda.synchronize()
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -340,10 +354,10 @@ def side_workloads(q, local, peak, steps):
                 ctx = q.Context(local, stream=stream)
                 ctx.set_schedule(sched, 0)
                 sb, t = ctx.alloc_sweep_buffers(md.descs, L)
-                l0 = ctx.launches
+                l0, c0 = ctx.launches, calls[0]
                 ms = timed(lambda: ctx.sweep_model(md.descs, L, md.macs, None, rcfg, sb))
                 r = {"ms_per_step": ms, "value": swept / (ms * 1e-3) / 1e9, "stages": ctx.stages,
-                     "launches_per_step": (ctx.launches - l0) // (steps + 3)}
+                     "launches_per_step": (ctx.launches - l0) // max(1, calls[0] - c0)}
                 g = ctx.sweep_graph(md.descs, L, md.macs, None, rcfg, sb)
                 gms = timed(g.launch)
                 g.close()
