@@ -1,6 +1,6 @@
 // Read-bandwidth ceiling probe: the same min/max reduction over one large fp32 array, fed by
 //  (a) plain 16-byte ld.global.nc loads with U loads in flight per thread,
-//  (b) a cp.async.bulk (1-D, no multicast, this GPU's memory only) + mbarrier shared-memory ring
+//  (b) a 1-D cp.async.bulk from this GPU's own memory into one CTA's shared memory + mbarrier ring
 //      with a producer warp and 8 consumer warps,
 //  (c) a per-thread cp.async (16-byte LDGSTS) ring.
 // Usage: read_probe [gigabytes=4] [reps=10] [only=<variant index or -1>]
