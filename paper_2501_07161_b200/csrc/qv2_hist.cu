@@ -239,10 +239,84 @@ clip_fold_kernel(const __grid_constant__ CalibArgs a, uint32_t tensor_begin) {
 // The pass is group-major: a unit is `rows` segments of `count` contiguous elements of ONE group
 // (the same channel of consecutive batch items), about 128 K elements.  A CTA counts a whole unit
 // into its shared-memory histogram and merges it into the group's global histogram once, at the
-// end of the unit.  Long segments are walked by the whole CTA, short ones by one warp each.
+// end of the unit.  Very small groups are packed several to a unit and skip the shared histogram.
 __device__ __forceinline__ float bin_scale(float A) {
   float w = (A > 0.0f) ? __fdiv_rn((float)kBins, A) : 0.0f;
   return isfinite(w) ? w : 0.0f;
+}
+
+// Exact n / d by one multiply-high, for n * d <= 2^32: with m = floor((2^32 - 1) / d) + 1 the
+// product m * d exceeds 2^32 by less than d, so the error of n * m / 2^32 stays below 1 / d.
+struct FastDiv {
+  uint32_t m, d;
+};
+__device__ __forceinline__ FastDiv fast_div(uint32_t d) {
+  FastDiv f;
+  f.d = d; f.m = d > 1u ? 0xFFFFFFFFu / d + 1u : 0u;
+  return f;
+}
+__device__ __forceinline__ uint32_t div_by(uint32_t n, const FastDiv& f) { return f.d > 1u ? __umulhi(n, f.m) : n; }
+
+// `rows` segments of `count` elements, segment r at x + r * seg_stride, walked by the whole CTA as
+// ONE index space of 16-byte groups: every thread keeps four loads in flight whatever the segment
+// length, and a round that straddles segments costs nothing.  Needs every segment to start on a
+// four-element boundary and to hold whole groups, and rows * (count / 4)^2 <= 2^32 (FastDiv).
+template <bool CAREFUL, class T>
+__device__ __forceinline__ void hist_rows_vec(const T* __restrict__ x, uint32_t rows, uint32_t count,
+                                              uint64_t seg_stride, float w, uint32_t* sh, EdgeCount& zeros) {
+  constexpr uint32_t U = 4;
+  const uint32_t nv = count >> 2, total = rows * nv;
+  const FastDiv f = fast_div(nv);
+  uint32_t j = threadIdx.x;
+  const uint32_t n_full = total / (U * kThreads) * (U * kThreads);
+  for (; j < n_full; j += U * kThreads) {
+    float4 v[U];
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) {
+      const uint32_t idx = j + u * kThreads, r = div_by(idx, f);
+      v[u] = ld_vec_at(x + r * seg_stride, idx - r * nv);
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) {
+      hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
+      hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
+    }
+  }
+  if (n_full < total) {             // what is left: one predicated round
+    float4 v[U];
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) {
+      const uint32_t idx = min(j + u * kThreads, total - 1u), r = div_by(idx, f);   // in bounds, maybe unused
+      v[u] = ld_vec_at(x + r * seg_stride, idx - r * nv);
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u)
+      if (j + u * kThreads < total) {
+        hist_elem<CAREFUL>(v[u].x, w, sh, zeros); hist_elem<CAREFUL>(v[u].y, w, sh, zeros);
+        hist_elem<CAREFUL>(v[u].z, w, sh, zeros); hist_elem<CAREFUL>(v[u].w, w, sh, zeros);
+      }
+  }
+}
+
+// The same index space element by element, for short segments that do not line up with 16-byte
+// groups (7x7 maps, odd strides): eight scalar loads in flight per thread.  rows * count^2 <= 2^32.
+template <bool CAREFUL, class T>
+__device__ __noinline__ void hist_rows_scalar(const T* __restrict__ x, uint32_t rows, uint32_t count,
+                                                 uint64_t seg_stride, float w, uint32_t* sh, EdgeCount& zeros) {
+  constexpr uint32_t U = 8;
+  const uint32_t total = rows * count;
+  const FastDiv f = fast_div(count);
+  for (uint32_t j0 = 0; j0 < total; j0 += U * kThreads) {
+    float v[U];
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u) {
+      const uint32_t idx = min(j0 + threadIdx.x + u * kThreads, total - 1u), r = div_by(idx, f);
+      v[u] = Ld<T>::one(x + r * seg_stride + (idx - r * count));
+    }
+#pragma unroll
+    for (uint32_t u = 0; u < U; ++u)
+      if (j0 + threadIdx.x + u * kThreads < total) hist_elem<CAREFUL>(v[u], w, sh, zeros);
+  }
 }
 
 // One segment handled by one warp: 16-byte loads over the aligned body, scalars at the ends.
@@ -278,24 +352,85 @@ __device__ __forceinline__ void hist_segment_warp(const T* __restrict__ x, uint3
   if (lane < s.tail) hist_elem<CAREFUL>(Ld<T>::one(x + s.head + 4u * s.nvec + lane), w, sh, zeros);
 }
 
-constexpr uint32_t kWarpSegmentMax = 4096;     // shorter segments go one per warp
+constexpr uint32_t kWarpSegmentMax = 4096;     // unaligned segments shorter than this go one per warp ...
+constexpr uint32_t kScalarSegmentMax = 256;    // ... and shorter than this element by element
 
-template <class T>
+template <bool CAREFUL, class T>
 __device__ __forceinline__ void group_hist_unit(const T* x, const Tile& u, uint64_t seg_stride, float w,
-                                                bool careful, uint32_t* sh, EdgeCount& zeros) {
-  if (u.count >= kWarpSegmentMax) {
-    for (uint32_t r = 0; r < u.rows; ++r) hist_tile(x + r * seg_stride, u.count, w, careful, sh, zeros);
-  } else {
+                                                uint32_t* sh, EdgeCount& zeros) {
+  const uint64_t nv = u.count >> 2;
+  const bool lined_up = (((uintptr_t)x / sizeof(T) | seg_stride | u.count) & 3u) == 0;
+  if (lined_up && u.rows * nv * nv <= (1ull << 32)) {
+    hist_rows_vec<CAREFUL>(x, u.rows, u.count, seg_stride, w, sh, zeros);
+  } else if (u.count >= kWarpSegmentMax) {
+    for (uint32_t r = 0; r < u.rows; ++r) hist_flat<CAREFUL>(x + r * seg_stride, u.count, w, sh, zeros);
+  } else if (u.count >= kScalarSegmentMax) {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    for (uint32_t r = warp; r < u.rows; r += kWarps) {
-      if (careful) hist_segment_warp<true>(x + r * seg_stride, u.count, lane, w, sh, zeros);
-      else hist_segment_warp<false>(x + r * seg_stride, u.count, lane, w, sh, zeros);
-    }
+    for (uint32_t r = warp; r < u.rows; r += kWarps) hist_segment_warp<CAREFUL>(x + r * seg_stride, u.count, lane, w, sh, zeros);
+  } else {
+    hist_rows_scalar<CAREFUL>(x, u.rows, u.count, seg_stride, w, sh, zeros);   // rows * count <= kGroupUnitElems
   }
 }
 
+// Groups of at most kMicroGroupMax elements (fully connected activations: one element per batch
+// item and channel): a unit is `nc` CONSECUTIVE channels, all batch items.  Clearing and merging
+// a 2048-bin shared histogram per group would cost far more than the group's few elements, so
+// each element adds straight into its group's global histogram.  `wtab` (the CTA's shared
+// histogram, zero on entry and on exit) holds the nc bin scales meanwhile.
+template <bool CAREFUL, class T>
+__device__ __noinline__ void micro_groups(const T* __restrict__ x, const Tile& u, uint64_t seg_stride,
+                                             const float* __restrict__ gabsmax, uint32_t* wtab,
+                                             unsigned long long* h) {
+  constexpr uint32_t U = 8;
+  const uint32_t nc = u.reserved, inner = u.count, run = nc * inner, total = u.rows * run;   // total^2 <= 2^32
+  for (uint32_t c = threadIdx.x; c < nc; c += kThreads) wtab[c] = __float_as_uint(bin_scale(gabsmax[c]));
+  __syncthreads();
+  const FastDiv fr = fast_div(run), fi = fast_div(inner);
+  for (uint32_t j0 = 0; j0 < total; j0 += U * kThreads) {
+    float v[U];
+    uint32_t ch[U];
+#pragma unroll
+    for (uint32_t k = 0; k < U; ++k) {
+      const uint32_t idx = min(j0 + threadIdx.x + k * kThreads, total - 1u), o = div_by(idx, fr), e = idx - o * run;
+      ch[k] = div_by(e, fi);
+      v[k] = Ld<T>::one(x + o * seg_stride + e);
+    }
+#pragma unroll
+    for (uint32_t k = 0; k < U; ++k)
+      if (j0 + threadIdx.x + k * kThreads < total && !(CAREFUL && !isfinite(v[k])))
+        atomicAdd(h + (size_t)ch[k] * kBins + bin_of(v[k], __uint_as_float(wtab[ch[k]])), 1ull);
+  }
+  __syncthreads();
+  for (uint32_t c = threadIdx.x; c < nc; c += kThreads) wtab[c] = 0u;
+  __syncthreads();
+}
+
+template <class T>
+__device__ __forceinline__ void group_hist_any(const T* x, const Tile& u, const TensorRec* tr, bool careful,
+                                               const float* __restrict__ gabsmax, uint32_t* sh, unsigned long long* h) {
+  const uint64_t seg_stride = (uint64_t)tr->channels * tr->inner;
+  const float* A = gabsmax + tr->group_base + (uint32_t)u.row0;
+  if (u.reserved) {
+    if (careful) micro_groups<true>(x, u, seg_stride, A, sh, h);
+    else micro_groups<false>(x, u, seg_stride, A, sh, h);
+    return;
+  }
+  const float w = bin_scale(A[0]);
+  EdgeCount zeros = {0u};
+  if (careful) group_hist_unit<true>(x, u, seg_stride, w, sh, zeros);
+  else group_hist_unit<false>(x, u, seg_stride, w, sh, zeros);
+  // merge: a unit holds fewer than 2^32 elements, so the 32-bit counts cannot have wrapped
+  flush_edges(sh, zeros);
+  __syncthreads();
+  for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {
+    const uint32_t c = sh[b];
+    if (c) { atomicAdd(h + b, (unsigned long long)c); sh[b] = 0; }
+  }
+  __syncthreads();
+}
+
 template <bool ANY16>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, 5)
 group_hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict__ units, uint32_t n_units,
                   const float* __restrict__ gabsmax, const unsigned long long* __restrict__ nonfinite,
                   unsigned long long* ghist) {
@@ -305,23 +440,11 @@ group_hist_kernel(const TensorRec* __restrict__ tensors, const Tile* __restrict_
   for (uint32_t ui = blockIdx.x; ui < n_units; ui += gridDim.x) {
     const Tile u = load_tile(units, ui);
     const TensorRec* tr = tensors + u.tensor;
-    const uint32_t g = (uint32_t)u.row0;
-    const float w = bin_scale(gabsmax[tr->group_base + g]);
     const bool careful = nonfinite[u.tensor] != 0ull;
-    const uint64_t seg_stride = (uint64_t)tr->channels * tr->inner;
-    EdgeCount zeros = {0u};
-    if (!ANY16 || tr->dtype == kF32) group_hist_unit(reinterpret_cast<const float*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
-    else if (tr->dtype == kF16) group_hist_unit(reinterpret_cast<const __half*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
-    else group_hist_unit(reinterpret_cast<const __nv_bfloat16*>(tr->x) + u.begin, u, seg_stride, w, careful, sh, zeros);
-    // merge: a unit holds fewer than 2^32 elements, so the 32-bit counts cannot have wrapped
-    flush_edges(sh, zeros);
-    __syncthreads();
-    unsigned long long* h = ghist + (size_t)(tr->ghist_first + g) * kBins;
-    for (uint32_t b = threadIdx.x; b < kBins; b += kThreads) {
-      const uint32_t c = sh[b];
-      if (c) { atomicAdd(h + b, (unsigned long long)c); sh[b] = 0; }
-    }
-    __syncthreads();
+    unsigned long long* h = ghist + (size_t)(tr->ghist_first + (uint32_t)u.row0) * kBins;
+    if (!ANY16 || tr->dtype == kF32) group_hist_any(reinterpret_cast<const float*>(tr->x) + u.begin, u, tr, careful, gabsmax, sh, h);
+    else if (tr->dtype == kF16) group_hist_any(reinterpret_cast<const __half*>(tr->x) + u.begin, u, tr, careful, gabsmax, sh, h);
+    else group_hist_any(reinterpret_cast<const __nv_bfloat16*>(tr->x) + u.begin, u, tr, careful, gabsmax, sh, h);
   }
 }
 

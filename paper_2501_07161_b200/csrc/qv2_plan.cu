@@ -26,6 +26,8 @@ static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t g
 // Tables larger than this many tiles (4 GB of records; two trillion elements) are refused before
 // any of them is generated.
 constexpr uint64_t kMaxTiles = 1ull << 27;
+constexpr uint64_t kMicroGroupMax = 2048;    // per-group histograms: groups this small are packed into micro units ...
+constexpr uint64_t kMicroUnitElems = 8192;   // ... of about this many elements (the kernel needs the square to fit 32 bits)
 
 static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const GridCaps& caps,
                               uint64_t chunk_bytes, uint32_t fold_mode, HostPlan* out) {
@@ -101,6 +103,9 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
       if (!r.per_channel) {
         cut_flat(t, 0, ne, 0, &out->tiles);
       } else if (d.inner >= kRowTileMin) {
+        // (Cutting a row into equal tiles, or dealing its 8192-element rounds evenly so that no
+        // tile is a sliver, was measured on 50176-element rows: the metrics kernel gains 3 %, the
+        // range kernel loses as much, the pass stays within 0.6 % either way.)
         for (uint64_t row = 0; row < rows; ++row)
           cut_flat(t, row * d.inner, d.inner, row % d.channels, &out->tiles);
       } else {
@@ -122,14 +127,26 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
         // ONE group, segment k starting at begin + k * channels * inner (the same channel of the
         // next batch item).  A unit holds about kGroupUnitElems elements so that a CTA merges its
         // shared-memory histogram once per unit; rows longer than kGroupSegMax are cut.
+        // Groups of at most kMicroGroupMax elements are packed instead: a unit is `reserved`
+        // consecutive channels (count = inner, rows = outer, begin at the first channel of batch
+        // item 0), about kMicroUnitElems elements and at most one bin-scale table of channels.
         const uint64_t per = kGroupUnitElems / d.inner ? kGroupUnitElems / d.inner : 1;   // rows per unit
+        const uint64_t group_elems = d.outer * d.inner;
+        const bool micro = group_elems <= kMicroGroupMax;
+        uint64_t pack = micro ? kMicroUnitElems / group_elems : 1;     // channels per micro unit
+        if (pack > kBins) pack = kBins;
         const uint64_t per_group = d.inner > kGroupSegMax
             ? d.outer * ((d.inner + kGroupSegMax - 1) / kGroupSegMax) : (d.outer + per - 1) / per;
         uint64_t total;
         if (mul_overflows(per_group, d.channels, &total) || out->ghist_tiles.size() + total > (1ull << 26))
           return QV2_ERR_SIZE;
-        for (uint64_t c = 0; c < d.channels; ++c) {
-          if (d.inner > kGroupSegMax) {
+        for (uint64_t c = 0; c < d.channels; c += pack) {
+          if (micro) {
+            Tile u;
+            u.begin = c * d.inner; u.row0 = c; u.count = (uint32_t)d.inner; u.tensor = t;
+            u.rows = (uint32_t)d.outer; u.reserved = (uint32_t)(d.channels - c < pack ? d.channels - c : pack);
+            out->ghist_tiles.push_back(u);
+          } else if (d.inner > kGroupSegMax) {
             for (uint64_t o = 0; o < d.outer; ++o)
               for (uint64_t off = 0; off < d.inner; off += kGroupSegMax) {
                 Tile u;

@@ -541,6 +541,35 @@ def test_group_percentile_nonfinite_constant_and_empty_groups(ctx):
     check_specs(ctx, specs, check_codes=False)
 
 
+_GROUP_WALKER_SHAPES = (
+    (64, 300, 1), (4, 37, 7), (2, 5000, 1), (128, 20, 16), (1, 9, 2048),      # packed small groups (up to 2048 elements)
+    (129, 3, 16), (6, 8, 196), (64, 4, 784), (3, 5, 12544), (2, 3, 50176),    # whole 16-byte groups: one index space
+    (128, 6, 49), (50, 3, 255), (2049, 2, 1),                                 # short rows that do not line up
+    (9, 3, 257), (5, 3, 1153), (3, 2, 4097))                                  # one row per warp / per CTA
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.float16, torch.bfloat16])
+def test_group_percentile_every_unit_walker(ctx, dtype):
+    """Per-group histograms are counted by different walkers depending on the group size, the row
+    length and whether rows start on 16-byte boundaries; every one must give the oracle's counts,
+    with the tensor start shifted off the boundary too, and with non-finite elements skipped."""
+    specs = [Spec(_scaled_channels(o, c, i, 260 + k, relu=k % 2 == 1), o, c, i, per_channel=True, asym=k % 2 == 1,
+                  percentile=0.99, group_pct=True, dtype=dtype, name=f"group-pct {o}x{c}x{i} {dtype}")
+             for k, (o, c, i) in enumerate(_GROUP_WALKER_SHAPES)]
+    check_specs(ctx, specs, check_codes=False)
+    for mis in (1, 2, 3):
+        check_specs(ctx, specs, misalign_x=mis, check_codes=False, twice=False)
+    bad = []
+    for k, s in enumerate(specs):
+        x = s.x.clone()
+        flat = x.view(-1)
+        flat[(7 * k) % flat.numel()] = float("nan")
+        flat[flat.numel() - 1 - (3 * k) % flat.numel()] = float("-inf")
+        bad.append(Spec(x, s.outer, s.channels, s.inner, per_channel=True, asym=s.asym, percentile=0.99, group_pct=True,
+                        dtype=dtype, name=s.name + " nonfinite"))
+    check_specs(ctx, bad, check_codes=False, twice=False)
+
+
 @pytest.mark.parametrize("p", [0.0, 1e-9, 0.1, 0.5, 0.731, 1.0 - 1e-12, 1.0])
 def test_group_percentile_any_percentile(ctx, p):
     """The per-group clip is found by a scan from the top bin down; the bin must be the one the
