@@ -626,7 +626,7 @@ def test_group_percentile_in_the_chained_pass_and_its_graph(ctx):
 
 
 # ------------------------------------------------- the row walkers and the row lengths at which they change
-@pytest.mark.parametrize("inner", [1, 2, 3, 4, 5, 9, 27, 49, 127, 128, 196, 319, 320, 321, 510, 511, 512, 513, 1021])
+@pytest.mark.parametrize("inner", [1, 2, 3, 4, 5, 7, 8, 9, 13, 27, 49, 127, 128, 196, 319, 320, 321, 510, 511, 512, 513, 1021])
 def test_short_rows_per_channel_all_modes(ctx, inner):
     """The range kernel walks rows below 320 elements lane-contiguously (32 consecutive elements per
     thread) and longer ones in per-warp chunks; the metrics kernel fetches parameters per 16-byte
@@ -661,6 +661,13 @@ def test_short_rows_with_nonfinite_elements_and_many_rows_per_tile(ctx):
     x[:, 7, :] = 0.0
     check_specs(ctx, [Spec(x, o, c, inner, per_channel=True), Spec(x, o, c, inner, per_channel=True, asym=True)],
                 check_codes=False)
+    o, c, inner = 4, 300, 50                      # rows that straddle 16-byte groups, a row without a finite element
+    z = _scaled_channels(o, c, inner, 502)
+    z[1, 17, :] = float("nan"); z[0, 17, :] = float("inf"); z[2, 17, :] = float("-inf"); z[3, 17, :] = float("nan")
+    z[3, 299, 49] = float("inf"); z[0, 0, 0] = float("nan"); z[2, 100, 3:5] = float("nan")
+    for mis in (0, 1, 3):
+        check_specs(ctx, [Spec(z, o, c, inner, per_channel=True), Spec(z, o, c, inner, per_channel=True, asym=True)],
+                    misalign_x=mis, check_codes=False, twice=False)
 
 
 # ----------------------------------------------------------------------- seeded random descriptor sets
