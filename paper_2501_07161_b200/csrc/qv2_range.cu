@@ -220,8 +220,10 @@ template <> struct LdCached<__nv_bfloat16> {
 // down to a single element and of any alignment take the same path.  Non-finite elements are
 // tested per element here (the flat path's redo-the-warp scheme would have to hold back every
 // publication until the warp has voted).  Out of line, so that the flat path keeps its registers.
-// The lane-contiguous loads cost eight times the L1 tag lookups of coalesced ones, which caps this
-// walker near 2.7 TB/s; below about 300 elements per row it still beats the per-warp chunks of
+// This walker runs near 2.7 TB/s.  The cap is the serial per-element walk, not the load pattern:
+// coalesced loads regrouped through shared memory gave the same times, and a coalesced variant
+// that reduces the run of lanes holding a row with warp votes was slower.  Below about 300
+// elements per row it still beats the per-warp chunks of
 // range_rows_tile (one round trip per row piece), above it does not: 32x256x196 takes 94 against
 // 120 us per 257 MB, 1000x512 36 against 24 us per 82 MB.  In a same-box A/B thresholds of 320 and
 // 640 gave the same times on ResNet-18/50 and MobileNet-v2 shapes, 128 and 1024 worse ones.
