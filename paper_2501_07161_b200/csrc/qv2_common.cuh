@@ -68,13 +68,17 @@ struct TensorRec {
 //  rows == 0: every element belongs to quantization group `row0` (0 for per-tensor tensors).
 //  rows  > 0: `rows` whole rows of `inner` elements starting at row `row0`; the group of row r
 //             is r % channels.
+// In the unit table of the per-group histograms a record means something else: `rows` segments
+// of `count` elements of group `row0`, segment k at begin + k * channels * inner; and when
+// `pack` > 0, `pack` consecutive groups row0, row0 + 1, ... taken together (count = inner,
+// rows = outer).  `pack` is 0 in the tile tables.
 struct Tile {
   uint64_t begin;
   uint64_t row0;
   uint32_t count;
   uint32_t tensor;
   uint32_t rows;
-  uint32_t reserved;
+  uint32_t pack;
 };
 static_assert(sizeof(Tile) == 32, "Tile is read as two 16-byte words");
 

@@ -79,7 +79,7 @@ __device__ __forceinline__ Tile load_tile(const Tile* tiles, uint32_t i) {
   Tile t;
   t.begin = (uint64_t)a.x | ((uint64_t)a.y << 32);
   t.row0 = (uint64_t)a.z | ((uint64_t)a.w << 32);
-  t.count = b.x; t.tensor = b.y; t.rows = b.z; t.reserved = b.w;
+  t.count = b.x; t.tensor = b.y; t.rows = b.z; t.pack = b.w;
   return t;
 }
 

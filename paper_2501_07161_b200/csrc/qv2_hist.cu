@@ -382,7 +382,7 @@ __device__ __noinline__ void micro_groups(const T* __restrict__ x, const Tile& u
                                              const float* __restrict__ gabsmax, uint32_t* wtab,
                                              unsigned long long* h) {
   constexpr uint32_t U = 8;
-  const uint32_t nc = u.reserved, inner = u.count, run = nc * inner, total = u.rows * run;   // total^2 <= 2^32
+  const uint32_t nc = u.pack, inner = u.count, run = nc * inner, total = u.rows * run;   // total^2 <= 2^32
   for (uint32_t c = threadIdx.x; c < nc; c += kThreads) wtab[c] = __float_as_uint(bin_scale(gabsmax[c]));
   __syncthreads();
   const FastDiv fr = fast_div(run), fi = fast_div(inner);
@@ -410,7 +410,7 @@ __device__ __forceinline__ void group_hist_any(const T* x, const Tile& u, const 
                                                const float* __restrict__ gabsmax, uint32_t* sh, unsigned long long* h) {
   const uint64_t seg_stride = (uint64_t)tr->channels * tr->inner;
   const float* A = gabsmax + tr->group_base + (uint32_t)u.row0;
-  if (u.reserved) {
+  if (u.pack) {
     if (careful) micro_groups<true>(x, u, seg_stride, A, sh, h);
     else micro_groups<false>(x, u, seg_stride, A, sh, h);
     return;

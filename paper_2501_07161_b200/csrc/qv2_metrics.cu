@@ -756,7 +756,7 @@ struct NoAllocJob {
 // The same decomposition as the host planner, evaluated on the fly for one tensor.
 __device__ __forceinline__ Tile noalloc_tile(const NoAllocJob& j, uint32_t ti) {
   Tile t;
-  t.tensor = 0; t.reserved = 0;
+  t.tensor = 0; t.pack = 0;
   if (j.cut == 0) {
     t.begin = (uint64_t)ti * kTileElems;
     const uint64_t left = j.tr.n_elems - t.begin;

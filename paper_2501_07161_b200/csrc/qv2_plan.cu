@@ -17,7 +17,7 @@ static void cut_flat(uint32_t tensor, uint64_t begin, uint64_t count, uint64_t g
   while (count > 0) {
     uint32_t c = count > kTileElems ? kTileElems : (uint32_t)count;
     Tile t;
-    t.begin = begin; t.row0 = group; t.count = c; t.tensor = tensor; t.rows = 0; t.reserved = 0;
+    t.begin = begin; t.row0 = group; t.count = c; t.tensor = tensor; t.rows = 0; t.pack = 0;
     tiles->push_back(t);
     begin += c; count -= c;
   }
@@ -117,7 +117,7 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
           uint64_t nr = rows - row < per ? rows - row : per;
           Tile tl;
           tl.begin = row * d.inner; tl.row0 = row; tl.count = (uint32_t)(nr * d.inner);
-          tl.tensor = t; tl.rows = (uint32_t)nr; tl.reserved = 0;
+          tl.tensor = t; tl.rows = (uint32_t)nr; tl.pack = 0;
           out->tiles.push_back(tl);
         }
       }
@@ -127,7 +127,7 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
         // ONE group, segment k starting at begin + k * channels * inner (the same channel of the
         // next batch item).  A unit holds about kGroupUnitElems elements so that a CTA merges its
         // shared-memory histogram once per unit; rows longer than kGroupSegMax are cut.
-        // Groups of at most kMicroGroupMax elements are packed instead: a unit is `reserved`
+        // Groups of at most kMicroGroupMax elements are packed instead: a unit is `pack`
         // consecutive channels (count = inner, rows = outer, begin at the first channel of batch
         // item 0), about kMicroUnitElems elements and at most one bin-scale table of channels.
         const uint64_t per = kGroupUnitElems / d.inner ? kGroupUnitElems / d.inner : 1;   // rows per unit
@@ -144,7 +144,7 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
           if (micro) {
             Tile u;
             u.begin = c * d.inner; u.row0 = c; u.count = (uint32_t)d.inner; u.tensor = t;
-            u.rows = (uint32_t)d.outer; u.reserved = (uint32_t)(d.channels - c < pack ? d.channels - c : pack);
+            u.rows = (uint32_t)d.outer; u.pack = (uint32_t)(d.channels - c < pack ? d.channels - c : pack);
             out->ghist_tiles.push_back(u);
           } else if (d.inner > kGroupSegMax) {
             for (uint64_t o = 0; o < d.outer; ++o)
@@ -152,14 +152,14 @@ static int build_plan_checked(const qv2_tensor_desc* descs, uint32_t n, const Gr
                 Tile u;
                 u.begin = (o * d.channels + c) * d.inner + off; u.row0 = c;
                 u.count = (uint32_t)(d.inner - off < kGroupSegMax ? d.inner - off : kGroupSegMax);
-                u.tensor = t; u.rows = 1; u.reserved = 0;
+                u.tensor = t; u.rows = 1; u.pack = 0;
                 out->ghist_tiles.push_back(u);
               }
           } else {
             for (uint64_t o = 0; o < d.outer; o += per) {
               Tile u;
               u.begin = (o * d.channels + c) * d.inner; u.row0 = c; u.count = (uint32_t)d.inner;
-              u.tensor = t; u.rows = (uint32_t)(d.outer - o < per ? d.outer - o : per); u.reserved = 0;
+              u.tensor = t; u.rows = (uint32_t)(d.outer - o < per ? d.outer - o : per); u.pack = 0;
               out->ghist_tiles.push_back(u);
             }
           }
